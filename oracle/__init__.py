@@ -1,0 +1,9 @@
+"""CPU oracle of the batched egocentric rasterizer -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper around ``pic_oracle.c`` (plain C, double precision, brute force).  Only the
+tests, the smoke check and the benchmark's CPU-baseline leg may import this package; the product
+package never does, and this package never imports the product.
+"""
+from .wrapper import build, render, step, f64_to_f16_bits, max_threads, OracleResult
+
+__all__ = ["build", "render", "step", "f64_to_f16_bits", "max_threads", "OracleResult"]

@@ -1,0 +1,405 @@
+/*
+ * pic_oracle.c -- TEST INFRASTRUCTURE, not product code.
+ *
+ * A plain, slow, double-precision CPU statement of what the batched egocentric rasterizer
+ * computes: for every requested (env, agent, camera) view and every pixel, a loop over ALL
+ * primitives of the environment (every map triangle, then the 12 triangles of every other
+ * active agent's box) -- no culling, no binning, no tiling.  It exists so that the CUDA path can
+ * be compared against an independent definition; it shares no code with that path and nothing
+ * in the product may call it (only tests, the smoke check and the benchmark's CPU-baseline leg).
+ *
+ * What is computed follows the paper's statement of the rasterizer (Sec. 3.2, Eq. 2: each
+ * image is a deterministic function of the surrounding agents, the map geometry and one
+ * camera of the ego-mounted rig; only the surroundings are drawn, never the ego itself) with the
+ * frame conventions of its camera-rig table (agent frame x forward, y left, z up, yaw about z;
+ * intrinsics given as a focal length in pixels, principal point at the image centre).  A rig row
+ * is (mount x, y, z, yaw, pitch, fx, fy).  The paper fixes no
+ * sampling, fill or depth rule; the ones used here are the steps O1..O9 below:
+ *
+ *  O1 camera      q = X - P_agent; q' = q - Rz(yaw_agent) m; X_c = (r.q', d.q', f.q') with
+ *                 f = (cos(pitch)cos(a), cos(pitch)sin(a), sin(pitch)), r = (sin a, -cos a, 0), d = f x r,
+ *                 a = yaw_agent + yaw_cam.  Pixel (u,v) samples the ray
+ *                 rho = ((u+0.5-W/2)/fx, (v+0.5-H/2)/fy, 1).
+ *  O2 background  world-z of the ray w = -rho_y cos(pitch) + sin(pitch); w<0 and camera above the
+ *                 ground: class ground, depth min(far, C_z/(-w)); else sky at depth far.
+ *  O3 primitives  map triangles in the given order (index 0..N-1), then box triangle t of agent b
+ *                 at index N + 12 b + t (ego and inactive agents skipped).
+ *  O4 coverage    N0=V1xV2, N1=V2xV0, N2=V0xV1, D=V0.N0 (sign-normalised to D>0), E_i = rho.N_i;
+ *                 covered iff every E_i>0, or E_i==0 on a top-left edge (N_i.x>0, or ==0 and
+ *                 N_i.y>0 -- fx, fy are positive so the division is dropped), and S=E0+E1+E2>0.
+ *  O5 depth       z = D/S, kept iff near <= z <= far.
+ *  O6 resolve     smallest z wins, exact ties go to the lower index; any kept fragment replaces
+ *                 the background.
+ *  O7 output      class u8, depth as f64 and rounded to binary16 (round-to-nearest-even).
+ *  O8 ambiguity   pixels where a 1e-5 relative perturbation of an edge function, a depth gap, a
+ *                 clip plane or the horizon could change the answer are flagged, so that a float32
+ *                 implementation may legitimately differ there (and only there).
+ *  O9 stepping    explicit-Euler kinematic bicycle update (pico_step).
+ *
+ * Parity pins: tests/test_oracle_*.py (closed forms, invariants, an independent ray caster,
+ * hand-counted tiny scenes, numpy's binary16 conversion).  No function here is unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define REL_TOL 1e-5
+
+typedef struct { double x, y, z; } v3;
+
+static v3 v3_sub(v3 a, v3 b) { v3 r = { a.x - b.x, a.y - b.y, a.z - b.z }; return r; }
+static v3 v3_cross(v3 a, v3 b) {
+    v3 r = { a.y * b.z - a.z * b.y, a.z * b.x - a.x * b.z, a.x * b.y - a.y * b.x };
+    return r;
+}
+static double v3_dot(v3 a, v3 b) { return a.x * b.x + a.y * b.y + a.z * b.z; }
+static double v3_norm(v3 a) { return sqrt(v3_dot(a, a)); }
+
+/* One primitive of a view after O1/O4 set-up. */
+typedef struct {
+    v3 N[3];          /* sign-normalised edge normals */
+    double D;         /* sign-normalised, > 0; 0 marks a skipped (degenerate / edge-on) primitive */
+    double band[3];   /* O8 edge band without the |rho| factor */
+    int32_t index;    /* global primitive index (O3) */
+    uint8_t cls;
+} prim_t;
+
+typedef struct {
+    v3 P;             /* agent position (z = 0) */
+    v3 mw;            /* Rz(yaw_agent) * mount */
+    v3 r, d, f;       /* camera basis in world coordinates */
+    double fx, fy, cx, cy, pitch, cz;
+} cam_t;
+
+/* O1: world point -> camera space. */
+static v3 to_camera(const cam_t* c, v3 X) {
+    v3 q = v3_sub(X, c->P);
+    v3 qp = v3_sub(q, c->mw);
+    v3 r = { v3_dot(c->r, qp), v3_dot(c->d, qp), v3_dot(c->f, qp) };
+    return r;
+}
+
+static void make_camera(cam_t* c, const float* pose, const float* cam, int H, int W) {
+    double th = (double)pose[2];
+    double mx = cam[0], my = cam[1], mz = cam[2], yaw = cam[3], pitch = cam[4];
+    double a = th + yaw;
+    c->P.x = pose[0]; c->P.y = pose[1]; c->P.z = 0.0;
+    c->mw.x = cos(th) * mx - sin(th) * my;
+    c->mw.y = sin(th) * mx + cos(th) * my;
+    c->mw.z = mz;
+    c->f.x = cos(pitch) * cos(a); c->f.y = cos(pitch) * sin(a); c->f.z = sin(pitch);
+    c->r.x = sin(a); c->r.y = -cos(a); c->r.z = 0.0;
+    c->d = v3_cross(c->f, c->r);
+    c->fx = cam[5];                       /* focal lengths in pixels, as given */
+    c->fy = cam[6];
+    c->cx = W / 2.0; c->cy = H / 2.0;
+    c->pitch = pitch;
+    c->cz = mz;
+}
+
+/* O4 set-up of one triangle given in camera space. */
+static void setup_prim(prim_t* p, v3 V0, v3 V1, v3 V2, int32_t index, uint8_t cls) {
+    p->N[0] = v3_cross(V1, V2);
+    p->N[1] = v3_cross(V2, V0);
+    p->N[2] = v3_cross(V0, V1);
+    p->D = v3_dot(V0, p->N[0]);
+    if (p->D < 0.0) {
+        for (int i = 0; i < 3; ++i) { p->N[i].x = -p->N[i].x; p->N[i].y = -p->N[i].y; p->N[i].z = -p->N[i].z; }
+        p->D = -p->D;
+    }
+    /* edge i is opposite vertex i: (V1,V2), (V2,V0), (V0,V1) */
+    double n0 = v3_norm(V0), n1 = v3_norm(V1), n2 = v3_norm(V2);
+    p->band[0] = REL_TOL * fmax(n1, n2) * v3_norm(v3_sub(V2, V1));
+    p->band[1] = REL_TOL * fmax(n2, n0) * v3_norm(v3_sub(V0, V2));
+    p->band[2] = REL_TOL * fmax(n0, n1) * v3_norm(v3_sub(V1, V0));
+    p->index = index;
+    p->cls = cls;
+}
+
+/* O3: the 12 triangles of agent b's box, in world coordinates. */
+static void box_triangles(const float* pose, const float* dim, v3 tri[12][3]) {
+    static const int face[6][4] = {
+        {0, 2, 6, 4},  /* rear  (-x) */
+        {1, 5, 7, 3},  /* front (+x) */
+        {0, 4, 5, 1},  /* right (-y) */
+        {2, 3, 7, 6},  /* left  (+y) */
+        {0, 1, 3, 2},  /* bottom     */
+        {4, 6, 7, 5},  /* top        */
+    };
+    double x = pose[0], y = pose[1], th = pose[2];
+    double hl = dim[0] / 2.0, hw = dim[1] / 2.0, h = dim[2];
+    v3 c[8];
+    for (int i = 0; i < 8; ++i) {
+        double sx = (i & 1) ? hl : -hl;
+        double sy = (i & 2) ? hw : -hw;
+        c[i].x = x + cos(th) * sx - sin(th) * sy;
+        c[i].y = y + sin(th) * sx + cos(th) * sy;
+        c[i].z = (i & 4) ? h : 0.0;
+    }
+    for (int f = 0; f < 6; ++f) {
+        tri[2 * f][0] = c[face[f][0]]; tri[2 * f][1] = c[face[f][1]]; tri[2 * f][2] = c[face[f][2]];
+        tri[2 * f + 1][0] = c[face[f][0]]; tri[2 * f + 1][1] = c[face[f][2]]; tri[2 * f + 1][2] = c[face[f][3]];
+    }
+}
+
+/* O7: double -> IEEE binary16 bits, round-to-nearest-even (default rounding mode assumed). */
+uint16_t pico_f64_to_f16(double z) {
+    uint16_t sign = 0;
+    if (z != z) return 0x7e00;
+    if (z < 0.0) { sign = 0x8000; z = -z; }
+    if (z == 0.0) return sign;
+    if (isinf(z)) return sign | 0x7c00;
+    int e;
+    (void)frexp(z, &e);               /* z = m 2^e, 0.5 <= m < 1  => exponent of the leading bit is e-1 */
+    int lead = e - 1;
+    if (lead < -14) lead = -14;       /* subnormal quantum 2^-24 */
+    double quantum = ldexp(1.0, lead - 10);
+    double r = nearbyint(z / quantum);   /* exact scaling, ties-to-even */
+    if (r >= 2048.0) { r /= 2.0; lead += 1; }
+    if (lead > 15) return sign | 0x7c00;
+    if (r < 1024.0) return sign | (uint16_t)r;     /* subnormal (lead == -14) */
+    return sign | (uint16_t)(((lead + 15) << 10) | ((int)r - 1024));
+}
+
+/* Sutherland-Hodgman clip of a convex polygon against a.x*X + a.y*Y + a.z*Z + w >= 0. */
+static int clip_poly(const v3* in, int n, v3 a, double w, v3* out) {
+    int m = 0;
+    for (int i = 0; i < n; ++i) {
+        v3 p = in[i], q = in[(i + 1) % n];
+        double dp = v3_dot(a, p) + w, dq = v3_dot(a, q) + w;
+        if (dp >= 0.0) out[m++] = p;
+        if ((dp >= 0.0) != (dq >= 0.0)) {
+            double t = dp / (dp - dq);
+            v3 x = { p.x + t * (q.x - p.x), p.y + t * (q.y - p.y), p.z + t * (q.z - p.z) };
+            out[m++] = x;
+        }
+    }
+    return m;
+}
+
+/* Does the camera-space triangle meet the view frustum (closed)?  Only used for the work counts. */
+static int meets_frustum(v3 V0, v3 V1, v3 V2, double tx, double ty, double near, double far) {
+    v3 a[16], b[16];
+    a[0] = V0; a[1] = V1; a[2] = V2;
+    int n = 3;
+    v3 pl[6] = { {0, 0, 1}, {0, 0, -1}, {1, 0, tx}, {-1, 0, tx}, {0, 1, ty}, {0, -1, ty} };
+    double w[6] = { -near, far, 0, 0, 0, 0 };
+    for (int i = 0; i < 6 && n > 0; ++i) {
+        n = clip_poly(a, n, pl[i], w[i], b);
+        memcpy(a, b, sizeof(v3) * (size_t)n);
+    }
+    return n > 0;
+}
+
+/*
+ * Render the listed views.  view_ids[i] = (e*A + a)*K + k.  Outputs are [n_views, H, W]:
+ *   out_class  u8      O6/O7 class
+ *   out_depth  f64     O5/O6 depth (metres along the optical axis)
+ *   out_f16    u16     O7 binary16 bits of the depth
+ *   out_index  i32     global index of the winning primitive, -1 for background
+ *   out_flag   u8      O8 bit mask: 1 edge, 2 depth gap, 4 near/far plane, 8 horizon
+ *   counts     i64 [n_views,4]: primitives meeting the frustum, primitives with >=1 kept
+ *              fragment, kept fragments, flagged pixels
+ * Any output pointer may be NULL.  Returns 0, or -1 on allocation failure.
+ */
+int pico_render(int E, int A, int K, int H, int W, double near, double far,
+                const int32_t* env_map_id, const int64_t* map_tri_offset,
+                const float* tri_xyz, const uint8_t* tri_class,
+                int agent_class, int sky_class, int ground_class,
+                const float* poses, const float* dims, const uint8_t* active, const float* rig,
+                int n_views, const int64_t* view_ids,
+                uint8_t* out_class, double* out_depth, uint16_t* out_f16, int32_t* out_index,
+                uint8_t* out_flag, int64_t* counts, int n_threads)
+{
+    (void)E;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+    int failed = 0;
+    for (int vi = 0; vi < n_views; ++vi) {
+        int64_t id = view_ids[vi];
+        int k = (int)(id % K);
+        int a = (int)((id / K) % A);
+        int e = (int)(id / ((int64_t)K * A));
+        size_t base = (size_t)vi * (size_t)H * (size_t)W;
+        const float* cam = rig + 7 * k;
+
+        /* inactive ego: sky everywhere */
+        if (active && !active[(size_t)e * A + a]) {
+            for (size_t p = 0; p < (size_t)H * W; ++p) {
+                if (out_class) out_class[base + p] = (uint8_t)sky_class;
+                if (out_depth) out_depth[base + p] = far;
+                if (out_f16) out_f16[base + p] = pico_f64_to_f16(far);
+                if (out_index) out_index[base + p] = -1;
+                if (out_flag) out_flag[base + p] = 0;
+            }
+            if (counts) memset(counts + 4 * (size_t)vi, 0, 4 * sizeof(int64_t));
+            continue;
+        }
+
+        cam_t c;
+        make_camera(&c, poses + 3 * ((size_t)e * A + a), cam, H, W);
+
+        /* O3 + O4 set-up of every primitive of the environment */
+        int m = env_map_id[e];
+        int64_t t0 = map_tri_offset[m], t1 = map_tri_offset[m + 1];
+        int64_t n_map = t1 - t0;
+        int64_t n_prim = n_map + 12 * (int64_t)A;
+        prim_t* prim = (prim_t*)malloc(sizeof(prim_t) * (size_t)n_prim);
+        uint8_t* hit = (uint8_t*)calloc((size_t)n_prim, 1);
+        if (!prim || !hit) { free(prim); free(hit); failed = 1; break; }
+        int64_t np = 0, t_vis = 0;
+        double tx = (W / 2.0) / c.fx, ty = (H / 2.0) / c.fy;
+        for (int64_t t = 0; t < n_map; ++t) {
+            const float* p = tri_xyz + 9 * (size_t)(t0 + t);
+            v3 X0 = { p[0], p[1], p[2] }, X1 = { p[3], p[4], p[5] }, X2 = { p[6], p[7], p[8] };
+            v3 V0 = to_camera(&c, X0), V1 = to_camera(&c, X1), V2 = to_camera(&c, X2);
+            setup_prim(&prim[np], V0, V1, V2, (int32_t)t, tri_class[t0 + t]);
+            if (prim[np].D != 0.0 && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
+            ++np;
+        }
+        for (int b = 0; b < A; ++b) {
+            if (b == a) continue;                                   /* the ego is never drawn */
+            if (active && !active[(size_t)e * A + b]) continue;
+            v3 tri[12][3];
+            box_triangles(poses + 3 * ((size_t)e * A + b), dims + 3 * ((size_t)e * A + b), tri);
+            for (int t = 0; t < 12; ++t) {
+                v3 V0 = to_camera(&c, tri[t][0]), V1 = to_camera(&c, tri[t][1]), V2 = to_camera(&c, tri[t][2]);
+                setup_prim(&prim[np], V0, V1, V2, (int32_t)(n_map + 12 * b + t), (uint8_t)agent_class);
+                if (prim[np].D != 0.0 && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
+                ++np;
+            }
+        }
+
+        int64_t n_frag = 0, n_flag = 0;
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : n_frag, n_flag)
+        for (int v = 0; v < H; ++v) {
+            for (int u = 0; u < W; ++u) {
+                v3 rho = { (u + 0.5 - c.cx) / c.fx, (v + 0.5 - c.cy) / c.fy, 1.0 };
+                double rho_n = v3_norm(rho);
+
+                /* O4-O6: nearest kept fragment */
+                double z_win = 0.0; int32_t i_win = -1; uint8_t c_win = 0;
+                for (int64_t j = 0; j < np; ++j) {
+                    const prim_t* p = &prim[j];
+                    if (p->D == 0.0) continue;
+                    int covered = 1;
+                    double S = 0.0;
+                    for (int i = 0; i < 3; ++i) {
+                        double Ei = v3_dot(rho, p->N[i]);
+                        S += Ei;
+                        if (Ei > 0.0) continue;
+                        if (Ei == 0.0 && (p->N[i].x > 0.0 || (p->N[i].x == 0.0 && p->N[i].y > 0.0))) continue;
+                        covered = 0;
+                    }
+                    if (!covered || !(S > 0.0)) continue;
+                    double z = p->D / S;
+                    if (z < near || z > far) continue;
+                    ++n_frag;
+                    if (!hit[j]) {
+#pragma omp atomic write
+                        hit[j] = 1;
+                    }
+                    if (i_win < 0 || z < z_win || (z == z_win && p->index < i_win)) {
+                        z_win = z; i_win = p->index; c_win = p->cls;
+                    }
+                }
+
+                /* O2: background */
+                double w = -rho.y * cos(c.pitch) + sin(c.pitch);
+                uint8_t cls; double depth;
+                if (i_win >= 0) { cls = c_win; depth = z_win; }
+                else if (w < 0.0 && c.cz > 0.0) { cls = (uint8_t)ground_class; depth = fmin(far, c.cz / (-w)); }
+                else { cls = (uint8_t)sky_class; depth = far; }
+
+                /* O8: ambiguity mask */
+                uint8_t flag = 0;
+                if (i_win < 0 && fabs(w) <= REL_TOL) flag |= 8;
+                for (int64_t j = 0; j < np; ++j) {
+                    const prim_t* p = &prim[j];
+                    if (p->D == 0.0) continue;
+                    double Ei[3], S = 0.0;
+                    int inside_band = 1, on_band = 0, covered = 1;
+                    for (int i = 0; i < 3; ++i) {
+                        Ei[i] = v3_dot(rho, p->N[i]);
+                        S += Ei[i];
+                        double band = p->band[i] * rho_n;
+                        if (Ei[i] < -band) inside_band = 0;
+                        if (fabs(Ei[i]) <= band) on_band = 1;
+                        if (!(Ei[i] > 0.0 ||
+                              (Ei[i] == 0.0 && (p->N[i].x > 0.0 || (p->N[i].x == 0.0 && p->N[i].y > 0.0)))))
+                            covered = 0;
+                    }
+                    if (!(S > 0.0)) continue;
+                    double z = p->D / S;
+                    int could_show = (i_win < 0) || (z <= (1.0 + REL_TOL) * z_win);
+                    /* (i) pixel centre within the band of p's boundary */
+                    if (inside_band && on_band && could_show &&
+                        z >= near * (1.0 - REL_TOL) && z <= far * (1.0 + REL_TOL)) flag |= 1;
+                    if (!covered) continue;
+                    /* (ii) a kept fragment of another class almost as near as the winner */
+                    if (i_win >= 0 && z >= near && z <= far && p->cls != c_win &&
+                        fabs(z - z_win) <= REL_TOL * z_win) flag |= 2;
+                    /* (iii) a covered fragment sitting on the near or far plane that matters */
+                    if ((fabs(z - near) <= REL_TOL * near || fabs(z - far) <= REL_TOL * far) && could_show) flag |= 4;
+                }
+                if (flag) ++n_flag;
+
+                size_t o = base + (size_t)v * W + u;
+                if (out_class) out_class[o] = cls;
+                if (out_depth) out_depth[o] = depth;
+                if (out_f16) out_f16[o] = pico_f64_to_f16(depth);
+                if (out_index) out_index[o] = i_win;
+                if (out_flag) out_flag[o] = flag;
+            }
+        }
+        if (counts) {
+            int64_t t_hit = 0;
+            for (int64_t j = 0; j < np; ++j) t_hit += hit[j];
+            counts[4 * (size_t)vi + 0] = t_vis;
+            counts[4 * (size_t)vi + 1] = t_hit;
+            counts[4 * (size_t)vi + 2] = n_frag;
+            counts[4 * (size_t)vi + 3] = n_flag;
+        }
+        free(prim);
+        free(hit);
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * O9: one explicit-Euler step of the kinematic bicycle model, everything from the old state:
+ *   x' = x + v cos(yaw) dt,  y' = y + v sin(yaw) dt,  yaw' = yaw + (v / wheelbase) tan(steer) dt,
+ *   v' = clamp(v + accel dt, 0, v_max).   state f64 [n,4] (x, y, yaw, v) in place;
+ *   actions f32 [n,2] (accel, steer); inactive agents do not move.
+ */
+void pico_step(double* state, const float* actions, const uint8_t* active, int64_t n,
+               double dt, double wheelbase, double v_max)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        if (active && !active[i]) continue;
+        double x = state[4 * i], y = state[4 * i + 1], th = state[4 * i + 2], v = state[4 * i + 3];
+        double acc = actions[2 * i], steer = actions[2 * i + 1];
+        state[4 * i + 0] = x + v * cos(th) * dt;
+        state[4 * i + 1] = y + v * sin(th) * dt;
+        state[4 * i + 2] = th + (v / wheelbase) * tan(steer) * dt;
+        double vn = v + acc * dt;
+        if (vn < 0.0) vn = 0.0;
+        if (vn > v_max) vn = v_max;
+        state[4 * i + 3] = vn;
+    }
+}
+
+int pico_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

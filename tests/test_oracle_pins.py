@@ -1,0 +1,510 @@
+"""Pins of the CPU oracle against things other than itself: closed forms worked by hand, values the
+paper prints (camera table), invariants, an independent world-space ray caster, hand-counted tiny
+scenes and a library binary16 conversion.  No GPU needed."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from scenes import make_config, make_rig, custom_scene, focal_px
+from tests.util import single_env, compare_images
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+CAR = (4.5, 1.9, 1.5)
+
+
+def ego(x=0.0, y=0.0, yaw=0.0, dims=CAR):
+    return (x, y, yaw) + tuple(dims)
+
+
+# ------------------------------------------------------------------------------------------------
+# closed form: empty scene = analytic ground plane below the horizon row, sky above
+# ------------------------------------------------------------------------------------------------
+def test_empty_scene_ground_sky_split():
+    s = single_env(np.zeros((0, 3, 3)), [], [ego()])
+    r = oracle.render(s)
+    cls, z = r.cls[0], r.depth[0]
+    assert (cls[:32] == 0).all() and (z[:32] == 100.0).all()
+    assert (cls[32:] == 1).all()
+    # camera 1.5 m high, fy = 32: the ray of row v drops (v - 31.5)/32 per metre -> z = 48 / (v - 31.5)
+    for v, zz in ((32, 96.0), (33, 32.0), (34, 19.2), (35, 13.714285714285714), (63, 1.5238095238095237)):
+        assert np.allclose(z[v], zz, rtol=1e-14, atol=0), (v, z[v, 0])
+    f16 = r.depth_f16[0]
+    assert f16[34, 0] == np.float16(19.203125) and f16[35, 5] == np.float16(13.7109375)
+    assert f16[63, 63] == np.float16(1.5234375) and f16[0, 0] == np.float16(100.0)
+    assert (r.index[0] == -1).all() and (r.flag[0] == 0).all()
+    assert r.counts[0].tolist() == [0, 0, 0, 0]
+
+
+def test_empty_scene_pitch_moves_horizon():
+    # pitch up by atan(0.25): horizon at v + 0.5 = 32 + 32*0.25 = 40 -> rows 0..39 sky, 40.. ground
+    phi = np.degrees(np.arctan(0.25))
+    s = single_env(np.zeros((0, 3, 3)), [], [ego()], rig=make_rig((0.0,), 90.0, 90.0, pitch_deg=phi))
+    r = oracle.render(s)
+    assert (r.cls[0][:40] == 0).all() and (r.cls[0][40:] == 1).all()
+    # row 40: ray (0, 8.5/32, 1) in camera axes; with tan(phi) = 1/4 its world slope per unit of
+    # horizontal travel is (1/4 - 8.5/32) / (1 + 8.5/128); depth along the axis follows from that
+    ry = 8.5 / 32
+    p32 = float(s.rig[0, 4])               # the pitch as the float32 the renderer is given
+    down_per_depth = ry * np.cos(p32) - np.sin(p32)   # metres of descent per metre of view depth
+    assert np.allclose(r.depth[0][40], 1.5 / down_per_depth, rtol=1e-12)
+    assert abs(r.depth[0][40, 0] - 1.5 / (ry * np.cos(np.arctan(0.25)) - np.sin(np.arctan(0.25)))) < 1e-3
+
+
+def test_empty_scene_wide_camera_far_clamp():
+    # 128 x 256, hfov 96, vfov 40: fy = 64 / tan(20 deg) = 175.8386; rows 64, 65 see the ground
+    # beyond the 150 m far plane (1.5 fy / 0.5 = 527.5 m, / 1.5 = 175.8 m), row 66 at 105.503 m
+    s = single_env(np.zeros((0, 3, 3)), [], [ego()], rig=make_rig((0.0,), 96.0, 40.0, 256, 128), H=128, W=256, far=150.0)
+    r = oracle.render(s)
+    assert (r.cls[0][:64] == 0).all() and (r.cls[0][64:] == 1).all()
+    assert (r.depth[0][64] == 150.0).all() and (r.depth[0][65] == 150.0).all()
+    assert np.allclose(r.depth[0][66], 105.503, rtol=1e-5)
+
+
+# ------------------------------------------------------------------------------------------------
+# closed form: one box straight ahead (all numbers exact in binary)
+# ------------------------------------------------------------------------------------------------
+def _one_box(width=1.9, height=1.5, mount_z=1.5):
+    rig = make_rig((0.0,), 90.0, 90.0, mount=(2.25, 0.0, mount_z))
+    return single_env(np.zeros((0, 3, 3)), [], [ego(), (12.5, 0.0, 0.0, 4.5, width, height)], rig=rig)
+
+
+def test_one_box_rectangle_and_depth():
+    # rear face 8 m ahead of the camera, 1.9 wide, 1.5 tall, camera at its top height:
+    # columns 32 +- 3.8 -> centres 28.5..35.5 ; rows 32..38 -> centres 32.5..37.5
+    r = oracle.render(_one_box(), view_ids=[0])
+    cls, z = r.cls[0], r.depth[0]
+    box = np.zeros((64, 64), bool)
+    box[32:38, 28:36] = True
+    assert (cls[box] == 4).all() and (cls[~box] != 4).all() and box.sum() == 48
+    assert np.allclose(z[box], 8.0, rtol=1e-13)
+    assert (r.depth_f16[0][box] == np.float16(8.0)).all()
+    assert set(np.unique(r.index[0][box])) <= {12 + 0, 12 + 1, 12 + 4, 12 + 5}  # rear face (agent 1) or an exact tie on its rim
+    # the second view (from the box towards nothing) never shows the ego itself
+    r1 = oracle.render(_one_box(), view_ids=[1])
+    assert (r1.cls[0] != 4).all()
+
+
+def test_fill_rule_left_and_top_edges_owned():
+    # width 1.75: vertical edges exactly on the centres of columns 28 and 35 -> 28 owned, 35 not
+    r = oracle.render(_one_box(width=1.75), view_ids=[0])
+    got = r.cls[0] == 4
+    want = np.zeros((64, 64), bool)
+    want[32:38, 28:35] = True
+    assert (got == want).all() and got.sum() == 42
+    # height 1.375: top edge exactly on the centre of row 32 (camera 0.125 above it) -> owned
+    r = oracle.render(_one_box(height=1.375), view_ids=[0])
+    want = np.zeros((64, 64), bool)
+    want[32:38, 28:36] = True
+    assert ((r.cls[0] == 4) == want).all()
+    # camera at 1.375: bottom edge exactly on the centre of row 37 -> not owned; top edge at
+    # 32 - 4*0.125 = 31.5 -> row 31 centre exactly on the top edge -> owned
+    r = oracle.render(_one_box(mount_z=1.375), view_ids=[0])
+    want = np.zeros((64, 64), bool)
+    want[31:37, 28:36] = True
+    assert ((r.cls[0] == 4) == want).all()
+
+
+def test_flat_map_depth_closed_form():
+    # pitch 0, camera 1.5 m high: road pixels of row v lie at 48/(v-31.5), markings 2 cm higher
+    s = make_config(0)
+    r = oracle.render(s)
+    v = np.broadcast_to(np.arange(64)[None, :, None], r.cls.shape)
+    road, mark = r.cls == 2, r.cls == 3
+    assert road.sum() > 1000 and mark.sum() > 20
+    assert np.allclose(r.depth[road], 48.0 / (v[road] - 31.5), rtol=1e-9)
+    assert np.allclose(r.depth[mark], 47.36 / (v[mark] - 31.5), rtol=1e-9)
+    assert (r.depth >= s.near).all() and (r.depth <= s.far).all()
+    assert (r.depth[r.cls == 0] == s.far).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# the paper's camera table: focal length <-> field of view, yaw sign
+# ------------------------------------------------------------------------------------------------
+def _golden_rig():
+    vals, cams = {}, {}
+    for line in open(os.path.join(HERE, "golden", "camera_rig.txt")):
+        t = line.split()
+        if not t or t[0].startswith("#"):
+            continue
+        if len(t) == 2:
+            vals[t[0]] = float(t[1])
+        else:
+            cams[t[0]] = tuple(float(x) for x in t[1:])
+    return vals, cams
+
+
+def test_paper_intrinsics_focal_vs_fov():
+    g, _ = _golden_rig()
+    # render at 1/10 of the sensor; the focal length scales with the resolution
+    W, H = int(g["sensor_width_px"]) // 10, int(g["sensor_height_px"]) // 10
+    s = single_env(np.zeros((0, 3, 3)), [], [ego()], rig=make_rig((0.0,), g["hfov_deg"], g["vfov_deg"], W, H), H=H, W=W)
+    r = oracle.render(s)
+    # ground depth of row v is C_z * fy / (v + 0.5 - H/2): read fy back from the image
+    v = H - 1
+    fy = r.depth[0][v, 0] * (v + 0.5 - H / 2) / 1.5
+    assert abs(fy * 10 - g["focal_px"]) < 2.0          # 38.5 deg is printed to 3 digits
+    # a wall edge at azimuth atan(0.25) to the right lands 0.25*fx right of centre
+    wall = [[(4.0, -1.0, -50.0), (400.0, -100.0, -50.0), (400.0, -100.0, 50.0)],
+            [(4.0, -1.0, -50.0), (400.0, -100.0, 50.0), (4.0, -1.0, 50.0)]]
+    far_wall = [[(50.0, -200.0, -50.0), (50.0, 200.0, 50.0), (50.0, 200.0, -50.0)],
+                [(50.0, -200.0, -50.0), (50.0, -200.0, 50.0), (50.0, 200.0, 50.0)]]
+    rig0 = make_rig((0.0,), g["hfov_deg"], g["vfov_deg"], W, H, mount=(0.0, 0.0, 1.5))
+    s = single_env(wall + far_wall, [5, 5, 6, 6], [ego()], rig=rig0, H=H, W=W, far=1000.0)
+    r = oracle.render(s)
+    row = r.cls[0][10]
+    # the near wall (class 5) is seen edge-on and covers nothing; the far wall fills the row
+    assert (row == 6).all()
+    # slant the near wall a little so that it occludes everything right of its leading edge
+    wall2 = [[(4.0, -1.0, -50.0), (400.0, -120.0, -50.0), (400.0, -120.0, 50.0)],
+             [(4.0, -1.0, -50.0), (400.0, -120.0, 50.0), (4.0, -1.0, 50.0)]]
+    wall3 = [[(4.0, -1.0, -50.0), (40.0, -10.0, 50.0), (40.0, -10.0, -50.0)],
+             [(4.0, -1.0, -50.0), (4.0, -1.0, 50.0), (40.0, -10.0, 50.0)]]
+    s = single_env(wall2 + wall3 + far_wall, [5, 5, 5, 5, 6, 6], [ego()], rig=rig0, H=H, W=W, far=1000.0)
+    r = oracle.render(s)
+    row = r.cls[0][10]
+    edge = np.flatnonzero(row == 5)
+    fx = (edge.min() - W / 2) / 0.25      # first column whose centre is right of the leading edge
+    assert abs(fx * 10 - g["focal_px"]) < 25.0   # one pixel of 1/10-scale image = 40 px of focal length
+    assert abs(2 * np.degrees(np.arctan(g["sensor_width_px"] / 2 / g["focal_px"])) - g["hfov_deg"]) < 0.05
+
+
+def test_paper_rig_yaw_sign_front_left_sees_left():
+    g, cams = _golden_rig()
+    W, H = int(g["render_width_px"]), int(g["render_height_px"])
+    rig = np.zeros((4, 7), np.float32)
+    for i, name in enumerate(("front", "front_left", "front_right", "back")):
+        x, y, z, yaw = cams[name]
+        rig[i] = (x, y, z, np.radians(yaw), 0.0, focal_px(W, g["hfov_deg"]), focal_px(H, g["vfov_deg"]))
+    # a second car 20 m down the optical axis of the front-left camera (ahead and to the LEFT, +y),
+    # heading along that axis, so its rear face is centred and fronto-parallel in that camera
+    b = np.radians(55.0)
+    cx_, cy_ = cams["front_left"][0], cams["front_left"][1]
+    s = single_env(np.zeros((0, 3, 3)), [], [ego(), (cx_ + 20 * np.cos(b), cy_ + 20 * np.sin(b), b) + CAR],
+                   rig=rig, H=H, W=W)
+    r = oracle.render(s, view_ids=[0, 1, 2, 3])
+    n4 = [(r.cls[i] == 4).sum() for i in range(4)]
+    assert n4[1] > 20 and n4[2] == 0 and n4[3] == 0
+    cols = np.flatnonzero((r.cls[1] == 4).any(axis=0))
+    assert abs(cols.mean() - (W - 1) / 2) <= 0.5     # centred in the front-left image
+    # and in the front camera (hfov 63.7 -> +-31.85 deg) a car at +20 deg is in the LEFT half
+    b = np.radians(20.0)
+    s = single_env(np.zeros((0, 3, 3)), [], [ego(), (20 * np.cos(b), 20 * np.sin(b), 0.0) + CAR], rig=rig, H=H, W=W)
+    r = oracle.render(s, view_ids=[0])
+    cols = np.flatnonzero((r.cls[0] == 4).any(axis=0))
+    assert len(cols) and cols.max() < W / 2
+
+
+# ------------------------------------------------------------------------------------------------
+# independent ray caster: world-space Moeller-Trumbore, no camera-space transform, no edge normals
+# ------------------------------------------------------------------------------------------------
+def _ray_cast(scene, e, a, k):
+    s = scene
+    x, y, th = (float(t) for t in s.poses[e, a])
+    mx, my, mz, yaw, pitch, fx, fy = (float(t) for t in s.rig[k])
+    az = th + yaw
+    fwd = np.array([np.cos(pitch) * np.cos(az), np.cos(pitch) * np.sin(az), np.sin(pitch)])
+    right = np.array([np.sin(az), -np.cos(az), 0.0])
+    down = np.cross(fwd, right)
+    origin = np.array([x + np.cos(th) * mx - np.sin(th) * my, y + np.sin(th) * mx + np.cos(th) * my, mz])
+    t0, t1 = s.map_slice(e)
+    tris = [(s.tri_xyz[i].astype(np.float64), int(s.tri_class[i])) for i in range(t0, t1)]
+    assert s.A == 1, "ray caster handles map triangles only"
+    cls = np.full((s.H, s.W), -1, int)
+    depth = np.full((s.H, s.W), np.inf)
+    for v in range(s.H):
+        for u in range(s.W):
+            d = fwd + (u + 0.5 - s.W / 2) / fx * right + (v + 0.5 - s.H / 2) / fy * down
+            for tri, c in tris:
+                e1, e2 = tri[1] - tri[0], tri[2] - tri[0]
+                pvec = np.cross(d, e2)
+                det = e1 @ pvec
+                if det == 0:
+                    continue
+                tvec = origin - tri[0]
+                uu = (tvec @ pvec) / det
+                qvec = np.cross(tvec, e1)
+                vv = (d @ qvec) / det
+                t = (e2 @ qvec) / det
+                if uu < 0 or vv < 0 or uu + vv > 1 or t < s.near or t > s.far:
+                    continue
+                if t < depth[v, u]:
+                    depth[v, u], cls[v, u] = t, c
+    return cls, depth
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_against_world_space_ray_caster(seed):
+    rng = np.random.default_rng(seed)
+    n = 12
+    # triangles scattered around a camera at the origin region, many crossing the camera plane
+    centre = rng.uniform(-6, 6, size=(n, 1, 3)) + np.array([4.0, 0.0, 1.0])
+    tris = centre + rng.uniform(-6, 6, size=(n, 3, 3))
+    classes = rng.integers(2, 9, size=n)
+    H, W = (12, 16) if seed % 2 else (16, 12)
+    rig = make_rig((float(rng.uniform(-180, 180)),), 80.0, 60.0, W, H, mount=(0.7, -0.3, 1.2),
+                   pitch_deg=float(rng.uniform(-20, 20)))
+    s = single_env(tris, classes, [ego(rng.uniform(-2, 2), rng.uniform(-2, 2), rng.uniform(-3, 3))],
+                   rig=rig, H=H, W=W, near=0.5, far=30.0)
+    r = oracle.render(s)
+    cls, depth = _ray_cast(s, 0, 0, 0)
+    hit = cls >= 0
+    ok = r.flag[0] != 0                       # either answer is acceptable on flagged pixels
+    assert hit.sum() > 20
+    assert (((r.index[0] >= 0) == hit) | ok).all()
+    assert ((r.cls[0] == cls) | ~hit | ok).all()
+    both = hit & (r.index[0] >= 0) & ~ok
+    assert np.allclose(r.depth[0][both], depth[both], rtol=1e-9)
+
+
+# ------------------------------------------------------------------------------------------------
+# hand-counted tiny scenes
+# ------------------------------------------------------------------------------------------------
+RIG0 = make_rig((0.0,), 90.0, 90.0, 8, 8, mount=(0.0, 0.0, 1.0))   # 8x8 image, fx = fy = 4, at (0,0,1) looking along +x
+RIG32 = make_rig((0.0,), 90.0, 90.0, 32, 32)
+RIG16 = make_rig((0.0,), 90.0, 90.0, 16, 16, mount=(0.0, 0.0, 1.0))
+
+
+def _wall(x, y0, y1, z0, z1):
+    """Rectangle in the plane x = const facing the camera: two triangles."""
+    return [[(x, y0, z0), (x, y1, z0), (x, y1, z1)], [(x, y0, z0), (x, y1, z1), (x, y0, z1)]]
+
+
+def test_single_triangle_hand_counted():
+    # 8x8 image, fx = fy = 4, wall triangle at x = 4: one pixel per metre, column = 4 - y, row = 4 - (z-1)
+    # vertices (y,z): (2,3) (-2,3) (2,-1) -> pixel-space corners (2,2) (6,2) (2,6): right triangle,
+    # centres (u+.5, v+.5) inside iff (u+.5-2) + (v+.5-2) < 4, i.e. u+v < 7 (u,v >= 2); hypotenuse is not top-left
+    tri = [[(4.0, 2.0, 3.0), (4.0, -2.0, 3.0), (4.0, 2.0, -1.0)]]
+    s = single_env(tri, [7], [ego()], rig=RIG0, H=8, W=8)
+    r = oracle.render(s)
+    want = np.zeros((8, 8), bool)
+    for v in range(2, 8):
+        for u in range(2, 8):
+            want[v, u] = (u + v) < 7
+    assert ((r.cls[0] == 7) == want).all() and want.sum() == 6
+    assert np.allclose(r.depth[0][want], 4.0)
+    assert r.counts[0, 0] == 1 and r.counts[0, 1] == 1 and r.counts[0, 2] == 6
+
+
+def test_two_walls_nearest_wins_and_occluded_box_is_invisible():
+    near_wall = _wall(4.0, -1.0, 1.0, 0.0, 2.0)     # covers columns 3..4, rows 3..4 of an 8x8 image
+    far_wall = _wall(8.0, -6.0, 6.0, -3.0, 5.0)     # covers columns 1..6, rows 2..5
+    s = single_env(far_wall + near_wall, [5, 5, 6, 6], [ego()], rig=RIG0, H=8, W=8)
+    r = oracle.render(s)
+    c = r.cls[0]
+    assert (c[3:5, 3:5] == 6).all() and (c == 6).sum() == 4
+    assert (c == 5).sum() == 6 * 4 - 4
+    assert np.allclose(r.depth[0][c == 6], 4.0) and np.allclose(r.depth[0][c == 5], 8.0)
+    # a car hidden behind the near wall changes nothing (occlusion is real)
+    wall = _wall(4.0, -3.9, 3.9, -2.9, 4.9)
+    s0 = single_env(wall, [6, 6], [ego()], rig=RIG0, H=8, W=8)
+    s1 = single_env(wall, [6, 6], [ego(), (10.0, 0.0, 0.3) + CAR], rig=RIG0, H=8, W=8)
+    r0, r1 = oracle.render(s0, view_ids=[0]), oracle.render(s1, view_ids=[0])
+    assert (r0.cls == r1.cls).all() and (r0.depth == r1.depth).all()
+    assert (r1.cls != 4).all()
+
+
+def test_exact_depth_tie_goes_to_lower_index():
+    a = _wall(4.0, -2.0, 2.0, -1.0, 3.0)
+    b = _wall(4.0, -1.0, 3.0, 0.0, 4.0)
+    for tris, classes, want in ((a + b, [5, 5, 6, 6], 5), (b + a, [6, 6, 5, 5], 6)):
+        s = single_env(tris, classes, [ego()], rig=RIG0, H=8, W=8)
+        r = oracle.render(s)
+        # overlap of the two walls: y in [-1,2] -> columns 2..4, z in [0,3] -> rows 2..4
+        assert (r.cls[0][2:5, 2:5] == want).all()
+        assert (r.flag[0][2:5, 2:5] & 2).all()      # and the tie is reported as a depth ambiguity
+
+
+def test_near_and_far_planes_inclusive():
+    s = single_env(_wall(0.5, -4, 4, -3, 5) , [5, 5], [ego()], rig=RIG0, H=8, W=8, near=0.5, far=100.0)
+    assert (oracle.render(s).cls[0] == 5).all()
+    s = single_env(_wall(0.4375, -4, 4, -3, 5), [5, 5], [ego()], rig=RIG0, H=8, W=8, near=0.5, far=100.0)
+    assert (oracle.render(s).cls[0] != 5).all()
+    s = single_env(_wall(64.0, -400, 400, -300, 500), [5, 5], [ego()], rig=RIG0, H=8, W=8, near=0.5, far=64.0)
+    assert (oracle.render(s).cls[0] == 5).all()
+    s = single_env(_wall(64.5, -400, 400, -300, 500), [5, 5], [ego()], rig=RIG0, H=8, W=8, near=0.5, far=64.0)
+    assert (oracle.render(s).cls[0] != 5).all()
+
+
+def test_triangle_through_camera_plane_needs_no_clipping():
+    # a ground-level strip from 10 m behind the camera to 20 m ahead, 2 m wide, 1 m below the camera
+    strip = [[(-10.0, -1.0, 0.0), (20.0, -1.0, 0.0), (20.0, 1.0, 0.0)], [(-10.0, -1.0, 0.0), (20.0, 1.0, 0.0), (-10.0, 1.0, 0.0)]]
+    s = single_env(strip, [2, 2], [ego()], rig=RIG16, H=16, W=16, near=0.5, far=100.0)
+    r = oracle.render(s)
+    fx = 8.0
+    for v in range(16):
+        for u in range(16):
+            ry = (v + 0.5 - 8) / fx
+            rx = (u + 0.5 - 8) / fx
+            inside = False
+            if ry > 0:
+                z = 1.0 / ry                       # ground hit at view depth z, lateral offset rx*z
+                inside = (0.5 <= z <= 20.0) and -1.0 <= rx * z < 1.0   # left edge owned, right edge not
+            assert (r.cls[0][v, u] == 2) == inside, (u, v)
+
+
+def test_frustum_counts():
+    def t_vis(tri, **kw):
+        s = single_env([tri], [5], [ego()], rig=RIG0, H=8, W=8, near=0.5, far=50.0, **kw)
+        return int(oracle.render(s).counts[0, 0])
+    assert t_vis([(4, -1, 0.5), (4, 1, 0.5), (4, 0, 1.5)]) == 1            # inside
+    assert t_vis([(-4, -1, 0.5), (-4, 1, 0.5), (-4, 0, 1.5)]) == 0         # behind
+    assert t_vis([(60, -1, 0.5), (60, 1, 0.5), (60, 0, 1.5)]) == 0         # beyond far
+    assert t_vis([(4, 10, 0.5), (4, 12, 0.5), (4, 11, 1.5)]) == 0          # off to the left
+    assert t_vis([(-4, 0, 0), (20, -1, 0), (20, 1, 0)]) == 1               # straddles the camera plane
+    assert t_vis([(10, -100, -100), (10, 100, -100), (10, 0, 200)]) == 1   # encloses the whole frustum
+    assert t_vis([(0.2, -0.1, 1.0), (0.3, 0.1, 1.0), (0.3, 0.0, 1.1)]) == 0  # in front of the near plane
+    assert t_vis([(4, 3.9, 1), (4, 12, 1), (4, 12, 2)]) == 1               # clips the left frustum side (y = x)
+    assert t_vis([(4, 4.1, 1), (4, 12, 1), (4, 12, 2)]) == 0
+
+
+# ------------------------------------------------------------------------------------------------
+# invariants
+# ------------------------------------------------------------------------------------------------
+def _small_world(seed=3):
+    rng = np.random.default_rng(seed)
+    gm_tris = []
+    for i in range(40):
+        c = np.array([rng.integers(-640, 640) / 16.0, rng.integers(-640, 640) / 16.0, 0.0])
+        gm_tris.append(c + np.round(rng.uniform(-8, 8, size=(3, 3)) * 16) / 16 * np.array([1, 1, 0.2]))
+    classes = rng.integers(2, 6, size=40)
+    agents = [ego(0.0, 0.0, 0.0)] + [(rng.integers(-300, 300) / 16.0, rng.integers(-300, 300) / 16.0,
+                                      float(np.float32(rng.uniform(-3, 3)))) + CAR for _ in range(5)]
+    return np.array(gm_tris), classes, agents
+
+
+def test_translation_by_powers_of_two_is_bit_exact():
+    tris, classes, agents = _small_world()
+    rig = make_rig((0.0, 90.0, 180.0, 270.0), 90.0, 90.0, 32, 32)
+    base = oracle.render(single_env(tris, classes, agents, rig=rig, H=32, W=32))
+    assert (base.cls == 4).sum() > 50 and (base.cls >= 2).sum() > 500
+    for dx, dy in ((256.0, -512.0), (-1024.0, 64.0)):
+        t2 = tris + np.array([dx, dy, 0.0])
+        a2 = [(a[0] + dx, a[1] + dy) + tuple(a[2:]) for a in agents]
+        moved = oracle.render(single_env(t2, classes, a2, rig=rig, H=32, W=32))
+        assert (moved.cls == base.cls).all() and (moved.index == base.index).all()
+        on_map = base.index < len(tris)           # map vertices minus the ego position is exact in binary
+        assert (moved.depth[on_map] == base.depth[on_map]).all()
+        assert np.allclose(moved.depth, base.depth, rtol=1e-11, atol=0)   # box corners round at 1e-16 * 1024
+
+
+def test_rotation_and_general_motion_leave_image_unchanged():
+    tris, classes, agents = _small_world(5)
+    rig = make_rig((0.0, 90.0), 90.0, 90.0, 32, 32)
+    base = oracle.render(single_env(tris, classes, agents, rig=rig, H=32, W=32))
+    for ang, dx, dy in ((np.pi / 2, 0.0, 0.0), (0.7, 13.25, -7.5)):
+        c, s_ = np.cos(ang), np.sin(ang)
+        R = np.array([[c, -s_, 0], [s_, c, 0], [0, 0, 1]])
+        t2 = tris @ R.T + np.array([dx, dy, 0.0])
+        a2 = [(c * a[0] - s_ * a[1] + dx, s_ * a[0] + c * a[1] + dy, a[2] + ang) + tuple(a[3:]) for a in agents]
+        moved = oracle.render(single_env(t2, classes, a2, rig=rig, H=32, W=32))
+        # inputs are re-rounded to float32, so equality holds off the flagged pixels, depth to ~1e-6
+        compare_images(base.cls, base.depth, base.flag | moved.flag, moved.cls, moved.depth, depth_rtol=1e-5,
+                       max_mismatch_frac=5e-3)
+
+
+def test_primitive_order_does_not_matter_without_ties():
+    tris, classes, agents = _small_world(7)
+    base = oracle.render(single_env(tris, classes, agents, rig=RIG32, H=32, W=32), view_ids=[0])
+    perm = np.random.default_rng(0).permutation(len(tris))
+    shuf = oracle.render(single_env(tris[perm], classes[perm], agents, rig=RIG32, H=32, W=32), view_ids=[0])
+    assert (base.cls == shuf.cls).all() and (base.depth == shuf.depth).all()
+
+
+def test_mirror_scene_mirrors_image():
+    tris, classes, agents = _small_world(11)
+    m = np.array([1.0, -1.0, 1.0])
+    base = oracle.render(single_env(tris, classes, agents, rig=RIG32, H=32, W=32), view_ids=[0])
+    a2 = [(a[0], -a[1], -a[2]) + tuple(a[3:]) for a in agents]
+    mir = oracle.render(single_env(tris * m, classes, a2, rig=RIG32, H=32, W=32), view_ids=[0])
+    flag = base.flag | mir.flag[:, :, ::-1]
+    diff = (base.cls != mir.cls[:, :, ::-1]) & (flag == 0)
+    assert diff.sum() == 0
+    same = base.cls == mir.cls[:, :, ::-1]
+    assert np.allclose(base.depth[same & (flag == 0)], mir.depth[:, :, ::-1][same & (flag == 0)], rtol=1e-6)
+
+
+def test_ego_excluded_inactive_and_other_envs():
+    # camera INSIDE the ego's own box (mount at the centre): the ego must not be drawn
+    rig = make_rig((0.0,), 90.0, 90.0, 16, 16, mount=(0.0, 0.0, 0.75))
+    s = single_env(np.zeros((0, 3, 3)), [], [ego(), (10.0, 0.0, 0.0) + CAR], rig=rig, H=16, W=16)
+    r = oracle.render(s)
+    assert (r.cls[0] == 4).sum() > 0 and (r.cls[0] == 4).sum() < 60      # only the other car
+    s1 = single_env(np.zeros((0, 3, 3)), [], [ego()], rig=rig, H=16, W=16)
+    assert (oracle.render(s1).cls != 4).all()
+    # inactive other agent is not drawn; inactive ego renders sky/far everywhere
+    s2 = single_env(np.zeros((0, 3, 3)), [], [ego(), (10.0, 0.0, 0.0) + CAR], rig=rig, H=16, W=16, active=[1, 0])
+    r2 = oracle.render(s2)
+    assert (r2.cls[0] != 4).all()
+    assert (r2.cls[1] == 0).all() and (r2.depth[1] == 100.0).all()
+    # two envs on one shared map: agents of env 1 never show up in env 0
+    poses = np.array([[[0, 0, 0]], [[10, 0, 0]]], np.float32)
+    dims = np.tile(np.array(CAR, np.float32), (2, 1, 1))
+    s3 = custom_scene(np.zeros((0, 3, 3)), [], poses, dims, rig, 16, 16)
+    assert (oracle.render(s3).cls != 4).all()
+
+
+def test_determinism():
+    s = make_config(0)
+    a, b = oracle.render(s, n_threads=1), oracle.render(s, n_threads=4)
+    assert (a.cls == b.cls).all() and (a.depth == b.depth).all() and (a.counts == b.counts).all()
+
+
+def test_flag_fraction_is_small_on_a_real_workload():
+    s = make_config(1, E=1)
+    r = oracle.render(s, view_ids=np.arange(0, 128, 5))
+    frac = (r.flag != 0).mean()
+    assert frac < 3e-3, frac
+
+
+# ------------------------------------------------------------------------------------------------
+# binary16 rounding against the library conversion
+# ------------------------------------------------------------------------------------------------
+def test_f16_rounding_matches_numpy():
+    rng = np.random.default_rng(0)
+    vals = np.concatenate([rng.uniform(0.4, 160.0, 20000), 2.0 ** rng.uniform(-26, 17, 5000),
+                           [0.0, 1.0, 100.0, 150.0, 65504.0, 65519.9, 65520.0, 1e-8, 6e-8, 2.0 ** -24, 2.0 ** -25,
+                            1.5 * 2.0 ** -24, 2.5 * 2.0 ** -24]])
+    # exact ties between neighbouring binary16 values
+    h = rng.integers(0x0001, 0x7bfe, 5000).astype(np.uint16)
+    lo, hi = h.view(np.float16).astype(np.float64), (h + 1).astype(np.uint16).view(np.float16).astype(np.float64)
+    vals = np.concatenate([vals, (lo + hi) / 2, -vals[:100]])
+    with np.errstate(over="ignore"):
+        want = vals.astype(np.float16).view(np.uint16)
+    got = np.array([oracle.f64_to_f16_bits(v) for v in vals], np.uint16)
+    assert (got == want).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# kinematic bicycle closed forms
+# ------------------------------------------------------------------------------------------------
+def test_bicycle_straight_line_and_clamps():
+    st = np.array([[1.0, 2.0, 0.5, 10.0], [0.0, 0.0, 0.0, 0.5], [0.0, 0.0, 0.0, 29.5]])
+    act = np.array([[1.0, 0.0], [-3.0, 0.0], [2.0, 0.0]], np.float32)
+    x = st.copy()
+    dist = 0.0
+    for n in range(20):
+        dist += x[0, 3] * 0.1
+        x = oracle.step(x, act, None, 0.1, 2.8, 30.0)
+    # v_t = 10 + 0.1 t ; travelled = sum_{t<20} v_t dt = 0.1*(200 + 0.1*190) = 21.9
+    assert np.isclose(dist, 21.9) and np.allclose(x[0], [1 + 21.9 * np.cos(0.5), 2 + 21.9 * np.sin(0.5), 0.5, 12.0])
+    assert x[1, 3] == 0.0 and np.isclose(x[1, 0], 0.05 + 0.02)       # 0.5, 0.2, 0 ... then stopped
+    assert x[2, 3] == 30.0
+
+
+def test_bicycle_constant_steer_heading_is_linear():
+    st = np.array([[0.0, 0.0, 0.25, 8.0]])
+    act = np.array([[0.0, 0.2]], np.float32)
+    x = st.copy()
+    for n in range(50):
+        x = oracle.step(x, act, None, 0.1, 2.8, 30.0)
+    delta = float(np.float32(0.2))
+    assert np.isclose(x[0, 2], 0.25 + 50 * (8.0 / 2.8) * np.tan(delta) * 0.1, rtol=1e-13)
+    assert x[0, 3] == 8.0
+    # one hand-worked step: x += v cos(yaw) dt from the OLD heading
+    y = oracle.step(np.array([[0.0, 0.0, np.pi / 2, 10.0]]), np.array([[0.0, 0.3]], np.float32), None, 0.1, 2.8, 30.0)
+    assert abs(y[0, 0]) < 1e-15 * 10 + 1e-15 and np.isclose(y[0, 1], 1.0)
+    # inactive agents do not move
+    z = oracle.step(st, act, np.array([0], np.uint8), 0.1, 2.8, 30.0)
+    assert (z == st).all()
