@@ -1,0 +1,168 @@
+/*
+ * pictura.h -- C ABI of the batched egocentric rasterizer (CUDA, sm_100a).
+ *
+ * The library renders, for every agent of every environment and every camera of an ego-mounted
+ * rig, a semantic-class image (u8) and a depth image (IEEE binary16) of the agent's surroundings:
+ * the triangles of the environment's map and the other agents as oriented 3-D boxes, under a
+ * pinhole projection with a z-buffer.  This is the rasterizer Phi of the paper (Sec. 3.2, Eq. 2:
+ * I_{i,k} = Phi(A_i, W_i, K_{i,k}); "only the surroundings are rendered"), with a class/depth
+ * output in place of the paper's shaded colour.
+ *
+ * Conventions (paper, table "Camera rig"): world z up; agent frame x forward, y left, z up; yaw
+ * counter-clockwise about z; a camera is mounted at `mount` in the agent frame, turned by `yaw`
+ * about z and pitched up by `pitch`; intrinsics are focal lengths in pixels with the principal
+ * point at the image centre.  Pixel (u, v) -- column u left to right, row v top to bottom,
+ * row-major storage -- samples the ray through (u + 0.5, v + 0.5).
+ *
+ * Per pixel: a primitive covers the pixel when the ray hits it (edge functions with a top-left
+ * fill rule on exact zeros, no geometric clipping); its depth z is the distance along the optical
+ * axis; fragments with near <= z <= far are kept; the smallest z wins, exact ties go to the lower
+ * primitive index (map triangles in the order given, then 12 triangles per agent box).  Pixels
+ * without a fragment show the analytic ground plane z = 0 (ground class, depth min(far, hit
+ * depth)) below the horizon and sky (sky class, depth far) above it.  An agent never sees its own
+ * box; agents of other environments are never visible; an inactive agent is not drawn and its
+ * own images are sky/far.  Arithmetic is float32; results agree with a double-precision
+ * evaluation except at pixels whose edge function, depth gap or clip plane is within 1e-5
+ * relative of a decision boundary.
+ *
+ * Memory: every pointer marked "dev" is device memory of the scene's CUDA device, owned by the
+ * caller; "host" pointers are ordinary host memory.  The library never takes ownership of a
+ * caller's buffer.  Unless stated otherwise calls are asynchronous on the given CUDA stream
+ * (a cudaStream_t passed as void*; NULL is the default stream) and allocate nothing.
+ *
+ * Errors: every call returns a pic_status; nothing throws, aborts or traps.  pic_last_error()
+ * returns a thread-local description of the last failure.  Device-detected conditions are
+ * accumulated in sticky flags read by pic_get_status().
+ */
+#ifndef PICTURA_H
+#define PICTURA_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pic_scene pic_scene; /* opaque; created and destroyed by the library */
+
+typedef enum {
+    PIC_OK = 0,
+    PIC_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, bad struct size, bad device  */
+    PIC_ERR_SHAPE = 2,       /* non-positive or unsupported sizes, inconsistent offsets        */
+    PIC_ERR_OOM = 3,         /* host or device allocation failed                                */
+    PIC_ERR_CUDA = 4,        /* a CUDA runtime call failed (see pic_last_error)                 */
+    PIC_ERR_CAPACITY = 5,    /* a fixed-size entry point was given more than it can hold        */
+    PIC_ERR_NONFINITE = 6    /* reserved for status flags                                       */
+} pic_status;
+
+/* Sticky device flags returned by pic_get_status. */
+#define PIC_FLAG_NONFINITE_POSE 0x1u /* a pose, size or action was NaN/Inf; that agent's output is unspecified */
+
+/* One pinhole camera of the rig, in the agent frame (x forward, y left, z up). */
+typedef struct {
+    float mount_x, mount_y, mount_z; /* metres                                                   */
+    float yaw;                       /* rad, counter-clockwise about z (left positive)           */
+    float pitch;                     /* rad, up positive; no roll                                */
+    float fx, fy;                    /* focal lengths in pixels: fx = (W/2)/tan(hfov/2), same for fy */
+} pic_camera;
+
+typedef struct {
+    uint32_t size;                 /* = sizeof(pic_scene_desc); rejects mismatched headers       */
+    int32_t E, A, K, H, W;         /* environments, agents/env, cameras/agent, image rows, cols  */
+    float near_z, far_z;           /* kept depth range, metres, 0 < near_z < far_z              */
+    int32_t num_maps;              /* M >= 1 maps                                                */
+    const int32_t* env_map_id;     /* host [E], values in [0,M); NULL: identity if M == E, else all 0 */
+    const int64_t* map_tri_offset; /* host [M+1], non-decreasing, [0] == 0                       */
+    const float* tri_xyz;          /* host [N,3,3] f32 world coordinates, N = map_tri_offset[M] */
+    const uint8_t* tri_class;      /* host [N] class id of each triangle                         */
+    uint8_t agent_class;           /* class written for agent boxes                              */
+    uint8_t sky_class;             /* background above the horizon                               */
+    uint8_t ground_class;          /* background below the horizon                               */
+    uint8_t reserved;
+    int32_t device;                /* CUDA device ordinal                                        */
+} pic_scene_desc;
+
+/*
+ * Build a scene: copies the map (the caller may free its arrays on return), builds the per-map
+ * culling hierarchy and allocates all device memory the scene will ever need, including the
+ * kinematic state [E,A,4] used by pic_step.  Synchronous.  At most 2^24 - 12*A triangles per map.
+ */
+pic_status pic_scene_create(const pic_scene_desc* desc, pic_scene** out);
+
+/* Free a scene and everything it owns.  Synchronises the device.  NULL is accepted. */
+pic_status pic_scene_destroy(pic_scene* scene);
+
+/*
+ * Render all E*A*K views (the rasterizer Phi, Eq. 2).
+ *   poses      dev f32 [E,A,3]   x, y, yaw of each agent (box centre on the ground plane)
+ *   dims       dev f32 [E,A,3]   box length (along heading), width, height
+ *   active     dev u8  [E,A] or NULL (all active)
+ *   rig        host    [K]       copied during the call
+ *   out_class  dev u8  [E,A,K,H,W]
+ *   out_depth  dev u16 [E,A,K,H,W] binary16 bit patterns
+ * out_class must be 16-byte aligned and out_depth 16-byte aligned.
+ */
+pic_status pic_render(pic_scene* scene, const float* poses, const float* dims, const uint8_t* active,
+                      const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth, void* cuda_stream);
+
+/*
+ * Same as pic_render with HOST inputs and outputs: copies poses/dims/active to the device, renders
+ * into staging buffers owned by the scene (allocated on first use: 3*E*A*K*H*W bytes) and copies
+ * both images back.  Returns after the copies completed (the stream is synchronised).  Host
+ * buffers may be pageable or pinned; pinned is faster.
+ */
+pic_status pic_render_host(pic_scene* scene, const float* poses, const float* dims, const uint8_t* active,
+                           const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth, void* cuda_stream);
+
+/*
+ * Kinematic state for pic_step: state dev f32 [E,A,4] = x, y, yaw, v; dims and active as in
+ * pic_render (copied into the scene).  pic_get_state copies the state out to dev memory.
+ */
+pic_status pic_set_state(pic_scene* scene, const float* state, const float* dims, const uint8_t* active,
+                         void* cuda_stream);
+pic_status pic_get_state(pic_scene* scene, float* state_out, void* cuda_stream);
+
+/*
+ * One simulator step: explicit-Euler kinematic bicycle update of every active agent, everything
+ * computed from the old state,
+ *     x += v cos(yaw) dt,  y += v sin(yaw) dt,  yaw += (v / wheelbase) tan(steer) dt,
+ *     v = clamp(v + accel dt, 0, v_max)            (dt 0.1 s, wheelbase 2.8 m, v_max 30 m/s),
+ * then a render of all views from the NEW state (the paper's loop: each agent acts, then is
+ * rendered for its neighbours, Sec. 1; its own dynamics use jerk actions and are not reproduced).
+ *   actions    dev f32 [E,A,2]   accel (m/s^2), steer (rad)
+ */
+pic_status pic_step(pic_scene* scene, const float* actions, const pic_camera* rig, uint8_t* out_class,
+                    uint16_t* out_depth, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, then read and clear the sticky device flags (PIC_FLAG_*) into *flags (host). */
+pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
+
+/*
+ * Options (all default 0):
+ *   PIC_OPT_BRUTE_FORCE   1: render with the exhaustive kernel (every primitive against every
+ *                         pixel tile, no culling hierarchy) -- a slow cross-check that shares the
+ *                         per-primitive arithmetic with the production kernel.
+ *   PIC_OPT_DEPTH32       value = dev f32* [E,A,K,H,W] (as uintptr) or 0: also write the float32
+ *                         depth the binary16 image was rounded from.
+ *   PIC_OPT_COUNTERS      value = dev u64* [8] (as uintptr) or 0: accumulate work counters
+ *                         (views, group tests, leaf tests, primitives tested, set up, small, large, fragments).
+ *   PIC_OPT_VIEW_FIRST,   render only views [first, first + count) (flat index (e*A + a)*K + k);
+ *   PIC_OPT_VIEW_COUNT    count 0 = through the last view.  Other views' pixels are left untouched.
+ */
+#define PIC_OPT_BRUTE_FORCE 1
+#define PIC_OPT_DEPTH32 2
+#define PIC_OPT_COUNTERS 3
+#define PIC_OPT_VIEW_FIRST 4
+#define PIC_OPT_VIEW_COUNT 5
+pic_status pic_scene_set_option(pic_scene* scene, int32_t option, uint64_t value);
+
+/* Thread-local, never NULL; valid until the next failing call on this thread. */
+const char* pic_last_error(void);
+
+/* Library version (major*10000 + minor*100 + patch). */
+int32_t pic_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PICTURA_H */

@@ -1,0 +1,11 @@
+"""B200-native batched egocentric rasterizer (class u8 + depth f16 per agent camera).
+
+The work is done by libpictura.so (hand-written CUDA for sm_100a, C ABI in include/pictura.h);
+this package is the thin Python binding used by the tests and the benchmark.
+"""
+from . import build
+from .binding import (Scene, PicError, load, EXPORTS, OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST,
+                      OPT_VIEW_COUNT, FLAG_NONFINITE_POSE)
+
+__all__ = ["Scene", "PicError", "load", "build", "EXPORTS", "OPT_BRUTE_FORCE", "OPT_DEPTH32", "OPT_COUNTERS",
+           "OPT_VIEW_FIRST", "OPT_VIEW_COUNT", "FLAG_NONFINITE_POSE"]

@@ -1,0 +1,240 @@
+"""Thin ctypes binding of libpictura.so: argument marshalling only.
+
+Every step of the rendering path runs inside the CUDA library; torch is used for device memory,
+streams and nothing else.  There is no CPU fallback: if the library cannot be loaded, or no CUDA
+device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+PIC_OK = 0
+STATUS_NAMES = {0: "PIC_OK", 1: "PIC_ERR_INVALID_ARG", 2: "PIC_ERR_SHAPE", 3: "PIC_ERR_OOM", 4: "PIC_ERR_CUDA",
+                5: "PIC_ERR_CAPACITY", 6: "PIC_ERR_NONFINITE"}
+OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT = 1, 2, 3, 4, 5
+FLAG_NONFINITE_POSE = 1
+
+EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
+           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_last_error", "pic_version"]
+
+
+class PicError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class pic_camera(C.Structure):
+    _fields_ = [("mount_x", C.c_float), ("mount_y", C.c_float), ("mount_z", C.c_float), ("yaw", C.c_float),
+                ("pitch", C.c_float), ("fx", C.c_float), ("fy", C.c_float)]
+
+
+class pic_scene_desc(C.Structure):
+    _fields_ = [("size", C.c_uint32), ("E", C.c_int32), ("A", C.c_int32), ("K", C.c_int32), ("H", C.c_int32),
+                ("W", C.c_int32), ("near_z", C.c_float), ("far_z", C.c_float), ("num_maps", C.c_int32),
+                ("env_map_id", C.c_void_p), ("map_tri_offset", C.c_void_p), ("tri_xyz", C.c_void_p),
+                ("tri_class", C.c_void_p), ("agent_class", C.c_uint8), ("sky_class", C.c_uint8),
+                ("ground_class", C.c_uint8), ("reserved", C.c_uint8), ("device", C.c_int32)]
+
+
+_lib = None
+
+
+def load(path: Optional[str] = None):
+    """Load libpictura.so (building it with nvcc first if it is missing or stale)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError(f"CUDA library {path} is missing; run paper_2607_26005_b200.build.build()")
+    lib = C.CDLL(path)
+    vp = C.c_void_p
+    lib.pic_scene_create.argtypes = [C.POINTER(pic_scene_desc), C.POINTER(vp)]
+    lib.pic_scene_destroy.argtypes = [vp]
+    lib.pic_render.argtypes = [vp, vp, vp, vp, C.POINTER(pic_camera), vp, vp, vp]
+    lib.pic_render_host.argtypes = [vp, vp, vp, vp, C.POINTER(pic_camera), vp, vp, vp]
+    lib.pic_set_state.argtypes = [vp, vp, vp, vp, vp]
+    lib.pic_get_state.argtypes = [vp, vp, vp]
+    lib.pic_step.argtypes = [vp, vp, C.POINTER(pic_camera), vp, vp, vp]
+    lib.pic_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
+    for name in EXPORTS:
+        getattr(lib, name).restype = C.c_int
+    lib.pic_last_error.restype = C.c_char_p
+    lib.pic_last_error.argtypes = []
+    lib.pic_version.restype = C.c_int32
+    lib.pic_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(lib, status: int):
+    if status != PIC_OK:
+        raise PicError(status, lib.pic_last_error().decode("utf-8", "replace"))
+
+
+def _rig_array(rig) -> "C.Array":
+    rig = np.asarray(rig, dtype=np.float32).reshape(-1, 7)
+    arr = (pic_camera * rig.shape[0])()
+    for k in range(rig.shape[0]):
+        arr[k] = pic_camera(*[float(v) for v in rig[k]])
+    return arr
+
+
+def _dev_ptr(t, dtype, numel: Optional[int] = None) -> int:
+    import torch
+    if t is None:
+        return 0
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("expected a CUDA torch tensor")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"expected a contiguous {dtype} tensor, got {t.dtype}")
+    if numel is not None and t.numel() != numel:
+        raise ValueError(f"expected {numel} elements, got {t.numel()}")
+    return t.data_ptr()
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class Scene:
+    """Owner of one pic_scene.  Arrays follow include/pictura.h; device tensors are torch CUDA tensors."""
+
+    def __init__(self, E: int, A: int, K: int, H: int, W: int, near: float, far: float, tri_xyz, tri_class,
+                 map_tri_offset=None, env_map_id=None, agent_class: int = 4, sky_class: int = 0,
+                 ground_class: int = 1, device: int = 0):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the rasterizer has no CPU path")
+        self._lib = load()
+        tri_xyz = np.ascontiguousarray(tri_xyz, dtype=np.float32).reshape(-1, 3, 3)
+        tri_class = np.ascontiguousarray(tri_class, dtype=np.uint8).reshape(-1)
+        if map_tri_offset is None:
+            map_tri_offset = [0, tri_xyz.shape[0]]
+        off = np.ascontiguousarray(map_tri_offset, dtype=np.int64)
+        emi = None if env_map_id is None else np.ascontiguousarray(env_map_id, dtype=np.int32)
+        d = pic_scene_desc()
+        d.size = C.sizeof(pic_scene_desc)
+        d.E, d.A, d.K, d.H, d.W = int(E), int(A), int(K), int(H), int(W)
+        d.near_z, d.far_z = float(near), float(far)
+        d.num_maps = int(off.shape[0] - 1)
+        d.env_map_id = None if emi is None else emi.ctypes.data
+        d.map_tri_offset = off.ctypes.data
+        d.tri_xyz = tri_xyz.ctypes.data
+        d.tri_class = tri_class.ctypes.data
+        d.agent_class, d.sky_class, d.ground_class = int(agent_class), int(sky_class), int(ground_class)
+        d.device = int(device)
+        handle = C.c_void_p()
+        _check(self._lib, self._lib.pic_scene_create(C.byref(d), C.byref(handle)))
+        self._h = handle
+        self.E, self.A, self.K, self.H, self.W = int(E), int(A), int(K), int(H), int(W)
+        self.device = torch.device("cuda", int(device))
+        self._keep = []   # tensors referenced by options
+
+    # -- shapes ---------------------------------------------------------------------------------
+    @property
+    def n_agents(self) -> int:
+        return self.E * self.A
+
+    @property
+    def image_shape(self) -> Tuple[int, int, int, int, int]:
+        return (self.E, self.A, self.K, self.H, self.W)
+
+    def alloc_outputs(self):
+        import torch
+        cls = torch.empty(self.image_shape, dtype=torch.uint8, device=self.device)
+        depth = torch.empty(self.image_shape, dtype=torch.float16, device=self.device)
+        return cls, depth
+
+    # -- calls ----------------------------------------------------------------------------------
+    def render(self, poses, dims, rig, active=None, out_class=None, out_depth=None, stream=None):
+        import torch
+        if out_class is None or out_depth is None:
+            out_class, out_depth = self.alloc_outputs()
+        n, npx = self.n_agents, self.n_agents * self.K * self.H * self.W
+        _check(self._lib, self._lib.pic_render(
+            self._h, _dev_ptr(poses, torch.float32, 3 * n), _dev_ptr(dims, torch.float32, 3 * n),
+            _dev_ptr(active, torch.uint8, n) if active is not None else None, _rig_array(rig),
+            _dev_ptr(out_class, torch.uint8, npx), _dev_ptr(out_depth, torch.float16, npx), _stream_ptr(stream)))
+        return out_class, out_depth
+
+    def render_host(self, poses: np.ndarray, dims: np.ndarray, rig, out_class: np.ndarray, out_depth: np.ndarray,
+                    active: Optional[np.ndarray] = None, stream=None):
+        """Host-buffer variant: numpy (or pinned torch CPU tensors viewed as numpy) in and out."""
+        def hp(a, dtype, numel):
+            if a is None:
+                return None
+            if a.dtype != dtype or not a.flags["C_CONTIGUOUS"] or a.size != numel:
+                raise TypeError(f"expected contiguous {dtype} array of {numel} elements")
+            return a.ctypes.data
+        n, npx = self.n_agents, self.n_agents * self.K * self.H * self.W
+        _check(self._lib, self._lib.pic_render_host(
+            self._h, hp(poses, np.float32, 3 * n), hp(dims, np.float32, 3 * n), hp(active, np.uint8, n),
+            _rig_array(rig), hp(out_class, np.uint8, npx), hp(out_depth, np.float16, npx), _stream_ptr(stream)))
+        return out_class, out_depth
+
+    def set_state(self, state, dims, active=None, stream=None):
+        import torch
+        n = self.n_agents
+        _check(self._lib, self._lib.pic_set_state(
+            self._h, _dev_ptr(state, torch.float32, 4 * n), _dev_ptr(dims, torch.float32, 3 * n),
+            _dev_ptr(active, torch.uint8, n) if active is not None else None, _stream_ptr(stream)))
+
+    def get_state(self, out=None, stream=None):
+        import torch
+        if out is None:
+            out = torch.empty((self.E, self.A, 4), dtype=torch.float32, device=self.device)
+        _check(self._lib, self._lib.pic_get_state(self._h, _dev_ptr(out, torch.float32, 4 * self.n_agents),
+                                                  _stream_ptr(stream)))
+        return out
+
+    def step(self, actions, rig, out_class=None, out_depth=None, stream=None):
+        import torch
+        if out_class is None or out_depth is None:
+            out_class, out_depth = self.alloc_outputs()
+        n, npx = self.n_agents, self.n_agents * self.K * self.H * self.W
+        _check(self._lib, self._lib.pic_step(
+            self._h, _dev_ptr(actions, torch.float32, 2 * n), _rig_array(rig), _dev_ptr(out_class, torch.uint8, npx),
+            _dev_ptr(out_depth, torch.float16, npx), _stream_ptr(stream)))
+        return out_class, out_depth
+
+    def status(self, stream=None) -> int:
+        flags = C.c_uint32(0)
+        _check(self._lib, self._lib.pic_get_status(self._h, C.byref(flags), _stream_ptr(stream)))
+        return int(flags.value)
+
+    def set_option(self, option: int, value) -> None:
+        import torch
+        if isinstance(value, torch.Tensor):
+            self._keep.append(value)
+            value = value.data_ptr()
+        _check(self._lib, self._lib.pic_scene_set_option(self._h, int(option), int(value)))
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self._lib.pic_scene_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()

@@ -1,0 +1,353 @@
+// C ABI of the rasterizer library: scene management, argument validation, launches.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/pictura.h"
+#include "pic_types.h"
+
+namespace pic {
+size_t render_smem_bytes();
+cudaError_t configure_kernels();
+cudaError_t launch_agents(int n, const float* poses, float* state, const float* actions, const float* dims,
+                          const uint8_t* active, AgentGeom* out, uint32_t* status, float dt, float wheelbase,
+                          float v_max, cudaStream_t stream);
+cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, cudaStream_t stream);
+}  // namespace pic
+
+namespace {
+
+constexpr float kDt = 0.1f, kWheelbase = 2.8f, kVMax = 30.0f;
+
+thread_local char g_err[512] = "";
+
+pic_status fail(pic_status st, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+#define CUDA_TRY(expr)                                                                                   \
+    do {                                                                                                 \
+        cudaError_t _e = (expr);                                                                         \
+        if (_e != cudaSuccess)                                                                           \
+            return fail(_e == cudaErrorMemoryAllocation ? PIC_ERR_OOM : PIC_ERR_CUDA, "%s: %s", #expr,   \
+                        cudaGetErrorString(_e));                                                         \
+    } while (0)
+
+}  // namespace
+
+struct pic_scene {
+    int E = 0, A = 0, K = 0, H = 0, W = 0;
+    float near_z = 0, far_z = 0;
+    int M = 0;
+    uint8_t cls_agent = 0, cls_sky = 0, cls_ground = 0;
+    int device = 0;
+    // device memory owned by the scene
+    int32_t* d_env_map = nullptr;
+    pic::MapInfo* d_maps = nullptr;
+    pic::Node* d_groups = nullptr;
+    pic::Node* d_leaves = nullptr;
+    pic::Prim* d_prims = nullptr;
+    pic::AgentGeom* d_agents = nullptr;
+    float* d_state = nullptr;       // [E*A*4]
+    float* d_dims = nullptr;        // [E*A*3]
+    uint8_t* d_active = nullptr;    // [E*A]
+    bool have_active = false;
+    uint32_t* d_status = nullptr;
+    // staging for pic_render_host
+    float* d_in_poses = nullptr;
+    float* d_in_dims = nullptr;
+    uint8_t* d_in_active = nullptr;
+    uint8_t* d_out_class = nullptr;
+    uint16_t* d_out_depth = nullptr;
+    // options
+    bool brute = false;
+    float* depth32 = nullptr;
+    unsigned long long* counters = nullptr;
+    long long view_first = 0, view_count = 0;
+    size_t n_prims = 0, n_leaves = 0, n_groups = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+void free_scene(pic_scene* s) {
+    cudaFree(s->d_env_map); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
+    cudaFree(s->d_agents); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
+    cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
+    cudaFree(s->d_out_depth);
+    delete s;
+}
+
+pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth,
+                       pic::RenderParams& P) {
+    if (!rig) return fail(PIC_ERR_INVALID_ARG, "rig is NULL");
+    if (!out_class || !out_depth) return fail(PIC_ERR_INVALID_ARG, "output pointer is NULL");
+    if ((reinterpret_cast<uintptr_t>(out_class) & 15u) || (reinterpret_cast<uintptr_t>(out_depth) & 15u))
+        return fail(PIC_ERR_INVALID_ARG, "output pointers must be 16-byte aligned");
+    std::memset(&P, 0, sizeof(P));
+    P.E = s->E; P.A = s->A; P.K = s->K; P.H = s->H; P.W = s->W;
+    P.tiles_x = (s->W + pic::TILE - 1) / pic::TILE;
+    P.tiles_y = (s->H + pic::TILE - 1) / pic::TILE;
+    P.near_z = s->near_z; P.far_z = s->far_z;
+    P.w_near = 1.0f / s->near_z; P.w_far = 1.0f / s->far_z;
+    P.cls_agent = s->cls_agent; P.cls_sky = s->cls_sky; P.cls_ground = s->cls_ground;
+    P.env_map = s->d_env_map; P.maps = s->d_maps; P.groups = s->d_groups; P.leaves = s->d_leaves; P.prims = s->d_prims;
+    P.agents = s->d_agents;
+    P.out_class = out_class; P.out_depth = out_depth; P.out_depth32 = s->depth32; P.counters = s->counters;
+    P.view_first = 0;
+    for (int k = 0; k < s->K; ++k) {
+        const pic_camera& c = rig[k];
+        const float vals[7] = {c.mount_x, c.mount_y, c.mount_z, c.yaw, c.pitch, c.fx, c.fy};
+        for (float v : vals)
+            if (!std::isfinite(v)) return fail(PIC_ERR_INVALID_ARG, "camera %d has a non-finite field", k);
+        if (!(c.fx > 0.f) || !(c.fy > 0.f)) return fail(PIC_ERR_INVALID_ARG, "camera %d: focal lengths must be positive", k);
+        pic::CamConst& o = P.cam[k];
+        o.mx = c.mount_x; o.my = c.mount_y; o.mz = c.mount_z;
+        o.cpsi = (float)std::cos((double)c.yaw); o.spsi = (float)std::sin((double)c.yaw);
+        o.cphi = (float)std::cos((double)c.pitch); o.sphi = (float)std::sin((double)c.pitch);
+        o.fx = c.fx; o.fy = c.fy;
+    }
+    return PIC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pic_last_error(void) { return g_err; }
+
+int32_t pic_version(void) { return 100; }
+
+pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
+    if (!d || !out) return fail(PIC_ERR_INVALID_ARG, "desc or out is NULL");
+    *out = nullptr;
+    if (d->size != sizeof(pic_scene_desc))
+        return fail(PIC_ERR_INVALID_ARG, "desc->size is %u, this library expects %zu", d->size, sizeof(pic_scene_desc));
+    if (d->E <= 0 || d->A <= 0 || d->K <= 0 || d->H <= 0 || d->W <= 0)
+        return fail(PIC_ERR_SHAPE, "E, A, K, H, W must be positive");
+    if (d->K > pic::MAX_CAMS) return fail(PIC_ERR_SHAPE, "at most %d cameras per rig", pic::MAX_CAMS);
+    if (d->H > 16384 || d->W > 16384) return fail(PIC_ERR_SHAPE, "images larger than 16384 pixels per side are not supported");
+    if ((long long)d->E * d->A > (1LL << 28)) return fail(PIC_ERR_SHAPE, "E*A too large");
+    if (!(d->near_z > 0.f) || !(d->far_z > d->near_z) || !std::isfinite(d->far_z))
+        return fail(PIC_ERR_INVALID_ARG, "need 0 < near_z < far_z < inf");
+    if (d->num_maps <= 0) return fail(PIC_ERR_SHAPE, "num_maps must be positive");
+    if (!d->map_tri_offset) return fail(PIC_ERR_INVALID_ARG, "map_tri_offset is NULL");
+    if (d->map_tri_offset[0] != 0) return fail(PIC_ERR_SHAPE, "map_tri_offset[0] must be 0");
+    for (int m = 0; m < d->num_maps; ++m)
+        if (d->map_tri_offset[m + 1] < d->map_tri_offset[m]) return fail(PIC_ERR_SHAPE, "map_tri_offset must be non-decreasing");
+    const int64_t n_tri = d->map_tri_offset[d->num_maps];
+    if (n_tri > 0 && (!d->tri_xyz || !d->tri_class)) return fail(PIC_ERR_INVALID_ARG, "triangle arrays are NULL");
+    for (int64_t i = 0; i < 9 * n_tri; ++i)
+        if (!std::isfinite(d->tri_xyz[i])) return fail(PIC_ERR_INVALID_ARG, "triangle %lld has a non-finite coordinate", (long long)(i / 9));
+    if (d->env_map_id) {
+        for (int e = 0; e < d->E; ++e)
+            if (d->env_map_id[e] < 0 || d->env_map_id[e] >= d->num_maps) return fail(PIC_ERR_SHAPE, "env_map_id[%d] out of range", e);
+    } else if (d->num_maps != 1 && d->num_maps != d->E) {
+        return fail(PIC_ERR_SHAPE, "env_map_id is NULL but num_maps is neither 1 nor E");
+    }
+    int n_dev = 0;
+    CUDA_TRY(cudaGetDeviceCount(&n_dev));
+    if (d->device < 0 || d->device >= n_dev) return fail(PIC_ERR_INVALID_ARG, "device %d does not exist", d->device);
+    DeviceGuard guard(d->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", d->device);
+    cudaDeviceProp prop;
+    CUDA_TRY(cudaGetDeviceProperties(&prop, d->device));
+    if (prop.major < 10) return fail(PIC_ERR_CUDA, "device %d is sm_%d%d; this library is built for sm_100a only", d->device, prop.major, prop.minor);
+    if ((size_t)prop.sharedMemPerBlockOptin < pic::render_smem_bytes())
+        return fail(PIC_ERR_CUDA, "device offers %zu bytes of shared memory per block, %zu needed", (size_t)prop.sharedMemPerBlockOptin, pic::render_smem_bytes());
+    CUDA_TRY(pic::configure_kernels());
+
+    char err[256] = "";
+    pic::HostHierarchy* hh = pic::build_hierarchy(d->num_maps, d->map_tri_offset, d->tri_xyz, d->tri_class, d->A, err, sizeof(err));
+    if (!hh) return fail(PIC_ERR_SHAPE, "%s", err);
+
+    pic_scene* s = new (std::nothrow) pic_scene();
+    if (!s) { pic::free_hierarchy(hh); return fail(PIC_ERR_OOM, "host allocation failed"); }
+    s->E = d->E; s->A = d->A; s->K = d->K; s->H = d->H; s->W = d->W;
+    s->near_z = d->near_z; s->far_z = d->far_z; s->M = d->num_maps;
+    s->cls_agent = d->agent_class; s->cls_sky = d->sky_class; s->cls_ground = d->ground_class;
+    s->device = d->device;
+
+    size_t np, nl, ng, nm;
+    const pic::Prim* prims = pic::hierarchy_prims(hh, &np);
+    const pic::Node* leaves = pic::hierarchy_leaves(hh, &nl);
+    const pic::Node* groups = pic::hierarchy_groups(hh, &ng);
+    const pic::MapInfo* maps = pic::hierarchy_maps(hh, &nm);
+    s->n_prims = np; s->n_leaves = nl; s->n_groups = ng;
+    const size_t n_agents = (size_t)d->E * d->A;
+    int32_t* env_map = new (std::nothrow) int32_t[d->E];
+    if (!env_map) { pic::free_hierarchy(hh); free_scene(s); return fail(PIC_ERR_OOM, "host allocation failed"); }
+    for (int e = 0; e < d->E; ++e) env_map[e] = d->env_map_id ? d->env_map_id[e] : (d->num_maps == 1 ? 0 : e);
+
+    cudaError_t ce = cudaSuccess;
+    auto dmalloc = [&](void** p, size_t bytes) { if (ce == cudaSuccess) ce = cudaMalloc(p, bytes ? bytes : 16); };
+    auto upload = [&](void* dst, const void* src, size_t bytes) {
+        if (ce == cudaSuccess && bytes) ce = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice);
+    };
+    dmalloc((void**)&s->d_env_map, sizeof(int32_t) * d->E);
+    dmalloc((void**)&s->d_maps, sizeof(pic::MapInfo) * nm);
+    dmalloc((void**)&s->d_groups, sizeof(pic::Node) * ng);
+    dmalloc((void**)&s->d_leaves, sizeof(pic::Node) * nl);
+    dmalloc((void**)&s->d_prims, sizeof(pic::Prim) * np);
+    dmalloc((void**)&s->d_agents, sizeof(pic::AgentGeom) * n_agents);
+    dmalloc((void**)&s->d_state, sizeof(float) * 4 * n_agents);
+    dmalloc((void**)&s->d_dims, sizeof(float) * 3 * n_agents);
+    dmalloc((void**)&s->d_active, n_agents);
+    dmalloc((void**)&s->d_status, sizeof(uint32_t));
+    upload(s->d_env_map, env_map, sizeof(int32_t) * d->E);
+    upload(s->d_maps, maps, sizeof(pic::MapInfo) * nm);
+    upload(s->d_groups, groups, sizeof(pic::Node) * ng);
+    upload(s->d_leaves, leaves, sizeof(pic::Node) * nl);
+    upload(s->d_prims, prims, sizeof(pic::Prim) * np);
+    if (ce == cudaSuccess) ce = cudaMemset(s->d_status, 0, sizeof(uint32_t));
+    if (ce == cudaSuccess) ce = cudaMemset(s->d_state, 0, sizeof(float) * 4 * n_agents);
+    if (ce == cudaSuccess) ce = cudaMemset(s->d_dims, 0, sizeof(float) * 3 * n_agents);
+    if (ce == cudaSuccess) ce = cudaMemset(s->d_active, 1, n_agents);
+    delete[] env_map;
+    pic::free_hierarchy(hh);
+    if (ce != cudaSuccess) {
+        free_scene(s);
+        return fail(ce == cudaErrorMemoryAllocation ? PIC_ERR_OOM : PIC_ERR_CUDA, "scene allocation/upload: %s", cudaGetErrorString(ce));
+    }
+    *out = s;
+    return PIC_OK;
+}
+
+pic_status pic_scene_destroy(pic_scene* s) {
+    if (!s) return PIC_OK;
+    DeviceGuard guard(s->device);
+    cudaDeviceSynchronize();
+    free_scene(s);
+    return PIC_OK;
+}
+
+pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    switch (option) {
+        case PIC_OPT_BRUTE_FORCE: s->brute = value != 0; return PIC_OK;
+        case PIC_OPT_DEPTH32: s->depth32 = reinterpret_cast<float*>(static_cast<uintptr_t>(value)); return PIC_OK;
+        case PIC_OPT_COUNTERS: s->counters = reinterpret_cast<unsigned long long*>(static_cast<uintptr_t>(value)); return PIC_OK;
+        case PIC_OPT_VIEW_FIRST:
+            if (value >= (uint64_t)s->E * s->A * s->K) return fail(PIC_ERR_INVALID_ARG, "first view out of range");
+            s->view_first = (long long)value; return PIC_OK;
+        case PIC_OPT_VIEW_COUNT: s->view_count = (long long)value; return PIC_OK;
+        default: return fail(PIC_ERR_INVALID_ARG, "unknown option %d", option);
+    }
+}
+
+static pic_status render_from(pic_scene* s, const float* poses, float* state, const float* actions, const float* dims,
+                              const uint8_t* active, const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth,
+                              cudaStream_t stream) {
+    pic::RenderParams P;
+    pic_status st = fill_params(s, rig, out_class, out_depth, P);
+    if (st != PIC_OK) return st;
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    const int n_agents = s->E * s->A;
+    CUDA_TRY(pic::launch_agents(n_agents, poses, state, actions, dims, active, s->d_agents, s->d_status, kDt, kWheelbase,
+                                kVMax, stream));
+    const long long total = (long long)s->E * s->A * s->K;
+    long long count = total - s->view_first;
+    if (s->view_count > 0 && s->view_count < count) count = s->view_count;
+    P.view_first = s->view_first;
+    CUDA_TRY(pic::launch_render(P, count, s->brute, stream));
+    return PIC_OK;
+}
+
+pic_status pic_render(pic_scene* s, const float* poses, const float* dims, const uint8_t* active, const pic_camera* rig,
+                      uint8_t* out_class, uint16_t* out_depth, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!poses || !dims) return fail(PIC_ERR_INVALID_ARG, "poses or dims is NULL");
+    return render_from(s, poses, nullptr, nullptr, dims, active, rig, out_class, out_depth, static_cast<cudaStream_t>(cuda_stream));
+}
+
+pic_status pic_render_host(pic_scene* s, const float* poses, const float* dims, const uint8_t* active,
+                           const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!poses || !dims || !out_class || !out_depth) return fail(PIC_ERR_INVALID_ARG, "a required host pointer is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t n_agents = (size_t)s->E * s->A;
+    const size_t n_px = n_agents * s->K * s->H * s->W;
+    if (!s->d_out_class) {
+        CUDA_TRY(cudaMalloc((void**)&s->d_in_poses, sizeof(float) * 3 * n_agents));
+        CUDA_TRY(cudaMalloc((void**)&s->d_in_dims, sizeof(float) * 3 * n_agents));
+        CUDA_TRY(cudaMalloc((void**)&s->d_in_active, n_agents));
+        CUDA_TRY(cudaMalloc((void**)&s->d_out_depth, sizeof(uint16_t) * n_px));
+        CUDA_TRY(cudaMalloc((void**)&s->d_out_class, n_px));
+    }
+    CUDA_TRY(cudaMemcpyAsync(s->d_in_poses, poses, sizeof(float) * 3 * n_agents, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(s->d_in_dims, dims, sizeof(float) * 3 * n_agents, cudaMemcpyHostToDevice, stream));
+    if (active) CUDA_TRY(cudaMemcpyAsync(s->d_in_active, active, n_agents, cudaMemcpyHostToDevice, stream));
+    pic_status st = render_from(s, s->d_in_poses, nullptr, nullptr, s->d_in_dims, active ? s->d_in_active : nullptr, rig,
+                                s->d_out_class, s->d_out_depth, stream);
+    if (st != PIC_OK) return st;
+    CUDA_TRY(cudaMemcpyAsync(out_class, s->d_out_class, n_px, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaMemcpyAsync(out_depth, s->d_out_depth, sizeof(uint16_t) * n_px, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return PIC_OK;
+}
+
+pic_status pic_set_state(pic_scene* s, const float* state, const float* dims, const uint8_t* active, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!state || !dims) return fail(PIC_ERR_INVALID_ARG, "state or dims is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t n = (size_t)s->E * s->A;
+    CUDA_TRY(cudaMemcpyAsync(s->d_state, state, sizeof(float) * 4 * n, cudaMemcpyDeviceToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(s->d_dims, dims, sizeof(float) * 3 * n, cudaMemcpyDeviceToDevice, stream));
+    if (active) CUDA_TRY(cudaMemcpyAsync(s->d_active, active, n, cudaMemcpyDeviceToDevice, stream));
+    else CUDA_TRY(cudaMemsetAsync(s->d_active, 1, n, stream));
+    return PIC_OK;
+}
+
+pic_status pic_get_state(pic_scene* s, float* state_out, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!state_out) return fail(PIC_ERR_INVALID_ARG, "state_out is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    const size_t n = (size_t)s->E * s->A;
+    CUDA_TRY(cudaMemcpyAsync(state_out, s->d_state, sizeof(float) * 4 * n, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
+    return PIC_OK;
+}
+
+pic_status pic_step(pic_scene* s, const float* actions, const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth,
+                    void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!actions) return fail(PIC_ERR_INVALID_ARG, "actions is NULL");
+    return render_from(s, nullptr, s->d_state, actions, s->d_dims, s->d_active, rig, out_class, out_depth,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+pic_status pic_get_status(pic_scene* s, uint32_t* flags, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!flags) return fail(PIC_ERR_INVALID_ARG, "flags is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    CUDA_TRY(cudaMemcpyAsync(flags, s->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaMemsetAsync(s->d_status, 0, sizeof(uint32_t), stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return PIC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,229 @@
+// Host-side construction of the per-map culling hierarchy (runs once, in pic_scene_create).
+//
+// Input triangles are first fused pairwise into planar convex quads where the input allows it
+// (two consecutive triangles of one class sharing an edge: road, marking and wall quads), then
+// sorted along a Morton curve and cut into leaves of up to 32 primitives; leaves are grouped by
+// 32.  Primitives much longer than the average get small leaves of their own, so that one long
+// road quad does not inflate the box of 31 lane markings.  The renderer tests group boxes, then
+// leaf boxes, then primitives against each view frustum.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "pic_types.h"
+
+namespace pic {
+
+struct HostHierarchy {
+    std::vector<Prim> prims;
+    std::vector<Node> leaves;
+    std::vector<Node> groups;
+    std::vector<MapInfo> maps;
+};
+
+namespace {
+
+struct D3 { double x, y, z; };
+inline D3 sub(D3 a, D3 b) { return {a.x - b.x, a.y - b.y, a.z - b.z}; }
+inline D3 cross(D3 a, D3 b) { return {a.y * b.z - a.z * b.y, a.z * b.x - a.x * b.z, a.x * b.y - a.y * b.x}; }
+inline double dot(D3 a, D3 b) { return a.x * b.x + a.y * b.y + a.z * b.z; }
+inline double norm(D3 a) { return std::sqrt(dot(a, a)); }
+
+struct F3 { float x, y, z; };
+inline bool same(F3 a, F3 b) { return a.x == b.x && a.y == b.y && a.z == b.z; }
+inline D3 d3(F3 a) { return {a.x, a.y, a.z}; }
+inline bool lex_less(F3 a, F3 b) {
+    if (a.x != b.x) return a.x < b.x;
+    if (a.y != b.y) return a.y < b.y;
+    return a.z < b.z;
+}
+
+// Try to fuse triangles a and b into the convex planar quad (q[0..3] in perimeter order).
+bool fuse_quad(const F3 a[3], const F3 b[3], F3 q[4]) {
+    for (int i = 0; i < 3; ++i) {
+        // candidate: a's vertex i is the one b does not share
+        F3 pa = a[i], s0 = a[(i + 1) % 3], s1 = a[(i + 2) % 3];
+        int j0 = -1, j1 = -1;
+        for (int j = 0; j < 3; ++j) {
+            if (same(b[j], s0)) j0 = j;
+            if (same(b[j], s1)) j1 = j;
+        }
+        if (j0 < 0 || j1 < 0 || j0 == j1) continue;
+        F3 pb = b[3 - j0 - j1];
+        if (same(pb, pa) || same(pb, s0) || same(pb, s1)) return false;
+        D3 P[4] = {d3(pa), d3(s0), d3(pb), d3(s1)};
+        D3 n = cross(sub(P[2], P[0]), sub(P[3], P[1]));
+        double nn = norm(n);
+        if (nn == 0.0) return false;
+        // coplanar: the two diagonals' common normal must be orthogonal to every side
+        double scale = 0.0;
+        for (int k = 0; k < 4; ++k) scale = std::max(scale, norm(sub(P[(k + 1) % 4], P[k])));
+        for (int k = 0; k < 4; ++k)
+            if (std::fabs(dot(n, sub(P[(k + 1) % 4], P[k]))) > 1e-7 * nn * scale) return false;
+        // strictly convex with one winding
+        for (int k = 0; k < 4; ++k) {
+            D3 e0 = sub(P[(k + 1) % 4], P[k]), e1 = sub(P[(k + 2) % 4], P[(k + 1) % 4]);
+            if (dot(cross(e0, e1), n) <= 1e-9 * nn * norm(e0) * norm(e1)) return false;
+        }
+        q[0] = pa; q[1] = s0; q[2] = pb; q[3] = s1;
+        return true;
+    }
+    return false;
+}
+
+inline uint64_t spread21(uint64_t v) {   // 21 bits -> every third bit
+    v &= 0x1fffffULL;
+    v = (v | v << 32) & 0x1f00000000ffffULL;
+    v = (v | v << 16) & 0x1f0000ff0000ffULL;
+    v = (v | v << 8) & 0x100f00f00f00f00fULL;
+    v = (v | v << 4) & 0x10c30c30c30c30c3ULL;
+    v = (v | v << 2) & 0x1249249249249249ULL;
+    return v;
+}
+
+struct Item { uint64_t code; uint32_t id; };
+
+void box_of_prim(const Prim& p, float lo[3], float hi[3]) {
+    int nv = (p.flags & 1u) ? 4 : 3;
+    for (int c = 0; c < 3; ++c) { lo[c] = p.v[c]; hi[c] = p.v[c]; }
+    for (int k = 1; k < nv; ++k)
+        for (int c = 0; c < 3; ++c) {
+            lo[c] = std::min(lo[c], p.v[3 * k + c]);
+            hi[c] = std::max(hi[c], p.v[3 * k + c]);
+        }
+}
+
+}  // namespace
+
+HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const float* tri_xyz,
+                               const uint8_t* tri_class, int agents_per_env, char* err, int err_len) {
+    HostHierarchy* h = new HostHierarchy();
+    h->maps.resize(num_maps);
+    std::vector<Prim> local;
+    std::vector<Item> items;
+    for (int m = 0; m < num_maps; ++m) {
+        int64_t t0 = tri_offset[m], t1 = tri_offset[m + 1];
+        int64_t n = t1 - t0;
+        if (n + 12LL * agents_per_env > (1LL << 24)) {
+            std::snprintf(err, err_len, "map %d has %lld triangles; at most 2^24 - 12*A are supported", m, (long long)n);
+            delete h;
+            return nullptr;
+        }
+        // ---- primitives: fuse consecutive triangle pairs into quads where possible
+        local.clear();
+        for (int64_t i = 0; i < n;) {
+            const F3* a = reinterpret_cast<const F3*>(tri_xyz + 9 * (t0 + i));
+            Prim p;
+            std::memset(&p, 0, sizeof(p));
+            F3 q[4];
+            bool quad = false;
+            if (i + 1 < n && tri_class[t0 + i] == tri_class[t0 + i + 1]) {
+                const F3* b = reinterpret_cast<const F3*>(tri_xyz + 9 * (t0 + i + 1));
+                quad = fuse_quad(a, b, q);
+            }
+            if (!quad) { q[0] = a[0]; q[1] = a[1]; q[2] = a[2]; q[3] = a[2]; }
+            for (int k = 0; k < 4; ++k) { p.v[3 * k] = q[k].x; p.v[3 * k + 1] = q[k].y; p.v[3 * k + 2] = q[k].z; }
+            p.key_lo = ((0xFFFFFFu - (uint32_t)i) << 8) | tri_class[t0 + i];
+            p.flags = quad ? 1u : 0u;
+            int nv = quad ? 4 : 3;
+            for (int k = 0; k < nv; ++k)
+                if (!lex_less(q[k], q[(k + 1) % nv])) p.flags |= 1u << (4 + k);
+            local.push_back(p);
+            i += quad ? 2 : 1;
+        }
+        // ---- classify long primitives, Morton-sort both classes
+        size_t np = local.size();
+        float mlo[3] = {0, 0, 0}, mhi[3] = {0, 0, 0};
+        std::vector<float> diag(np);
+        double mean_diag = 0.0;
+        for (size_t i = 0; i < np; ++i) {
+            float lo[3], hi[3];
+            box_of_prim(local[i], lo, hi);
+            for (int c = 0; c < 3; ++c) {
+                if (i == 0 || lo[c] < mlo[c]) mlo[c] = lo[c];
+                if (i == 0 || hi[c] > mhi[c]) mhi[c] = hi[c];
+            }
+            double dx = hi[0] - lo[0], dy = hi[1] - lo[1], dz = hi[2] - lo[2];
+            diag[i] = (float)std::sqrt(dx * dx + dy * dy + dz * dz);
+            mean_diag += diag[i];
+        }
+        if (np) mean_diag /= (double)np;
+        double extent = std::max({(double)mhi[0] - mlo[0], (double)mhi[1] - mlo[1], (double)mhi[2] - mlo[2], 1e-30});
+        items.clear();
+        for (size_t i = 0; i < np; ++i) {
+            float lo[3], hi[3];
+            box_of_prim(local[i], lo, hi);
+            uint64_t code = 0;
+            for (int c = 0; c < 3; ++c) {
+                double u = ((0.5 * ((double)lo[c] + hi[c])) - mlo[c]) / extent;
+                uint64_t g = (uint64_t)std::min(2097151.0, std::max(0.0, u * 2097152.0));
+                code |= spread21(g) << c;
+            }
+            bool is_long = diag[i] > 4.0 * mean_diag;
+            items.push_back({code | (is_long ? (1ULL << 63) : 0ULL), (uint32_t)i});
+        }
+        std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
+            return a.code != b.code ? a.code < b.code : a.id < b.id;
+        });
+        // ---- leaves
+        MapInfo& mi = h->maps[m];
+        std::memset(&mi, 0, sizeof(mi));
+        mi.n_tris = (uint32_t)n;
+        mi.prim_begin = (uint32_t)h->prims.size();
+        size_t leaf_begin = h->leaves.size();
+        size_t i = 0;
+        while (i < np) {
+            bool is_long = (items[i].code >> 63) != 0;
+            size_t cap = is_long ? LONG_LEAF_PRIMS : LEAF_PRIMS;
+            size_t j = i;
+            Node leaf;
+            leaf.first = (uint32_t)h->prims.size();
+            while (j < np && j - i < cap && ((items[j].code >> 63) != 0) == is_long) {
+                const Prim& p = local[items[j].id];
+                float lo[3], hi[3];
+                box_of_prim(p, lo, hi);
+                for (int c = 0; c < 3; ++c) {
+                    leaf.lo[c] = (j == i) ? lo[c] : std::min(leaf.lo[c], lo[c]);
+                    leaf.hi[c] = (j == i) ? hi[c] : std::max(leaf.hi[c], hi[c]);
+                }
+                h->prims.push_back(p);
+                ++j;
+            }
+            leaf.count = (uint32_t)(j - i);
+            h->leaves.push_back(leaf);
+            i = j;
+        }
+        mi.prim_end = (uint32_t)h->prims.size();
+        // ---- groups of consecutive leaves
+        mi.group_begin = (uint32_t)h->groups.size();
+        size_t leaf_end = h->leaves.size();
+        for (size_t l = leaf_begin; l < leaf_end; l += GROUP_LEAVES) {
+            Node g;
+            g.first = (uint32_t)l;
+            g.count = (uint32_t)std::min<size_t>(GROUP_LEAVES, leaf_end - l);
+            for (uint32_t k = 0; k < g.count; ++k)
+                for (int c = 0; c < 3; ++c) {
+                    g.lo[c] = (k == 0) ? h->leaves[l + k].lo[c] : std::min(g.lo[c], h->leaves[l + k].lo[c]);
+                    g.hi[c] = (k == 0) ? h->leaves[l + k].hi[c] : std::max(g.hi[c], h->leaves[l + k].hi[c]);
+                }
+            h->groups.push_back(g);
+        }
+        mi.group_end = (uint32_t)h->groups.size();
+        if (h->prims.size() > 0xFFFFFFF0ull) {
+            std::snprintf(err, err_len, "more than 2^32 primitives in one scene");
+            delete h;
+            return nullptr;
+        }
+    }
+    return h;
+}
+
+void free_hierarchy(HostHierarchy* h) { delete h; }
+const Prim* hierarchy_prims(const HostHierarchy* h, size_t* n) { *n = h->prims.size(); return h->prims.data(); }
+const Node* hierarchy_leaves(const HostHierarchy* h, size_t* n) { *n = h->leaves.size(); return h->leaves.data(); }
+const Node* hierarchy_groups(const HostHierarchy* h, size_t* n) { *n = h->groups.size(); return h->groups.data(); }
+const MapInfo* hierarchy_maps(const HostHierarchy* h, size_t* n) { *n = h->maps.size(); return h->maps.data(); }
+
+}  // namespace pic

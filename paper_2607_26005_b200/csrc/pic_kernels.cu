@@ -1,0 +1,797 @@
+// CUDA kernels of the batched egocentric rasterizer (sm_100a).
+//
+// One CTA renders one tile (up to 64 x 64 pixels) of one view.  The z-buffer lives in shared
+// memory as one 64-bit key per pixel:
+//     key = float_bits(1/z) << 32 | (0xFFFFFF - primitive index) << 8 | class
+// so "nearest fragment wins, ties to the lower index" is a plain unsigned max, independent of
+// the order in which primitives are processed; 0 means "no fragment" (background).
+//
+// Steps per tile (letters as in the scope table of the design notes):
+//   (a) cull      group boxes -> leaf boxes -> primitives against the tile frustum; survivors are
+//                 compacted into a candidate list with warp ballots; agent boxes are culled the same way
+//   (c) set-up    per candidate: camera-space vertices, 3-4 edge functions, 1/z plane
+//       small     primitives whose pixel box holds few pixel centres are rasterized at once by
+//                 their thread with a shared-memory atomic max
+//   (b) binning   the others are tested against the 8 x 8 pixel blocks of the tile (trivial
+//                 reject / trivial accept with the same float32 edge functions) into bit masks
+//   (c) raster    each warp owns blocks; a lane owns two pixels, keeps their keys in registers
+//                 and walks the block's mask
+//   (d) store     keys -> class u8 + depth binary16, 16 pixels per thread, 128-bit stores
+//
+// All arithmetic that decides a pixel is written with explicit round-to-nearest intrinsics so that
+// every kernel (production and exhaustive) evaluates bit-identical expressions.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pic_types.h"
+
+namespace pic {
+
+constexpr int LCAP = 128;         // binned primitives per pass (one mask bit each)
+constexpr int LWORDS = LCAP / 64;
+constexpr int CCAP = 512;         // candidate list entries
+constexpr int LEAFCAP = 1024;     // visible leaves per batch of 32 groups
+constexpr int REC = 17;           // words per set-up record (odd: conflict-free per-lane reads)
+constexpr int SMALL_MAX_PIXELS = 16;   // pixel centres in the box of a "small" primitive
+constexpr float ZPROJ_FRAC = 0.5f;     // vertices nearer than this * near are not projected
+
+struct __align__(16) Cam {
+    float px, py;              // ego position
+    float mwx, mwy, mwz;       // mount in world axes
+    float rx, ry;              // right   (rz = 0)
+    float dx, dy, dz;          // down
+    float fx_, fy_, fz_;       // forward
+    float focx, focy;          // focal lengths
+    float cx, cy;              // principal point
+};
+
+struct PrimEq {
+    float nx[4], ny[4], nz[4];   // E_i = nx*rx + ny*ry + nz, sign-normalised (inside: E_i > 0)
+    float wx, wy, wz;            // 1/z = wx*rx + wy*ry + wz
+    uint32_t tl;                 // bit i: exact zeros of edge i belong to the primitive
+};
+
+struct V3 { float x, y, z; };
+
+__device__ __forceinline__ float fm(float a, float b, float c) { return __fmaf_rn(a, b, c); }
+__device__ __forceinline__ float mul(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ float sub(float a, float b) { return __fsub_rn(a, b); }
+__device__ __forceinline__ float add(float a, float b) { return __fadd_rn(a, b); }
+
+__device__ __forceinline__ V3 vsub(V3 a, V3 b) { return {sub(a.x, b.x), sub(a.y, b.y), sub(a.z, b.z)}; }
+__device__ __forceinline__ V3 vcross(V3 a, V3 b) {
+    return {fm(a.y, b.z, -mul(a.z, b.y)), fm(a.z, b.x, -mul(a.x, b.z)), fm(a.x, b.y, -mul(a.y, b.x))};
+}
+__device__ __forceinline__ float vdot(V3 a, V3 b) { return fm(a.x, b.x, fm(a.y, b.y, mul(a.z, b.z))); }
+
+// World point -> camera space: subtract the ego position first (keeps float32 accurate far from
+// the origin), then the mount, then rotate.
+__device__ __forceinline__ V3 to_camera(const Cam& c, float X, float Y, float Z) {
+    float qx = sub(sub(X, c.px), c.mwx);
+    float qy = sub(sub(Y, c.py), c.mwy);
+    float qz = sub(Z, c.mwz);
+    V3 r;
+    r.x = fm(c.rx, qx, mul(c.ry, qy));
+    r.y = fm(c.dx, qx, fm(c.dy, qy, mul(c.dz, qz)));
+    r.z = fm(c.fx_, qx, fm(c.fy_, qy, mul(c.fz_, qz)));
+    return r;
+}
+
+// Ego-relative vector (already minus ego position) -> camera space, without the mount offset.
+__device__ __forceinline__ V3 rotate_to_camera(const Cam& c, float qx, float qy, float qz) {
+    V3 r;
+    r.x = fm(c.rx, qx, mul(c.ry, qy));
+    r.y = fm(c.dx, qx, fm(c.dy, qy, mul(c.dz, qz)));
+    r.z = fm(c.fx_, qx, fm(c.fy_, qy, mul(c.fz_, qz)));
+    return r;
+}
+
+__device__ __forceinline__ void make_camera(Cam& c, const AgentGeom& ego, const CamConst& k, int W, int H) {
+    float ca = fm(ego.c, k.cpsi, -mul(ego.s, k.spsi));
+    float sa = fm(ego.s, k.cpsi, mul(ego.c, k.spsi));
+    c.px = ego.x; c.py = ego.y;
+    c.mwx = fm(ego.c, k.mx, -mul(ego.s, k.my));
+    c.mwy = fm(ego.s, k.mx, mul(ego.c, k.my));
+    c.mwz = k.mz;
+    c.rx = sa; c.ry = -ca;
+    c.fx_ = mul(k.cphi, ca); c.fy_ = mul(k.cphi, sa); c.fz_ = k.sphi;
+    c.dx = mul(k.sphi, ca); c.dy = mul(k.sphi, sa); c.dz = -k.cphi;
+    c.focx = k.fx; c.focy = k.fy;
+    c.cx = 0.5f * (float)W; c.cy = 0.5f * (float)H;
+}
+
+// Edge functions and reciprocal-depth plane of a primitive given in camera space.
+// Returns false for degenerate / edge-on primitives (D == 0), which cover nothing.
+__device__ __forceinline__ bool prim_equations(const V3 (&V)[4], bool quad, uint32_t flags, PrimEq& q) {
+    const int n = quad ? 4 : 3;
+    V3 N[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (i < n) {
+            const V3 a = V[i];
+            const V3 b = (i == 3 || (i == 2 && !quad)) ? V[0] : V[(i + 1) & 3];
+            if ((flags >> (4 + i)) & 1u) {       // evaluate in the canonical direction b -> a, then negate
+                V3 t = vcross(b, vsub(a, b));
+                N[i] = {-t.x, -t.y, -t.z};
+            } else {
+                N[i] = vcross(a, vsub(b, a));
+            }
+        } else {
+            N[i] = {0.f, 0.f, 1.f};              // triangles: a fourth edge that is always inside
+        }
+    }
+    V3 P = quad ? vcross(vsub(V[2], V[0]), vsub(V[3], V[1])) : vcross(vsub(V[1], V[0]), vsub(V[2], V[0]));
+    float D = vdot(P, V[0]);
+    if (!(D != 0.f)) return false;               // also drops NaN
+    const float s = D < 0.f ? -1.f : 1.f;
+    uint32_t tl = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float sx = (i < n) ? mul(s, N[i].x) : 0.f, sy = (i < n) ? mul(s, N[i].y) : 0.f, sz = (i < n) ? mul(s, N[i].z) : 1.f;
+        q.nx[i] = sx; q.ny[i] = sy; q.nz[i] = sz;
+        if (sx > 0.f || (sx == 0.f && sy > 0.f)) tl |= 1u << i;
+    }
+    q.tl = tl;
+    q.wx = __fdiv_rn(P.x, D); q.wy = __fdiv_rn(P.y, D); q.wz = __fdiv_rn(P.z, D);
+    return true;
+}
+
+// Fragment of a primitive at the ray (rx, ry, 1): the high key word (bits of 1/z), or 0 if the
+// pixel is not covered or the depth is outside [near, far].
+__device__ __forceinline__ uint32_t fragment(const PrimEq& q, float rx, float ry, float w_near, float w_far) {
+    bool in = true;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float e = fm(q.nx[i], rx, fm(q.ny[i], ry, q.nz[i]));
+        in = in && (e > 0.f || (e == 0.f && ((q.tl >> i) & 1u)));
+    }
+    float w = fm(q.wx, rx, fm(q.wy, ry, q.wz));
+    in = in && (w >= w_far) && (w <= w_near);
+    return in ? __float_as_uint(w) : 0u;
+}
+
+__device__ __forceinline__ unsigned long long make_key(uint32_t wbits, uint32_t key_lo) {
+    return ((unsigned long long)wbits << 32) | key_lo;
+}
+
+// ------------------------------------------------------------------------------------------------
+// agent kernel: poses/dims/active -> AgentGeom (optionally after one kinematic-bicycle step)
+// ------------------------------------------------------------------------------------------------
+__global__ void agent_kernel(int n, const float* __restrict__ poses, int pose_stride, float* state,
+                             const float* __restrict__ actions, const float* __restrict__ dims,
+                             const uint8_t* __restrict__ active, AgentGeom* __restrict__ out, uint32_t* status,
+                             float dt, float wheelbase, float v_max) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    bool act = active ? active[i] != 0 : true;
+    float x, y, th;
+    if (state) {                                   // pic_step: update the scene's own state in place
+        float v;
+        x = state[4 * i]; y = state[4 * i + 1]; th = state[4 * i + 2]; v = state[4 * i + 3];
+        if (actions && act) {
+            float acc = actions[2 * i], steer = actions[2 * i + 1];
+            float s, c;
+            sincosf(th, &s, &c);
+            float nx = fm(mul(v, c), dt, x);
+            float ny = fm(mul(v, s), dt, y);
+            float nth = fm(mul(__fdiv_rn(v, wheelbase), tanf(steer)), dt, th);
+            float nv = fminf(fmaxf(fm(acc, dt, v), 0.f), v_max);
+            x = nx; y = ny; th = nth; v = nv;
+            state[4 * i] = x; state[4 * i + 1] = y; state[4 * i + 2] = th; state[4 * i + 3] = v;
+        }
+    } else {
+        x = poses[pose_stride * i]; y = poses[pose_stride * i + 1]; th = poses[pose_stride * i + 2];
+    }
+    float l = dims[3 * i], w = dims[3 * i + 1], h = dims[3 * i + 2];
+    if (!(isfinite(x) && isfinite(y) && isfinite(th) && isfinite(l) && isfinite(w) && isfinite(h))) {
+        atomicOr(status, 1u);
+        act = false;
+        x = y = th = 0.f; l = w = h = 1.f;
+    }
+    AgentGeom g;
+    g.x = x; g.y = y;
+    sincosf(th, &g.s, &g.c);
+    g.hl = 0.5f * l; g.hw = 0.5f * w; g.h = h;
+    g.active = act ? 1u : 0u;
+    out[i] = g;
+}
+
+// ------------------------------------------------------------------------------------------------
+// shared-memory layout of a render CTA
+// ------------------------------------------------------------------------------------------------
+struct __align__(16) TileSmem {
+    unsigned long long key[TILE * TILE];      // 32 KB
+    float rec[LCAP * REC];                    // set-up records of binned primitives
+    unsigned long long bin_any[64][LWORDS];   // per 8x8 block: primitives to test
+    unsigned long long bin_full[64][LWORDS];  // per 8x8 block: primitives covering the whole block in range
+    uint2 cand[CCAP];                         // (primitive id | box face item, packed pixel box)
+    uint32_t leaf[LEAFCAP];
+    uint32_t grp[32];
+    float ray_x[TILE], ray_y[TILE];           // ray coordinates of the tile's pixel columns / rows
+    float plane[6][4];                        // tile frustum in ego-relative world space: n.x, n.y, n.z, offset
+    Cam cam;
+    int n_cand, n_large, n_leaf, n_grp;
+    unsigned long long cnt[8];
+};
+
+struct TileCtx {
+    int x0, y0, tw, th;          // tile origin and size in pixels
+    float w_near, w_far, near_z, far_z;
+};
+
+// Is the box [lo,hi] (world) possibly inside the tile frustum?  Conservative.
+__device__ __forceinline__ bool box_visible(const TileSmem& s, const Node& b) {
+    // ego-relative centre and half size
+    float cx = sub(mul(0.5f, add(b.lo[0], b.hi[0])), s.cam.px);
+    float cy = sub(mul(0.5f, add(b.lo[1], b.hi[1])), s.cam.py);
+    float cz = mul(0.5f, add(b.lo[2], b.hi[2]));
+    float hx = mul(0.5f, sub(b.hi[0], b.lo[0])), hy = mul(0.5f, sub(b.hi[1], b.lo[1])), hz = mul(0.5f, sub(b.hi[2], b.lo[2]));
+    bool vis = true;
+#pragma unroll
+    for (int p = 0; p < 6; ++p) {
+        float nx = s.plane[p][0], ny = s.plane[p][1], nz = s.plane[p][2], d = s.plane[p][3];
+        float dist = fm(nx, cx, fm(ny, cy, fm(nz, cz, d)));
+        float reach = fm(fabsf(nx), hx, fm(fabsf(ny), hy, mul(fabsf(nz), hz)));
+        // slack: float32 rounding of the terms above, far below any real distance
+        float slack = fm(1e-5f, add(add(fabsf(mul(nx, cx)), fabsf(mul(ny, cy))), add(fabsf(mul(nz, cz)), add(fabsf(d), reach))), 1e-4f);
+        vis = vis && (add(dist, reach) >= -slack);
+    }
+    return vis;
+}
+
+// Pixel box (inclusive, tile coordinates) of camera-space vertices, or the whole tile when a
+// vertex is too close to the camera plane to project.  Returns false if the primitive cannot
+// touch any pixel centre of the tile or lies entirely before near / beyond far.
+// (Triangles pass their third vertex twice.)
+__device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const V3 (&V)[4], uint32_t& packed) {
+    constexpr int n = 4;
+    float zmin = V[0].z, zmax = V[0].z;
+#pragma unroll
+    for (int i = 1; i < n; ++i) { zmin = fminf(zmin, V[i].z); zmax = fmaxf(zmax, V[i].z); }
+    if (!(zmax >= t.near_z * 0.9999f) || !(zmin <= t.far_z * 1.0001f)) return false;
+    int bx0 = 0, by0 = 0, bx1 = t.tw - 1, by1 = t.th - 1;
+    if (zmin >= t.near_z * ZPROJ_FRAC) {
+        float sx0 = 3e38f, sx1 = -3e38f, sy0 = 3e38f, sy1 = -3e38f;
+#pragma unroll
+        for (int i = 0; i < n; ++i) {
+            float iz = __frcp_rn(V[i].z);
+            float sx = fm(c.focx, mul(V[i].x, iz), c.cx), sy = fm(c.focy, mul(V[i].y, iz), c.cy);
+            sx0 = fminf(sx0, sx); sx1 = fmaxf(sx1, sx); sy0 = fminf(sy0, sy); sy1 = fmaxf(sy1, sy);
+        }
+        // pixel centres u + 0.5 in [sx0, sx1], widened by 1/256 pixel against rounding
+        const float m = 0.00390625f;
+        float fx0 = ceilf(sx0 - 0.5f - m) - (float)t.x0, fx1 = floorf(sx1 - 0.5f + m) - (float)t.x0;
+        float fy0 = ceilf(sy0 - 0.5f - m) - (float)t.y0, fy1 = floorf(sy1 - 0.5f + m) - (float)t.y0;
+        if (!(fx0 <= fx1) || !(fy0 <= fy1)) return false;
+        if (fx1 < 0.f || fy1 < 0.f || fx0 > (float)(t.tw - 1) || fy0 > (float)(t.th - 1)) return false;
+        bx0 = (int)fmaxf(fx0, 0.f); by0 = (int)fmaxf(fy0, 0.f);
+        bx1 = (int)fminf(fx1, (float)(t.tw - 1)); by1 = (int)fminf(fy1, (float)(t.th - 1));
+    } else {
+        // frustum side planes through the camera centre, valid for any sign of z
+        float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
+        bool ol = true, orr = true, ou = true, od = true;
+#pragma unroll
+        for (int i = 0; i < n; ++i) {
+            float X = mul(V[i].x, c.focx), Y = mul(V[i].y, c.focy), Z = V[i].z;
+            ol = ol && (X < mul(Z, l) - 1e-4f * (fabsf(X) + fabsf(mul(Z, l))));
+            orr = orr && (X > mul(Z, r) + 1e-4f * (fabsf(X) + fabsf(mul(Z, r))));
+            ou = ou && (Y < mul(Z, u) - 1e-4f * (fabsf(Y) + fabsf(mul(Z, u))));
+            od = od && (Y > mul(Z, d) + 1e-4f * (fabsf(Y) + fabsf(mul(Z, d))));
+        }
+        if (ol || orr || ou || od) return false;
+    }
+    packed = (uint32_t)bx0 | ((uint32_t)by0 << 8) | ((uint32_t)bx1 << 16) | ((uint32_t)by1 << 24);
+    return true;
+}
+
+__device__ __forceinline__ void load_prim(const Prim* __restrict__ p, float (&v)[12], uint32_t& key_lo, uint32_t& flags) {
+    const float4* q = reinterpret_cast<const float4*>(p);
+    float4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2);
+    uint4 d = __ldg(reinterpret_cast<const uint4*>(q + 3));
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    v[8] = c.x; v[9] = c.y; v[10] = c.z; v[11] = c.w;
+    key_lo = d.x; flags = d.y;
+}
+
+// Box corner i (bit0 +x, bit1 +y, bit2 top) of agent g in camera space.
+__device__ __forceinline__ V3 box_corner(const Cam& c, const AgentGeom& g, int i) {
+    float sx = (i & 1) ? g.hl : -g.hl, sy = (i & 2) ? g.hw : -g.hw;
+    float qx = add(sub(g.x, c.px), fm(g.c, sx, -mul(g.s, sy)));
+    float qy = add(sub(g.y, c.py), fm(g.s, sx, mul(g.c, sy)));
+    float qz = (i & 4) ? g.h : 0.f;
+    return rotate_to_camera(c, sub(qx, c.mwx), sub(qy, c.mwy), sub(qz, c.mwz));
+}
+
+// Faces of a box as corner quadruples (perimeter order) -- rear, front, right, left, bottom, top.
+__constant__ uint8_t kFace[6][4] = {{0, 2, 6, 4}, {1, 5, 7, 3}, {0, 4, 5, 1}, {2, 3, 7, 6}, {0, 1, 3, 2}, {4, 6, 7, 5}};
+
+__device__ __forceinline__ uint32_t face_flags(int f) {
+    uint32_t fl = 1u;   // quad
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        if (!(kFace[f][k] < kFace[f][(k + 1) & 3])) fl |= 1u << (4 + k);   // canonical: lower corner index first
+    return fl;
+}
+
+// Rasterize a small primitive from its thread: loop over its pixel box, atomic max per fragment.
+__device__ __forceinline__ int raster_small(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, uint32_t box) {
+    int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    int frags = 0;
+    for (int y = by0; y <= by1; ++y) {
+        float ry = s.ray_y[y];
+        for (int x = bx0; x <= bx1; ++x) {
+            uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
+            if (wb) {
+                unsigned long long k = make_key(wb, key_lo);
+                unsigned long long* addr = &s.key[y * TILE + x];
+                if (k > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, k);
+                ++frags;
+            }
+        }
+    }
+    return frags;
+}
+
+__device__ __forceinline__ void store_record(float* r, const PrimEq& q, uint32_t key_lo, uint32_t box) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { r[i] = q.nx[i]; r[4 + i] = q.ny[i]; r[8 + i] = q.nz[i]; }
+    r[12] = q.wx; r[13] = q.wy; r[14] = q.wz;
+    r[15] = __uint_as_float(key_lo);
+    // the pixel box needs 6 bits per coordinate; the top-left bits ride along
+    uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    r[16] = __uint_as_float(bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24));
+}
+
+// Set up one candidate (already culled to the tile): small ones are rasterized at once, the others
+// are appended to the binned list.  `slot_base` + rank within the CTA pass is reserved by the caller.
+__device__ __forceinline__ void emit_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
+                                          uint32_t key_lo, uint32_t box, int& frags, int& n_small, int& n_set) {
+    PrimEq q;
+    if (!prim_equations(V, quad, flags, q)) return;
+    ++n_set;
+    int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    int area = (bx1 - bx0 + 1) * (by1 - by0 + 1);
+    if (area <= SMALL_MAX_PIXELS) {
+        frags += raster_small(s, t, q, key_lo, box);
+        ++n_small;
+    } else {
+        int slot = atomicAdd(&s.n_large, 1);     // the caller guarantees room
+        store_record(&s.rec[slot * REC], q, key_lo, box);
+    }
+}
+
+// (b) binning: test every binned primitive against the 8x8 blocks its pixel box touches.
+__device__ void bin_large(TileSmem& s, const TileCtx& t) {
+    const int n = s.n_large;
+    for (int i = threadIdx.x; i < 64 * LWORDS; i += NTHREADS) { (&s.bin_any[0][0])[i] = 0ull; (&s.bin_full[0][0])[i] = 0ull; }
+    __syncthreads();
+    // work item = (primitive, block row)
+    for (int item = threadIdx.x; item < n * 8; item += NTHREADS) {
+        const int p = item >> 3, brow = item & 7;
+        const float* r = &s.rec[p * REC];
+        const uint32_t bw = __float_as_uint(r[16]);
+        const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
+        if (brow < (by0 >> 3) || brow > (by1 >> 3)) continue;
+        // rows of this block row that exist in the tile
+        const int ya = brow * 8, yb = min(brow * 8 + 7, t.th - 1);
+        const float rya = s.ray_y[ya], ryb = s.ray_y[yb];
+        float tmin[4], tmax[4], nx[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float ny = r[4 + e], nz = r[8 + e];
+            float ta = fm(ny, rya, nz), tb = fm(ny, ryb, nz);
+            tmin[e] = fminf(ta, tb); tmax[e] = fmaxf(ta, tb);
+            nx[e] = r[e];
+        }
+        const float wx = r[12], wy = r[13], wz = r[14];
+        const float wa = fm(wy, rya, wz), wb = fm(wy, ryb, wz);
+        const float wtmin = fminf(wa, wb), wtmax = fmaxf(wa, wb);
+        for (int bcol = bx0 >> 3; bcol <= (bx1 >> 3); ++bcol) {
+            const int xa = bcol * 8, xb = min(bcol * 8 + 7, t.tw - 1);
+            const float rxa = s.ray_x[xa], rxb = s.ray_x[xb];    // rxa < rxb
+            bool reject = false, full = true;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                // fma is monotone in each argument, so the block's extreme values are at its corners
+                float emax = fm(nx[e], nx[e] >= 0.f ? rxb : rxa, tmax[e]);
+                float emin = fm(nx[e], nx[e] >= 0.f ? rxa : rxb, tmin[e]);
+                reject = reject || (emax < 0.f);
+                full = full && (emin > 0.f);
+            }
+            float wmax = fm(wx, wx >= 0.f ? rxb : rxa, wtmax), wmin = fm(wx, wx >= 0.f ? rxa : rxb, wtmin);
+            reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
+            full = full && (wmin >= t.w_far) && (wmax <= t.w_near);
+            if (reject) continue;
+            const int blk = brow * 8 + bcol;
+            atomicOr(&s.bin_any[blk][p >> 6], 1ull << (p & 63));
+            if (full) atomicOr(&s.bin_full[blk][p >> 6], 1ull << (p & 63));
+        }
+    }
+    __syncthreads();
+}
+
+// (c) raster of the binned primitives: a warp owns an 8x8 block, a lane two horizontally adjacent
+// pixels whose keys stay in registers while the block's primitives are walked.
+__device__ int raster_large(TileSmem& s, const TileCtx& t) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int frags = 0;
+    for (int blk = warp; blk < 64; blk += NTHREADS / 32) {
+        bool some = false;
+#pragma unroll
+        for (int w = 0; w < LWORDS; ++w) some = some || (s.bin_any[blk][w] != 0ull);
+        if (!some) continue;
+        const int x = (blk & 7) * 8 + (lane & 3) * 2, y = (blk >> 3) * 8 + (lane >> 2);
+        const float rx0 = s.ray_x[x], rx1 = s.ray_x[x + 1], ry = s.ray_y[y];
+        ulonglong2 kk = *reinterpret_cast<ulonglong2*>(&s.key[y * TILE + x]);
+#pragma unroll 1
+        for (int w = 0; w < LWORDS; ++w) {
+        unsigned long long any = s.bin_any[blk][w];
+        const unsigned long long fullm = s.bin_full[blk][w];
+        while (any) {
+            const int pb = __ffsll((long long)any) - 1;
+            any &= any - 1;
+            const int p = w * 64 + pb;
+            const float* r = &s.rec[p * REC];
+            const uint32_t key_lo = __float_as_uint(r[15]);
+            const float wt = fm(r[13], ry, r[14]);
+            const float w0 = fm(r[12], rx0, wt), w1 = fm(r[12], rx1, wt);
+            bool in0 = true, in1 = true;
+            if (!((fullm >> pb) & 1ull)) {
+                const uint32_t tl = __float_as_uint(r[16]) >> 24;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float te = fm(r[4 + e], ry, r[8 + e]);
+                    const float e0 = fm(r[e], rx0, te), e1 = fm(r[e], rx1, te);
+                    const bool own = (tl >> e) & 1u;
+                    in0 = in0 && (e0 > 0.f || (e0 == 0.f && own));
+                    in1 = in1 && (e1 > 0.f || (e1 == 0.f && own));
+                }
+                in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
+                in1 = in1 && (w1 >= t.w_far) && (w1 <= t.w_near);
+            }
+            if (in0) { unsigned long long k = make_key(__float_as_uint(w0), key_lo); if (k > kk.x) kk.x = k; ++frags; }
+            if (in1) { unsigned long long k = make_key(__float_as_uint(w1), key_lo); if (k > kk.y) kk.y = k; ++frags; }
+        }
+        }
+        *reinterpret_cast<ulonglong2*>(&s.key[y * TILE + x]) = kk;
+    }
+    return frags;
+}
+
+// Flush the binned list: bin, raster, reset.  Must be called by all threads of the CTA.
+__device__ __forceinline__ int flush_large(TileSmem& s, const TileCtx& t) {
+    __syncthreads();
+    int frags = 0;
+    if (s.n_large > 0) {
+        bin_large(s, t);
+        frags = raster_large(s, t);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) s.n_large = 0;
+    __syncthreads();
+    return frags;
+}
+
+// (d) keys -> class / depth images.
+__device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderParams& P, size_t view, bool ego_active) {
+    const Cam& c = s.cam;
+    const size_t img = (size_t)P.H * P.W;
+    uint8_t* oc = P.out_class + view * img;
+    uint16_t* od = P.out_depth + view * img;
+    float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
+    const float cphi = -c.dz, sphi = c.fz_;
+    const bool vec = (t.tw % 16 == 0) && (P.W % 16 == 0) && o32 == nullptr;
+    const int segs_per_row = (t.tw + 15) / 16;
+    for (int seg = threadIdx.x; seg < t.th * segs_per_row; seg += NTHREADS) {
+        const int y = seg / segs_per_row, xs = (seg % segs_per_row) * 16;
+        // background of this row: analytic ground plane below the horizon, sky above
+        const float wr = fm(-s.ray_y[y], cphi, sphi);
+        uint32_t bg_cls = P.cls_sky;
+        float bg_z = P.far_z;
+        if (wr < 0.f && c.mwz > 0.f) { bg_cls = P.cls_ground; bg_z = fminf(P.far_z, __fdiv_rn(c.mwz, -wr)); }
+        if (!ego_active) { bg_cls = P.cls_sky; bg_z = P.far_z; }
+        const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + xs;
+        if (vec) {
+            uint32_t cw[4];
+            uint32_t dw[8];
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+                ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(&s.key[y * TILE + xs + j]);
+                float z0 = kk.x ? __frcp_rn(__uint_as_float((uint32_t)(kk.x >> 32))) : bg_z;
+                float z1 = kk.y ? __frcp_rn(__uint_as_float((uint32_t)(kk.y >> 32))) : bg_z;
+                uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bg_cls, c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bg_cls;
+                __half2 h = __floats2half2_rn(z0, z1);
+                dw[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                if ((j & 3) == 0) cw[j >> 2] = c0 | (c1 << 8); else cw[j >> 2] |= (c0 << 16) | (c1 << 24);
+            }
+            *reinterpret_cast<uint4*>(oc + o) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            *reinterpret_cast<uint4*>(od + o) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
+            *reinterpret_cast<uint4*>(od + o + 8) = make_uint4(dw[4], dw[5], dw[6], dw[7]);
+        } else {
+            for (int j = 0; j < 16 && xs + j < t.tw; ++j) {
+                unsigned long long k = s.key[y * TILE + xs + j];
+                float z = k ? __frcp_rn(__uint_as_float((uint32_t)(k >> 32))) : bg_z;
+                oc[o + j] = (uint8_t)(k ? (uint32_t)(k & 0xff) : bg_cls);
+                od[o + j] = __half_as_ushort(__float2half_rn(z));
+                if (o32) o32[o + j] = z;
+            }
+        }
+    }
+}
+
+// Common prologue: tile geometry, camera, ray tables, frustum planes, cleared keys.
+// Returns false when the ego is inactive (the tile is then all sky).
+__device__ bool tile_prologue(TileSmem& s, TileCtx& t, const RenderParams& P, size_t& view, int& e, int& a) {
+    const int tiles = P.tiles_x * P.tiles_y;
+    const long long job = blockIdx.x;
+    view = (size_t)(P.view_first + job / tiles);
+    const int tile = (int)(job % tiles);
+    const int k = (int)(view % P.K);
+    a = (int)((view / P.K) % P.A);
+    e = (int)(view / ((size_t)P.K * P.A));
+    t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
+    t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
+    t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
+    const AgentGeom ego = P.agents[(size_t)e * P.A + a];
+    if (threadIdx.x == 0) {
+        make_camera(s.cam, ego, P.cam[k], P.W, P.H);
+        s.n_cand = 0; s.n_large = 0; s.n_leaf = 0; s.n_grp = 0;
+    }
+    if (threadIdx.x < 8) s.cnt[threadIdx.x] = 0ull;
+    for (int i = threadIdx.x; i < TILE * TILE / 2; i += NTHREADS)
+        reinterpret_cast<ulonglong2*>(s.key)[i] = make_ulonglong2(0ull, 0ull);
+    __syncthreads();
+    const Cam& c = s.cam;
+    if (threadIdx.x < TILE) {
+        const int i = threadIdx.x;
+        s.ray_x[i] = __fdiv_rn(sub(add((float)(t.x0 + i), 0.5f), c.cx), c.focx);
+        s.ray_y[i] = __fdiv_rn(sub(add((float)(t.y0 + i), 0.5f), c.cy), c.focy);
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 70) {
+        // frustum planes n.(q - m_w) >= 0 with q = X - P_ego; stored as n and offset -n.m_w (+ near/far)
+        const int p = threadIdx.x - 64;
+        float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
+        float nx, ny, nz, off = 0.f;
+        const float Rx = c.rx, Ry = c.ry, Dx = c.dx, Dy = c.dy, Dz = c.dz, Fx = c.fx_, Fy = c.fy_, Fz = c.fz_;
+        switch (p) {
+            case 0: nx = Fx; ny = Fy; nz = Fz; off = -P.near_z * 0.999f; break;                                       // z >= near
+            case 1: nx = -Fx; ny = -Fy; nz = -Fz; off = P.far_z * 1.001f; break;                                      // z <= far
+            case 2: nx = c.focx * Rx - l * Fx; ny = c.focx * Ry - l * Fy; nz = -l * Fz; break;                        // x f >= z l
+            case 3: nx = r * Fx - c.focx * Rx; ny = r * Fy - c.focx * Ry; nz = r * Fz; break;                         // x f <= z r
+            case 4: nx = c.focy * Dx - u * Fx; ny = c.focy * Dy - u * Fy; nz = c.focy * Dz - u * Fz; break;           // y f >= z u
+            default: nx = d * Fx - c.focy * Dx; ny = d * Fy - c.focy * Dy; nz = d * Fz - c.focy * Dz; break;          // y f <= z d
+        }
+        s.plane[p][0] = nx; s.plane[p][1] = ny; s.plane[p][2] = nz;
+        s.plane[p][3] = off - (nx * c.mwx + ny * c.mwy + nz * c.mwz);
+    }
+    __syncthreads();
+    return ego.active != 0;
+}
+
+__device__ __forceinline__ void add_counters(TileSmem& s, const RenderParams& P) {
+    __syncthreads();
+    if (P.counters && threadIdx.x < 8 && s.cnt[threadIdx.x]) atomicAdd(&P.counters[threadIdx.x], s.cnt[threadIdx.x]);
+}
+
+// Drain the candidate list: dense set-up, one candidate per thread per pass.
+// Candidate .x: bit 31 set -> box face item (agent << 3 | face), else primitive id.
+__device__ void drain_candidates(TileSmem& s, const TileCtx& t, const RenderParams& P, int e, uint32_t n_map_tris) {
+    __syncthreads();
+    const int n = s.n_cand;
+    int frags = 0, n_small = 0, n_set = 0;
+    for (int base = 0; base < n; base += NTHREADS) {
+        __syncthreads();                                                  // n_large is stable and uniform here
+        if (s.n_large + min(NTHREADS, n - base) > LCAP) frags += flush_large(s, t);   // room for this pass
+        const int i = base + threadIdx.x;
+        if (i < n) {
+            const uint2 cd = s.cand[i];
+            V3 V[4];
+            bool quad;
+            uint32_t flags, key_lo;
+            if (cd.x & 0x80000000u) {
+                const int b = (cd.x & 0x7fffffffu) >> 3, f = cd.x & 7;
+                const AgentGeom g = P.agents[(size_t)e * P.A + b];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, kFace[f][k]);
+                quad = true;
+                flags = face_flags(f);
+                key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+            } else {
+                float v[12];
+                load_prim(P.prims + cd.x, v, key_lo, flags);
+                quad = flags & 1u;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) V[k] = to_camera(s.cam, v[3 * k], v[3 * k + 1], v[3 * k + 2]);
+            }
+            emit_prim(s, t, V, quad, flags, key_lo, cd.y, frags, n_small, n_set);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) s.n_cand = 0;
+    if (P.counters) {
+        atomicAdd(&s.cnt[4], (unsigned long long)n_set);
+        atomicAdd(&s.cnt[5], (unsigned long long)n_small);
+        atomicAdd(&s.cnt[7], (unsigned long long)frags);
+    }
+    __syncthreads();
+}
+
+// Warp-aggregated append of one candidate per participating lane.
+__device__ __forceinline__ void push_candidate(TileSmem& s, bool keep, uint32_t id, uint32_t box) {
+    const unsigned m = __ballot_sync(0xffffffffu, keep);
+    if (!m) return;
+    const int lane = threadIdx.x & 31;
+    int base = 0;
+    if (lane == 0) base = atomicAdd(&s.n_cand, __popc(m));
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if (keep) s.cand[base + __popc(m & ((1u << lane) - 1u))] = make_uint2(id, box);
+}
+
+// ------------------------------------------------------------------------------------------------
+// production kernel
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NTHREADS) render_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& s = *reinterpret_cast<TileSmem*>(smem_raw);
+    TileCtx t;
+    size_t view; int e, a;
+    const bool ego_active = tile_prologue(s, t, P, view, e, a);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int NW = NTHREADS / 32;
+    if (ego_active) {
+        const MapInfo mi = P.maps[P.env_map[e]];
+        unsigned long long c_grp = 0, c_leaf = 0, c_prim = 0;
+        // ---- (a) map: groups -> leaves -> primitives
+        for (uint32_t g0 = mi.group_begin; g0 < mi.group_end; g0 += 32) {
+            if (warp == 0) {
+                const uint32_t g = g0 + lane;
+                bool vis = false;
+                if (g < mi.group_end) { vis = box_visible(s, P.groups[g]); ++c_grp; }
+                const unsigned m = __ballot_sync(0xffffffffu, vis);
+                if (vis) s.grp[__popc(m & ((1u << lane) - 1u))] = g;
+                if (lane == 0) { s.n_grp = __popc(m); s.n_leaf = 0; }
+            }
+            __syncthreads();
+            const int ng = s.n_grp;
+            for (int i = warp; i < ng; i += NW) {
+                const Node g = P.groups[s.grp[i]];
+                bool vis = false;
+                if (lane < (int)g.count) { vis = box_visible(s, P.leaves[g.first + lane]); ++c_leaf; }
+                const unsigned m = __ballot_sync(0xffffffffu, vis);
+                int base = 0;
+                if (lane == 0 && m) base = atomicAdd(&s.n_leaf, __popc(m));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                if (vis) s.leaf[base + __popc(m & ((1u << lane) - 1u))] = g.first + lane;
+            }
+            __syncthreads();
+            const int nl = s.n_leaf;
+            // rounds of NW leaves: each adds at most NW*32 candidates
+            for (int l0 = 0; l0 < nl; l0 += NW) {
+                if (s.n_cand + NW * 32 > CCAP) drain_candidates(s, t, P, e, mi.n_tris);   // uniform
+                const int li = l0 + warp;
+                if (li < nl) {
+                    const Node lf = P.leaves[s.leaf[li]];
+                    bool keep = false;
+                    uint32_t box = 0;
+                    if (lane < (int)lf.count) {
+                        float v[12]; uint32_t key_lo, flags;
+                        load_prim(P.prims + lf.first + lane, v, key_lo, flags);
+                        V3 V[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) V[k] = to_camera(s.cam, v[3 * k], v[3 * k + 1], v[3 * k + 2]);
+                        keep = pixel_box(s.cam, t, V, box);
+                        ++c_prim;
+                    }
+                    push_candidate(s, keep, lf.first + lane, box);
+                }
+                __syncthreads();
+            }
+        }
+        // ---- (a) other agents' boxes: cull per box, one item per possibly visible face
+        for (int b0 = 0; b0 < P.A; b0 += NTHREADS / 8) {
+            // 16 boxes per round -> at most 96 face items
+            if (s.n_cand + (NTHREADS / 8) * 6 > CCAP) drain_candidates(s, t, P, e, mi.n_tris);
+            const int b = b0 + (threadIdx.x >> 3), f = threadIdx.x & 7;
+            bool keep = false;
+            uint32_t box = 0;
+            if (b < P.A && b != a && f < 6) {
+                const AgentGeom g = P.agents[(size_t)e * P.A + b];
+                if (g.active) {
+                    V3 V[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, kFace[f][k]);
+                    keep = pixel_box(s.cam, t, V, box);
+                    ++c_prim;
+                }
+            }
+            push_candidate(s, keep, 0x80000000u | ((uint32_t)b << 3) | (uint32_t)f, box);
+            __syncthreads();
+        }
+        drain_candidates(s, t, P, e, mi.n_tris);
+        int frags = flush_large(s, t);
+        if (P.counters) {
+            atomicAdd(&s.cnt[1], c_grp); atomicAdd(&s.cnt[2], c_leaf); atomicAdd(&s.cnt[3], c_prim);
+            atomicAdd(&s.cnt[7], (unsigned long long)frags);
+            if (threadIdx.x == 0) s.cnt[0] = 1;
+        }
+    }
+    __syncthreads();
+    store_tile(s, t, P, view, ego_active);
+    add_counters(s, P);
+}
+
+// ------------------------------------------------------------------------------------------------
+// exhaustive kernel: every primitive of the map and every face of every other box against every
+// pixel of the tile; no hierarchy, no frustum or pixel-box culling, no binning.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NTHREADS) render_brute_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& s = *reinterpret_cast<TileSmem*>(smem_raw);
+    TileCtx t;
+    size_t view; int e, a;
+    const bool ego_active = tile_prologue(s, t, P, view, e, a);
+    if (ego_active) {
+        const MapInfo mi = P.maps[P.env_map[e]];
+        const uint32_t full = 0u | (0u << 8) | ((uint32_t)(t.tw - 1) << 16) | ((uint32_t)(t.th - 1) << 24);
+        const uint32_t n_items = (mi.prim_end - mi.prim_begin) + 6u * (uint32_t)P.A;
+        for (uint32_t i = threadIdx.x; i < n_items; i += NTHREADS) {
+            V3 V[4]; bool quad; uint32_t flags, key_lo;
+            if (i < mi.prim_end - mi.prim_begin) {
+                float v[12];
+                load_prim(P.prims + mi.prim_begin + i, v, key_lo, flags);
+                quad = flags & 1u;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) V[k] = to_camera(s.cam, v[3 * k], v[3 * k + 1], v[3 * k + 2]);
+            } else {
+                const uint32_t j = i - (mi.prim_end - mi.prim_begin);
+                const int b = (int)(j / 6u), f = (int)(j % 6u);
+                if (b == a) continue;
+                const AgentGeom g = P.agents[(size_t)e * P.A + b];
+                if (!g.active) continue;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, kFace[f][k]);
+                quad = true; flags = face_flags(f);
+                key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+            }
+            PrimEq q;
+            if (!prim_equations(V, quad, flags, q)) continue;
+            raster_small(s, t, q, key_lo, full);
+        }
+    }
+    __syncthreads();
+    store_tile(s, t, P, view, ego_active);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host-side launchers (called from the C ABI)
+// ------------------------------------------------------------------------------------------------
+size_t render_smem_bytes() { return sizeof(TileSmem); }
+
+cudaError_t configure_kernels() {
+    cudaError_t err = cudaFuncSetAttribute(render_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(render_brute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+}
+
+cudaError_t launch_agents(int n, const float* poses, float* state, const float* actions, const float* dims,
+                          const uint8_t* active, AgentGeom* out, uint32_t* status, float dt, float wheelbase,
+                          float v_max, cudaStream_t stream) {
+    if (n <= 0) return cudaSuccess;
+    agent_kernel<<<(n + 127) / 128, 128, 0, stream>>>(n, poses, 3, state, actions, dims, active, out, status, dt,
+                                                      wheelbase, v_max);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, cudaStream_t stream) {
+    if (n_views <= 0) return cudaSuccess;
+    const long long blocks = n_views * P.tiles_x * P.tiles_y;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (brute)
+        render_brute_kernel<<<(unsigned)blocks, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    else
+        render_kernel<<<(unsigned)blocks, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    return cudaGetLastError();
+}
+
+}  // namespace pic

@@ -1,0 +1,85 @@
+// Device/host data layout of the rasterizer library (internal).
+#pragma once
+#include <stdint.h>
+
+namespace pic {
+
+constexpr int TILE = 64;        // a view is rendered in tiles of up to TILE x TILE pixels (one CTA each)
+constexpr int NTHREADS = 128;   // threads per render CTA
+constexpr int MAX_CAMS = 16;    // cameras per rig
+constexpr int LEAF_PRIMS = 32;  // primitives per leaf (one per lane)
+constexpr int LONG_LEAF_PRIMS = 4;   // long primitives get small leaves so their boxes stay tight
+constexpr int GROUP_LEAVES = 32;     // leaves per group (one per lane)
+
+// Map primitive in hierarchy order: a triangle, or a planar convex quad fused from two consecutive
+// triangles of the input that share an edge (same class).  64 bytes, read as four 128-bit loads.
+struct Prim {
+    float v[12];        // 4 vertices xyz in perimeter order (triangle: the 4th repeats the 3rd)
+    uint32_t key_lo;    // (0xFFFFFF - primitive index) << 8 | class : low half of the z-buffer key
+    uint32_t flags;     // bit 0: quad; bits 4..7: edge i runs against its canonical direction
+    uint32_t pad[2];
+};
+static_assert(sizeof(Prim) == 64, "Prim must be 64 bytes");
+
+// Axis-aligned box of a leaf (over primitives) or a group (over leaves); 32 bytes.
+struct Node {
+    float lo[3];
+    uint32_t first;
+    float hi[3];
+    uint32_t count;
+};
+static_assert(sizeof(Node) == 32, "Node must be 32 bytes");
+
+struct MapInfo {
+    uint32_t group_begin, group_end;   // range in the groups array
+    uint32_t n_tris;                   // triangles of the map as given (box indices start here)
+    uint32_t prim_begin;               // first primitive (used by the exhaustive kernel)
+    uint32_t prim_end;
+    uint32_t pad[3];
+};
+
+// Per-agent geometry written once per render by the agent kernel; 32 bytes.
+struct AgentGeom {
+    float x, y;       // box centre on the ground plane
+    float c, s;       // cos, sin of the heading
+    float hl, hw, h;  // half length, half width, height
+    uint32_t active;
+};
+
+struct CamConst {
+    float mx, my, mz;
+    float cpsi, spsi, cphi, sphi;   // cos/sin of the camera yaw and pitch (rounded from double)
+    float fx, fy;
+};
+
+struct RenderParams {
+    int32_t E, A, K, H, W;
+    int32_t tiles_x, tiles_y;
+    float near_z, far_z;
+    float w_near, w_far;            // 1/near, 1/far: kept range of the reciprocal depth
+    uint32_t cls_agent, cls_sky, cls_ground;
+    const int32_t* env_map;
+    const MapInfo* maps;
+    const Node* groups;
+    const Node* leaves;
+    const Prim* prims;
+    const AgentGeom* agents;
+    uint8_t* out_class;
+    uint16_t* out_depth;
+    float* out_depth32;             // optional
+    unsigned long long* counters;   // optional [8]
+    long long view_first;           // render views [view_first, view_first + gridDim / tiles)
+    CamConst cam[MAX_CAMS];
+};
+
+// Host-side result of the hierarchy build for all maps of a scene.
+struct HostHierarchy;
+HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const float* tri_xyz,
+                               const uint8_t* tri_class, int agents_per_env, char* err, int err_len);
+void free_hierarchy(HostHierarchy*);
+const Prim* hierarchy_prims(const HostHierarchy*, size_t* n);
+const Node* hierarchy_leaves(const HostHierarchy*, size_t* n);
+const Node* hierarchy_groups(const HostHierarchy*, size_t* n);
+const MapInfo* hierarchy_maps(const HostHierarchy*, size_t* n);
+
+}  // namespace pic
