@@ -148,13 +148,24 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *                         (views, group tests, leaf tests, primitives tested, set up, small, large, fragments).
  *   PIC_OPT_VIEW_FIRST,   render only views [first, first + count) (flat index (e*A + a)*K + k);
  *   PIC_OPT_VIEW_COUNT    count 0 = through the last view.  Other views' pixels are left untouched.
+ *   PIC_OPT_TIMING        1: bracket every render-kernel launch with CUDA events on its stream
+ *                         (up to 1024 launches between two pic_get_kernel_times calls); 0: off.
+ *                         Turning it on creates the events (allocates), so do it outside timed code.
  */
 #define PIC_OPT_BRUTE_FORCE 1
 #define PIC_OPT_DEPTH32 2
 #define PIC_OPT_COUNTERS 3
 #define PIC_OPT_VIEW_FIRST 4
 #define PIC_OPT_VIEW_COUNT 5
+#define PIC_OPT_TIMING 6
 pic_status pic_scene_set_option(pic_scene* scene, int32_t option, uint64_t value);
+
+/*
+ * Device time of each render-kernel launch recorded since the last call (PIC_OPT_TIMING on), in
+ * milliseconds, oldest first: waits for the last recorded launch, writes min(*n, capacity) values
+ * to ms (host) and the number recorded to *n, then forgets them.
+ */
+pic_status pic_get_kernel_times(pic_scene* scene, float* ms, int32_t capacity, int32_t* n);
 
 /* Thread-local, never NULL; valid until the next failing call on this thread. */
 const char* pic_last_error(void);

@@ -17,11 +17,12 @@ from . import build as _build
 PIC_OK = 0
 STATUS_NAMES = {0: "PIC_OK", 1: "PIC_ERR_INVALID_ARG", 2: "PIC_ERR_SHAPE", 3: "PIC_ERR_OOM", 4: "PIC_ERR_CUDA",
                 5: "PIC_ERR_CAPACITY", 6: "PIC_ERR_NONFINITE"}
-OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT = 1, 2, 3, 4, 5
+OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_TIMING = 1, 2, 3, 4, 5, 6
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_last_error", "pic_version"]
+           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times",
+           "pic_last_error", "pic_version"]
 
 
 class PicError(RuntimeError):
@@ -66,6 +67,7 @@ def load(path: Optional[str] = None):
     lib.pic_step.argtypes = [vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     lib.pic_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
+    lib.pic_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32, C.POINTER(C.c_int32)]
     for name in EXPORTS:
         getattr(lib, name).restype = C.c_int
     lib.pic_last_error.restype = C.c_char_p
@@ -214,6 +216,13 @@ class Scene:
         flags = C.c_uint32(0)
         _check(self._lib, self._lib.pic_get_status(self._h, C.byref(flags), _stream_ptr(stream)))
         return int(flags.value)
+
+    def kernel_times(self) -> np.ndarray:
+        """Milliseconds of each render-kernel launch since the last call (OPT_TIMING must be on)."""
+        buf = (C.c_float * 1024)()
+        n = C.c_int32(0)
+        _check(self._lib, self._lib.pic_get_kernel_times(self._h, buf, 1024, C.byref(n)))
+        return np.array(buf[:min(int(n.value), 1024)], dtype=np.float64)
 
     def set_option(self, option: int, value) -> None:
         import torch

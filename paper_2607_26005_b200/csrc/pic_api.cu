@@ -22,6 +22,7 @@ cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, 
 namespace {
 
 constexpr float kDt = 0.1f, kWheelbase = 2.8f, kVMax = 30.0f;
+constexpr int kMaxTimed = 1024;
 
 thread_local char g_err[512] = "";
 
@@ -72,6 +73,9 @@ struct pic_scene {
     float* depth32 = nullptr;
     unsigned long long* counters = nullptr;
     long long view_first = 0, view_count = 0;
+    bool timing = false;
+    cudaEvent_t* ev = nullptr;      // 2 * kMaxTimed events
+    int n_timed = 0;
     size_t n_prims = 0, n_leaves = 0, n_groups = 0;
 };
 
@@ -92,6 +96,10 @@ void free_scene(pic_scene* s) {
     cudaFree(s->d_agents); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
+    if (s->ev) {
+        for (int i = 0; i < 2 * kMaxTimed; ++i) if (s->ev[i]) cudaEventDestroy(s->ev[i]);
+        delete[] s->ev;
+    }
     delete s;
 }
 
@@ -248,6 +256,18 @@ pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
             if (value >= (uint64_t)s->E * s->A * s->K) return fail(PIC_ERR_INVALID_ARG, "first view out of range");
             s->view_first = (long long)value; return PIC_OK;
         case PIC_OPT_VIEW_COUNT: s->view_count = (long long)value; return PIC_OK;
+        case PIC_OPT_TIMING: {
+            if (value && !s->ev) {
+                DeviceGuard guard(s->device);
+                if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+                s->ev = new (std::nothrow) cudaEvent_t[2 * kMaxTimed]();
+                if (!s->ev) return fail(PIC_ERR_OOM, "host allocation failed");
+                for (int i = 0; i < 2 * kMaxTimed; ++i) CUDA_TRY(cudaEventCreate(&s->ev[i]));
+            }
+            s->timing = value != 0;
+            s->n_timed = 0;
+            return PIC_OK;
+        }
         default: return fail(PIC_ERR_INVALID_ARG, "unknown option %d", option);
     }
 }
@@ -267,7 +287,10 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
     long long count = total - s->view_first;
     if (s->view_count > 0 && s->view_count < count) count = s->view_count;
     P.view_first = s->view_first;
+    const bool timed = s->timing && s->n_timed < kMaxTimed;
+    if (timed) CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed], stream));
     CUDA_TRY(pic::launch_render(P, count, s->brute, stream));
+    if (timed) { CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed + 1], stream)); ++s->n_timed; }
     return PIC_OK;
 }
 
@@ -336,6 +359,20 @@ pic_status pic_step(pic_scene* s, const float* actions, const pic_camera* rig, u
     if (!actions) return fail(PIC_ERR_INVALID_ARG, "actions is NULL");
     return render_from(s, nullptr, s->d_state, actions, s->d_dims, s->d_active, rig, out_class, out_depth,
                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+pic_status pic_get_kernel_times(pic_scene* s, float* ms, int32_t capacity, int32_t* n) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!n || (capacity > 0 && !ms)) return fail(PIC_ERR_INVALID_ARG, "ms or n is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    *n = s->n_timed;
+    for (int i = 0; i < s->n_timed; ++i) {
+        CUDA_TRY(cudaEventSynchronize(s->ev[2 * i + 1]));
+        if (i < capacity) CUDA_TRY(cudaEventElapsedTime(&ms[i], s->ev[2 * i], s->ev[2 * i + 1]));
+    }
+    s->n_timed = 0;
+    return PIC_OK;
 }
 
 pic_status pic_get_status(pic_scene* s, uint32_t* flags, void* cuda_stream) {
