@@ -12,6 +12,7 @@
 
 namespace pic {
 size_t render_smem_bytes();
+int render_list_caps(int which);
 cudaError_t configure_kernels();
 cudaError_t launch_agents(int n, const float* poses, float* state, const float* actions, const float* dims,
                           const uint8_t* active, AgentGeom* out, uint32_t* status, float dt, float wheelbase,
@@ -73,6 +74,7 @@ struct pic_scene {
     float* depth32 = nullptr;
     unsigned long long* counters = nullptr;
     long long view_first = 0, view_count = 0;
+    int med_cap = 1 << 30, large_cap = 1 << 30;
     bool timing = false;
     cudaEvent_t* ev = nullptr;      // 2 * kMaxTimed events
     int n_timed = 0;
@@ -120,6 +122,7 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.agents = s->d_agents;
     P.out_class = out_class; P.out_depth = out_depth; P.out_depth32 = s->depth32; P.counters = s->counters;
     P.view_first = 0;
+    P.med_cap = s->med_cap; P.large_cap = s->large_cap;
     for (int k = 0; k < s->K; ++k) {
         const pic_camera& c = rig[k];
         const float vals[7] = {c.mount_x, c.mount_y, c.mount_z, c.yaw, c.pitch, c.fx, c.fy};
@@ -256,6 +259,8 @@ pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
             if (value >= (uint64_t)s->E * s->A * s->K) return fail(PIC_ERR_INVALID_ARG, "first view out of range");
             s->view_first = (long long)value; return PIC_OK;
         case PIC_OPT_VIEW_COUNT: s->view_count = (long long)value; return PIC_OK;
+        case PIC_OPT_LIST_CAPS:
+            s->med_cap = (int)(value & 0xffffu); s->large_cap = (int)((value >> 16) & 0xffffu); return PIC_OK;
         case PIC_OPT_TIMING: {
             if (value && !s->ev) {
                 DeviceGuard guard(s->device);

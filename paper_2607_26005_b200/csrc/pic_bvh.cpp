@@ -211,8 +211,8 @@ HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const fl
             h->groups.push_back(g);
         }
         mi.group_end = (uint32_t)h->groups.size();
-        if (h->prims.size() > 0xFFFFFFF0ull) {
-            std::snprintf(err, err_len, "more than 2^32 primitives in one scene");
+        if (h->prims.size() >= (1ull << 28)) {
+            std::snprintf(err, err_len, "more than 2^28 primitives in one scene");
             delete h;
             return nullptr;
         }

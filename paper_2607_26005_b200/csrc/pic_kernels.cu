@@ -6,13 +6,15 @@
 // so "nearest fragment wins, ties to the lower index" is a plain unsigned max, independent of
 // the order in which primitives are processed; 0 means "no fragment" (background).
 //
-// Steps per tile (letters as in the scope table of the design notes):
-//   (a) cull      group boxes -> leaf boxes -> primitives against the tile frustum; survivors are
-//                 compacted into a candidate list with warp ballots; agent boxes are culled the same way
-//   (c) set-up    per candidate: camera-space vertices, 3-4 edge functions, 1/z plane
-//       small     primitives whose pixel box holds few pixel centres are rasterized at once by
+// Steps per tile:
+//   (a) cull      group boxes -> leaf boxes (compacted with warp ballots) -> primitives against the
+//                 tile frustum and the pixel grid; other agents' boxes are culled as spheres and
+//                 only their camera-facing faces are kept
+//   (c) set-up    per survivor: camera-space vertices, 3-4 edge functions, 1/z plane
+//       tiny      primitives whose pixel box holds <= 4 pixel centres are rasterized at once by
 //                 their thread with a shared-memory atomic max
-//   (b) binning   the others are tested against the 8 x 8 pixel blocks of the tile (trivial
+//       medium    pixel boxes up to 64 centres: one warp per primitive, a lane per pixel, atomic max
+//   (b) binning   larger ones are tested against the 8 x 8 pixel blocks of the tile (trivial
 //                 reject / trivial accept with the same float32 edge functions) into bit masks
 //   (c) raster    each warp owns blocks; a lane owns two pixels, keeps their keys in registers
 //                 and walks the block's mask
@@ -28,12 +30,15 @@
 
 namespace pic {
 
-constexpr int LCAP = 128;         // binned primitives per pass (one mask bit each)
-constexpr int LWORDS = LCAP / 64;
-constexpr int CCAP = 512;         // candidate list entries
-constexpr int LEAFCAP = 1024;     // visible leaves per batch of 32 groups
+constexpr int NW = NTHREADS / 32;
+constexpr int LCAP = 64;          // binned (large) primitives per tile pass: one mask bit each
+constexpr int MCAP = 64;          // medium primitives (warp-cooperative raster) per tile pass
+constexpr int GROUP_BATCH = 16;   // groups examined per batch
+constexpr int LEAFCAP = GROUP_BATCH * GROUP_LEAVES;   // visible leaves per batch
+constexpr int FACECAP = 6 * NTHREADS;                 // box-face items per round of NTHREADS boxes
 constexpr int REC = 17;           // words per set-up record (odd: conflict-free per-lane reads)
-constexpr int SMALL_MAX_PIXELS = 16;   // pixel centres in the box of a "small" primitive
+constexpr int TINY_MAX_PIXELS = 4;     // pixel centres in the box of a primitive rasterized by its own thread
+constexpr int MEDIUM_MAX_PIXELS = 64;  // ... rasterized by one warp with atomics; larger ones are binned
 constexpr float ZPROJ_FRAC = 0.5f;     // vertices nearer than this * near are not projected
 
 struct __align__(16) Cam {
@@ -197,45 +202,71 @@ __global__ void agent_kernel(int n, const float* __restrict__ poses, int pose_st
     out[i] = g;
 }
 
+
 // ------------------------------------------------------------------------------------------------
 // shared-memory layout of a render CTA
 // ------------------------------------------------------------------------------------------------
 struct __align__(16) TileSmem {
-    unsigned long long key[TILE * TILE];      // 32 KB
-    float rec[LCAP * REC];                    // set-up records of binned primitives
-    unsigned long long bin_any[64][LWORDS];   // per 8x8 block: primitives to test
-    unsigned long long bin_full[64][LWORDS];  // per 8x8 block: primitives covering the whole block in range
-    uint2 cand[CCAP];                         // (primitive id | box face item, packed pixel box)
-    uint32_t leaf[LEAFCAP];
-    uint32_t grp[32];
+    unsigned long long key[TILE * TILE];      // 32 KB, 16-byte chunks XOR-swizzled by row (key_index)
+    float rec_l[LCAP * REC];                  // set-up records of binned primitives
+    float rec_m[MCAP * REC];                  // set-up records of medium primitives
+    unsigned long long bin_any[64];           // per 8x8 block: binned primitives to test
+    unsigned long long bin_full[64];          // per 8x8 block: primitives covering the whole block, depth in range
+    union {
+        uint32_t leaf[LEAFCAP];               // visible leaves of the batch: first primitive << 4 | count
+        uint32_t face[LEAFCAP];               // box-face items: agent << 3 | face
+    };
+    uint32_t grp[GROUP_BATCH];
     float ray_x[TILE], ray_y[TILE];           // ray coordinates of the tile's pixel columns / rows
-    float plane[6][4];                        // tile frustum in ego-relative world space: n.x, n.y, n.z, offset
+    float plane[6][4];                        // tile frustum, ego-relative world space, unit normals: n, offset
+    float side[4][4];                         // the four side planes in camera space, unit normals
     Cam cam;
-    int n_cand, n_large, n_leaf, n_grp;
-    unsigned long long cnt[8];
+    int n_large, n_med, n_leaf, n_grp, n_face;
+    uint32_t touched[2];                      // 8x8 blocks that may hold a fragment (rows 0-3, rows 4-7)
+    unsigned long long cnt[16];
 };
 
 struct TileCtx {
     int x0, y0, tw, th;          // tile origin and size in pixels
     float w_near, w_far, near_z, far_z;
+    int med_cap, large_cap;
 };
+
+// Keys are stored so that both an 8x8 block (raster) and 16-pixel row segments (store) spread over
+// all banks: the 16-byte chunk holding pixels (2c, 2c+1) of row y sits at chunk c ^ (y & 7).
+__device__ __forceinline__ int key_index(int x, int y) {
+    return (y << 6) | ((((x >> 1) ^ (y & 7)) << 1) | (x & 1));
+}
+
+// Bit mask of the 8x8 blocks touched by a pixel box (inclusive).
+__device__ __forceinline__ unsigned long long block_mask(int bx0, int by0, int bx1, int by1) {
+    const int c0 = bx0 >> 3, c1 = bx1 >> 3, r0 = by0 >> 3, r1 = by1 >> 3;
+    const unsigned long long row = (unsigned long long)(((2u << c1) - (1u << c0)) & 0xffu);
+    const unsigned long long rows = (0x0101010101010101ull >> (8 * (7 - (r1 - r0)))) << (8 * r0);
+    return row * rows;
+}
+
+__device__ __forceinline__ void mark_touched(TileSmem& s, unsigned long long m) {
+    const uint32_t lo = (uint32_t)m, hi = (uint32_t)(m >> 32);
+    if (lo & ~s.touched[0]) atomicOr(&s.touched[0], lo);
+    if (hi & ~s.touched[1]) atomicOr(&s.touched[1], hi);
+}
 
 // Is the box [lo,hi] (world) possibly inside the tile frustum?  Conservative.
 __device__ __forceinline__ bool box_visible(const TileSmem& s, const Node& b) {
-    // ego-relative centre and half size
-    float cx = sub(mul(0.5f, add(b.lo[0], b.hi[0])), s.cam.px);
-    float cy = sub(mul(0.5f, add(b.lo[1], b.hi[1])), s.cam.py);
-    float cz = mul(0.5f, add(b.lo[2], b.hi[2]));
-    float hx = mul(0.5f, sub(b.hi[0], b.lo[0])), hy = mul(0.5f, sub(b.hi[1], b.lo[1])), hz = mul(0.5f, sub(b.hi[2], b.lo[2]));
+    const float ax = sub(b.lo[0], s.cam.px), bx = sub(b.hi[0], s.cam.px);
+    const float ay = sub(b.lo[1], s.cam.py), by = sub(b.hi[1], s.cam.py);
+    const float cx = 0.5f * (ax + bx), cy = 0.5f * (ay + by), cz = 0.5f * (b.lo[2] + b.hi[2]);
+    const float hx = 0.5f * (bx - ax), hy = 0.5f * (by - ay), hz = 0.5f * (b.hi[2] - b.lo[2]);
+    // rounding of the few float32 operations below, far under any real distance
+    const float slack = 1e-3f + 4e-6f * (fabsf(cx) + fabsf(cy) + fabsf(cz) + hx + hy + hz);
     bool vis = true;
 #pragma unroll
     for (int p = 0; p < 6; ++p) {
-        float nx = s.plane[p][0], ny = s.plane[p][1], nz = s.plane[p][2], d = s.plane[p][3];
-        float dist = fm(nx, cx, fm(ny, cy, fm(nz, cz, d)));
-        float reach = fm(fabsf(nx), hx, fm(fabsf(ny), hy, mul(fabsf(nz), hz)));
-        // slack: float32 rounding of the terms above, far below any real distance
-        float slack = fm(1e-5f, add(add(fabsf(mul(nx, cx)), fabsf(mul(ny, cy))), add(fabsf(mul(nz, cz)), add(fabsf(d), reach))), 1e-4f);
-        vis = vis && (add(dist, reach) >= -slack);
+        const float nx = s.plane[p][0], ny = s.plane[p][1], nz = s.plane[p][2], d = s.plane[p][3];
+        const float dist = nx * cx + ny * cy + nz * cz + d;
+        const float reach = fabsf(nx) * hx + fabsf(ny) * hy + fabsf(nz) * hz;
+        vis = vis && (dist + reach >= -slack);
     }
     return vis;
 }
@@ -255,7 +286,7 @@ __device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const 
         float sx0 = 3e38f, sx1 = -3e38f, sy0 = 3e38f, sy1 = -3e38f;
 #pragma unroll
         for (int i = 0; i < n; ++i) {
-            float iz = __frcp_rn(V[i].z);
+            float iz = __fdividef(1.0f, V[i].z);
             float sx = fm(c.focx, mul(V[i].x, iz), c.cx), sy = fm(c.focy, mul(V[i].y, iz), c.cy);
             sx0 = fminf(sx0, sx); sx1 = fmaxf(sx1, sx); sy0 = fminf(sy0, sy); sy1 = fmaxf(sy1, sy);
         }
@@ -303,33 +334,43 @@ __device__ __forceinline__ V3 box_corner(const Cam& c, const AgentGeom& g, int i
     return rotate_to_camera(c, sub(qx, c.mwx), sub(qy, c.mwy), sub(qz, c.mwz));
 }
 
-// Faces of a box as corner quadruples (perimeter order) -- rear, front, right, left, bottom, top.
-__constant__ uint8_t kFace[6][4] = {{0, 2, 6, 4}, {1, 5, 7, 3}, {0, 4, 5, 1}, {2, 3, 7, 6}, {0, 1, 3, 2}, {4, 6, 7, 5}};
+// Faces of a box as corner quadruples in perimeter order, one nibble per corner:
+// rear (-x), front (+x), right (-y), left (+y), bottom, top.
+__device__ __forceinline__ uint32_t face_corners(int f) {
+    const uint32_t tab[6] = {0x4620u, 0x3751u, 0x1540u, 0x6732u, 0x2310u, 0x5764u};
+    uint32_t r = tab[0];
+#pragma unroll
+    for (int i = 1; i < 6; ++i) r = (f == i) ? tab[i] : r;
+    return r;
+}
 
-__device__ __forceinline__ uint32_t face_flags(int f) {
+__device__ __forceinline__ uint32_t face_flags(uint32_t corners) {
     uint32_t fl = 1u;   // quad
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-        if (!(kFace[f][k] < kFace[f][(k + 1) & 3])) fl |= 1u << (4 + k);   // canonical: lower corner index first
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t a = (corners >> (4 * k)) & 7u, b = (corners >> (4 * ((k + 1) & 3))) & 7u;
+        if (!(a < b)) fl |= 1u << (4 + k);     // canonical direction: lower corner index first
+    }
     return fl;
 }
 
-// Rasterize a small primitive from its thread: loop over its pixel box, atomic max per fragment.
-__device__ __forceinline__ int raster_small(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, uint32_t box) {
-    int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+// Rasterize a primitive from one thread: loop over its pixel box, atomic max per fragment.
+__device__ __forceinline__ int raster_in_thread(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, uint32_t box) {
+    const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
     int frags = 0;
     for (int y = by0; y <= by1; ++y) {
-        float ry = s.ray_y[y];
+        const float ry = s.ray_y[y];
         for (int x = bx0; x <= bx1; ++x) {
-            uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
+            const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
             if (wb) {
-                unsigned long long k = make_key(wb, key_lo);
-                unsigned long long* addr = &s.key[y * TILE + x];
+                const unsigned long long k = make_key(wb, key_lo);
+                unsigned long long* addr = &s.key[key_index(x, y)];
                 if (k > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, k);
                 ++frags;
             }
         }
     }
+    if (frags) mark_touched(s, block_mask(bx0, by0, bx1, by1));
     return frags;
 }
 
@@ -339,37 +380,84 @@ __device__ __forceinline__ void store_record(float* r, const PrimEq& q, uint32_t
     r[12] = q.wx; r[13] = q.wy; r[14] = q.wz;
     r[15] = __uint_as_float(key_lo);
     // the pixel box needs 6 bits per coordinate; the top-left bits ride along
-    uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
     r[16] = __uint_as_float(bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24));
 }
 
-// Set up one candidate (already culled to the tile): small ones are rasterized at once, the others
-// are appended to the binned list.  `slot_base` + rank within the CTA pass is reserved by the caller.
-__device__ __forceinline__ void emit_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
-                                          uint32_t key_lo, uint32_t box, int& frags, int& n_small, int& n_set) {
+struct Tally { int tested, setup, tiny, medium, large, fallback, frags; };
+
+// Cull one primitive against the tile, set it up, and route it by the size of its pixel box.
+__device__ __forceinline__ void process_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
+                                             uint32_t key_lo, Tally& n) {
+    ++n.tested;
+    uint32_t box;
+    if (!pixel_box(s.cam, t, V, box)) return;
     PrimEq q;
     if (!prim_equations(V, quad, flags, q)) return;
-    ++n_set;
-    int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
-    int area = (bx1 - bx0 + 1) * (by1 - by0 + 1);
-    if (area <= SMALL_MAX_PIXELS) {
-        frags += raster_small(s, t, q, key_lo, box);
-        ++n_small;
-    } else {
-        int slot = atomicAdd(&s.n_large, 1);     // the caller guarantees room
-        store_record(&s.rec[slot * REC], q, key_lo, box);
+    ++n.setup;
+    const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    const int area = (bx1 - bx0 + 1) * (by1 - by0 + 1);
+    if (area <= TINY_MAX_PIXELS) {
+        n.frags += raster_in_thread(s, t, q, key_lo, box);
+        ++n.tiny;
+        return;
     }
+    if (area <= MEDIUM_MAX_PIXELS) {
+        const int slot = atomicAdd(&s.n_med, 1);
+        if (slot < t.med_cap) { store_record(&s.rec_m[slot * REC], q, key_lo, box); ++n.medium; return; }
+    } else {
+        const int slot = atomicAdd(&s.n_large, 1);
+        if (slot < t.large_cap) { store_record(&s.rec_l[slot * REC], q, key_lo, box); ++n.large; return; }
+    }
+    // list full: correct but slow
+    n.frags += raster_in_thread(s, t, q, key_lo, box);
+    ++n.fallback;
 }
 
-// (b) binning: test every binned primitive against the 8x8 blocks its pixel box touches.
+// Medium primitives: one warp per primitive, lanes tile its pixel box 8 x 4 at a time.
+__device__ int raster_medium(TileSmem& s, const TileCtx& t) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = min(s.n_med, t.med_cap);
+    int frags = 0;
+    for (int p = warp; p < n; p += NW) {
+        const float* r = &s.rec_m[p * REC];
+        PrimEq q;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { q.nx[i] = r[i]; q.ny[i] = r[4 + i]; q.nz[i] = r[8 + i]; }
+        q.wx = r[12]; q.wy = r[13]; q.wz = r[14];
+        const uint32_t key_lo = __float_as_uint(r[15]);
+        const uint32_t bw = __float_as_uint(r[16]);
+        q.tl = bw >> 24;
+        const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
+        bool any = false;
+        for (int yy = by0; yy <= by1; yy += 4) {
+            const int y = yy + (lane >> 3);
+            for (int xx = bx0; xx <= bx1; xx += 8) {
+                const int x = xx + (lane & 7);
+                if (x <= bx1 && y <= by1) {
+                    const uint32_t wb = fragment(q, s.ray_x[x], s.ray_y[y], t.w_near, t.w_far);
+                    if (wb) {
+                        const unsigned long long k = make_key(wb, key_lo);
+                        unsigned long long* addr = &s.key[key_index(x, y)];
+                        if (k > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, k);
+                        any = true;
+                        ++frags;
+                    }
+                }
+            }
+        }
+        if (__any_sync(0xffffffffu, any) && lane == 0) mark_touched(s, block_mask(bx0, by0, bx1, by1));
+    }
+    return frags;
+}
+
+// (b) binning: test every large primitive against the 8x8 blocks its pixel box touches.
+// Work item = (primitive, block row).  The caller synchronises before and after.
 __device__ void bin_large(TileSmem& s, const TileCtx& t) {
-    const int n = s.n_large;
-    for (int i = threadIdx.x; i < 64 * LWORDS; i += NTHREADS) { (&s.bin_any[0][0])[i] = 0ull; (&s.bin_full[0][0])[i] = 0ull; }
-    __syncthreads();
-    // work item = (primitive, block row)
+    const int n = min(s.n_large, t.large_cap);
     for (int item = threadIdx.x; item < n * 8; item += NTHREADS) {
         const int p = item >> 3, brow = item & 7;
-        const float* r = &s.rec[p * REC];
+        const float* r = &s.rec_l[p * REC];
         const uint32_t bw = __float_as_uint(r[16]);
         const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
         if (brow < (by0 >> 3) || brow > (by1 >> 3)) continue;
@@ -379,36 +467,40 @@ __device__ void bin_large(TileSmem& s, const TileCtx& t) {
         float tmin[4], tmax[4], nx[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            float ny = r[4 + e], nz = r[8 + e];
-            float ta = fm(ny, rya, nz), tb = fm(ny, ryb, nz);
+            const float ny = r[4 + e], nz = r[8 + e];
+            const float ta = fm(ny, rya, nz), tb = fm(ny, ryb, nz);
             tmin[e] = fminf(ta, tb); tmax[e] = fmaxf(ta, tb);
             nx[e] = r[e];
         }
         const float wx = r[12], wy = r[13], wz = r[14];
         const float wa = fm(wy, rya, wz), wb = fm(wy, ryb, wz);
         const float wtmin = fminf(wa, wb), wtmax = fmaxf(wa, wb);
+        unsigned long long any = 0ull, full = 0ull;
         for (int bcol = bx0 >> 3; bcol <= (bx1 >> 3); ++bcol) {
             const int xa = bcol * 8, xb = min(bcol * 8 + 7, t.tw - 1);
             const float rxa = s.ray_x[xa], rxb = s.ray_x[xb];    // rxa < rxb
-            bool reject = false, full = true;
+            bool reject = false, inside = true;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 // fma is monotone in each argument, so the block's extreme values are at its corners
-                float emax = fm(nx[e], nx[e] >= 0.f ? rxb : rxa, tmax[e]);
-                float emin = fm(nx[e], nx[e] >= 0.f ? rxa : rxb, tmin[e]);
+                const float emax = fm(nx[e], nx[e] >= 0.f ? rxb : rxa, tmax[e]);
+                const float emin = fm(nx[e], nx[e] >= 0.f ? rxa : rxb, tmin[e]);
                 reject = reject || (emax < 0.f);
-                full = full && (emin > 0.f);
+                inside = inside && (emin > 0.f);
             }
-            float wmax = fm(wx, wx >= 0.f ? rxb : rxa, wtmax), wmin = fm(wx, wx >= 0.f ? rxa : rxb, wtmin);
+            const float wmax = fm(wx, wx >= 0.f ? rxb : rxa, wtmax), wmin = fm(wx, wx >= 0.f ? rxa : rxb, wtmin);
             reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
-            full = full && (wmin >= t.w_far) && (wmax <= t.w_near);
+            inside = inside && (wmin >= t.w_far) && (wmax <= t.w_near);
             if (reject) continue;
-            const int blk = brow * 8 + bcol;
-            atomicOr(&s.bin_any[blk][p >> 6], 1ull << (p & 63));
-            if (full) atomicOr(&s.bin_full[blk][p >> 6], 1ull << (p & 63));
+            any |= 1ull << bcol;
+            if (inside) full |= 1ull << bcol;
+        }
+        for (; any; any &= any - 1) {
+            const int bcol = __ffsll((long long)any) - 1;
+            atomicOr(&s.bin_any[brow * 8 + bcol], 1ull << p);
+            if ((full >> bcol) & 1ull) atomicOr(&s.bin_full[brow * 8 + bcol], 1ull << p);
         }
     }
-    __syncthreads();
 }
 
 // (c) raster of the binned primitives: a warp owns an 8x8 block, a lane two horizontally adjacent
@@ -416,28 +508,23 @@ __device__ void bin_large(TileSmem& s, const TileCtx& t) {
 __device__ int raster_large(TileSmem& s, const TileCtx& t) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int frags = 0;
-    for (int blk = warp; blk < 64; blk += NTHREADS / 32) {
-        bool some = false;
-#pragma unroll
-        for (int w = 0; w < LWORDS; ++w) some = some || (s.bin_any[blk][w] != 0ull);
-        if (!some) continue;
+    for (int blk = warp; blk < 64; blk += NW) {
+        unsigned long long any = s.bin_any[blk];
+        if (!any) continue;
+        const unsigned long long fullm = s.bin_full[blk];
         const int x = (blk & 7) * 8 + (lane & 3) * 2, y = (blk >> 3) * 8 + (lane >> 2);
         const float rx0 = s.ray_x[x], rx1 = s.ray_x[x + 1], ry = s.ray_y[y];
-        ulonglong2 kk = *reinterpret_cast<ulonglong2*>(&s.key[y * TILE + x]);
-#pragma unroll 1
-        for (int w = 0; w < LWORDS; ++w) {
-        unsigned long long any = s.bin_any[blk][w];
-        const unsigned long long fullm = s.bin_full[blk][w];
+        ulonglong2* kp = reinterpret_cast<ulonglong2*>(&s.key[key_index(x, y)]);
+        ulonglong2 kk = *kp;
         while (any) {
-            const int pb = __ffsll((long long)any) - 1;
+            const int p = __ffsll((long long)any) - 1;
             any &= any - 1;
-            const int p = w * 64 + pb;
-            const float* r = &s.rec[p * REC];
+            const float* r = &s.rec_l[p * REC];
             const uint32_t key_lo = __float_as_uint(r[15]);
             const float wt = fm(r[13], ry, r[14]);
             const float w0 = fm(r[12], rx0, wt), w1 = fm(r[12], rx1, wt);
             bool in0 = true, in1 = true;
-            if (!((fullm >> pb) & 1ull)) {
+            if (!((fullm >> p) & 1ull)) {
                 const uint32_t tl = __float_as_uint(r[16]) >> 24;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -450,27 +537,18 @@ __device__ int raster_large(TileSmem& s, const TileCtx& t) {
                 in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
                 in1 = in1 && (w1 >= t.w_far) && (w1 <= t.w_near);
             }
-            if (in0) { unsigned long long k = make_key(__float_as_uint(w0), key_lo); if (k > kk.x) kk.x = k; ++frags; }
-            if (in1) { unsigned long long k = make_key(__float_as_uint(w1), key_lo); if (k > kk.y) kk.y = k; ++frags; }
+            if (in0) { const unsigned long long k = make_key(__float_as_uint(w0), key_lo); if (k > kk.x) kk.x = k; ++frags; }
+            if (in1) { const unsigned long long k = make_key(__float_as_uint(w1), key_lo); if (k > kk.y) kk.y = k; ++frags; }
         }
-        }
-        *reinterpret_cast<ulonglong2*>(&s.key[y * TILE + x]) = kk;
+        *kp = kk;
     }
     return frags;
 }
 
-// Flush the binned list: bin, raster, reset.  Must be called by all threads of the CTA.
-__device__ __forceinline__ int flush_large(TileSmem& s, const TileCtx& t) {
-    __syncthreads();
-    int frags = 0;
-    if (s.n_large > 0) {
-        bin_large(s, t);
-        frags = raster_large(s, t);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) s.n_large = 0;
-    __syncthreads();
-    return frags;
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
 }
 
 // (d) keys -> class / depth images.
@@ -483,6 +561,7 @@ __device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderPara
     const float cphi = -c.dz, sphi = c.fz_;
     const bool vec = (t.tw % 16 == 0) && (P.W % 16 == 0) && o32 == nullptr;
     const int segs_per_row = (t.tw + 15) / 16;
+    const unsigned long long touched = ((unsigned long long)s.touched[1] << 32) | s.touched[0];
     for (int seg = threadIdx.x; seg < t.th * segs_per_row; seg += NTHREADS) {
         const int y = seg / segs_per_row, xs = (seg % segs_per_row) * 16;
         // background of this row: analytic ground plane below the horizon, sky above
@@ -492,26 +571,37 @@ __device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderPara
         if (wr < 0.f && c.mwz > 0.f) { bg_cls = P.cls_ground; bg_z = fminf(P.far_z, __fdiv_rn(c.mwz, -wr)); }
         if (!ego_active) { bg_cls = P.cls_sky; bg_z = P.far_z; }
         const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + xs;
+        const bool empty = ((touched >> ((y >> 3) * 8 + (xs >> 3))) & 3ull) == 0ull;   // both blocks of the segment
         if (vec) {
             uint32_t cw[4];
             uint32_t dw[8];
+            if (empty) {
+                const uint32_t c4 = bg_cls * 0x01010101u;
+                const __half2 h = __floats2half2_rn(bg_z, bg_z);
+                const uint32_t d2 = *reinterpret_cast<const uint32_t*>(&h);
 #pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-                ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(&s.key[y * TILE + xs + j]);
-                float z0 = kk.x ? __frcp_rn(__uint_as_float((uint32_t)(kk.x >> 32))) : bg_z;
-                float z1 = kk.y ? __frcp_rn(__uint_as_float((uint32_t)(kk.y >> 32))) : bg_z;
-                uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bg_cls, c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bg_cls;
-                __half2 h = __floats2half2_rn(z0, z1);
-                dw[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
-                if ((j & 3) == 0) cw[j >> 2] = c0 | (c1 << 8); else cw[j >> 2] |= (c0 << 16) | (c1 << 24);
+                for (int j = 0; j < 4; ++j) cw[j] = c4;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) dw[j] = d2;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(&s.key[key_index(xs + j, y)]);
+                    const float z0 = kk.x ? fast_rcp(__uint_as_float((uint32_t)(kk.x >> 32))) : bg_z;
+                    const float z1 = kk.y ? fast_rcp(__uint_as_float((uint32_t)(kk.y >> 32))) : bg_z;
+                    const uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bg_cls, c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bg_cls;
+                    const __half2 h = __floats2half2_rn(z0, z1);
+                    dw[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                    if ((j & 3) == 0) cw[j >> 2] = c0 | (c1 << 8); else cw[j >> 2] |= (c0 << 16) | (c1 << 24);
+                }
             }
             *reinterpret_cast<uint4*>(oc + o) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
             *reinterpret_cast<uint4*>(od + o) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
             *reinterpret_cast<uint4*>(od + o + 8) = make_uint4(dw[4], dw[5], dw[6], dw[7]);
         } else {
             for (int j = 0; j < 16 && xs + j < t.tw; ++j) {
-                unsigned long long k = s.key[y * TILE + xs + j];
-                float z = k ? __frcp_rn(__uint_as_float((uint32_t)(k >> 32))) : bg_z;
+                const unsigned long long k = s.key[key_index(xs + j, y)];
+                const float z = k ? fast_rcp(__uint_as_float((uint32_t)(k >> 32))) : bg_z;
                 oc[o + j] = (uint8_t)(k ? (uint32_t)(k & 0xff) : bg_cls);
                 od[o + j] = __half_as_ushort(__float2half_rn(z));
                 if (o32) o32[o + j] = z;
@@ -533,12 +623,15 @@ __device__ bool tile_prologue(TileSmem& s, TileCtx& t, const RenderParams& P, si
     t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
     t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
     t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
+    t.med_cap = min(MCAP, P.med_cap); t.large_cap = min(LCAP, P.large_cap);
     const AgentGeom ego = P.agents[(size_t)e * P.A + a];
     if (threadIdx.x == 0) {
         make_camera(s.cam, ego, P.cam[k], P.W, P.H);
-        s.n_cand = 0; s.n_large = 0; s.n_leaf = 0; s.n_grp = 0;
+        s.n_large = 0; s.n_med = 0; s.n_leaf = 0; s.n_grp = 0; s.n_face = 0;
+        s.touched[0] = 0u; s.touched[1] = 0u;
     }
-    if (threadIdx.x < 8) s.cnt[threadIdx.x] = 0ull;
+    if (threadIdx.x < 16) s.cnt[threadIdx.x] = 0ull;
+    if (threadIdx.x < 64) { s.bin_any[threadIdx.x] = 0ull; s.bin_full[threadIdx.x] = 0ull; }
     for (int i = threadIdx.x; i < TILE * TILE / 2; i += NTHREADS)
         reinterpret_cast<ulonglong2*>(s.key)[i] = make_ulonglong2(0ull, 0ull);
     __syncthreads();
@@ -549,105 +642,56 @@ __device__ bool tile_prologue(TileSmem& s, TileCtx& t, const RenderParams& P, si
         s.ray_y[i] = __fdiv_rn(sub(add((float)(t.y0 + i), 0.5f), c.cy), c.focy);
     }
     if (threadIdx.x >= 64 && threadIdx.x < 70) {
-        // frustum planes n.(q - m_w) >= 0 with q = X - P_ego; stored as n and offset -n.m_w (+ near/far)
+        // frustum planes n.(q - m_w) >= 0 with q = X - P_ego; unit normals, offset -n.m_w (+ near/far)
         const int p = threadIdx.x - 64;
-        float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
-        float nx, ny, nz, off = 0.f;
+        const float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
+        float nx, ny, nz, off = 0.f, sx = 0.f, sy = 0.f, sz = 0.f;
         const float Rx = c.rx, Ry = c.ry, Dx = c.dx, Dy = c.dy, Dz = c.dz, Fx = c.fx_, Fy = c.fy_, Fz = c.fz_;
         switch (p) {
             case 0: nx = Fx; ny = Fy; nz = Fz; off = -P.near_z * 0.999f; break;                                       // z >= near
             case 1: nx = -Fx; ny = -Fy; nz = -Fz; off = P.far_z * 1.001f; break;                                      // z <= far
-            case 2: nx = c.focx * Rx - l * Fx; ny = c.focx * Ry - l * Fy; nz = -l * Fz; break;                        // x f >= z l
-            case 3: nx = r * Fx - c.focx * Rx; ny = r * Fy - c.focx * Ry; nz = r * Fz; break;                         // x f <= z r
-            case 4: nx = c.focy * Dx - u * Fx; ny = c.focy * Dy - u * Fy; nz = c.focy * Dz - u * Fz; break;           // y f >= z u
-            default: nx = d * Fx - c.focy * Dx; ny = d * Fy - c.focy * Dy; nz = d * Fz - c.focy * Dz; break;          // y f <= z d
+            case 2: nx = c.focx * Rx - l * Fx; ny = c.focx * Ry - l * Fy; nz = -l * Fz; sx = c.focx; sz = -l; break;  // x f >= z l
+            case 3: nx = r * Fx - c.focx * Rx; ny = r * Fy - c.focx * Ry; nz = r * Fz; sx = -c.focx; sz = r; break;   // x f <= z r
+            case 4: nx = c.focy * Dx - u * Fx; ny = c.focy * Dy - u * Fy; nz = c.focy * Dz - u * Fz; sy = c.focy; sz = -u; break;   // y f >= z u
+            default: nx = d * Fx - c.focy * Dx; ny = d * Fy - c.focy * Dy; nz = d * Fz - c.focy * Dz; sy = -c.focy; sz = d; break;  // y f <= z d
         }
+        const float inv = rsqrtf(nx * nx + ny * ny + nz * nz);
+        nx *= inv; ny *= inv; nz *= inv;
         s.plane[p][0] = nx; s.plane[p][1] = ny; s.plane[p][2] = nz;
         s.plane[p][3] = off - (nx * c.mwx + ny * c.mwy + nz * c.mwz);
+        if (p >= 2) {
+            const float is = rsqrtf(sx * sx + sy * sy + sz * sz);
+            s.side[p - 2][0] = sx * is; s.side[p - 2][1] = sy * is; s.side[p - 2][2] = sz * is; s.side[p - 2][3] = 0.f;
+        }
     }
     __syncthreads();
     return ego.active != 0;
 }
 
-__device__ __forceinline__ void add_counters(TileSmem& s, const RenderParams& P) {
-    __syncthreads();
-    if (P.counters && threadIdx.x < 8 && s.cnt[threadIdx.x]) atomicAdd(&P.counters[threadIdx.x], s.cnt[threadIdx.x]);
-}
-
-// Drain the candidate list: dense set-up, one candidate per thread per pass.
-// Candidate .x: bit 31 set -> box face item (agent << 3 | face), else primitive id.
-__device__ void drain_candidates(TileSmem& s, const TileCtx& t, const RenderParams& P, int e, uint32_t n_map_tris) {
-    __syncthreads();
-    const int n = s.n_cand;
-    int frags = 0, n_small = 0, n_set = 0;
-    for (int base = 0; base < n; base += NTHREADS) {
-        __syncthreads();                                                  // n_large is stable and uniform here
-        if (s.n_large + min(NTHREADS, n - base) > LCAP) frags += flush_large(s, t);   // room for this pass
-        const int i = base + threadIdx.x;
-        if (i < n) {
-            const uint2 cd = s.cand[i];
-            V3 V[4];
-            bool quad;
-            uint32_t flags, key_lo;
-            if (cd.x & 0x80000000u) {
-                const int b = (cd.x & 0x7fffffffu) >> 3, f = cd.x & 7;
-                const AgentGeom g = P.agents[(size_t)e * P.A + b];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, kFace[f][k]);
-                quad = true;
-                flags = face_flags(f);
-                key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
-            } else {
-                float v[12];
-                load_prim(P.prims + cd.x, v, key_lo, flags);
-                quad = flags & 1u;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) V[k] = to_camera(s.cam, v[3 * k], v[3 * k + 1], v[3 * k + 2]);
-            }
-            emit_prim(s, t, V, quad, flags, key_lo, cd.y, frags, n_small, n_set);
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) s.n_cand = 0;
-    if (P.counters) {
-        atomicAdd(&s.cnt[4], (unsigned long long)n_set);
-        atomicAdd(&s.cnt[5], (unsigned long long)n_small);
-        atomicAdd(&s.cnt[7], (unsigned long long)frags);
-    }
-    __syncthreads();
-}
-
-// Warp-aggregated append of one candidate per participating lane.
-__device__ __forceinline__ void push_candidate(TileSmem& s, bool keep, uint32_t id, uint32_t box) {
-    const unsigned m = __ballot_sync(0xffffffffu, keep);
-    if (!m) return;
-    const int lane = threadIdx.x & 31;
-    int base = 0;
-    if (lane == 0) base = atomicAdd(&s.n_cand, __popc(m));
-    base = __shfl_sync(0xffffffffu, base, 0);
-    if (keep) s.cand[base + __popc(m & ((1u << lane) - 1u))] = make_uint2(id, box);
-}
-
 // ------------------------------------------------------------------------------------------------
 // production kernel
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(NTHREADS) render_kernel(const __grid_constant__ RenderParams P) {
+__global__ void __launch_bounds__(NTHREADS, 4) render_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& s = *reinterpret_cast<TileSmem*>(smem_raw);
     TileCtx t;
     size_t view; int e, a;
+    const bool count = P.counters != nullptr;
+    long long c0 = count ? clock64() : 0;
     const bool ego_active = tile_prologue(s, t, P, view, e, a);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int NW = NTHREADS / 32;
+    Tally n = {0, 0, 0, 0, 0, 0, 0};
+    int n_grp_tests = 0, n_leaf_tests = 0;
+    long long c1 = 0, c2 = 0, c3 = 0, c4 = 0, c5 = 0;
+    if (count) c1 = clock64();
     if (ego_active) {
         const MapInfo mi = P.maps[P.env_map[e]];
-        unsigned long long c_grp = 0, c_leaf = 0, c_prim = 0;
-        // ---- (a) map: groups -> leaves -> primitives
-        for (uint32_t g0 = mi.group_begin; g0 < mi.group_end; g0 += 32) {
+        // ---- (a)+(c) map: groups -> leaves -> primitives, set up as they survive
+        for (uint32_t g0 = mi.group_begin; g0 < mi.group_end; g0 += GROUP_BATCH) {
             if (warp == 0) {
                 const uint32_t g = g0 + lane;
                 bool vis = false;
-                if (g < mi.group_end) { vis = box_visible(s, P.groups[g]); ++c_grp; }
+                if (lane < GROUP_BATCH && g < mi.group_end) { vis = box_visible(s, P.groups[g]); ++n_grp_tests; }
                 const unsigned m = __ballot_sync(0xffffffffu, vis);
                 if (vis) s.grp[__popc(m & ((1u << lane) - 1u))] = g;
                 if (lane == 0) { s.n_grp = __popc(m); s.n_leaf = 0; }
@@ -657,68 +701,119 @@ __global__ void __launch_bounds__(NTHREADS) render_kernel(const __grid_constant_
             for (int i = warp; i < ng; i += NW) {
                 const Node g = P.groups[s.grp[i]];
                 bool vis = false;
-                if (lane < (int)g.count) { vis = box_visible(s, P.leaves[g.first + lane]); ++c_leaf; }
+                Node lf;
+                if (lane < (int)g.count) { lf = P.leaves[g.first + lane]; vis = box_visible(s, lf); ++n_leaf_tests; }
                 const unsigned m = __ballot_sync(0xffffffffu, vis);
                 int base = 0;
                 if (lane == 0 && m) base = atomicAdd(&s.n_leaf, __popc(m));
                 base = __shfl_sync(0xffffffffu, base, 0);
-                if (vis) s.leaf[base + __popc(m & ((1u << lane) - 1u))] = g.first + lane;
+                if (vis) s.leaf[base + __popc(m & ((1u << lane) - 1u))] = (lf.first << 4) | lf.count;
             }
             __syncthreads();
             const int nl = s.n_leaf;
-            // rounds of NW leaves: each adds at most NW*32 candidates
-            for (int l0 = 0; l0 < nl; l0 += NW) {
-                if (s.n_cand + NW * 32 > CCAP) drain_candidates(s, t, P, e, mi.n_tris);   // uniform
-                const int li = l0 + warp;
-                if (li < nl) {
-                    const Node lf = P.leaves[s.leaf[li]];
-                    bool keep = false;
-                    uint32_t box = 0;
-                    if (lane < (int)lf.count) {
-                        float v[12]; uint32_t key_lo, flags;
-                        load_prim(P.prims + lf.first + lane, v, key_lo, flags);
-                        V3 V[4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) V[k] = to_camera(s.cam, v[3 * k], v[3 * k + 1], v[3 * k + 2]);
-                        keep = pixel_box(s.cam, t, V, box);
-                        ++c_prim;
-                    }
-                    push_candidate(s, keep, lf.first + lane, box);
-                }
-                __syncthreads();
-            }
-        }
-        // ---- (a) other agents' boxes: cull per box, one item per possibly visible face
-        for (int b0 = 0; b0 < P.A; b0 += NTHREADS / 8) {
-            // 16 boxes per round -> at most 96 face items
-            if (s.n_cand + (NTHREADS / 8) * 6 > CCAP) drain_candidates(s, t, P, e, mi.n_tris);
-            const int b = b0 + (threadIdx.x >> 3), f = threadIdx.x & 7;
-            bool keep = false;
-            uint32_t box = 0;
-            if (b < P.A && b != a && f < 6) {
-                const AgentGeom g = P.agents[(size_t)e * P.A + b];
-                if (g.active) {
+            // LEAF_PRIMS threads per leaf, no barrier inside this loop
+            for (int i = threadIdx.x; i < nl * LEAF_PRIMS; i += NTHREADS) {
+                const uint32_t lf = s.leaf[i / LEAF_PRIMS];
+                const uint32_t k = i % LEAF_PRIMS;
+                if (k < (lf & 15u)) {
+                    float v[12]; uint32_t key_lo, flags;
+                    load_prim(P.prims + (lf >> 4) + k, v, key_lo, flags);
                     V3 V[4];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, kFace[f][k]);
-                    keep = pixel_box(s.cam, t, V, box);
-                    ++c_prim;
+                    for (int j = 0; j < 4; ++j) V[j] = to_camera(s.cam, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
+                    process_prim(s, t, V, flags & 1u, flags, key_lo, n);
                 }
             }
-            push_candidate(s, keep, 0x80000000u | ((uint32_t)b << 3) | (uint32_t)f, box);
+            __syncthreads();       // the leaf list is reused by the next batch and by the face items
+        }
+        if (count) c2 = clock64();
+        // ---- (a)+(c) other agents: sphere cull per box, camera-facing faces become items
+        const Cam& c = s.cam;
+        for (int b0 = 0; b0 < P.A; b0 += LEAFCAP / 8) {
+            for (int b = b0 + threadIdx.x; b < min(P.A, b0 + LEAFCAP / 8); b += NTHREADS) {
+                if (b == a) continue;
+                const AgentGeom g = P.agents[(size_t)e * P.A + b];
+                if (!g.active) continue;
+                const float hh = 0.5f * g.h;
+                const V3 ctr = rotate_to_camera(c, sub(sub(g.x, c.px), c.mwx), sub(sub(g.y, c.py), c.mwy), sub(hh, c.mwz));
+                const float rad = sqrtf(g.hl * g.hl + g.hw * g.hw + hh * hh) * 1.0001f + 1e-4f;
+                bool vis = (ctr.z + rad >= t.near_z * 0.999f) && (ctr.z - rad <= t.far_z * 1.001f);
+#pragma unroll
+                for (int p = 0; p < 4; ++p)
+                    vis = vis && (s.side[p][0] * ctr.x + s.side[p][1] * ctr.y + s.side[p][2] * ctr.z >= -rad);
+                if (!vis) continue;
+                // camera position in the box frame decides which faces can face the camera; near
+                // the near plane (or inside the box) every face is kept
+                uint32_t faces = 0x3fu;
+                if (ctr.z - rad > t.near_z * 1.01f) {
+                    const float dx = sub(c.mwx, sub(g.x, c.px)), dy = sub(c.mwy, sub(g.y, c.py));
+                    const float u = g.c * dx + g.s * dy, v = g.c * dy - g.s * dx;
+                    const float eps = 1e-4f * (1.f + fabsf(dx) + fabsf(dy));
+                    faces = 0u;
+                    if (u < -g.hl + eps) faces |= 1u;          // rear
+                    if (u > g.hl - eps) faces |= 2u;           // front
+                    if (v < -g.hw + eps) faces |= 4u;          // right
+                    if (v > g.hw - eps) faces |= 8u;           // left
+                    if (c.mwz < eps) faces |= 16u;             // bottom
+                    if (c.mwz > g.h - eps) faces |= 32u;       // top
+                }
+                const int nf = __popc(faces);
+                int slot = atomicAdd(&s.n_face, nf);
+                for (; faces; faces &= faces - 1) s.face[slot++] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
+            }
+            __syncthreads();
+            const int nf = s.n_face;
+            for (int i = threadIdx.x; i < nf; i += NTHREADS) {
+                const uint32_t it = s.face[i];
+                const int b = (int)(it >> 3), f = (int)(it & 7u);
+                const AgentGeom g = P.agents[(size_t)e * P.A + b];
+                const uint32_t corners = face_corners(f);
+                V3 V[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) V[k] = box_corner(c, g, (corners >> (4 * k)) & 7u);
+                const uint32_t key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+                process_prim(s, t, V, true, face_flags(corners), key_lo, n);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) s.n_face = 0;
             __syncthreads();
         }
-        drain_candidates(s, t, P, e, mi.n_tris);
-        int frags = flush_large(s, t);
-        if (P.counters) {
-            atomicAdd(&s.cnt[1], c_grp); atomicAdd(&s.cnt[2], c_leaf); atomicAdd(&s.cnt[3], c_prim);
-            atomicAdd(&s.cnt[7], (unsigned long long)frags);
-            if (threadIdx.x == 0) s.cnt[0] = 1;
-        }
+        if (count) c3 = clock64();
+        // ---- medium primitives (atomics) and binning of the large ones, then the block raster
+        n.frags += raster_medium(s, t);
+        bin_large(s, t);
+        __syncthreads();
+        if (threadIdx.x < 64 && s.bin_any[threadIdx.x]) mark_touched(s, 1ull << threadIdx.x);
+        if (count) c4 = clock64();
+        n.frags += raster_large(s, t);
     }
     __syncthreads();
+    if (count) c5 = clock64();
     store_tile(s, t, P, view, ego_active);
-    add_counters(s, P);
+    if (count) {
+        atomicAdd(&s.cnt[1], (unsigned long long)n_grp_tests);
+        atomicAdd(&s.cnt[2], (unsigned long long)n_leaf_tests);
+        atomicAdd(&s.cnt[3], (unsigned long long)n.tested);
+        atomicAdd(&s.cnt[4], (unsigned long long)n.setup);
+        atomicAdd(&s.cnt[5], (unsigned long long)n.tiny);
+        atomicAdd(&s.cnt[6], (unsigned long long)n.medium);
+        atomicAdd(&s.cnt[7], (unsigned long long)n.large);
+        atomicAdd(&s.cnt[8], (unsigned long long)n.fallback);
+        atomicAdd(&s.cnt[9], (unsigned long long)n.frags);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const long long c6 = clock64();
+            s.cnt[0] = 1;
+            s.cnt[10] = (unsigned long long)(c1 - c0);
+            if (ego_active) {
+                s.cnt[11] = (unsigned long long)(c2 - c1); s.cnt[12] = (unsigned long long)(c3 - c2);
+                s.cnt[13] = (unsigned long long)(c4 - c3); s.cnt[14] = (unsigned long long)(c5 - c4);
+            }
+            s.cnt[15] = (unsigned long long)(c6 - c5);
+        }
+        __syncthreads();
+        if (threadIdx.x < 16 && s.cnt[threadIdx.x]) atomicAdd(&P.counters[threadIdx.x], s.cnt[threadIdx.x]);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -749,14 +844,15 @@ __global__ void __launch_bounds__(NTHREADS) render_brute_kernel(const __grid_con
                 if (b == a) continue;
                 const AgentGeom g = P.agents[(size_t)e * P.A + b];
                 if (!g.active) continue;
+                const uint32_t corners = face_corners(f);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, kFace[f][k]);
-                quad = true; flags = face_flags(f);
+                for (int k = 0; k < 4; ++k) V[k] = box_corner(s.cam, g, (corners >> (4 * k)) & 7u);
+                quad = true; flags = face_flags(corners);
                 key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
             }
             PrimEq q;
             if (!prim_equations(V, quad, flags, q)) continue;
-            raster_small(s, t, q, key_lo, full);
+            raster_in_thread(s, t, q, key_lo, full);
         }
     }
     __syncthreads();
@@ -767,6 +863,7 @@ __global__ void __launch_bounds__(NTHREADS) render_brute_kernel(const __grid_con
 // host-side launchers (called from the C ABI)
 // ------------------------------------------------------------------------------------------------
 size_t render_smem_bytes() { return sizeof(TileSmem); }
+int render_list_caps(int which) { return which == 0 ? MCAP : LCAP; }
 
 cudaError_t configure_kernels() {
     cudaError_t err = cudaFuncSetAttribute(render_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));

@@ -7,8 +7,8 @@ namespace pic {
 constexpr int TILE = 64;        // a view is rendered in tiles of up to TILE x TILE pixels (one CTA each)
 constexpr int NTHREADS = 128;   // threads per render CTA
 constexpr int MAX_CAMS = 16;    // cameras per rig
-constexpr int LEAF_PRIMS = 32;  // primitives per leaf (one per lane)
-constexpr int LONG_LEAF_PRIMS = 4;   // long primitives get small leaves so their boxes stay tight
+constexpr int LEAF_PRIMS = 8;   // primitives per leaf (8 threads per leaf in the cull pass)
+constexpr int LONG_LEAF_PRIMS = 8;   // long primitives get leaves of their own so the others' boxes stay tight
 constexpr int GROUP_LEAVES = 32;     // leaves per group (one per lane)
 
 // Map primitive in hierarchy order: a triangle, or a planar convex quad fused from two consecutive
@@ -67,7 +67,8 @@ struct RenderParams {
     uint8_t* out_class;
     uint16_t* out_depth;
     float* out_depth32;             // optional
-    unsigned long long* counters;   // optional [8]
+    unsigned long long* counters;   // optional [16]
+    int32_t med_cap, large_cap;     // usable entries of the medium / large lists (debug: shrink to force the fallback)
     long long view_first;           // render views [view_first, view_first + gridDim / tiles)
     CamConst cam[MAX_CAMS];
 };

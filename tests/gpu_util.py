@@ -23,19 +23,21 @@ class GpuRun:
         self.active = torch.from_numpy(np.ascontiguousarray(s.active)).to(self.dev)
 
     def render(self, brute: bool = False, depth32: bool = True, poses=None, view_first: int = 0, view_count: int = 0,
-               counters: bool = False):
+               counters: bool = False, list_caps=None):
         """Returns (class u8 [V,H,W], depth f16 [V,H,W], depth32 f32 [V,H,W] or None[, counters]) as numpy."""
         torch, pic, s = self.torch, self.pic, self.s
         cls, dep = self.scene.alloc_outputs()
         cls.fill_(255)
         dep.fill_(-1.0)
         d32 = torch.full(self.scene.image_shape, -1.0, dtype=torch.float32, device=self.dev) if depth32 else None
-        cnt = torch.zeros(8, dtype=torch.int64, device=self.dev) if counters else None
+        cnt = torch.zeros(16, dtype=torch.int64, device=self.dev) if counters else None
         self.scene.set_option(pic.OPT_BRUTE_FORCE, 1 if brute else 0)
         self.scene.set_option(pic.OPT_DEPTH32, d32 if depth32 else 0)
         self.scene.set_option(pic.OPT_COUNTERS, cnt if counters else 0)
         self.scene.set_option(pic.OPT_VIEW_FIRST, view_first)
         self.scene.set_option(pic.OPT_VIEW_COUNT, view_count)
+        if list_caps is not None:
+            self.scene.set_option(pic.OPT_LIST_CAPS, int(list_caps[0]) | (int(list_caps[1]) << 16))
         p = self.poses if poses is None else torch.from_numpy(np.ascontiguousarray(poses, dtype=np.float32)).to(self.dev)
         self.scene.render(p, self.dims, s.rig, active=self.active, out_class=cls, out_depth=dep)
         torch.cuda.synchronize()
@@ -44,6 +46,7 @@ class GpuRun:
         self.scene.set_option(pic.OPT_BRUTE_FORCE, 0)
         self.scene.set_option(pic.OPT_VIEW_FIRST, 0)
         self.scene.set_option(pic.OPT_VIEW_COUNT, 0)
+        self.scene.set_option(pic.OPT_LIST_CAPS, 0xffff | (0xffff << 16))
         V = s.E * s.A * s.K
         out = (cls.cpu().numpy().reshape(V, s.H, s.W), dep.cpu().numpy().reshape(V, s.H, s.W),
                d32.cpu().numpy().reshape(V, s.H, s.W) if depth32 else None)
