@@ -145,13 +145,13 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *   PIC_OPT_DEPTH32       value = dev f32* [E,A,K,H,W] (as uintptr) or 0: also write the float32
  *                         depth the binary16 image was rounded from.
  *   PIC_OPT_COUNTERS      value = dev u64* [16] (as uintptr) or 0: accumulate work counters (tiles,
- *                         group tests, leaf tests, primitives tested, set up, tiny, medium, large,
- *                         list-overflow fallbacks, fragments, then SM cycles of six phases of thread 0).
+ *                         group tests, leaf tests, primitives tested, set up, rasterized by their
+ *                         thread, records, record-list overflows, records classified per cell, cells visited).
  *   PIC_OPT_VIEW_FIRST,   render only views [first, first + count) (flat index (e*A + a)*K + k);
  *   PIC_OPT_VIEW_COUNT    count 0 = through the last view.  Other views' pixels are left untouched.
- *   PIC_OPT_LIST_CAPS     value = medium | large << 16: usable entries of the kernel's two
- *                         per-tile primitive lists (default: all).  Overflowing primitives take a
- *                         slower path with identical results; shrinking the lists tests that path.
+ *   PIC_OPT_DEBUG_FLAGS   bit 0: rasterize large primitives without the per-cell trivial
+ *                         accept/reject; bit 1: shrink the per-tile record list to 2 entries so that
+ *                         the overflow path runs.  Both leave the images unchanged (tests rely on it).
  *   PIC_OPT_TIMING        1: bracket every render-kernel launch with CUDA events on its stream
  *                         (up to 1024 launches between two pic_get_kernel_times calls); 0: off.
  *                         Turning it on creates the events (allocates), so do it outside timed code.
@@ -162,7 +162,7 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
 #define PIC_OPT_VIEW_FIRST 4
 #define PIC_OPT_VIEW_COUNT 5
 #define PIC_OPT_TIMING 6
-#define PIC_OPT_LIST_CAPS 7
+#define PIC_OPT_DEBUG_FLAGS 7
 pic_status pic_scene_set_option(pic_scene* scene, int32_t option, uint64_t value);
 
 /*

@@ -11,12 +11,11 @@
 #include "pic_types.h"
 
 namespace pic {
-size_t render_smem_bytes();
-int render_list_caps(int which);
+size_t max_smem_bytes();
 cudaError_t configure_kernels();
-cudaError_t launch_agents(int n, const float* poses, float* state, const float* actions, const float* dims,
-                          const uint8_t* active, AgentGeom* out, uint32_t* status, float dt, float wheelbase,
-                          float v_max, cudaStream_t stream);
+cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses, float* state, const float* actions,
+                         const float* dims, const uint8_t* active, AgentGeom* agents_out, ViewCam* cams_out,
+                         float* tables, uint32_t* status, float dt, float wheelbase, float v_max, cudaStream_t stream);
 cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, cudaStream_t stream);
 }  // namespace pic
 
@@ -58,6 +57,8 @@ struct pic_scene {
     pic::Node* d_leaves = nullptr;
     pic::Prim* d_prims = nullptr;
     pic::AgentGeom* d_agents = nullptr;
+    pic::ViewCam* d_cams = nullptr;   // [E*A*K]
+    float* d_tables = nullptr;        // per-camera ray and background tables, K*(W+3H) words
     float* d_state = nullptr;       // [E*A*4]
     float* d_dims = nullptr;        // [E*A*3]
     uint8_t* d_active = nullptr;    // [E*A]
@@ -74,7 +75,7 @@ struct pic_scene {
     float* depth32 = nullptr;
     unsigned long long* counters = nullptr;
     long long view_first = 0, view_count = 0;
-    int med_cap = 1 << 30, large_cap = 1 << 30;
+    int debug_flags = 0;
     bool timing = false;
     cudaEvent_t* ev = nullptr;      // 2 * kMaxTimed events
     int n_timed = 0;
@@ -95,7 +96,7 @@ struct DeviceGuard {
 
 void free_scene(pic_scene* s) {
     cudaFree(s->d_env_map); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
-    cudaFree(s->d_agents); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
+    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
     if (s->ev) {
@@ -120,9 +121,14 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.cls_agent = s->cls_agent; P.cls_sky = s->cls_sky; P.cls_ground = s->cls_ground;
     P.env_map = s->d_env_map; P.maps = s->d_maps; P.groups = s->d_groups; P.leaves = s->d_leaves; P.prims = s->d_prims;
     P.agents = s->d_agents;
+    P.cams = s->d_cams;
+    P.rig.ray_x = s->d_tables;
+    P.rig.ray_y = P.rig.ray_x + (size_t)s->K * s->W;
+    P.rig.bg_z = P.rig.ray_y + (size_t)s->K * s->H;
+    P.rig.bg_cls = reinterpret_cast<const uint32_t*>(P.rig.bg_z + (size_t)s->K * s->H);
     P.out_class = out_class; P.out_depth = out_depth; P.out_depth32 = s->depth32; P.counters = s->counters;
     P.view_first = 0;
-    P.med_cap = s->med_cap; P.large_cap = s->large_cap;
+    P.debug_flags = s->debug_flags;
     for (int k = 0; k < s->K; ++k) {
         const pic_camera& c = rig[k];
         const float vals[7] = {c.mount_x, c.mount_y, c.mount_z, c.yaw, c.pitch, c.fx, c.fy};
@@ -181,8 +187,8 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     cudaDeviceProp prop;
     CUDA_TRY(cudaGetDeviceProperties(&prop, d->device));
     if (prop.major < 10) return fail(PIC_ERR_CUDA, "device %d is sm_%d%d; this library is built for sm_100a only", d->device, prop.major, prop.minor);
-    if ((size_t)prop.sharedMemPerBlockOptin < pic::render_smem_bytes())
-        return fail(PIC_ERR_CUDA, "device offers %zu bytes of shared memory per block, %zu needed", (size_t)prop.sharedMemPerBlockOptin, pic::render_smem_bytes());
+    if ((size_t)prop.sharedMemPerBlockOptin < pic::max_smem_bytes())
+        return fail(PIC_ERR_CUDA, "device offers %zu bytes of shared memory per block, %zu needed", (size_t)prop.sharedMemPerBlockOptin, pic::max_smem_bytes());
     CUDA_TRY(pic::configure_kernels());
 
     char err[256] = "";
@@ -218,6 +224,8 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_leaves, sizeof(pic::Node) * nl);
     dmalloc((void**)&s->d_prims, sizeof(pic::Prim) * np);
     dmalloc((void**)&s->d_agents, sizeof(pic::AgentGeom) * n_agents);
+    dmalloc((void**)&s->d_cams, sizeof(pic::ViewCam) * n_agents * d->K);
+    dmalloc((void**)&s->d_tables, sizeof(float) * (size_t)d->K * ((size_t)d->W + 3 * (size_t)d->H));
     dmalloc((void**)&s->d_state, sizeof(float) * 4 * n_agents);
     dmalloc((void**)&s->d_dims, sizeof(float) * 3 * n_agents);
     dmalloc((void**)&s->d_active, n_agents);
@@ -259,8 +267,7 @@ pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
             if (value >= (uint64_t)s->E * s->A * s->K) return fail(PIC_ERR_INVALID_ARG, "first view out of range");
             s->view_first = (long long)value; return PIC_OK;
         case PIC_OPT_VIEW_COUNT: s->view_count = (long long)value; return PIC_OK;
-        case PIC_OPT_LIST_CAPS:
-            s->med_cap = (int)(value & 0xffffu); s->large_cap = (int)((value >> 16) & 0xffffu); return PIC_OK;
+        case PIC_OPT_DEBUG_FLAGS: s->debug_flags = (int)value; return PIC_OK;
         case PIC_OPT_TIMING: {
             if (value && !s->ev) {
                 DeviceGuard guard(s->device);
@@ -286,8 +293,8 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
     DeviceGuard guard(s->device);
     if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
     const int n_agents = s->E * s->A;
-    CUDA_TRY(pic::launch_agents(n_agents, poses, state, actions, dims, active, s->d_agents, s->d_status, kDt, kWheelbase,
-                                kVMax, stream));
+    CUDA_TRY(pic::launch_setup(P, n_agents, poses, state, actions, dims, active, s->d_agents, s->d_cams, s->d_tables,
+                               s->d_status, kDt, kWheelbase, kVMax, stream));
     const long long total = (long long)s->E * s->A * s->K;
     long long count = total - s->view_first;
     if (s->view_count > 0 && s->view_count < count) count = s->view_count;

@@ -1,0 +1,499 @@
+// Production render kernel of the batched egocentric rasterizer (sm_100a).
+//
+// One CTA of 128 threads renders one tile (up to 64 x 64 pixels) of one view.  The z-buffer lives
+// in shared memory as one 64-bit key per pixel,
+//     key = float_bits(1/z) << 32 | (0xFFFFFF - primitive index) << 8 | class,
+// so "nearest fragment wins, exact ties go to the lower index" is an unsigned max that does not
+// depend on the order in which primitives arrive; 0 means "no fragment" (background).
+//
+// Four phases separated by one barrier each:
+//   1 (a) cull      every warp tests the map's group boxes against the tile frustum, then takes
+//                   its share of the visible groups and tests their leaf boxes; visible leaves
+//                   are compacted into a list with warp ballots.  Other agents' boxes are culled as
+//                   spheres; only their camera-facing faces become items.
+//   2 (c) set-up    one thread per candidate (8 per visible leaf, 1 per face item): camera-space
+//                   vertices, pixel box, 3-4 edge functions + 1/z plane.  Primitives whose pixel
+//                   box holds <= 4 pixel centres are rasterized at once by their thread (atomic
+//                   max); the others leave a 17-word record.
+//   3 (b)+(c)       one warp per record: primitives covering many pixels first classify the
+//                   tile's 16 x 4 pixel cells (trivial reject / trivial accept from the same
+//                   float32 edge functions, two cells per lane), then the warp walks the surviving
+//                   cells, a lane per pixel pair, atomic max per fragment.
+//   4 (d) store     keys -> class u8 + depth binary16; a thread converts 16 pixels and issues
+//                   128-bit stores; 8 x 8 blocks no primitive touched are written without reading keys.
+//
+// Cameras (one 64-byte record per view) and per-camera ray / background tables are prepared by
+// the agent and rig kernels, so the prologue is a few loads.
+#include "pic_device.cuh"
+
+namespace pic {
+
+constexpr int NTHREADS = 128;
+constexpr int NW = NTHREADS / 32;
+constexpr int RCAP = 96;          // records (primitives rasterized by a warp) per tile
+constexpr int REC = 17;           // words per record
+constexpr int GROUP_BATCH = 16;   // groups examined per round
+constexpr int LEAFCAP = GROUP_BATCH * GROUP_LEAVES;   // visible leaves per round
+constexpr int BOX_ROUND = 64;     // boxes examined per round
+constexpr int FACECAP = 6 * BOX_ROUND;
+constexpr int TINY_MAX_PIXELS = 4;         // pixel centres in the box of a primitive rasterized by its own thread
+constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large classify cells before rasterizing
+
+struct __align__(16) TileSmem {
+    unsigned long long key[TILE * TILE];      // 32 KB, 16-byte chunks XOR-swizzled by row (key_index)
+    float rec[RCAP * REC];
+    uint32_t leaf[LEAFCAP];                   // visible leaves of the round: first primitive << 4 | count
+    uint32_t face[FACECAP];                   // box-face items of the round: agent << 3 | face
+    float ray_x[TILE], ray_y[TILE];           // ray coordinates of the tile's pixel columns / rows
+    float plane[6][4];                        // tile frustum, ego-relative world space, unit normals: n, offset
+    float side[4][4];                         // the four side planes in camera space, unit normals
+    Cam cam;
+    int n_rec, n_leaf, n_face;
+    uint32_t touched[2];                      // 8x8 blocks that may hold a fragment (rows 0-3, rows 4-7)
+    unsigned long long cnt[16];
+};
+
+// Keys are stored so that a 16 x 4 cell (raster) and 16-pixel row segments (store) spread over
+// all banks: the 16-byte chunk holding pixels (2c, 2c+1) of row y sits at chunk c ^ (y & 7).
+__device__ __forceinline__ int key_index(int x, int y) {
+    return (y << 6) | ((((x >> 1) ^ (y & 7)) << 1) | (x & 1));
+}
+
+// Bit mask of the 8x8 blocks touched by a pixel box (inclusive).
+__device__ __forceinline__ unsigned long long block_mask(int bx0, int by0, int bx1, int by1) {
+    const int c0 = bx0 >> 3, c1 = bx1 >> 3, r0 = by0 >> 3, r1 = by1 >> 3;
+    const unsigned long long row = (unsigned long long)(((2u << c1) - (1u << c0)) & 0xffu);
+    const unsigned long long rows = (0x0101010101010101ull >> (8 * (7 - (r1 - r0)))) << (8 * r0);
+    return row * rows;
+}
+
+__device__ __forceinline__ void mark_touched(TileSmem& s, unsigned long long m) {
+    const uint32_t lo = (uint32_t)m, hi = (uint32_t)(m >> 32);
+    if (lo & ~s.touched[0]) atomicOr(&s.touched[0], lo);
+    if (hi & ~s.touched[1]) atomicOr(&s.touched[1], hi);
+}
+
+// Is the box [lo,hi] (world) possibly inside the tile frustum?  Conservative.
+__device__ __forceinline__ bool box_visible(const TileSmem& s, const Node& b) {
+    const float ax = sub(b.lo[0], s.cam.px), bx = sub(b.hi[0], s.cam.px);
+    const float ay = sub(b.lo[1], s.cam.py), by = sub(b.hi[1], s.cam.py);
+    const float cx = 0.5f * (ax + bx), cy = 0.5f * (ay + by), cz = 0.5f * (b.lo[2] + b.hi[2]);
+    const float hx = 0.5f * (bx - ax), hy = 0.5f * (by - ay), hz = 0.5f * (b.hi[2] - b.lo[2]);
+    // rounding of the few float32 operations below, far under any real distance
+    const float slack = 1e-3f + 4e-6f * (fabsf(cx) + fabsf(cy) + fabsf(cz) + hx + hy + hz);
+    bool vis = true;
+#pragma unroll
+    for (int p = 0; p < 6; ++p) {
+        const float nx = s.plane[p][0], ny = s.plane[p][1], nz = s.plane[p][2], d = s.plane[p][3];
+        const float dist = nx * cx + ny * cy + nz * cz + d;
+        const float reach = fabsf(nx) * hx + fabsf(ny) * hy + fabsf(nz) * hz;
+        vis = vis && (dist + reach >= -slack);
+    }
+    return vis;
+}
+
+__device__ __forceinline__ void put_fragment(TileSmem& s, int x, int y, uint32_t wbits, uint32_t key_lo) {
+    const unsigned long long k = make_key(wbits, key_lo);
+    unsigned long long* addr = &s.key[key_index(x, y)];
+    if (k > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, k);
+}
+
+// Rasterize a primitive from one thread: loop over its pixel box, atomic max per fragment.
+__device__ __forceinline__ int raster_in_thread(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, uint32_t box) {
+    const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    int frags = 0;
+    for (int y = by0; y <= by1; ++y) {
+        const float ry = s.ray_y[y];
+        for (int x = bx0; x <= bx1; ++x) {
+            const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
+            if (wb) { put_fragment(s, x, y, wb, key_lo); ++frags; }
+        }
+    }
+    if (frags) mark_touched(s, block_mask(bx0, by0, bx1, by1));
+    return frags;
+}
+
+struct Tally { int grp, leaf, tested, setup, tiny, recs, fallback, classified, cells; };
+
+// Phase 2 body: cull one primitive against the tile, set it up, rasterize it or leave a record.
+__device__ __forceinline__ void process_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
+                                             uint32_t key_lo, int rec_cap, Tally& n) {
+    ++n.tested;
+    uint32_t box;
+    if (!pixel_box(s.cam, t, V, box)) return;
+    PrimEq q;
+    if (!prim_equations(V, quad, flags, q)) return;
+    ++n.setup;
+    const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    if ((bx1 - bx0 + 1) * (by1 - by0 + 1) > TINY_MAX_PIXELS) {
+        const int slot = atomicAdd(&s.n_rec, 1);
+        if (slot < rec_cap) {
+            float* r = &s.rec[slot * REC];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { r[i] = q.nx[i]; r[4 + i] = q.ny[i]; r[8 + i] = q.nz[i]; }
+            r[12] = q.wx; r[13] = q.wy; r[14] = q.wz;
+            r[15] = __uint_as_float(key_lo);
+            // the pixel box needs 6 bits per coordinate; the top-left bits ride along
+            r[16] = __uint_as_float((uint32_t)bx0 | ((uint32_t)by0 << 6) | ((uint32_t)bx1 << 12) | ((uint32_t)by1 << 18) | (q.tl << 24));
+            ++n.recs;
+            return;
+        }
+        ++n.fallback;          // list full: correct but slow
+    } else {
+        ++n.tiny;
+    }
+    raster_in_thread(s, t, q, key_lo, box);
+}
+
+// One 16 x 4 cell at (xx, yy): every lane tests its two pixels.  `inside`: the cell is known to
+// be covered and in range.  Returns whether any lane produced a fragment.
+__device__ __forceinline__ bool raster_cell(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, int xx, int yy,
+                                            bool inside, int lane) {
+    const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
+    const float rx0 = s.ray_x[x], rx1 = s.ray_x[x + 1], ry = s.ray_y[y];
+    const float wt = fm(q.wy, ry, q.wz);
+    const float w0 = fm(q.wx, rx0, wt), w1 = fm(q.wx, rx1, wt);
+    bool in0 = true, in1 = true;
+    if (!inside) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float te = fm(q.ny[e], ry, q.nz[e]);
+            const float e0 = fm(q.nx[e], rx0, te), e1 = fm(q.nx[e], rx1, te);
+            const bool own = (q.tl >> e) & 1u;
+            in0 = in0 && (e0 > 0.f || (e0 == 0.f && own));
+            in1 = in1 && (e1 > 0.f || (e1 == 0.f && own));
+        }
+        in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
+        in1 = in1 && (w1 >= t.w_far) && (w1 <= t.w_near);
+    }
+    if (in0 || in1) {
+        unsigned long long* addr = &s.key[key_index(x, y)];
+        ulonglong2 cur;
+        cur.x = *reinterpret_cast<volatile unsigned long long*>(addr);
+        cur.y = *reinterpret_cast<volatile unsigned long long*>(addr + 1);
+        const unsigned long long k0 = make_key(__float_as_uint(w0), key_lo), k1 = make_key(__float_as_uint(w1), key_lo);
+        if (in0 && k0 > cur.x) atomicMax(addr, k0);
+        if (in1 && k1 > cur.y) atomicMax(addr + 1, k1);
+    }
+    return __any_sync(0xffffffffu, in0 || in1);
+}
+
+// Phase 3: one warp per record.
+__device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool classify, Tally& n) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int p = warp; p < n_rec; p += NW) {
+        const float* r = &s.rec[p * REC];
+        PrimEq q;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { q.nx[i] = r[i]; q.ny[i] = r[4 + i]; q.nz[i] = r[8 + i]; }
+        q.wx = r[12]; q.wy = r[13]; q.wz = r[14];
+        const uint32_t key_lo = __float_as_uint(r[15]);
+        const uint32_t bw = __float_as_uint(r[16]);
+        q.tl = bw >> 24;
+        const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
+        unsigned long long touched = 0ull;     // 8x8 blocks
+        if (classify && (bx1 - bx0 + 1) * (by1 - by0 + 1) >= CLASSIFY_MIN_PIXELS) {
+            // (b) every lane classifies two of the tile's 64 cells: reject / partly covered / inside
+            ++n.classified;
+            unsigned any[2], full[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int cell = lane + 32 * h;
+                const int xa = (cell & 3) * 16, xb = xa + 15, ya = (cell >> 2) * 4, yb = ya + 3;
+                bool reject = xb < bx0 || xa > bx1 || yb < by0 || ya > by1;
+                bool inside = !reject;
+                if (!reject) {
+                    const float rxa = s.ray_x[xa], rxb = s.ray_x[xb], rya = s.ray_y[ya], ryb = s.ray_y[yb];   // rxa < rxb, rya < ryb
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        // fma is monotone in each argument, so the cell's extreme values are at its corners
+                        const float ta = fm(q.ny[e], rya, q.nz[e]), tb = fm(q.ny[e], ryb, q.nz[e]);
+                        const float emax = fm(q.nx[e], q.nx[e] >= 0.f ? rxb : rxa, fmaxf(ta, tb));
+                        const float emin = fm(q.nx[e], q.nx[e] >= 0.f ? rxa : rxb, fminf(ta, tb));
+                        reject = reject || (emax < 0.f);
+                        inside = inside && (emin > 0.f);
+                    }
+                    const float wa = fm(q.wy, rya, q.wz), wb = fm(q.wy, ryb, q.wz);
+                    const float wmax = fm(q.wx, q.wx >= 0.f ? rxb : rxa, fmaxf(wa, wb));
+                    const float wmin = fm(q.wx, q.wx >= 0.f ? rxa : rxb, fminf(wa, wb));
+                    reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
+                    inside = inside && (wmin >= t.w_far) && (wmax <= t.w_near);
+                }
+                any[h] = __ballot_sync(0xffffffffu, !reject);
+                full[h] = __ballot_sync(0xffffffffu, !reject && inside);
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                for (unsigned m = any[h]; m; m &= m - 1) {
+                    const int cell = __ffs(m) - 1 + 32 * h;
+                    const int xx = (cell & 3) * 16, yy = (cell >> 2) * 4;
+                    ++n.cells;
+                    if (raster_cell(s, t, q, key_lo, xx, yy, (full[h] >> (cell & 31)) & 1u, lane))
+                        touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
+                }
+        } else {
+            for (int yy = by0 & ~3; yy <= by1; yy += 4)
+                for (int xx = bx0 & ~15; xx <= bx1; xx += 16) {
+                    ++n.cells;
+                    if (raster_cell(s, t, q, key_lo, xx, yy, false, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
+                }
+        }
+        if (lane == 0 && touched) mark_touched(s, touched);
+    }
+}
+
+// (d) keys -> class / depth images.
+__device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderParams& P, size_t view, int k, bool ego_active) {
+    const size_t img = (size_t)P.H * P.W;
+    uint8_t* oc = P.out_class + view * img;
+    uint16_t* od = P.out_depth + view * img;
+    float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
+    const bool vec_ok = (P.W % 16 == 0) && o32 == nullptr;
+    const unsigned long long touched = ((unsigned long long)s.touched[1] << 32) | s.touched[0];
+    const int segs_per_row = (t.tw + 15) >> 4;
+    const int n_seg = t.th * segs_per_row;
+    for (int seg = threadIdx.x; seg < n_seg; seg += NTHREADS) {
+        const int y = (segs_per_row == 4) ? (seg >> 2) : seg / segs_per_row;
+        const int xs = (seg - y * segs_per_row) * 16;
+        uint32_t bg_cls = P.cls_sky;
+        float bg_z = P.far_z;
+        if (ego_active) { bg_cls = __ldg(P.rig.bg_cls + (size_t)k * P.H + t.y0 + y); bg_z = __ldg(P.rig.bg_z + (size_t)k * P.H + t.y0 + y); }
+        const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + xs;
+        const bool empty = ((touched >> ((y >> 3) * 8 + (xs >> 3))) & 3ull) == 0ull;   // both blocks of the segment
+        if (vec_ok && xs + 16 <= t.tw) {
+            uint32_t cw[4], dw[8];
+            if (empty) {
+                const uint32_t c4 = bg_cls * 0x01010101u;
+                const __half2 h = __floats2half2_rn(bg_z, bg_z);
+                const uint32_t d2 = *reinterpret_cast<const uint32_t*>(&h);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) cw[j] = c4;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) dw[j] = d2;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(&s.key[key_index(xs + j, y)]);
+                    const float z0 = kk.x ? fast_rcp(__uint_as_float((uint32_t)(kk.x >> 32))) : bg_z;
+                    const float z1 = kk.y ? fast_rcp(__uint_as_float((uint32_t)(kk.y >> 32))) : bg_z;
+                    const uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bg_cls, c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bg_cls;
+                    const __half2 h = __floats2half2_rn(z0, z1);
+                    dw[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                    if ((j & 3) == 0) cw[j >> 2] = c0 | (c1 << 8); else cw[j >> 2] |= (c0 << 16) | (c1 << 24);
+                }
+            }
+            *reinterpret_cast<uint4*>(oc + o) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            *reinterpret_cast<uint4*>(od + o) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
+            *reinterpret_cast<uint4*>(od + o + 8) = make_uint4(dw[4], dw[5], dw[6], dw[7]);
+        } else {
+            for (int j = 0; j < 16 && xs + j < t.tw; ++j) {
+                const unsigned long long key = empty ? 0ull : s.key[key_index(xs + j, y)];
+                const float z = key ? fast_rcp(__uint_as_float((uint32_t)(key >> 32))) : bg_z;
+                oc[o + j] = (uint8_t)(key ? (uint32_t)(key & 0xff) : bg_cls);
+                od[o + j] = __half_as_ushort(__float2half_rn(z));
+                if (o32) o32[o + j] = z;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& s = *reinterpret_cast<TileSmem*>(smem_raw);
+    const int tiles = P.tiles_x * P.tiles_y;
+    const long long job = blockIdx.x;
+    const size_t view = (size_t)(P.view_first + job / tiles);
+    const int tile = (int)(job % tiles);
+    const int k = (int)(view % P.K);
+    const int a = (int)((view / P.K) % P.A);
+    const int e = (int)(view / ((size_t)P.K * P.A));
+    TileCtx t;
+    t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
+    t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
+    t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool ego_active = P.agents[(size_t)e * P.A + a].active != 0;
+    const bool classify = !(P.debug_flags & 1);
+    const int rec_cap = (P.debug_flags & 2) ? 2 : RCAP;
+    Tally n = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+
+    // ---- prologue: camera, ray tables, frustum planes, cleared keys
+    if (threadIdx.x < 7) {
+        Cam c;
+        load_camera(c, P.cams[view], P.cam[k], P.W, P.H);
+        if (threadIdx.x == 6) {
+            s.cam = c;
+            s.n_rec = 0; s.n_leaf = 0; s.n_face = 0;
+            s.touched[0] = 0u; s.touched[1] = 0u;
+        } else {
+            // frustum planes n.(q - m_w) >= 0 with q = X - P_ego; unit normals, offset -n.m_w (+ near/far)
+            const int p = threadIdx.x;
+            const float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
+            float nx, ny, nz, off = 0.f, sx = 0.f, sy = 0.f, sz = 0.f;
+            const float Rx = c.rx, Ry = c.ry, Dx = c.dx, Dy = c.dy, Dz = c.dz, Fx = c.fx_, Fy = c.fy_, Fz = c.fz_;
+            switch (p) {
+                case 0: nx = Fx; ny = Fy; nz = Fz; off = -P.near_z * 0.999f; break;                                       // z >= near
+                case 1: nx = -Fx; ny = -Fy; nz = -Fz; off = P.far_z * 1.001f; break;                                      // z <= far
+                case 2: nx = c.focx * Rx - l * Fx; ny = c.focx * Ry - l * Fy; nz = -l * Fz; sx = c.focx; sz = -l; break;  // x f >= z l
+                case 3: nx = r * Fx - c.focx * Rx; ny = r * Fy - c.focx * Ry; nz = r * Fz; sx = -c.focx; sz = r; break;   // x f <= z r
+                case 4: nx = c.focy * Dx - u * Fx; ny = c.focy * Dy - u * Fy; nz = c.focy * Dz - u * Fz; sy = c.focy; sz = -u; break;
+                default: nx = d * Fx - c.focy * Dx; ny = d * Fy - c.focy * Dy; nz = d * Fz - c.focy * Dz; sy = -c.focy; sz = d; break;
+            }
+            const float inv = rsqrtf(nx * nx + ny * ny + nz * nz);
+            nx *= inv; ny *= inv; nz *= inv;
+            s.plane[p][0] = nx; s.plane[p][1] = ny; s.plane[p][2] = nz;
+            s.plane[p][3] = off - (nx * c.mwx + ny * c.mwy + nz * c.mwz);
+            if (p >= 2) {
+                const float is = rsqrtf(sx * sx + sy * sy + sz * sz);
+                s.side[p - 2][0] = sx * is; s.side[p - 2][1] = sy * is; s.side[p - 2][2] = sz * is; s.side[p - 2][3] = 0.f;
+            }
+        }
+    } else if (threadIdx.x >= 32 && threadIdx.x < 48) {
+        s.cnt[threadIdx.x - 32] = 0ull;
+    } else if (threadIdx.x >= 64) {
+        // columns / rows past the image edge (ragged tiles) continue the same formula, so the
+        // tables stay monotone for the cell classification
+        const int i = threadIdx.x - 64;
+        const CamConst& ck = P.cam[k];
+        s.ray_x[i] = (t.x0 + i < P.W) ? __ldg(P.rig.ray_x + (size_t)k * P.W + t.x0 + i)
+                                      : __fdiv_rn(sub(add((float)(t.x0 + i), 0.5f), 0.5f * (float)P.W), ck.fx);
+        s.ray_y[i] = (t.y0 + i < P.H) ? __ldg(P.rig.ray_y + (size_t)k * P.H + t.y0 + i)
+                                      : __fdiv_rn(sub(add((float)(t.y0 + i), 0.5f), 0.5f * (float)P.H), ck.fy);
+    }
+    for (int i = threadIdx.x; i < TILE * TILE / 2; i += NTHREADS)
+        reinterpret_cast<ulonglong2*>(s.key)[i] = make_ulonglong2(0ull, 0ull);
+    __syncthreads();
+
+    if (ego_active) {
+        const Cam& c = s.cam;
+        const MapInfo mi = P.maps[P.env_map[e]];
+        const uint32_t n_groups = mi.group_end - mi.group_begin;
+        const int n_rounds = max((int)((n_groups + GROUP_BATCH - 1) / GROUP_BATCH), (P.A + BOX_ROUND - 1) / BOX_ROUND);
+        for (int round = 0; round < n_rounds; ++round) {
+            // ---- phase 1 (a): hierarchy and boxes of this round
+            const uint32_t g0 = mi.group_begin + (uint32_t)round * GROUP_BATCH;
+            if (g0 < mi.group_end) {
+                const uint32_t g = g0 + lane;
+                bool vis = false;
+                Node gn;
+                if (lane < GROUP_BATCH && g < mi.group_end) { gn = P.groups[g]; vis = box_visible(s, gn); if (warp == 0) ++n.grp; }
+                unsigned gm = __ballot_sync(0xffffffffu, vis);
+                // warp w takes the visible groups w, w + NW, ...
+                for (int i = 0; gm; gm &= gm - 1, ++i) {
+                    if ((i & (NW - 1)) != warp) continue;
+                    const int src = __ffs(gm) - 1;
+                    const uint32_t first = __shfl_sync(0xffffffffu, gn.first, src);
+                    const uint32_t cnt = __shfl_sync(0xffffffffu, gn.count, src);
+                    bool lvis = false;
+                    Node lf;
+                    if (lane < (int)cnt) { lf = P.leaves[first + lane]; lvis = box_visible(s, lf); ++n.leaf; }
+                    const unsigned lm = __ballot_sync(0xffffffffu, lvis);
+                    int base = 0;
+                    if (lane == 0 && lm) base = atomicAdd(&s.n_leaf, __popc(lm));
+                    base = __shfl_sync(0xffffffffu, base, 0);
+                    if (lvis) s.leaf[base + __popc(lm & ((1u << lane) - 1u))] = (lf.first << 4) | lf.count;
+                }
+            }
+            for (int b = round * BOX_ROUND + threadIdx.x; b < min(P.A, (round + 1) * BOX_ROUND); b += NTHREADS) {
+                if (b == a) continue;
+                const AgentGeom g = P.agents[(size_t)e * P.A + b];
+                if (!g.active) continue;
+                const float hh = 0.5f * g.h;
+                const V3 ctr = rotate_to_camera(c, sub(sub(g.x, c.px), c.mwx), sub(sub(g.y, c.py), c.mwy), sub(hh, c.mwz));
+                const float rad = sqrtf(g.hl * g.hl + g.hw * g.hw + hh * hh) * 1.0001f + 1e-4f;
+                bool vis = (ctr.z + rad >= t.near_z * 0.999f) && (ctr.z - rad <= t.far_z * 1.001f);
+#pragma unroll
+                for (int p = 0; p < 4; ++p)
+                    vis = vis && (s.side[p][0] * ctr.x + s.side[p][1] * ctr.y + s.side[p][2] * ctr.z >= -rad);
+                if (!vis) continue;
+                // the camera position in the box frame decides which faces can face the camera;
+                // near the near plane (or inside the box) every face is kept
+                uint32_t faces = 0x3fu;
+                if (ctr.z - rad > t.near_z * 1.01f) {
+                    const float dx = sub(c.mwx, sub(g.x, c.px)), dy = sub(c.mwy, sub(g.y, c.py));
+                    const float u = g.c * dx + g.s * dy, v = g.c * dy - g.s * dx;
+                    const float eps = 1e-4f * (1.f + fabsf(dx) + fabsf(dy));
+                    faces = 0u;
+                    if (u < -g.hl + eps) faces |= 1u;          // rear
+                    if (u > g.hl - eps) faces |= 2u;           // front
+                    if (v < -g.hw + eps) faces |= 4u;          // right
+                    if (v > g.hw - eps) faces |= 8u;           // left
+                    if (c.mwz < eps) faces |= 16u;             // bottom
+                    if (c.mwz > g.h - eps) faces |= 32u;       // top
+                }
+                int slot = atomicAdd(&s.n_face, __popc(faces));
+                for (; faces; faces &= faces - 1) s.face[slot++] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
+            }
+            __syncthreads();
+            // ---- phase 2 (c): one thread per candidate primitive
+            const int nl = s.n_leaf, nf = s.n_face;
+            const int n_items = nl * LEAF_PRIMS + nf;
+            for (int i = threadIdx.x; i < n_items; i += NTHREADS) {
+                V3 V[4];
+                uint32_t key_lo, flags;
+                if (i < nl * LEAF_PRIMS) {
+                    const uint32_t lf = s.leaf[i / LEAF_PRIMS];
+                    const uint32_t j = i % LEAF_PRIMS;
+                    if (j >= (lf & 15u)) continue;
+                    float v[12];
+                    load_prim(P.prims + (lf >> 4) + j, v, key_lo, flags);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
+                } else {
+                    const uint32_t it = s.face[i - nl * LEAF_PRIMS];
+                    const int b = (int)(it >> 3), f = (int)(it & 7u);
+                    const AgentGeom g = P.agents[(size_t)e * P.A + b];
+                    const uint32_t corners = face_corners(f);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
+                    key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+                    flags = face_flags(corners);
+                }
+                process_prim(s, t, V, flags & 1u, flags, key_lo, rec_cap, n);
+            }
+            __syncthreads();
+            if (round + 1 < n_rounds) {
+                // the lists are reused by the next round; records are rasterized now if they might overflow
+                const int n_rec = min(s.n_rec, rec_cap);
+                if (n_rec > rec_cap / 2) raster_records(s, t, n_rec, classify, n);
+                __syncthreads();
+                if (threadIdx.x == 0) { s.n_leaf = 0; s.n_face = 0; if (n_rec > rec_cap / 2) s.n_rec = 0; }
+                __syncthreads();
+            }
+        }
+        // ---- phase 3 (b)+(c): one warp per record
+        raster_records(s, t, min(s.n_rec, rec_cap), classify, n);
+        __syncthreads();
+    }
+    // ---- phase 4 (d)
+    store_tile(s, t, P, view, k, ego_active);
+    if (P.counters) {
+        const int vals[9] = {n.grp, n.leaf, n.tested, n.setup, n.tiny, n.recs, n.fallback, n.classified, n.cells};
+#pragma unroll
+        for (int i = 0; i < 9; ++i) {
+            // classified / cells are counted by every lane of a warp alike
+            const int v = (i >= 7 && lane != 0) ? 0 : vals[i];
+            const int sum = __reduce_add_sync(0xffffffffu, v);
+            if (lane == 0 && sum) atomicAdd(&s.cnt[1 + i], (unsigned long long)sum);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s.cnt[0] = 1;
+        __syncthreads();
+        if (threadIdx.x < 16 && s.cnt[threadIdx.x]) atomicAdd(&P.counters[threadIdx.x], s.cnt[threadIdx.x]);
+    }
+}
+
+size_t render_smem_bytes() { return sizeof(TileSmem); }
+
+cudaError_t configure_render_kernel() {
+    return cudaFuncSetAttribute(render_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+}
+
+cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, cudaStream_t stream) {
+    const long long blocks = n_views * P.tiles_x * P.tiles_y;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    render_kernel<<<(unsigned)blocks, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    return cudaGetLastError();
+}
+
+}  // namespace pic

@@ -5,7 +5,6 @@
 namespace pic {
 
 constexpr int TILE = 64;        // a view is rendered in tiles of up to TILE x TILE pixels (one CTA each)
-constexpr int NTHREADS = 128;   // threads per render CTA
 constexpr int MAX_CAMS = 16;    // cameras per rig
 constexpr int LEAF_PRIMS = 8;   // primitives per leaf (8 threads per leaf in the cull pass)
 constexpr int LONG_LEAF_PRIMS = 8;   // long primitives get leaves of their own so the others' boxes stay tight
@@ -52,6 +51,26 @@ struct CamConst {
     float fx, fy;
 };
 
+// Per-view camera written by the agent kernel: ego position, mount and rotation rows; 64 bytes.
+struct ViewCam {
+    float px, py;              // ego position
+    float mwx, mwy, mwz;       // mount in world axes
+    float rx, ry;              // right   (rz = 0)
+    float dx, dy, dz;          // down
+    float fx, fy, fz;          // forward
+    float pad[3];
+};
+static_assert(sizeof(ViewCam) == 64, "ViewCam must be 64 bytes");
+
+// Per-camera tables shared by all views of a call: ray coordinates of pixel columns / rows and the
+// background (analytic ground plane / sky) of every row.
+struct RigTables {
+    const float* ray_x;        // [K][W]
+    const float* ray_y;        // [K][H]
+    const float* bg_z;         // [K][H] background depth
+    const uint32_t* bg_cls;    // [K][H] background class
+};
+
 struct RenderParams {
     int32_t E, A, K, H, W;
     int32_t tiles_x, tiles_y;
@@ -64,11 +83,13 @@ struct RenderParams {
     const Node* leaves;
     const Prim* prims;
     const AgentGeom* agents;
+    const ViewCam* cams;            // [E*A*K]
+    RigTables rig;
     uint8_t* out_class;
     uint16_t* out_depth;
     float* out_depth32;             // optional
     unsigned long long* counters;   // optional [16]
-    int32_t med_cap, large_cap;     // usable entries of the medium / large lists (debug: shrink to force the fallback)
+    int32_t debug_flags;            // bit 0: no per-cell trivial accept/reject, bit 1: record list of 2 entries (forces the overflow path)
     long long view_first;           // render views [view_first, view_first + gridDim / tiles)
     CamConst cam[MAX_CAMS];
 };

@@ -23,7 +23,7 @@ class GpuRun:
         self.active = torch.from_numpy(np.ascontiguousarray(s.active)).to(self.dev)
 
     def render(self, brute: bool = False, depth32: bool = True, poses=None, view_first: int = 0, view_count: int = 0,
-               counters: bool = False, list_caps=None):
+               counters: bool = False, debug_flags: int = 0):
         """Returns (class u8 [V,H,W], depth f16 [V,H,W], depth32 f32 [V,H,W] or None[, counters]) as numpy."""
         torch, pic, s = self.torch, self.pic, self.s
         cls, dep = self.scene.alloc_outputs()
@@ -36,8 +36,7 @@ class GpuRun:
         self.scene.set_option(pic.OPT_COUNTERS, cnt if counters else 0)
         self.scene.set_option(pic.OPT_VIEW_FIRST, view_first)
         self.scene.set_option(pic.OPT_VIEW_COUNT, view_count)
-        if list_caps is not None:
-            self.scene.set_option(pic.OPT_LIST_CAPS, int(list_caps[0]) | (int(list_caps[1]) << 16))
+        self.scene.set_option(pic.OPT_DEBUG_FLAGS, int(debug_flags))
         p = self.poses if poses is None else torch.from_numpy(np.ascontiguousarray(poses, dtype=np.float32)).to(self.dev)
         self.scene.render(p, self.dims, s.rig, active=self.active, out_class=cls, out_depth=dep)
         torch.cuda.synchronize()
@@ -46,7 +45,7 @@ class GpuRun:
         self.scene.set_option(pic.OPT_BRUTE_FORCE, 0)
         self.scene.set_option(pic.OPT_VIEW_FIRST, 0)
         self.scene.set_option(pic.OPT_VIEW_COUNT, 0)
-        self.scene.set_option(pic.OPT_LIST_CAPS, 0xffff | (0xffff << 16))
+        self.scene.set_option(pic.OPT_DEBUG_FLAGS, 0)
         V = s.E * s.A * s.K
         out = (cls.cpu().numpy().reshape(V, s.H, s.W), dep.cpu().numpy().reshape(V, s.H, s.W),
                d32.cpu().numpy().reshape(V, s.H, s.W) if depth32 else None)
