@@ -152,6 +152,8 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *   PIC_OPT_DEBUG_FLAGS   bit 0: rasterize large primitives without the per-cell trivial
  *                         accept/reject; bit 1: shrink the per-tile record list to 2 entries so that
  *                         the overflow path runs.  Both leave the images unchanged (tests rely on it).
+ *                         Bits 4-7: leave the render kernel after phase n = 1..3 (profiling aid;
+ *                         the images are then incomplete).
  *   PIC_OPT_TIMING        1: bracket every render-kernel launch with CUDA events on its stream
  *                         (up to 1024 launches between two pic_get_kernel_times calls); 0: off.
  *                         Turning it on creates the events (allocates), so do it outside timed code.

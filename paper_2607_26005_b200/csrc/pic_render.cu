@@ -30,12 +30,13 @@ namespace pic {
 
 constexpr int NTHREADS = 128;
 constexpr int NW = NTHREADS / 32;
-constexpr int RCAP = 96;          // records (primitives rasterized by a warp) per tile
+constexpr int RCAP = 64;          // records (primitives rasterized by a warp) per tile
 constexpr int REC = 17;           // words per record
 constexpr int GROUP_BATCH = 16;   // groups examined per round
 constexpr int LEAFCAP = GROUP_BATCH * GROUP_LEAVES;   // visible leaves per round
 constexpr int BOX_ROUND = 64;     // boxes examined per round
 constexpr int FACECAP = 6 * BOX_ROUND;
+constexpr int SCAP = 128;         // candidates that survive the pixel-box test, per round
 constexpr int TINY_MAX_PIXELS = 4;         // pixel centres in the box of a primitive rasterized by its own thread
 constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large classify cells before rasterizing
 
@@ -44,13 +45,13 @@ struct __align__(16) TileSmem {
     float rec[RCAP * REC];
     uint32_t leaf[LEAFCAP];                   // visible leaves of the round: first primitive << 4 | count
     uint32_t face[FACECAP];                   // box-face items of the round: agent << 3 | face
+    uint2 surv[SCAP];                         // candidates whose pixel box holds a pixel centre: (item, box)
     float ray_x[TILE], ray_y[TILE];           // ray coordinates of the tile's pixel columns / rows
     float plane[6][4];                        // tile frustum, ego-relative world space, unit normals: n, offset
     float side[4][4];                         // the four side planes in camera space, unit normals
     Cam cam;
-    int n_rec, n_leaf, n_face;
+    int n_rec, n_leaf, n_face, n_surv;
     uint32_t touched[2];                      // 8x8 blocks that may hold a fragment (rows 0-3, rows 4-7)
-    unsigned long long cnt[16];
 };
 
 // Keys are stored so that a 16 x 4 cell (raster) and 16-pixel row segments (store) spread over
@@ -115,12 +116,9 @@ __device__ __forceinline__ int raster_in_thread(TileSmem& s, const TileCtx& t, c
 
 struct Tally { int grp, leaf, tested, setup, tiny, recs, fallback, classified, cells; };
 
-// Phase 2 body: cull one primitive against the tile, set it up, rasterize it or leave a record.
-__device__ __forceinline__ void process_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
-                                             uint32_t key_lo, int rec_cap, Tally& n) {
-    ++n.tested;
-    uint32_t box;
-    if (!pixel_box(s.cam, t, V, box)) return;
+// Phase 2b body: set a surviving primitive up, rasterize it (tiny) or leave a record.
+__device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
+                                           uint32_t key_lo, uint32_t box, int rec_cap, Tally& n) {
     PrimEq q;
     if (!prim_equations(V, quad, flags, q)) return;
     ++n.setup;
@@ -145,8 +143,34 @@ __device__ __forceinline__ void process_prim(TileSmem& s, const TileCtx& t, cons
     raster_in_thread(s, t, q, key_lo, box);
 }
 
-// One 16 x 4 cell at (xx, yy): every lane tests its two pixels.  `inside`: the cell is known to
-// be covered and in range.  Returns whether any lane produced a fragment.
+// Candidate `i` of the round: a primitive of a visible leaf or a box-face item, in camera space.
+__device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderParams& P, int i, int nl, int e, uint32_t n_map_tris,
+                                                V3 (&V)[4], uint32_t& key_lo, uint32_t& flags) {
+    const Cam& c = s.cam;
+    if (i < nl * LEAF_PRIMS) {
+        const uint32_t lf = s.leaf[i / LEAF_PRIMS];
+        const uint32_t j = i % LEAF_PRIMS;
+        if (j >= (lf & 15u)) return false;
+        float v[12];
+        load_prim(P.prims + (lf >> 4) + j, v, key_lo, flags);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
+    } else {
+        const uint32_t it = s.face[i - nl * LEAF_PRIMS];
+        const int b = (int)(it >> 3), f = (int)(it & 7u);
+        const AgentGeom g = P.agents[(size_t)e * P.A + b];
+        const uint32_t corners = face_corners(f);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
+        key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+        flags = face_flags(corners);
+    }
+    return true;
+}
+
+// One 16 x 4 cell at (xx, yy): every lane tests its two pixels and updates their keys with plain
+// loads and stores -- in phase 3 the rows of a cell belong to exactly one warp.  `inside`: the
+// cell is known to be covered and in range.  Returns whether any lane produced a fragment.
 __device__ __forceinline__ bool raster_cell(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, int xx, int yy,
                                             bool inside, int lane) {
     const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
@@ -167,79 +191,76 @@ __device__ __forceinline__ bool raster_cell(TileSmem& s, const TileCtx& t, const
         in1 = in1 && (w1 >= t.w_far) && (w1 <= t.w_near);
     }
     if (in0 || in1) {
-        unsigned long long* addr = &s.key[key_index(x, y)];
-        ulonglong2 cur;
-        cur.x = *reinterpret_cast<volatile unsigned long long*>(addr);
-        cur.y = *reinterpret_cast<volatile unsigned long long*>(addr + 1);
+        ulonglong2* kp = reinterpret_cast<ulonglong2*>(&s.key[key_index(x, y)]);
+        ulonglong2 kk = *kp;
         const unsigned long long k0 = make_key(__float_as_uint(w0), key_lo), k1 = make_key(__float_as_uint(w1), key_lo);
-        if (in0 && k0 > cur.x) atomicMax(addr, k0);
-        if (in1 && k1 > cur.y) atomicMax(addr + 1, k1);
+        if (in0 && k0 > kk.x) kk.x = k0;
+        if (in1 && k1 > kk.y) kk.y = k1;
+        *kp = kk;
     }
     return __any_sync(0xffffffffu, in0 || in1);
 }
 
-// Phase 3: one warp per record.
+// Phase 3: every warp walks all records but rasterizes only the bands (4 pixel rows) it owns --
+// band b belongs to warp b % NW -- so keys are updated without atomics and the bands of a large
+// primitive are shared out evenly.
 __device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool classify, Tally& n) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int p = warp; p < n_rec; p += NW) {
+    unsigned long long touched = 0ull;     // 8x8 blocks
+    for (int p = 0; p < n_rec; ++p) {
         const float* r = &s.rec[p * REC];
+        const uint32_t bw = __float_as_uint(r[16]);
+        const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
+        // first band of this warp at or after the box's first band
+        const int band0 = by0 >> 2, band1 = by1 >> 2;
+        int first = band0 + ((warp - band0) & (NW - 1));
+        if (first > band1) continue;
         PrimEq q;
 #pragma unroll
         for (int i = 0; i < 4; ++i) { q.nx[i] = r[i]; q.ny[i] = r[4 + i]; q.nz[i] = r[8 + i]; }
         q.wx = r[12]; q.wy = r[13]; q.wz = r[14];
         const uint32_t key_lo = __float_as_uint(r[15]);
-        const uint32_t bw = __float_as_uint(r[16]);
         q.tl = bw >> 24;
-        const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
-        unsigned long long touched = 0ull;     // 8x8 blocks
         if (classify && (bx1 - bx0 + 1) * (by1 - by0 + 1) >= CLASSIFY_MIN_PIXELS) {
-            // (b) every lane classifies two of the tile's 64 cells: reject / partly covered / inside
-            ++n.classified;
-            unsigned any[2], full[2];
+            // (b) lanes 0..15 classify this warp's 16 cells: reject / partly covered / inside
+            if (warp == 0) ++n.classified;
+            const int band = (lane >> 2) * NW + warp, col = lane & 3;
+            const int xa = col * 16, xb = xa + 15, ya = band * 4, yb = ya + 3;
+            bool reject = lane >= 16 || xb < bx0 || xa > bx1 || yb < by0 || ya > by1;
+            bool inside = !reject;
+            if (!reject) {
+                const float rxa = s.ray_x[xa], rxb = s.ray_x[xb], rya = s.ray_y[ya], ryb = s.ray_y[yb];   // rxa < rxb, rya < ryb
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int cell = lane + 32 * h;
-                const int xa = (cell & 3) * 16, xb = xa + 15, ya = (cell >> 2) * 4, yb = ya + 3;
-                bool reject = xb < bx0 || xa > bx1 || yb < by0 || ya > by1;
-                bool inside = !reject;
-                if (!reject) {
-                    const float rxa = s.ray_x[xa], rxb = s.ray_x[xb], rya = s.ray_y[ya], ryb = s.ray_y[yb];   // rxa < rxb, rya < ryb
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        // fma is monotone in each argument, so the cell's extreme values are at its corners
-                        const float ta = fm(q.ny[e], rya, q.nz[e]), tb = fm(q.ny[e], ryb, q.nz[e]);
-                        const float emax = fm(q.nx[e], q.nx[e] >= 0.f ? rxb : rxa, fmaxf(ta, tb));
-                        const float emin = fm(q.nx[e], q.nx[e] >= 0.f ? rxa : rxb, fminf(ta, tb));
-                        reject = reject || (emax < 0.f);
-                        inside = inside && (emin > 0.f);
-                    }
-                    const float wa = fm(q.wy, rya, q.wz), wb = fm(q.wy, ryb, q.wz);
-                    const float wmax = fm(q.wx, q.wx >= 0.f ? rxb : rxa, fmaxf(wa, wb));
-                    const float wmin = fm(q.wx, q.wx >= 0.f ? rxa : rxb, fminf(wa, wb));
-                    reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
-                    inside = inside && (wmin >= t.w_far) && (wmax <= t.w_near);
+                for (int e = 0; e < 4; ++e) {
+                    // fma is monotone in each argument, so the cell's extreme values are at its corners
+                    const float ta = fm(q.ny[e], rya, q.nz[e]), tb = fm(q.ny[e], ryb, q.nz[e]);
+                    const float emax = fm(q.nx[e], q.nx[e] >= 0.f ? rxb : rxa, fmaxf(ta, tb));
+                    const float emin = fm(q.nx[e], q.nx[e] >= 0.f ? rxa : rxb, fminf(ta, tb));
+                    reject = reject || (emax < 0.f);
+                    inside = inside && (emin > 0.f);
                 }
-                any[h] = __ballot_sync(0xffffffffu, !reject);
-                full[h] = __ballot_sync(0xffffffffu, !reject && inside);
+                const float wa = fm(q.wy, rya, q.wz), wb = fm(q.wy, ryb, q.wz);
+                const float wmax = fm(q.wx, q.wx >= 0.f ? rxb : rxa, fmaxf(wa, wb));
+                const float wmin = fm(q.wx, q.wx >= 0.f ? rxa : rxb, fminf(wa, wb));
+                reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
+                inside = inside && (wmin >= t.w_far) && (wmax <= t.w_near);
             }
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-                for (unsigned m = any[h]; m; m &= m - 1) {
-                    const int cell = __ffs(m) - 1 + 32 * h;
-                    const int xx = (cell & 3) * 16, yy = (cell >> 2) * 4;
-                    ++n.cells;
-                    if (raster_cell(s, t, q, key_lo, xx, yy, (full[h] >> (cell & 31)) & 1u, lane))
-                        touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
-                }
+            const unsigned full = __ballot_sync(0xffffffffu, !reject && inside);
+            for (unsigned m = __ballot_sync(0xffffffffu, !reject); m; m &= m - 1) {
+                const int cell = __ffs(m) - 1;
+                const int xx = (cell & 3) * 16, yy = ((cell >> 2) * NW + warp) * 4;
+                ++n.cells;
+                if (raster_cell(s, t, q, key_lo, xx, yy, (full >> cell) & 1u, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
+            }
         } else {
-            for (int yy = by0 & ~3; yy <= by1; yy += 4)
+            for (int band = first; band <= band1; band += NW)
                 for (int xx = bx0 & ~15; xx <= bx1; xx += 16) {
                     ++n.cells;
-                    if (raster_cell(s, t, q, key_lo, xx, yy, false, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
+                    if (raster_cell(s, t, q, key_lo, xx, band * 4, false, lane)) touched |= 3ull << ((band >> 1) * 8 + (xx >> 3));
                 }
         }
-        if (lane == 0 && touched) mark_touched(s, touched);
     }
+    if (lane == 0 && touched) mark_touched(s, touched);
 }
 
 // (d) keys -> class / depth images.
@@ -301,21 +322,32 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& s = *reinterpret_cast<TileSmem*>(smem_raw);
     const int tiles = P.tiles_x * P.tiles_y;
-    const long long job = blockIdx.x;
-    const size_t view = (size_t)(P.view_first + job / tiles);
-    const int tile = (int)(job % tiles);
-    const int k = (int)(view % P.K);
-    const int a = (int)((view / P.K) % P.A);
-    const int e = (int)(view / ((size_t)P.K * P.A));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool classify = !(P.debug_flags & 1);
+    const int rec_cap = (P.debug_flags & 2) ? 2 : RCAP;
+    const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave after phase `stop` (image incomplete)
+    Tally n = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    // grid: x = tile + tiles * camera, y = agent, z = env; a 1-D grid (gridDim.y == 0 is impossible,
+    // so "linear" is flagged by P.linear) serves view sub-ranges
+    int tile, k, a, e;
+    if (P.linear) {
+        const unsigned job = blockIdx.x;
+        const unsigned v = (unsigned)P.view_first + job / (unsigned)tiles;
+        tile = (int)(job % (unsigned)tiles);
+        k = (int)(v % (unsigned)P.K);
+        a = (int)((v / (unsigned)P.K) % (unsigned)P.A);
+        e = (int)(v / ((unsigned)P.K * (unsigned)P.A));
+    } else {
+        k = (int)(blockIdx.x / (unsigned)tiles);
+        tile = (int)(blockIdx.x - (unsigned)k * (unsigned)tiles);
+        a = (int)blockIdx.y; e = (int)blockIdx.z;
+    }
+    const size_t view = ((size_t)e * P.A + a) * P.K + k;
     TileCtx t;
     t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
     t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
     t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool ego_active = P.agents[(size_t)e * P.A + a].active != 0;
-    const bool classify = !(P.debug_flags & 1);
-    const int rec_cap = (P.debug_flags & 2) ? 2 : RCAP;
-    Tally n = {0, 0, 0, 0, 0, 0, 0, 0, 0};
 
     // ---- prologue: camera, ray tables, frustum planes, cleared keys
     if (threadIdx.x < 7) {
@@ -323,7 +355,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         load_camera(c, P.cams[view], P.cam[k], P.W, P.H);
         if (threadIdx.x == 6) {
             s.cam = c;
-            s.n_rec = 0; s.n_leaf = 0; s.n_face = 0;
+            s.n_rec = 0; s.n_leaf = 0; s.n_face = 0; s.n_surv = 0;
             s.touched[0] = 0u; s.touched[1] = 0u;
         } else {
             // frustum planes n.(q - m_w) >= 0 with q = X - P_ego; unit normals, offset -n.m_w (+ near/far)
@@ -348,8 +380,6 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                 s.side[p - 2][0] = sx * is; s.side[p - 2][1] = sy * is; s.side[p - 2][2] = sz * is; s.side[p - 2][3] = 0.f;
             }
         }
-    } else if (threadIdx.x >= 32 && threadIdx.x < 48) {
-        s.cnt[threadIdx.x - 32] = 0ull;
     } else if (threadIdx.x >= 64) {
         // columns / rows past the image edge (ragged tiles) continue the same formula, so the
         // tables stay monotone for the cell classification
@@ -364,7 +394,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         reinterpret_cast<ulonglong2*>(s.key)[i] = make_ulonglong2(0ull, 0ull);
     __syncthreads();
 
-    if (ego_active) {
+    if (ego_active && stop != 1) {
         const Cam& c = s.cam;
         const MapInfo mi = P.maps[P.env_map[e]];
         const uint32_t n_groups = mi.group_end - mi.group_begin;
@@ -425,31 +455,37 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                 for (; faces; faces &= faces - 1) s.face[slot++] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
             }
             __syncthreads();
-            // ---- phase 2 (c): one thread per candidate primitive
+            // ---- phase 2a (a): one thread per candidate: camera space, pixel box; survivors are compacted
             const int nl = s.n_leaf, nf = s.n_face;
-            const int n_items = nl * LEAF_PRIMS + nf;
-            for (int i = threadIdx.x; i < n_items; i += NTHREADS) {
+            const int n_items = (stop == 2) ? 0 : nl * LEAF_PRIMS + nf;
+            for (int i0 = 0; i0 < n_items; i0 += NTHREADS) {
+                const int i = i0 + threadIdx.x;
+                V3 V[4];
+                uint32_t key_lo, flags, box = 0;
+                bool keep = false;
+                if (i < n_items && fetch_candidate(s, P, i, nl, e, mi.n_tris, V, key_lo, flags)) {
+                    ++n.tested;
+                    keep = pixel_box(c, t, V, box);
+                }
+                const unsigned m = __ballot_sync(0xffffffffu, keep);
+                int base = 0;
+                if (lane == 0 && m) base = atomicAdd(&s.n_surv, __popc(m));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                if (keep) {
+                    const int slot = base + __popc(m & ((1u << lane) - 1u));
+                    if (slot < SCAP) s.surv[slot] = make_uint2((uint32_t)i, box);
+                    else setup_prim(s, t, V, flags & 1u, flags, key_lo, box, rec_cap, n);     // list full
+                }
+            }
+            __syncthreads();
+            // ---- phase 2b (c): one thread per survivor: edge functions, 1/z plane, tiny raster or record
+            const int ns = (stop == 3) ? 0 : min(s.n_surv, SCAP);
+            for (int j = threadIdx.x; j < ns; j += NTHREADS) {
+                const uint2 sv = s.surv[j];
                 V3 V[4];
                 uint32_t key_lo, flags;
-                if (i < nl * LEAF_PRIMS) {
-                    const uint32_t lf = s.leaf[i / LEAF_PRIMS];
-                    const uint32_t j = i % LEAF_PRIMS;
-                    if (j >= (lf & 15u)) continue;
-                    float v[12];
-                    load_prim(P.prims + (lf >> 4) + j, v, key_lo, flags);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
-                } else {
-                    const uint32_t it = s.face[i - nl * LEAF_PRIMS];
-                    const int b = (int)(it >> 3), f = (int)(it & 7u);
-                    const AgentGeom g = P.agents[(size_t)e * P.A + b];
-                    const uint32_t corners = face_corners(f);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
-                    key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
-                    flags = face_flags(corners);
-                }
-                process_prim(s, t, V, flags & 1u, flags, key_lo, rec_cap, n);
+                fetch_candidate(s, P, (int)sv.x, nl, e, mi.n_tris, V, key_lo, flags);
+                setup_prim(s, t, V, flags & 1u, flags, key_lo, sv.y, rec_cap, n);
             }
             __syncthreads();
             if (round + 1 < n_rounds) {
@@ -457,12 +493,13 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                 const int n_rec = min(s.n_rec, rec_cap);
                 if (n_rec > rec_cap / 2) raster_records(s, t, n_rec, classify, n);
                 __syncthreads();
-                if (threadIdx.x == 0) { s.n_leaf = 0; s.n_face = 0; if (n_rec > rec_cap / 2) s.n_rec = 0; }
+                if (threadIdx.x == 0) { s.n_leaf = 0; s.n_face = 0; s.n_surv = 0; if (n_rec > rec_cap / 2) s.n_rec = 0; }
                 __syncthreads();
             }
         }
         // ---- phase 3 (b)+(c): one warp per record
-        raster_records(s, t, min(s.n_rec, rec_cap), classify, n);
+        if (stop == 0 || stop > 5) raster_records(s, t, min(s.n_rec, rec_cap), classify, n);
+        if (stop == 5 && threadIdx.x == 0) { s.touched[0] = 0xffffffffu; s.touched[1] = 0xffffffffu; }
         __syncthreads();
     }
     // ---- phase 4 (d)
@@ -474,25 +511,32 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             // classified / cells are counted by every lane of a warp alike
             const int v = (i >= 7 && lane != 0) ? 0 : vals[i];
             const int sum = __reduce_add_sync(0xffffffffu, v);
-            if (lane == 0 && sum) atomicAdd(&s.cnt[1 + i], (unsigned long long)sum);
+            if (lane == 0 && sum) atomicAdd(&P.counters[1 + i], (unsigned long long)sum);
         }
-        __syncthreads();
-        if (threadIdx.x == 0) s.cnt[0] = 1;
-        __syncthreads();
-        if (threadIdx.x < 16 && s.cnt[threadIdx.x]) atomicAdd(&P.counters[threadIdx.x], s.cnt[threadIdx.x]);
+        if (threadIdx.x == 0) atomicAdd(&P.counters[0], 1ull);
     }
 }
 
+static_assert(sizeof(TileSmem) <= 44 * 1024, "TileSmem must leave room for 5 CTAs per SM (228 KB, 1 KB reserved per CTA)");
 size_t render_smem_bytes() { return sizeof(TileSmem); }
 
 cudaError_t configure_render_kernel() {
     return cudaFuncSetAttribute(render_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
 }
 
-cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, cudaStream_t stream) {
-    const long long blocks = n_views * P.tiles_x * P.tiles_y;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    render_kernel<<<(unsigned)blocks, NTHREADS, sizeof(TileSmem), stream>>>(P);
+cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cudaStream_t stream) {
+    RenderParams P = P0;
+    const long long tiles = (long long)P.tiles_x * P.tiles_y;
+    const bool whole = P.view_first == 0 && n_views == (long long)P.E * P.A * P.K;
+    if (whole && tiles * P.K <= 0x7fffffffLL && P.A <= 65535 && P.E <= 65535) {
+        P.linear = 0;
+        render_kernel<<<dim3((unsigned)(tiles * P.K), (unsigned)P.A, (unsigned)P.E), NTHREADS, sizeof(TileSmem), stream>>>(P);
+    } else {
+        const long long blocks = n_views * tiles;
+        if (blocks > 0x7fffffffLL || (long long)P.E * P.A * P.K > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+        P.linear = 1;
+        render_kernel<<<(unsigned)blocks, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    }
     return cudaGetLastError();
 }
 
