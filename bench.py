@@ -53,6 +53,22 @@ def _peaks():
     return FALLBACK_HBM_GBS, "fallback", 1965.0
 
 
+def env_offset(rank: int, envs_per_rank: int) -> int:
+    """First environment of the full (weak-scaled) workload rendered by `rank`: ranks take disjoint,
+    consecutive slices; there is no exchange between them."""
+    return rank * envs_per_rank
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of a list of floats over all ranks (timing rule: slowest rank counts)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
 def _oracle_sample(scene, n_views: int, seed: int = 0):
     """Time the oracle on a seeded sample of views; returns (seconds, views, counts[n,4])."""
     import oracle
@@ -171,7 +187,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
 
     E = args.envs
     t_gen = time.perf_counter()
-    s = make_config(CFG, E=E, env_offset=rank * E)
+    s = make_config(CFG, E=E, env_offset=env_offset(rank, E))
     t_gen = time.perf_counter() - t_gen
     scene = pic.Scene(s.E, s.A, s.K, s.H, s.W, s.near, s.far, s.tri_xyz, s.tri_class, map_tri_offset=s.map_tri_offset,
                       env_map_id=s.env_map_id, agent_class=s.agent_class, sky_class=s.sky_class,
@@ -231,11 +247,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, dev)
 
     if rank == 0:
         agents = s.E * s.A * world
@@ -287,7 +299,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "agent-steps/s", "h2d_bytes_per_step": 25 * s.E * s.A,
                     "d2h_bytes_per_step": 3 * px, "steps": n_e2e, "entry": "pic_render_host, pinned host buffers"},
-            "gpu_launches": 2 * args.steps,
+            "gpu_launches": 3 * args.steps,
             "roofline": roof,
             "cpu_baseline": {"value": cpu_value, "unit": "agent-steps/s", "cores": min(cores, 64), "kind": "oracle",
                              "sample": f"{len(or_views)} seeded views of this workload in {t_or:.1f} s"},

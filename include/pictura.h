@@ -174,6 +174,17 @@ pic_status pic_scene_set_option(pic_scene* scene, int32_t option, uint64_t value
  */
 pic_status pic_get_kernel_times(pic_scene* scene, float* ms, int32_t capacity, int32_t* n);
 
+/*
+ * Host-only: run the scene builder's map preprocessing (pairing of triangles into planar quads,
+ * Morton-ordered leaves of up to 8 primitives, groups of 32 leaves) on the maps of `desc` without
+ * touching a GPU, and report what it produced.  Only num_maps, map_tri_offset, tri_xyz, tri_class
+ * and A of `desc` are read.  out[0..7] = primitives, of which quads, leaves, groups, largest leaf,
+ * primitives lying outside their leaf box, leaves lying outside their group box, triangles accounted
+ * for (2 per quad + 1 per triangle primitive; equals the input count).  Useful for sizing and
+ * for checking the hierarchy's invariants (out[5] == out[6] == 0).
+ */
+pic_status pic_map_stats(const pic_scene_desc* desc, int64_t out[8]);
+
 /* Thread-local, never NULL; valid until the next failing call on this thread. */
 const char* pic_last_error(void);
 

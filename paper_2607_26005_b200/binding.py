@@ -21,7 +21,7 @@ OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times",
+           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats",
            "pic_last_error", "pic_version"]
 
 
@@ -68,6 +68,7 @@ def load(path: Optional[str] = None):
     lib.pic_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
     lib.pic_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32, C.POINTER(C.c_int32)]
+    lib.pic_map_stats.argtypes = [C.POINTER(pic_scene_desc), C.POINTER(C.c_int64)]
     for name in EXPORTS:
         getattr(lib, name).restype = C.c_int
     lib.pic_last_error.restype = C.c_char_p
@@ -109,6 +110,28 @@ def _stream_ptr(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return int(stream.cuda_stream)
+
+
+def map_stats(tri_xyz, tri_class, map_tri_offset=None, A: int = 0) -> dict:
+    """Host-only statistics of the scene builder's map preprocessing (no GPU needed)."""
+    lib = load()
+    tri_xyz = np.ascontiguousarray(tri_xyz, dtype=np.float32).reshape(-1, 3, 3)
+    tri_class = np.ascontiguousarray(tri_class, dtype=np.uint8).reshape(-1)
+    if map_tri_offset is None:
+        map_tri_offset = [0, tri_xyz.shape[0]]
+    off = np.ascontiguousarray(map_tri_offset, dtype=np.int64)
+    d = pic_scene_desc()
+    d.size = C.sizeof(pic_scene_desc)
+    d.A = int(A)
+    d.num_maps = int(off.shape[0] - 1)
+    d.map_tri_offset = off.ctypes.data
+    d.tri_xyz = tri_xyz.ctypes.data
+    d.tri_class = tri_class.ctypes.data
+    out = (C.c_int64 * 8)()
+    _check(lib, lib.pic_map_stats(C.byref(d), out))
+    names = ["primitives", "quads", "leaves", "groups", "largest_leaf", "prims_outside_leaf", "leaves_outside_group",
+             "triangles"]
+    return dict(zip(names, [int(v) for v in out]))
 
 
 class Scene:

@@ -249,6 +249,51 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     return PIC_OK;
 }
 
+pic_status pic_map_stats(const pic_scene_desc* d, int64_t out[8]) {
+    if (!d || !out) return fail(PIC_ERR_INVALID_ARG, "desc or out is NULL");
+    if (d->size != sizeof(pic_scene_desc)) return fail(PIC_ERR_INVALID_ARG, "desc->size mismatch");
+    if (d->num_maps <= 0 || !d->map_tri_offset || d->map_tri_offset[0] != 0) return fail(PIC_ERR_SHAPE, "bad map offsets");
+    for (int m = 0; m < d->num_maps; ++m)
+        if (d->map_tri_offset[m + 1] < d->map_tri_offset[m]) return fail(PIC_ERR_SHAPE, "map_tri_offset must be non-decreasing");
+    if (d->map_tri_offset[d->num_maps] > 0 && (!d->tri_xyz || !d->tri_class)) return fail(PIC_ERR_INVALID_ARG, "triangle arrays are NULL");
+    char err[256] = "";
+    pic::HostHierarchy* hh = pic::build_hierarchy(d->num_maps, d->map_tri_offset, d->tri_xyz, d->tri_class, d->A > 0 ? d->A : 0, err, sizeof(err));
+    if (!hh) return fail(PIC_ERR_SHAPE, "%s", err);
+    size_t np, nl, ng, nm;
+    const pic::Prim* prims = pic::hierarchy_prims(hh, &np);
+    const pic::Node* leaves = pic::hierarchy_leaves(hh, &nl);
+    const pic::Node* groups = pic::hierarchy_groups(hh, &ng);
+    pic::hierarchy_maps(hh, &nm);
+    int64_t quads = 0, largest = 0, prim_out = 0, leaf_out = 0, tris = 0;
+    for (size_t i = 0; i < np; ++i) { const bool q = prims[i].flags & 1u; quads += q; tris += q ? 2 : 1; }
+    for (size_t l = 0; l < nl; ++l) {
+        const pic::Node& lf = leaves[l];
+        if ((int64_t)lf.count > largest) largest = lf.count;
+        for (uint32_t k = 0; k < lf.count; ++k) {
+            const pic::Prim& p = prims[lf.first + k];
+            const int nv = (p.flags & 1u) ? 4 : 3;
+            bool inside = true;
+            for (int v = 0; v < nv; ++v)
+                for (int c = 0; c < 3; ++c)
+                    inside = inside && p.v[3 * v + c] >= lf.lo[c] && p.v[3 * v + c] <= lf.hi[c];
+            prim_out += !inside;
+        }
+    }
+    for (size_t g = 0; g < ng; ++g) {
+        const pic::Node& gr = groups[g];
+        for (uint32_t k = 0; k < gr.count; ++k) {
+            const pic::Node& lf = leaves[gr.first + k];
+            bool inside = true;
+            for (int c = 0; c < 3; ++c) inside = inside && lf.lo[c] >= gr.lo[c] && lf.hi[c] <= gr.hi[c];
+            leaf_out += !inside;
+        }
+    }
+    out[0] = (int64_t)np; out[1] = quads; out[2] = (int64_t)nl; out[3] = (int64_t)ng; out[4] = largest;
+    out[5] = prim_out; out[6] = leaf_out; out[7] = tris;
+    pic::free_hierarchy(hh);
+    return PIC_OK;
+}
+
 pic_status pic_scene_destroy(pic_scene* s) {
     if (!s) return PIC_OK;
     DeviceGuard guard(s->device);
