@@ -185,6 +185,50 @@ pic_status pic_get_kernel_times(pic_scene* scene, float* ms, int32_t capacity, i
  */
 pic_status pic_map_stats(const pic_scene_desc* desc, int64_t out[8]);
 
+/*
+ * pic_render_static -- render without a scene object and without any allocation.
+ * (The paper has no counterpart; this entry point exists for callers of this library.)
+ *
+ * Who needs it: code that is not allowed to obtain device memory at the point where it wants
+ * images -- a process whose memory pool was sized and locked at start-up, a real-time loop that
+ * must not enter the allocator, a plug-in running under a host application that owns the heap, or
+ * a tool that must keep working when the device is nearly full.  pic_scene_create allocates (map
+ * copy, hierarchy, per-agent and per-view buffers), so those callers cannot use the scene API.
+ *
+ * What it does: the same image definition as pic_render, computed by a variant of the exhaustive
+ * kernel that reads the caller's triangles directly (one map shared by all environments, every
+ * triangle against every pixel -- meant for small batches and small maps).  Per-agent geometry,
+ * per-view cameras, per-camera tables and the status word live in one fixed device array that is
+ * part of the library image (about 420 KB on every device that loads the library, until exit).
+ * The call itself uses no cudaMalloc/cudaFree and no allocating library routine.
+ *
+ * Limits (PIC_ERR_CAPACITY beyond them): E*A <= PIC_STATIC_MAX_AGENTS, E*A*K <= PIC_STATIC_MAX_VIEWS,
+ * H, W <= PIC_STATIC_MAX_SIDE, n_tris <= PIC_STATIC_MAX_TRIS, K <= 16.
+ *
+ *   tri_xyz    dev f32 [n_tris,3,3], tri_class dev u8 [n_tris]   (may be NULL when n_tris == 0)
+ *   poses, dims, active, rig, out_class, out_depth: as in pic_render (outputs need no alignment)
+ * Renders on the CURRENT device, asynchronously on `cuda_stream`.  The first call on a device looks
+ * up the array's device address and sets a kernel attribute; make that first call outside any
+ * stream capture.  All calls on a device share the one array and it keeps the previous call's
+ * contents: the call clears what must start at zero itself, but two calls whose kernels overlap
+ * on the GPU (different streams, or several host threads) race on it -- serialise them.
+ * A non-finite pose or size makes that agent inactive (its images are sky), as in pic_render.
+ */
+#define PIC_STATIC_MAX_AGENTS 1024
+#define PIC_STATIC_MAX_VIEWS 4096
+#define PIC_STATIC_MAX_SIDE 512
+#define PIC_STATIC_MAX_TRIS 65536
+typedef struct {
+    uint32_t size;                 /* = sizeof(pic_static_desc)                                  */
+    int32_t E, A, K, H, W;
+    int32_t n_tris;
+    float near_z, far_z;
+    uint8_t agent_class, sky_class, ground_class, reserved;
+} pic_static_desc;
+pic_status pic_render_static(const pic_static_desc* desc, const float* tri_xyz, const uint8_t* tri_class,
+                             const float* poses, const float* dims, const uint8_t* active, const pic_camera* rig,
+                             uint8_t* out_class, uint16_t* out_depth, void* cuda_stream);
+
 /* Thread-local, never NULL; valid until the next failing call on this thread. */
 const char* pic_last_error(void);
 

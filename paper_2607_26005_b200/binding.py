@@ -21,7 +21,7 @@ OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats",
+           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static",
            "pic_last_error", "pic_version"]
 
 
@@ -42,6 +42,13 @@ class pic_scene_desc(C.Structure):
                 ("env_map_id", C.c_void_p), ("map_tri_offset", C.c_void_p), ("tri_xyz", C.c_void_p),
                 ("tri_class", C.c_void_p), ("agent_class", C.c_uint8), ("sky_class", C.c_uint8),
                 ("ground_class", C.c_uint8), ("reserved", C.c_uint8), ("device", C.c_int32)]
+
+
+class pic_static_desc(C.Structure):
+    _fields_ = [("size", C.c_uint32), ("E", C.c_int32), ("A", C.c_int32), ("K", C.c_int32), ("H", C.c_int32),
+                ("W", C.c_int32), ("n_tris", C.c_int32), ("near_z", C.c_float), ("far_z", C.c_float),
+                ("agent_class", C.c_uint8), ("sky_class", C.c_uint8), ("ground_class", C.c_uint8),
+                ("reserved", C.c_uint8)]
 
 
 _lib = None
@@ -69,6 +76,7 @@ def load(path: Optional[str] = None):
     lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
     lib.pic_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32, C.POINTER(C.c_int32)]
     lib.pic_map_stats.argtypes = [C.POINTER(pic_scene_desc), C.POINTER(C.c_int64)]
+    lib.pic_render_static.argtypes = [C.POINTER(pic_static_desc), vp, vp, vp, vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = C.c_int
     lib.pic_last_error.restype = C.c_char_p
@@ -132,6 +140,30 @@ def map_stats(tri_xyz, tri_class, map_tri_offset=None, A: int = 0) -> dict:
     names = ["primitives", "quads", "leaves", "groups", "largest_leaf", "prims_outside_leaf", "leaves_outside_group",
              "triangles"]
     return dict(zip(names, [int(v) for v in out]))
+
+
+def render_static(E: int, A: int, K: int, H: int, W: int, near: float, far: float, tri_xyz, tri_class, poses, dims,
+                  rig, out_class, out_depth, active=None, agent_class: int = 4, sky_class: int = 0,
+                  ground_class: int = 1, stream=None):
+    """pic_render_static: render on the current device without a scene and without allocating.
+    tri_xyz (f32 [N,3,3]), tri_class (u8 [N]), poses, dims, active and the outputs are CUDA tensors
+    the caller already owns; nothing is allocated here either."""
+    import torch
+    lib = load()
+    n, npx = E * A, E * A * K * H * W
+    n_tris = 0 if tri_xyz is None else int(tri_xyz.shape[0])
+    d = pic_static_desc()
+    d.size = C.sizeof(pic_static_desc)
+    d.E, d.A, d.K, d.H, d.W, d.n_tris = int(E), int(A), int(K), int(H), int(W), n_tris
+    d.near_z, d.far_z = float(near), float(far)
+    d.agent_class, d.sky_class, d.ground_class = int(agent_class), int(sky_class), int(ground_class)
+    _check(lib, lib.pic_render_static(
+        C.byref(d), _dev_ptr(tri_xyz, torch.float32, 9 * n_tris) if n_tris else None,
+        _dev_ptr(tri_class, torch.uint8, n_tris) if n_tris else None, _dev_ptr(poses, torch.float32, 3 * n),
+        _dev_ptr(dims, torch.float32, 3 * n), _dev_ptr(active, torch.uint8, n) if active is not None else None,
+        _rig_array(rig), _dev_ptr(out_class, torch.uint8, npx), _dev_ptr(out_depth, torch.float16, npx),
+        _stream_ptr(stream)))
+    return out_class, out_depth
 
 
 class Scene:

@@ -34,6 +34,15 @@ pic_status fail(pic_status st, const char* fmt, ...) {
     return st;
 }
 
+}  // namespace
+
+namespace pic {
+// lets the other translation units of the library report through pic_last_error()
+void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+}  // namespace pic
+
+namespace {
+
 #define CUDA_TRY(expr)                                                                                   \
     do {                                                                                                 \
         cudaError_t _e = (expr);                                                                         \
