@@ -390,8 +390,9 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         s.ray_y[i] = (t.y0 + i < P.H) ? __ldg(P.rig.ray_y + (size_t)k * P.H + t.y0 + i)
                                       : __fdiv_rn(sub(add((float)(t.y0 + i), 0.5f), 0.5f * (float)P.H), ck.fy);
     }
-    for (int i = threadIdx.x; i < TILE * TILE / 2; i += NTHREADS)
-        reinterpret_cast<ulonglong2*>(s.key)[i] = make_ulonglong2(0ull, 0ull);
+#pragma unroll
+    for (int i = 0; i < TILE * TILE / 2 / NTHREADS; ++i)
+        reinterpret_cast<ulonglong2*>(s.key)[i * NTHREADS + threadIdx.x] = make_ulonglong2(0ull, 0ull);
     __syncthreads();
 
     if (ego_active && stop != 1) {
@@ -424,7 +425,8 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                     if (lvis) s.leaf[base + __popc(lm & ((1u << lane) - 1u))] = (lf.first << 4) | lf.count;
                 }
             }
-            for (int b = round * BOX_ROUND + threadIdx.x; b < min(P.A, (round + 1) * BOX_ROUND); b += NTHREADS) {
+            // boxes are taken from the last thread down: the first warps are busier with the visible groups
+            for (int b = round * BOX_ROUND + (NTHREADS - 1 - (int)threadIdx.x); b < min(P.A, (round + 1) * BOX_ROUND); b += NTHREADS) {
                 if (b == a) continue;
                 const AgentGeom g = P.agents[(size_t)e * P.A + b];
                 if (!g.active) continue;
