@@ -229,6 +229,17 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
     scene.set_option(pic.OPT_TIMING, 0)
     flags = scene.status()
 
+    # ---- context: plain fill of the output tensors (torch memset kernels), the write-only HBM rate on this machine
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    out_dep.zero_(); out_cls.zero_()
+    f0.record(stream)
+    for _ in range(3):
+        out_dep.zero_(); out_cls.zero_()
+    f1.record(stream)
+    torch.cuda.synchronize()
+    fill_gbs = 3 * (out_dep.numel() * 2 + out_cls.numel()) / (f0.elapsed_time(f1) * 1e-3) / 1e9
+
     # ---- end to end through the host-buffer entry point (pinned host memory)
     n_e2e = max(1, min(args.steps, 3))
     h_poses = torch.from_numpy(s.poses.copy()).pin_memory()
@@ -285,7 +296,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
             "traffic": None if NCU_DRAM_BYTES_PER_VIEW is None else NCU_DRAM_BYTES_PER_VIEW * s.E * s.A * s.K,
             "kernel": "render_kernel", "kernel_ms": k_ms, "kernel_launches_timed": int(len(kt)),
             "algorithmic_bytes": alg_bytes, "t_hbm_ms": 1e3 * t_hbm, "t_alu_ms": 1e3 * t_alu,
-            "alg_lane_ops_per_view": float(n_alg_view)})
+            "alg_lane_ops_per_view": float(n_alg_view), "write_only_fill_gbs": fill_gbs})
         line = {
             "metric": "agent_steps_per_s", "value": value, "unit": "agent-steps/s",
             "images_per_s": views / (ms_step * 1e-3), "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -4,7 +4,7 @@ from __future__ import annotations
 import numpy as np
 
 
-class GpuRun:
+class CudaRun:
     """Creates the library scene for a scenes.Scene and renders it through the C ABI."""
 
     def __init__(self, scene, device: int = 0):
@@ -57,13 +57,13 @@ class GpuRun:
         self.scene.close()
 
 
-def check_against_oracle(scene, view_ids=None, gpu: GpuRun = None, **kw):
+def check_against_oracle(scene, view_ids=None, gpu: CudaRun = None, **kw):
     """Render `view_ids` with the oracle and all views with the CUDA path; apply the acceptance rule."""
     import oracle
     from tests.util import compare_images
     own = gpu is None
     if own:
-        gpu = GpuRun(scene)
+        gpu = CudaRun(scene)
     try:
         cls, d16, d32 = gpu.render()
         if view_ids is None:

@@ -23,7 +23,7 @@ def gu():
 
 def _sample_and_check(gu, s, n_oracle, n_brute, seed):
     import oracle
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         V = s.E * s.A * s.K
         cls, d16, _ = g.render(depth32=False)
@@ -60,7 +60,7 @@ def test_config4_full_hundred_steps(gu):
     import torch
     import oracle
     s = make_config(4)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         dev = g.dev
         g.scene.set_state(torch.from_numpy(s.state()).to(dev), g.dims, g.active)
@@ -103,7 +103,7 @@ def test_many_large_primitives_overflow_the_lists(gu):
     tris = centre + rng.uniform(-5, 5, size=(n, 3, 3))
     s = single_env(tris, rng.integers(2, 9, size=n), [(0, 0, 0) + CAR], near=0.5, far=60.0)
     st = gu.check_against_oracle(s, max_mismatch_frac=1e-3)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         *_, cnt = g.render(counters=True)
         assert cnt[7] > 0, "expected the record list to overflow in this scene"
@@ -126,7 +126,7 @@ def test_many_agents_and_groups_take_several_rounds(gu):
                      54, 96, near=0.5, far=150.0)
     views = np.arange(0, 2 * A, 13)
     st = gu.check_against_oracle(s, view_ids=views)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         a, b = g.render(), g.render(brute=True)
         assert (a[0] == b[0]).all() and (a[2] == b[2]).all()

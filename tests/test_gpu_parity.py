@@ -135,7 +135,7 @@ def test_cfg_sampled_views(gu, cfg, E, n_sample):
 def test_production_kernel_equals_exhaustive_kernel(gu, cfg, E):
     """Culling, binning and the small/large split must not change a single bit."""
     s = make_config(cfg, E=E)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         V = s.E * s.A * s.K
         count = V if cfg != 3 else 64
@@ -157,7 +157,7 @@ def test_production_kernel_equals_exhaustive_kernel(gu, cfg, E):
 def test_determinism_and_host_entry_point(gu):
     import torch
     s = make_config(1, E=2)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         a = g.render(depth32=False)
         b = g.render(depth32=False)
@@ -174,7 +174,7 @@ def test_determinism_and_host_entry_point(gu):
 
 def test_counters_are_plausible(gu):
     s = make_config(2, E=1)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         *_, cnt = g.render(counters=True)
         V = s.E * s.A * s.K
@@ -194,7 +194,7 @@ def test_step_state_and_images(gu):
     import torch
     import oracle
     s = make_config(4, E=2)
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         dev = g.dev
         st64 = s.state().astype(np.float64)
@@ -246,7 +246,7 @@ def test_error_codes(gu):
     with pytest.raises(pic.PicError):
         pic.Scene(2, 1, 1, 8, 8, 0.5, 100.0, np.zeros((2, 3, 3)), [2, 2], map_tri_offset=[0, 2], env_map_id=[0, 1])
     s = single_env(np.zeros((0, 3, 3)), [], [ego()], H=16, W=16, rig=make_rig((0.0,), 90.0, 90.0, 16, 16))
-    g = gu.GpuRun(s)
+    g = gu.CudaRun(s)
     try:
         cls, dep = g.scene.alloc_outputs()
         bad_rig = s.rig.copy(); bad_rig[0, 5] = 0.0
