@@ -261,3 +261,21 @@ def test_error_codes(gu):
         assert (cls.cpu().numpy() == 0).all()          # that agent is treated as inactive: sky
     finally:
         g.close()
+
+
+def test_environment_to_map_assignment_and_tied_boxes(gu):
+    a = np.array(_wall(6.0, -20, 20, -10, 10), np.float32)
+    b = np.array(_wall(9.0, -20, 20, -10, 10), np.float32)
+    rig = make_rig((0.0, 180.0), 90.0, 90.0, 16, 16, mount=(0.0, 0.0, 1.0))
+    poses = np.zeros((3, 1, 3), np.float32)
+    dims = np.tile(np.array(CAR, np.float32), (3, 1, 1))
+    s = custom_scene(np.concatenate([a, b]), [5, 5, 6, 6], poses, dims, rig, 16, 16, env_map_id=[1, 0, 1],
+                     map_tri_offset=[0, 2, 4])
+    st = gu.check_against_oracle(s)
+    cls = st["gpu"][0]
+    assert (cls[0] == 6).all() and (cls[2] == 5).all() and (cls[4] == 6).all()
+    # identical boxes at one pose: exact ties everywhere on them, resolved identically on both sides
+    agents = [ego(), (12.5, 0.0, 0.0) + CAR, (12.5, 0.0, 0.0) + CAR]
+    s = single_env([[(50.0, -1.0, 0.0), (51.0, -1.0, 0.0), (51.0, 1.0, 0.0)]], [2], agents)
+    st = gu.check_against_oracle(s)
+    assert (st["gpu"][0] == st["ref"].cls).all()

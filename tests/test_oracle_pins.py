@@ -508,3 +508,58 @@ def test_bicycle_constant_steer_heading_is_linear():
     # inactive agents do not move
     z = oracle.step(st, act, np.array([0], np.uint8), 0.1, 2.8, 30.0)
     assert (z == st).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# further pins: ambiguity mask semantics, box indices, map selection per environment
+# ------------------------------------------------------------------------------------------------
+def test_ambiguity_mask_flags_only_near_boundaries():
+    # a wall whose left edge passes a given distance (in pixels) from the centres of column 3
+    def wall_with_left_edge_offset(eps_px):
+        # 8x8 image, fx = 4, wall at x = 4: image column coordinate = 4 - y ; left edge at u = 3.5 + eps
+        y_left = 4.0 - (3.5 + eps_px)
+        return _wall(4.0, -1.5, y_left, 0.0, 2.0)
+    for eps, want_flag in ((1e-7, True), (-1e-7, True), (1e-2, False), (-1e-2, False)):
+        s = single_env(wall_with_left_edge_offset(eps), [5, 5], [ego()], rig=RIG0, H=8, W=8)
+        r = oracle.render(s)
+        col3 = r.flag[0][3:5, 3] & 1          # rows 3, 4 see the wall (z in [0,2] -> rows 3..4)
+        assert bool(col3.all()) == want_flag, (eps, r.flag[0])
+        # pixels well inside or well outside are never flagged for an edge
+        assert (r.flag[0][3:5, 4] & 1).sum() == 0 and (r.flag[0][:, 0] & 1).sum() == 0
+    # a second surface 1e-6 relative behind the first, other class: depth ambiguity, and only there
+    s = single_env(_wall(4.0, -1, 1, 0, 2) + _wall(4.0 * (1 + 1e-6), -1, 1, 0, 2), [5, 5, 6, 6], [ego()], rig=RIG0, H=8, W=8)
+    r = oracle.render(s)
+    assert (r.cls[0][3:5, 3:5] == 5).all() and (r.flag[0][3:5, 3:5] & 2).all() and (r.flag[0][0:2] & 2).sum() == 0
+    s = single_env(_wall(4.0, -1, 1, 0, 2) + _wall(4.1, -1, 1, 0, 2), [5, 5, 6, 6], [ego()], rig=RIG0, H=8, W=8)
+    assert (oracle.render(s).flag[0] & 2).sum() == 0
+
+
+def test_box_primitive_indices_and_tie_between_identical_boxes():
+    # two identical boxes at the same pose: every pixel is an exact tie, the lower agent index wins,
+    # and the winning index is N + 12 b + t with N map triangles
+    tri = [[(50.0, -1.0, 0.0), (51.0, -1.0, 0.0), (51.0, 1.0, 0.0)]]      # one map triangle, far away
+    agents = [ego(), (12.5, 0.0, 0.0) + CAR, (12.5, 0.0, 0.0) + CAR]
+    s = single_env(tri, [2], agents)
+    r = oracle.render(s, view_ids=[0])
+    on_box = r.cls[0] == 4
+    assert on_box.sum() == 48
+    idx = r.index[0][on_box]
+    assert idx.min() >= 1 + 12 * 1 and idx.max() < 1 + 12 * 2            # agent 1's triangles only
+    assert set(np.unique(idx)) <= {1 + 12 + 0, 1 + 12 + 1, 1 + 12 + 4, 1 + 12 + 5}   # rear face, or a tie on its rim
+    # agent 2's camera sits on the front face of both boxes and looks away: nothing of them is in range
+    r2 = oracle.render(s, view_ids=[2])
+    assert (r2.cls[0] != 4).all()
+
+
+def test_each_environment_sees_its_own_map():
+    # two maps: a class-5 wall and a class-6 wall; env_map_id swaps them
+    a = np.array(_wall(6.0, -20, 20, -10, 10), np.float32)
+    b = np.array(_wall(9.0, -20, 20, -10, 10), np.float32)
+    poses = np.zeros((3, 1, 3), np.float32)
+    dims = np.tile(np.array(CAR, np.float32), (3, 1, 1))
+    s = custom_scene(np.concatenate([a, b]), [5, 5, 6, 6], poses, dims, RIG16, 16, 16,
+                     env_map_id=[1, 0, 1], map_tri_offset=[0, 2, 4])
+    r = oracle.render(s)
+    assert (r.cls[0] == 6).all() and (r.cls[1] == 5).all() and (r.cls[2] == 6).all()
+    assert np.allclose(r.depth[0], 9.0) and np.allclose(r.depth[1], 6.0)
+    assert (r.index[0] < 2).all()             # indices restart at 0 in every map
