@@ -6,20 +6,22 @@
 // so "nearest fragment wins, exact ties go to the lower index" is an unsigned max that does not
 // depend on the order in which primitives arrive; 0 means "no fragment" (background).
 //
-// Four phases separated by one barrier each:
-//   1 (a) cull      every warp tests the map's group boxes against the tile frustum, then takes
+// Phases, each ended by one CTA barrier:
+//   1  (a) cull     every warp tests the map's group boxes against the tile frustum, then takes
 //                   its share of the visible groups and tests their leaf boxes; visible leaves
 //                   are compacted into a list with warp ballots.  Other agents' boxes are culled as
 //                   spheres; only their camera-facing faces become items.
-//   2 (c) set-up    one thread per candidate (8 per visible leaf, 1 per face item): camera-space
-//                   vertices, pixel box, 3-4 edge functions + 1/z plane.  Primitives whose pixel
-//                   box holds <= 4 pixel centres are rasterized at once by their thread (atomic
-//                   max); the others leave a 17-word record.
-//   3 (b)+(c)       one warp per record: primitives covering many pixels first classify the
-//                   tile's 16 x 4 pixel cells (trivial reject / trivial accept from the same
-//                   float32 edge functions, two cells per lane), then the warp walks the surviving
-//                   cells, a lane per pixel pair, atomic max per fragment.
-//   4 (d) store     keys -> class u8 + depth binary16; a thread converts 16 pixels and issues
+//   2a (a) cull     one thread per candidate (8 per visible leaf, 1 per face item): camera-space
+//                   vertices and pixel box; candidates whose box holds no pixel centre of the tile
+//                   stop here, the survivors are compacted again.
+//   2b (c) set-up   one thread per survivor: 3-4 edge functions + 1/z plane.  Primitives whose
+//                   pixel box holds <= 4 pixel centres are rasterized at once by their thread
+//                   (atomic max); the others leave a 17-word record.
+//   3  (b)+(c)      bands of 4 pixel rows belong to warp (band mod 4); every warp walks the records
+//                   and rasterizes its own bands, a lane per pixel pair, plain loads and stores.
+//                   Primitives covering many pixels first classify the warp's 16 x 4 pixel cells
+//                   (trivial reject / trivial accept from the same float32 edge functions).
+//   4  (d) store    keys -> class u8 + depth binary16; a thread converts 16 pixels and issues
 //                   128-bit stores; 8 x 8 blocks no primitive touched are written without reading keys.
 //
 // Cameras (one 64-byte record per view) and per-camera ray / background tables are prepared by
