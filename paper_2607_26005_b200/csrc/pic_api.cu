@@ -62,6 +62,7 @@ struct pic_scene {
     // device memory owned by the scene
     int32_t* d_env_map = nullptr;
     pic::MapInfo* d_maps = nullptr;
+    pic::MapInfo* d_env_maps = nullptr;   // [E]
     pic::Node* d_groups = nullptr;
     pic::Node* d_leaves = nullptr;
     pic::Prim* d_prims = nullptr;
@@ -104,7 +105,7 @@ struct DeviceGuard {
 };
 
 void free_scene(pic_scene* s) {
-    cudaFree(s->d_env_map); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
+    cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
     cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
@@ -128,7 +129,7 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.near_z = s->near_z; P.far_z = s->far_z;
     P.w_near = 1.0f / s->near_z; P.w_far = 1.0f / s->far_z;
     P.cls_agent = s->cls_agent; P.cls_sky = s->cls_sky; P.cls_ground = s->cls_ground;
-    P.env_map = s->d_env_map; P.maps = s->d_maps; P.groups = s->d_groups; P.leaves = s->d_leaves; P.prims = s->d_prims;
+    P.env_map = s->d_env_map; P.env_maps = s->d_env_maps; P.maps = s->d_maps; P.groups = s->d_groups; P.leaves = s->d_leaves; P.prims = s->d_prims;
     P.agents = s->d_agents;
     P.cams = s->d_cams;
     P.rig.ray_x = s->d_tables;
@@ -229,6 +230,7 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     };
     dmalloc((void**)&s->d_env_map, sizeof(int32_t) * d->E);
     dmalloc((void**)&s->d_maps, sizeof(pic::MapInfo) * nm);
+    dmalloc((void**)&s->d_env_maps, sizeof(pic::MapInfo) * d->E);
     dmalloc((void**)&s->d_groups, sizeof(pic::Node) * ng);
     dmalloc((void**)&s->d_leaves, sizeof(pic::Node) * nl);
     dmalloc((void**)&s->d_prims, sizeof(pic::Prim) * np);
@@ -241,6 +243,15 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_status, sizeof(uint32_t));
     upload(s->d_env_map, env_map, sizeof(int32_t) * d->E);
     upload(s->d_maps, maps, sizeof(pic::MapInfo) * nm);
+    {
+        pic::MapInfo* per_env = new (std::nothrow) pic::MapInfo[d->E];
+        if (!per_env) { if (ce == cudaSuccess) ce = cudaErrorMemoryAllocation; }
+        else {
+            for (int e = 0; e < d->E; ++e) per_env[e] = maps[env_map[e]];
+            upload(s->d_env_maps, per_env, sizeof(pic::MapInfo) * d->E);
+            delete[] per_env;
+        }
+    }
     upload(s->d_groups, groups, sizeof(pic::Node) * ng);
     upload(s->d_leaves, leaves, sizeof(pic::Node) * nl);
     upload(s->d_prims, prims, sizeof(pic::Prim) * np);

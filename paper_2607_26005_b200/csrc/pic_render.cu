@@ -350,6 +350,12 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
     t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
     const bool ego_active = P.agents[(size_t)e * P.A + a].active != 0;
+    // issued now so that their latency overlaps the prologue: the map of this environment, the
+    // group box this lane tests first, and the background of the two rows this thread stores
+    const MapInfo mi = P.env_maps[e];
+    Node gn0;
+    gn0.first = 0; gn0.count = 0;
+    if (lane < GROUP_BATCH && mi.group_begin + lane < mi.group_end) gn0 = P.groups[mi.group_begin + lane];
 
     // ---- prologue: camera, ray tables, frustum planes, cleared keys
     if (threadIdx.x < 7) {
@@ -399,7 +405,6 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
 
     if (ego_active && stop != 1) {
         const Cam& c = s.cam;
-        const MapInfo mi = P.maps[P.env_map[e]];
         const uint32_t n_groups = mi.group_end - mi.group_begin;
         const int n_rounds = max((int)((n_groups + GROUP_BATCH - 1) / GROUP_BATCH), (P.A + BOX_ROUND - 1) / BOX_ROUND);
         for (int round = 0; round < n_rounds; ++round) {
@@ -409,7 +414,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                 const uint32_t g = g0 + lane;
                 bool vis = false;
                 Node gn;
-                if (lane < GROUP_BATCH && g < mi.group_end) { gn = P.groups[g]; vis = box_visible(s, gn); if (warp == 0) ++n.grp; }
+                if (lane < GROUP_BATCH && g < mi.group_end) { gn = (round == 0) ? gn0 : P.groups[g]; vis = box_visible(s, gn); if (warp == 0) ++n.grp; }
                 unsigned gm = __ballot_sync(0xffffffffu, vis);
                 // warp w takes the visible groups w, w + NW, ...
                 for (int i = 0; gm; gm &= gm - 1, ++i) {

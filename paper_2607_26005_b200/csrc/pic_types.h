@@ -78,6 +78,7 @@ struct RenderParams {
     float w_near, w_far;            // 1/near, 1/far: kept range of the reciprocal depth
     uint32_t cls_agent, cls_sky, cls_ground;
     const int32_t* env_map;
+    const MapInfo* env_maps;        // [E] the MapInfo of each environment's map (one load instead of two)
     const MapInfo* maps;
     const Node* groups;
     const Node* leaves;
