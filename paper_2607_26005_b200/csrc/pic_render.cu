@@ -171,23 +171,26 @@ __device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderP
 }
 
 // One 16 x 4 cell at (xx, yy): every lane tests its two pixels and updates their keys with plain
-// loads and stores -- in phase 3 the rows of a cell belong to exactly one warp.  `inside`: the
-// cell is known to be covered and in range.  Returns whether any lane produced a fragment.
+// loads and stores -- in phase 3 the rows of a cell belong to exactly one warp.  `need`: the edges
+// that still have to be tested on this cell (0: the cell is known to be covered and in depth
+// range; the range test rides on the edge tests).  Returns whether any lane produced a fragment.
 __device__ __forceinline__ bool raster_cell(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, int xx, int yy,
-                                            bool inside, int lane) {
+                                            uint32_t need, int lane) {
     const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
     const float rx0 = s.ray_x[x], rx1 = s.ray_x[x + 1], ry = s.ray_y[y];
     const float wt = fm(q.wy, ry, q.wz);
     const float w0 = fm(q.wx, rx0, wt), w1 = fm(q.wx, rx1, wt);
     bool in0 = true, in1 = true;
-    if (!inside) {
+    if (need) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const float te = fm(q.ny[e], ry, q.nz[e]);
-            const float e0 = fm(q.nx[e], rx0, te), e1 = fm(q.nx[e], rx1, te);
-            const bool own = (q.tl >> e) & 1u;
-            in0 = in0 && (e0 > 0.f || (e0 == 0.f && own));
-            in1 = in1 && (e1 > 0.f || (e1 == 0.f && own));
+            if ((need >> e) & 1u) {          // warp-uniform: edges known to be positive on the whole cell are skipped
+                const float te = fm(q.ny[e], ry, q.nz[e]);
+                const float e0 = fm(q.nx[e], rx0, te), e1 = fm(q.nx[e], rx1, te);
+                const bool own = (q.tl >> e) & 1u;
+                in0 = in0 && (e0 > 0.f || (e0 == 0.f && own));
+                in1 = in1 && (e1 > 0.f || (e1 == 0.f && own));
+            }
         }
         in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
         in1 = in1 && (w1 >= t.w_far) && (w1 <= t.w_near);
@@ -229,7 +232,7 @@ __device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool cl
             const int band = (lane >> 2) * NW + warp, col = lane & 3;
             const int xa = col * 16, xb = xa + 15, ya = band * 4, yb = ya + 3;
             bool reject = lane >= 16 || xb < bx0 || xa > bx1 || yb < by0 || ya > by1;
-            bool inside = !reject;
+            uint32_t need = 0u;
             if (!reject) {
                 const float rxa = s.ray_x[xa], rxb = s.ray_x[xb], rya = s.ray_y[ya], ryb = s.ray_y[yb];   // rxa < rxb, rya < ryb
 #pragma unroll
@@ -239,26 +242,27 @@ __device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool cl
                     const float emax = fm(q.nx[e], q.nx[e] >= 0.f ? rxb : rxa, fmaxf(ta, tb));
                     const float emin = fm(q.nx[e], q.nx[e] >= 0.f ? rxa : rxb, fminf(ta, tb));
                     reject = reject || (emax < 0.f);
-                    inside = inside && (emin > 0.f);
+                    if (!(emin > 0.f)) need |= 1u << e;
                 }
                 const float wa = fm(q.wy, rya, q.wz), wb = fm(q.wy, ryb, q.wz);
                 const float wmax = fm(q.wx, q.wx >= 0.f ? rxb : rxa, fmaxf(wa, wb));
                 const float wmin = fm(q.wx, q.wx >= 0.f ? rxa : rxb, fminf(wa, wb));
                 reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
-                inside = inside && (wmin >= t.w_far) && (wmax <= t.w_near);
+                // the depth range test rides on the edge tests: if it is still needed, so is one edge
+                if (need == 0u && !((wmin >= t.w_far) && (wmax <= t.w_near))) need = 1u;
             }
-            const unsigned full = __ballot_sync(0xffffffffu, !reject && inside);
             for (unsigned m = __ballot_sync(0xffffffffu, !reject); m; m &= m - 1) {
                 const int cell = __ffs(m) - 1;
                 const int xx = (cell & 3) * 16, yy = ((cell >> 2) * NW + warp) * 4;
+                const uint32_t need_c = __shfl_sync(0xffffffffu, need, cell);
                 ++n.cells;
-                if (raster_cell(s, t, q, key_lo, xx, yy, (full >> cell) & 1u, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
+                if (raster_cell(s, t, q, key_lo, xx, yy, need_c, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
             }
         } else {
             for (int band = first; band <= band1; band += NW)
                 for (int xx = bx0 & ~15; xx <= bx1; xx += 16) {
                     ++n.cells;
-                    if (raster_cell(s, t, q, key_lo, xx, band * 4, false, lane)) touched |= 3ull << ((band >> 1) * 8 + (xx >> 3));
+                    if (raster_cell(s, t, q, key_lo, xx, band * 4, 0xFu, lane)) touched |= 3ull << ((band >> 1) * 8 + (xx >> 3));
                 }
         }
     }
