@@ -33,7 +33,11 @@
  *  O7 output      class u8, depth as f64 and rounded to binary16 (round-to-nearest-even).
  *  O8 ambiguity   pixels where a 1e-5 relative perturbation of an edge function, a depth gap, a
  *                 clip plane or the horizon could change the answer are flagged, so that a float32
- *                 implementation may legitimately differ there (and only there).
+ *                 implementation may legitimately differ there (and only there); so are pixels whose
+ *                 winning primitive lies in a plane that passes the camera centre at less than 1/200
+ *                 of its farthest vertex's distance (bit 16, informative): depth there is
+ *                 ill-conditioned in float32 -- the per-pixel kappa output lets a comparison widen
+ *                 its depth tolerance to 5e-7 * kappa, and depth gaps are judged with that width.
  *  O9 stepping    explicit-Euler kinematic bicycle update (pico_step).
  *
  * Parity pins: tests/test_oracle_*.py (closed forms, invariants, an independent ray caster,
@@ -48,6 +52,8 @@
 #endif
 
 #define REL_TOL 1e-5
+#define GRAZING_KAPPA 200.0
+#define DEPTH_KAPPA 5e-7      /* relative depth uncertainty of a float32 renderer per unit of kappa */
 
 typedef struct { double x, y, z; } v3;
 
@@ -64,6 +70,7 @@ typedef struct {
     v3 N[3];          /* sign-normalised edge normals */
     double D;         /* sign-normalised, > 0; 0 marks a skipped (degenerate / edge-on) primitive */
     double band[3];   /* O8 edge band without the |rho| factor */
+    double kappa;     /* O8 (v): max|V_i| |N| / D, how close the primitive's plane passes by the camera centre */
     int32_t index;    /* global primitive index (O3) */
     uint8_t cls;
 } prim_t;
@@ -116,6 +123,10 @@ static void setup_prim(prim_t* p, v3 V0, v3 V1, v3 V2, int32_t index, uint8_t cl
     p->band[0] = REL_TOL * fmax(n1, n2) * v3_norm(v3_sub(V2, V1));
     p->band[1] = REL_TOL * fmax(n2, n0) * v3_norm(v3_sub(V0, V2));
     p->band[2] = REL_TOL * fmax(n0, n1) * v3_norm(v3_sub(V1, V0));
+    {
+        v3 Nn = v3_cross(v3_sub(V1, V0), v3_sub(V2, V0));
+        p->kappa = (p->D > 0.0) ? fmax(n0, fmax(n1, n2)) * v3_norm(Nn) / p->D : 0.0;
+    }
     p->index = index;
     p->cls = cls;
 }
@@ -201,7 +212,9 @@ static int meets_frustum(v3 V0, v3 V1, v3 V2, double tx, double ty, double near,
  *   out_depth  f64     O5/O6 depth (metres along the optical axis)
  *   out_f16    u16     O7 binary16 bits of the depth
  *   out_index  i32     global index of the winning primitive, -1 for background
- *   out_flag   u8      O8 bit mask: 1 edge, 2 depth gap, 4 near/far plane, 8 horizon
+ *   out_flag   u8      O8 bit mask: 1 edge, 2 depth gap, 4 near/far plane, 8 horizon, 16 grazing plane (informative)
+ *   out_kappa  f64     conditioning of the winner's depth: max|V_i| |N| / D of its plane (0 for background);
+ *                      a float32 renderer's depth may be off by about 5e-7 * kappa relative
  *   counts     i64 [n_views,4]: primitives meeting the frustum, primitives with >=1 kept
  *              fragment, kept fragments, flagged pixels
  * Any output pointer may be NULL.  Returns 0, or -1 on allocation failure.
@@ -213,7 +226,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 const float* poses, const float* dims, const uint8_t* active, const float* rig,
                 int n_views, const int64_t* view_ids,
                 uint8_t* out_class, double* out_depth, uint16_t* out_f16, int32_t* out_index,
-                uint8_t* out_flag, int64_t* counts, int n_threads)
+                uint8_t* out_flag, double* out_kappa, int64_t* counts, int n_threads)
 {
     (void)E;
 #ifdef _OPENMP
@@ -238,6 +251,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 if (out_f16) out_f16[base + p] = pico_f64_to_f16(far);
                 if (out_index) out_index[base + p] = -1;
                 if (out_flag) out_flag[base + p] = 0;
+                if (out_kappa) out_kappa[base + p] = 0.0;
             }
             if (counts) memset(counts + 4 * (size_t)vi, 0, 4 * sizeof(int64_t));
             continue;
@@ -285,7 +299,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 double rho_n = v3_norm(rho);
 
                 /* O4-O6: nearest kept fragment */
-                double z_win = 0.0; int32_t i_win = -1; uint8_t c_win = 0;
+                double z_win = 0.0, k_win = 0.0; int32_t i_win = -1; uint8_t c_win = 0;
                 for (int64_t j = 0; j < np; ++j) {
                     const prim_t* p = &prim[j];
                     if (p->D == 0.0) continue;
@@ -307,7 +321,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                         hit[j] = 1;
                     }
                     if (i_win < 0 || z < z_win || (z == z_win && p->index < i_win)) {
-                        z_win = z; i_win = p->index; c_win = p->cls;
+                        z_win = z; i_win = p->index; c_win = p->cls; k_win = p->kappa;
                     }
                 }
 
@@ -321,6 +335,10 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 /* O8: ambiguity mask */
                 uint8_t flag = 0;
                 if (i_win < 0 && fabs(w) <= REL_TOL) flag |= 8;
+                /* (v) the winner's plane grazes the camera centre: a 6e-8 relative change of its
+                   camera-space vertices (float32 spacing) moves the depth by more than half the
+                   1e-4 tolerance */
+                if (i_win >= 0 && k_win > GRAZING_KAPPA) flag |= 16;
                 for (int64_t j = 0; j < np; ++j) {
                     const prim_t* p = &prim[j];
                     if (p->D == 0.0) continue;
@@ -345,7 +363,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                     if (!covered) continue;
                     /* (ii) a kept fragment of another class almost as near as the winner */
                     if (i_win >= 0 && z >= near && z <= far && p->cls != c_win &&
-                        fabs(z - z_win) <= REL_TOL * z_win) flag |= 2;
+                        fabs(z - z_win) <= fmax(REL_TOL, DEPTH_KAPPA * fmax(p->kappa, k_win)) * z_win) flag |= 2;
                     /* (iii) a covered fragment sitting on the near or far plane that matters */
                     if ((fabs(z - near) <= REL_TOL * near || fabs(z - far) <= REL_TOL * far) && could_show) flag |= 4;
                 }
@@ -357,6 +375,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 if (out_f16) out_f16[o] = pico_f64_to_f16(depth);
                 if (out_index) out_index[o] = i_win;
                 if (out_flag) out_flag[o] = flag;
+                if (out_kappa) out_kappa[o] = (i_win >= 0) ? k_win : 0.0;
             }
         }
         if (counts) {

@@ -32,7 +32,7 @@ def _load():
         p = C.c_void_p
         lib.pico_render.restype = C.c_int
         lib.pico_render.argtypes = [C.c_int] * 5 + [C.c_double] * 2 + [p] * 4 + [C.c_int] * 3 + [p] * 4 + \
-                                   [C.c_int, p] + [p] * 6 + [C.c_int]
+                                   [C.c_int, p] + [p] * 7 + [C.c_int]
         lib.pico_step.restype = None
         lib.pico_step.argtypes = [p, p, p, C.c_int64, C.c_double, C.c_double, C.c_double]
         lib.pico_f64_to_f16.restype = C.c_uint16
@@ -58,6 +58,7 @@ class OracleResult:
     depth_f16: np.ndarray    # f16 [n,H,W]
     index: np.ndarray        # i32 [n,H,W]  winning primitive, -1 background
     flag: np.ndarray         # u8  [n,H,W]  ambiguity mask bits
+    kappa: np.ndarray        # f64 [n,H,W]  conditioning of the winner's depth (0 for background)
     counts: np.ndarray       # i64 [n,4]    in-frustum prims, prims with a kept fragment, kept fragments, flagged px
 
 
@@ -84,14 +85,15 @@ def render(scene, view_ids: Optional[Sequence[int]] = None, poses: Optional[np.n
     f16 = np.empty((n, s.H, s.W), np.uint16)
     index = np.empty((n, s.H, s.W), np.int32)
     flag = np.empty((n, s.H, s.W), np.uint8)
+    kappa = np.empty((n, s.H, s.W), np.float64)
     counts = np.zeros((n, 4), np.int64)
     rc = lib.pico_render(s.E, s.A, s.K, s.H, s.W, float(s.near), float(s.far), _ptr(emi), _ptr(off), _ptr(tri),
                          _ptr(tcl), int(s.agent_class), int(s.sky_class), int(s.ground_class), _ptr(poses),
                          _ptr(dims), _ptr(active), _ptr(rig), n, _ptr(view_ids), _ptr(cls), _ptr(depth),
-                         _ptr(f16), _ptr(index), _ptr(flag), _ptr(counts), int(n_threads))
+                         _ptr(f16), _ptr(index), _ptr(flag), _ptr(kappa), _ptr(counts), int(n_threads))
     if rc != 0:
         raise MemoryError("pico_render failed")
-    return OracleResult(view_ids, cls, depth, f16.view(np.float16), index, flag, counts)
+    return OracleResult(view_ids, cls, depth, f16.view(np.float16), index, flag, kappa, counts)
 
 
 def step(state: np.ndarray, actions: np.ndarray, active: Optional[np.ndarray], dt: float, wheelbase: float,

@@ -96,9 +96,28 @@ __device__ __forceinline__ void load_camera(Cam& c, const ViewCam& v, const CamC
     c.cx = 0.5f * (float)W; c.cy = 0.5f * (float)H;
 }
 
-// Edge functions and reciprocal-depth plane of a primitive given in camera space.
+// Plane normal of a primitive from its camera-space vertices (used for box faces, whose corners are
+// a few metres apart).
+__device__ __forceinline__ V3 plane_normal(const V3 (&V)[4], bool quad) {
+    return quad ? vcross(vsub(V[2], V[0]), vsub(V[3], V[1])) : vcross(vsub(V[1], V[0]), vsub(V[2], V[0]));
+}
+
+// Plane normal of a map primitive: the cross product is taken between WORLD-space edge vectors
+// (differences of nearby coordinates, exact to a float32 ulp of the edge) and then rotated into
+// camera space.  Differencing camera-space vertices instead would carry the rounding of the
+// vertex distance into the edge and tilt the plane of a small, distant primitive.
+__device__ __forceinline__ V3 plane_normal_world(const Cam& c, const float (&v)[12], bool quad) {
+    V3 d1, d2;
+    if (quad) { d1 = {sub(v[6], v[0]), sub(v[7], v[1]), sub(v[8], v[2])}; d2 = {sub(v[9], v[3]), sub(v[10], v[4]), sub(v[11], v[5])}; }
+    else      { d1 = {sub(v[3], v[0]), sub(v[4], v[1]), sub(v[5], v[2])}; d2 = {sub(v[6], v[0]), sub(v[7], v[1]), sub(v[8], v[2])}; }
+    const V3 nw = vcross(d1, d2);
+    return rotate_to_camera(c, nw.x, nw.y, nw.z);
+}
+
+// Edge functions and reciprocal-depth plane of a primitive given in camera space, with its plane
+// normal P (same orientation as the vertex order).
 // Returns false for degenerate / edge-on primitives (D == 0), which cover nothing.
-__device__ __forceinline__ bool prim_equations(const V3 (&V)[4], bool quad, uint32_t flags, PrimEq& q) {
+__device__ __forceinline__ bool prim_equations(const V3 (&V)[4], bool quad, uint32_t flags, const V3 P, PrimEq& q) {
     const int n = quad ? 4 : 3;
     V3 N[4];
 #pragma unroll
@@ -116,7 +135,6 @@ __device__ __forceinline__ bool prim_equations(const V3 (&V)[4], bool quad, uint
             N[i] = {0.f, 0.f, 1.f};              // triangles: a fourth edge that is always inside
         }
     }
-    V3 P = quad ? vcross(vsub(V[2], V[0]), vsub(V[3], V[1])) : vcross(vsub(V[1], V[0]), vsub(V[2], V[0]));
     float D = vdot(P, V[0]);
     if (!(D != 0.f)) return false;               // also drops NaN
     const float s = D < 0.f ? -1.f : 1.f;

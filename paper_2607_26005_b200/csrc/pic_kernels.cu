@@ -125,13 +125,14 @@ __global__ void __launch_bounds__(BRUTE_THREADS) render_brute_kernel(const __gri
         const uint32_t n_map = mi.prim_end - mi.prim_begin;
         const uint32_t n_items = n_map + 6u * (uint32_t)P.A;
         for (uint32_t i = threadIdx.x; i < n_items; i += BRUTE_THREADS) {
-            V3 V[4]; bool quad; uint32_t flags, key_lo;
+            V3 V[4], Pn; bool quad; uint32_t flags, key_lo;
             if (i < n_map) {
                 float v[12];
                 load_prim(P.prims + mi.prim_begin + i, v, key_lo, flags);
                 quad = flags & 1u;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
+                Pn = plane_normal_world(c, v, quad);
             } else {
                 const uint32_t j = i - n_map;
                 const int b = (int)(j / 6u), f = (int)(j % 6u);
@@ -143,9 +144,10 @@ __global__ void __launch_bounds__(BRUTE_THREADS) render_brute_kernel(const __gri
                 for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
                 quad = true; flags = face_flags(corners);
                 key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+                Pn = plane_normal(V, true);
             }
             PrimEq q;
-            if (!prim_equations(V, quad, flags, q)) continue;
+            if (!prim_equations(V, quad, flags, Pn, q)) continue;
             for (int y = 0; y < t.th; ++y) {
                 const float ry = s.ray_y[y];
                 for (int x = 0; x < t.tw; ++x) {

@@ -120,9 +120,9 @@ struct Tally { int grp, leaf, tested, setup, tiny, recs, fallback, classified, c
 
 // Phase 2b body: set a surviving primitive up, rasterize it (tiny) or leave a record.
 __device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
-                                           uint32_t key_lo, uint32_t box, int rec_cap, Tally& n) {
+                                           const V3 Pn, uint32_t key_lo, uint32_t box, int rec_cap, Tally& n) {
     PrimEq q;
-    if (!prim_equations(V, quad, flags, q)) return;
+    if (!prim_equations(V, quad, flags, Pn, q)) return;
     ++n.setup;
     const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
     if ((bx1 - bx0 + 1) * (by1 - by0 + 1) > TINY_MAX_PIXELS) {
@@ -147,7 +147,7 @@ __device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const 
 
 // Candidate `i` of the round: a primitive of a visible leaf or a box-face item, in camera space.
 __device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderParams& P, int i, int nl, int e, uint32_t n_map_tris,
-                                                V3 (&V)[4], uint32_t& key_lo, uint32_t& flags) {
+                                                V3 (&V)[4], V3& Pn, uint32_t& key_lo, uint32_t& flags, bool want_plane) {
     const Cam& c = s.cam;
     if (i < nl * LEAF_PRIMS) {
         const uint32_t lf = s.leaf[i / LEAF_PRIMS];
@@ -157,6 +157,7 @@ __device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderP
         load_prim(P.prims + (lf >> 4) + j, v, key_lo, flags);
 #pragma unroll
         for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
+        if (want_plane) Pn = plane_normal_world(c, v, flags & 1u);
     } else {
         const uint32_t it = s.face[i - nl * LEAF_PRIMS];
         const int b = (int)(it >> 3), f = (int)(it & 7u);
@@ -166,6 +167,7 @@ __device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderP
         for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
         key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
         flags = face_flags(corners);
+        if (want_plane) Pn = plane_normal(V, true);
     }
     return true;
 }
@@ -473,10 +475,10 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             const int n_items = (stop == 2) ? 0 : nl * LEAF_PRIMS + nf;
             for (int i0 = 0; i0 < n_items; i0 += NTHREADS) {
                 const int i = i0 + threadIdx.x;
-                V3 V[4];
+                V3 V[4], Pn;
                 uint32_t key_lo, flags, box = 0;
                 bool keep = false;
-                if (i < n_items && fetch_candidate(s, P, i, nl, e, mi.n_tris, V, key_lo, flags)) {
+                if (i < n_items && fetch_candidate(s, P, i, nl, e, mi.n_tris, V, Pn, key_lo, flags, false)) {
                     ++n.tested;
                     keep = pixel_box(c, t, V, box);
                 }
@@ -487,7 +489,10 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                 if (keep) {
                     const int slot = base + __popc(m & ((1u << lane) - 1u));
                     if (slot < SCAP) s.surv[slot] = make_uint2((uint32_t)i, box);
-                    else setup_prim(s, t, V, flags & 1u, flags, key_lo, box, rec_cap, n);     // list full
+                    else {                                                                  // list full (rare)
+                        fetch_candidate(s, P, i, nl, e, mi.n_tris, V, Pn, key_lo, flags, true);
+                        setup_prim(s, t, V, flags & 1u, flags, Pn, key_lo, box, rec_cap, n);
+                    }
                 }
             }
             __syncthreads();
@@ -495,10 +500,10 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             const int ns = (stop == 3) ? 0 : min(s.n_surv, SCAP);
             for (int j = threadIdx.x; j < ns; j += NTHREADS) {
                 const uint2 sv = s.surv[j];
-                V3 V[4];
+                V3 V[4], Pn;
                 uint32_t key_lo, flags;
-                fetch_candidate(s, P, (int)sv.x, nl, e, mi.n_tris, V, key_lo, flags);
-                setup_prim(s, t, V, flags & 1u, flags, key_lo, sv.y, rec_cap, n);
+                fetch_candidate(s, P, (int)sv.x, nl, e, mi.n_tris, V, Pn, key_lo, flags, true);
+                setup_prim(s, t, V, flags & 1u, flags, Pn, key_lo, sv.y, rec_cap, n);
             }
             __syncthreads();
             if (round + 1 < n_rounds) {

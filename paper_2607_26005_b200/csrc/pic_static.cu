@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(kThreads) render_static_kernel(const __grid_co
     if (ego.active) {
         const uint32_t n_items = S.n_tris + 6u * (uint32_t)P.A;
         for (uint32_t i = threadIdx.x; i < n_items; i += kThreads) {
-            V3 V[4]; bool quad; uint32_t flags, key_lo;
+            V3 V[4], Pn; bool quad; uint32_t flags, key_lo;
             if (i < S.n_tris) {
                 const float* p = S.tri_xyz + 9 * (size_t)i;
                 float v[9];
@@ -108,6 +108,10 @@ __global__ void __launch_bounds__(kThreads) render_static_kernel(const __grid_co
 #pragma unroll
                 for (int j = 0; j < 3; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
                 V[3] = V[2];
+                {
+                    const float v12[12] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], v[8], v[6], v[7], v[8]};
+                    Pn = plane_normal_world(c, v12, false);
+                }
                 quad = false;
                 flags = 0u;
                 // an edge shared by two triangles is evaluated in the same direction by both
@@ -126,9 +130,10 @@ __global__ void __launch_bounds__(kThreads) render_static_kernel(const __grid_co
                 for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
                 quad = true; flags = face_flags(corners);
                 key_lo = ((0xFFFFFFu - (S.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+                Pn = plane_normal(V, true);
             }
             PrimEq q;
-            if (!prim_equations(V, quad, flags, q)) continue;
+            if (!prim_equations(V, quad, flags, Pn, q)) continue;
             for (int y = 0; y < t.th; ++y) {
                 const float ry = s.ray_y[y];
                 for (int x = 0; x < t.tw; ++x) {

@@ -70,7 +70,8 @@ def check_against_oracle(scene, view_ids=None, gpu: CudaRun = None, **kw):
             view_ids = np.arange(scene.E * scene.A * scene.K)
         view_ids = np.asarray(view_ids, dtype=np.int64)
         ref = oracle.render(scene, view_ids)
-        stats = compare_images(ref.cls, ref.depth, ref.flag, cls[view_ids], d32[view_ids], d16[view_ids], **kw)
+        stats = compare_images(ref.cls, ref.depth, ref.flag, cls[view_ids], d32[view_ids], d16[view_ids],
+                               ref_kappa=ref.kappa, **kw)
         stats["ref"] = ref
         stats["gpu"] = (cls, d16, d32)
         return stats

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 from scenes import make_config, make_rig, make_actions, custom_scene, DT, WHEELBASE, V_MAX
-from tests.util import single_env, compare_images
+from tests.util import single_env, compare_images, assert_same_as_exhaustive
 
 pytestmark = pytest.mark.gpu
 CAR = (4.5, 1.9, 1.5)
@@ -31,11 +31,12 @@ def _sample_and_check(gu, s, n_oracle, n_brute, seed):
         rng = np.random.default_rng(seed)
         views = np.sort(rng.choice(V, size=n_oracle, replace=False))
         ref = oracle.render(s, views)
-        st = compare_images(ref.cls, ref.depth, ref.flag, cls[views], None, d16[views])
+        st = compare_images(ref.cls, ref.depth, ref.flag, cls[views], None, d16[views], ref_kappa=ref.kappa)
         first = int(rng.integers(0, V - n_brute))
-        b = g.render(brute=True, depth32=False, view_first=first, view_count=n_brute)
-        assert (b[0][first:first + n_brute] == cls[first:first + n_brute]).all()
-        assert (b[1][first:first + n_brute].view(np.uint16) == d16[first:first + n_brute].view(np.uint16)).all()
+        a = g.render(view_first=first, view_count=n_brute)
+        b = g.render(brute=True, view_first=first, view_count=n_brute)
+        assert_same_as_exhaustive(a, b, slice(first, first + n_brute))
+        assert (a[0][first:first + n_brute] == cls[first:first + n_brute]).all()
         return st
     finally:
         g.close()
@@ -107,8 +108,7 @@ def test_many_large_primitives_overflow_the_lists(gu):
     try:
         *_, cnt = g.render(counters=True)
         assert cnt[7] > 0, "expected the record list to overflow in this scene"
-        a, b = g.render(), g.render(brute=True)
-        assert (a[0] == b[0]).all() and (a[2] == b[2]).all()
+        assert_same_as_exhaustive(g.render(), g.render(brute=True))
     finally:
         g.close()
 
@@ -128,8 +128,7 @@ def test_many_agents_and_groups_take_several_rounds(gu):
     st = gu.check_against_oracle(s, view_ids=views)
     g = gu.CudaRun(s)
     try:
-        a, b = g.render(), g.render(brute=True)
-        assert (a[0] == b[0]).all() and (a[2] == b[2]).all()
+        assert_same_as_exhaustive(g.render(), g.render(brute=True))
     finally:
         g.close()
 

@@ -563,3 +563,25 @@ def test_each_environment_sees_its_own_map():
     assert (r.cls[0] == 6).all() and (r.cls[1] == 5).all() and (r.cls[2] == 6).all()
     assert np.allclose(r.depth[0], 9.0) and np.allclose(r.depth[1], 6.0)
     assert (r.index[0] < 2).all()             # indices restart at 0 in every map
+
+
+def test_grazing_plane_flag():
+    # a huge ground-parallel sheet 5 cm below the camera: its plane passes the camera centre at
+    # 0.05 m while its vertices are up to 85 m away (ratio 1 700) -> every pixel showing it is flagged
+    # (only the first row below the horizon sees it beyond the near plane: z = 0.05 / (0.5/8) = 0.8 m)
+    sheet = [[(0.25, -60.0, 0.95), (60.0, -60.0, 0.95), (60.0, 60.0, 0.95)], [(0.25, -60.0, 0.95), (60.0, 60.0, 0.95), (0.25, 60.0, 0.95)]]
+    s = single_env(sheet, [5, 5], [ego()], rig=RIG16, H=16, W=16, far=100.0)
+    r = oracle.render(s)
+    on = r.cls[0] == 5
+    assert on.sum() == 16 and on[8].all() and np.allclose(r.depth[0][8], 0.8)
+    assert (r.flag[0][on] & 16).all() and (r.flag[0][~on] & 16).sum() == 0
+    assert np.allclose(r.kappa[0][on], np.sqrt(60.0 ** 2 + 60.0 ** 2 + 0.05 ** 2) / 0.05, rtol=1e-6) and (r.kappa[0][~on] == 0).all()
+    # the same sheet 1 m below the camera (ratio ~85) is an ordinary road: never flagged as grazing
+    road = [[(1.0, -60.0, 0.0), (60.0, -60.0, 0.0), (60.0, 60.0, 0.0)], [(1.0, -60.0, 0.0), (60.0, 60.0, 0.0), (1.0, 60.0, 0.0)]]
+    s = single_env(road, [2, 2], [ego()], rig=RIG16, H=16, W=16, far=100.0)
+    r = oracle.render(s)
+    assert (r.cls[0] == 2).sum() > 50 and (r.flag[0] & 16).sum() == 0
+    assert np.allclose(r.kappa[0][r.cls[0] == 2], np.sqrt(7201.0), rtol=1e-9)       # farthest vertex / 1 m
+    # and none of the benchmark workloads' pixels are (camera 1.5 m above the roads)
+    r = oracle.render(make_config(0))
+    assert (r.flag & 16).sum() == 0
