@@ -33,7 +33,7 @@ namespace pic {
 constexpr int NTHREADS = 128;
 constexpr int NW = NTHREADS / 32;
 constexpr int RCAP = 64;          // records (primitives rasterized by a warp) per tile
-constexpr int REC = 17;           // words per record
+constexpr int REC = 20;           // words per record (17 used; 16-byte aligned for vector access)
 constexpr int GROUP_BATCH = 16;   // groups examined per round
 constexpr int LEAFCAP = GROUP_BATCH * GROUP_LEAVES;   // visible leaves per round
 constexpr int BOX_ROUND = 64;     // boxes examined per round
@@ -44,7 +44,7 @@ constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large cl
 
 struct __align__(16) TileSmem {
     unsigned long long key[TILE * TILE];      // 32 KB, 16-byte chunks XOR-swizzled by row (key_index)
-    float rec[RCAP * REC];
+    float4 rec[RCAP * REC / 4];
     uint32_t leaf[LEAFCAP];                   // visible leaves of the round: first primitive << 4 | count
     uint32_t face[FACECAP];                   // box-face items of the round: agent << 3 | face
     uint2 surv[SCAP];                         // candidates whose pixel box holds a pixel centre: (item, box)
@@ -128,13 +128,13 @@ __device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const 
     if ((bx1 - bx0 + 1) * (by1 - by0 + 1) > TINY_MAX_PIXELS) {
         const int slot = atomicAdd(&s.n_rec, 1);
         if (slot < rec_cap) {
-            float* r = &s.rec[slot * REC];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { r[i] = q.nx[i]; r[4 + i] = q.ny[i]; r[8 + i] = q.nz[i]; }
-            r[12] = q.wx; r[13] = q.wy; r[14] = q.wz;
-            r[15] = __uint_as_float(key_lo);
+            float4* r = &s.rec[slot * (REC / 4)];
+            r[0] = make_float4(q.nx[0], q.nx[1], q.nx[2], q.nx[3]);
+            r[1] = make_float4(q.ny[0], q.ny[1], q.ny[2], q.ny[3]);
+            r[2] = make_float4(q.nz[0], q.nz[1], q.nz[2], q.nz[3]);
+            r[3] = make_float4(q.wx, q.wy, q.wz, __uint_as_float(key_lo));
             // the pixel box needs 6 bits per coordinate; the top-left bits ride along
-            r[16] = __uint_as_float((uint32_t)bx0 | ((uint32_t)by0 << 6) | ((uint32_t)bx1 << 12) | ((uint32_t)by1 << 18) | (q.tl << 24));
+            r[4].x = __uint_as_float((uint32_t)bx0 | ((uint32_t)by0 << 6) | ((uint32_t)bx1 << 12) | ((uint32_t)by1 << 18) | (q.tl << 24));
             ++n.recs;
             return;
         }
@@ -215,18 +215,20 @@ __device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool cl
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     unsigned long long touched = 0ull;     // 8x8 blocks
     for (int p = 0; p < n_rec; ++p) {
-        const float* r = &s.rec[p * REC];
-        const uint32_t bw = __float_as_uint(r[16]);
+        const float4* r = &s.rec[p * (REC / 4)];
+        const uint32_t bw = __float_as_uint(r[4].x);
         const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
         // first band of this warp at or after the box's first band
         const int band0 = by0 >> 2, band1 = by1 >> 2;
         int first = band0 + ((warp - band0) & (NW - 1));
         if (first > band1) continue;
         PrimEq q;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { q.nx[i] = r[i]; q.ny[i] = r[4 + i]; q.nz[i] = r[8 + i]; }
-        q.wx = r[12]; q.wy = r[13]; q.wz = r[14];
-        const uint32_t key_lo = __float_as_uint(r[15]);
+        const float4 r0 = r[0], r1 = r[1], r2 = r[2], r3 = r[3];
+        q.nx[0] = r0.x; q.nx[1] = r0.y; q.nx[2] = r0.z; q.nx[3] = r0.w;
+        q.ny[0] = r1.x; q.ny[1] = r1.y; q.ny[2] = r1.z; q.ny[3] = r1.w;
+        q.nz[0] = r2.x; q.nz[1] = r2.y; q.nz[2] = r2.z; q.nz[3] = r2.w;
+        q.wx = r3.x; q.wy = r3.y; q.wz = r3.z;
+        const uint32_t key_lo = __float_as_uint(r3.w);
         q.tl = bw >> 24;
         if (classify && (bx1 - bx0 + 1) * (by1 - by0 + 1) >= CLASSIFY_MIN_PIXELS) {
             // (b) lanes 0..15 classify this warp's 16 cells: reject / partly covered / inside
