@@ -2,9 +2,9 @@
 //
 // Input triangles are first fused pairwise into planar convex quads where the input allows it
 // (two consecutive triangles of one class sharing an edge: road, marking and wall quads), then
-// sorted along a Morton curve and cut into leaves of up to 32 primitives; leaves are grouped by
-// 32.  Primitives much longer than the average get small leaves of their own, so that one long
-// road quad does not inflate the box of 31 lane markings.  The renderer tests group boxes, then
+// sorted along a Morton curve and cut into leaves of up to LEAF_PRIMS primitives; leaves are
+// grouped by GROUP_LEAVES.  Primitives much longer than the average get leaves of their own, so
+// that one long road quad does not inflate the box of its neighbouring lane markings.  The renderer tests group boxes, then
 // leaf boxes, then primitives against each view frustum.
 #include <algorithm>
 #include <cmath>

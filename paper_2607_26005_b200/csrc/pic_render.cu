@@ -70,14 +70,15 @@ __device__ __forceinline__ unsigned long long block_mask(int bx0, int by0, int b
     return row * rows;
 }
 
-__device__ __forceinline__ void mark_touched(TileSmem& s, unsigned long long m) {
+__device__ __forceinline__ void mark_touched(uint32_t* touched, unsigned long long m) {
     const uint32_t lo = (uint32_t)m, hi = (uint32_t)(m >> 32);
-    if (lo & ~s.touched[0]) atomicOr(&s.touched[0], lo);
-    if (hi & ~s.touched[1]) atomicOr(&s.touched[1], hi);
+    if (lo & ~touched[0]) atomicOr(&touched[0], lo);
+    if (hi & ~touched[1]) atomicOr(&touched[1], hi);
 }
 
 // Is the box [lo,hi] (world) possibly inside the tile frustum?  Conservative.
-__device__ __forceinline__ bool box_visible(const TileSmem& s, const Node& b) {
+template <class S>
+__device__ __forceinline__ bool box_visible(const S& s, const Node& b) {
     const float ax = sub(b.lo[0], s.cam.px), bx = sub(b.hi[0], s.cam.px);
     const float ay = sub(b.lo[1], s.cam.py), by = sub(b.hi[1], s.cam.py);
     const float cx = 0.5f * (ax + bx), cy = 0.5f * (ay + by), cz = 0.5f * (b.lo[2] + b.hi[2]);
@@ -95,14 +96,16 @@ __device__ __forceinline__ bool box_visible(const TileSmem& s, const Node& b) {
     return vis;
 }
 
-__device__ __forceinline__ void put_fragment(TileSmem& s, int x, int y, uint32_t wbits, uint32_t key_lo) {
+template <class S>
+__device__ __forceinline__ void put_fragment(S& s, int x, int y, uint32_t wbits, uint32_t key_lo) {
     const unsigned long long k = make_key(wbits, key_lo);
     unsigned long long* addr = &s.key[key_index(x, y)];
     if (k > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, k);
 }
 
 // Rasterize a primitive from one thread: loop over its pixel box, atomic max per fragment.
-__device__ __forceinline__ int raster_in_thread(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, uint32_t box) {
+template <class S>
+__device__ __forceinline__ int raster_in_thread(S& s, uint32_t* touched, const TileCtx& t, const PrimEq& q, uint32_t key_lo, uint32_t box) {
     const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
     int frags = 0;
     for (int y = by0; y <= by1; ++y) {
@@ -112,15 +115,75 @@ __device__ __forceinline__ int raster_in_thread(TileSmem& s, const TileCtx& t, c
             if (wb) { put_fragment(s, x, y, wb, key_lo); ++frags; }
         }
     }
-    if (frags) mark_touched(s, block_mask(bx0, by0, bx1, by1));
+    if (frags) mark_touched(touched, block_mask(bx0, by0, bx1, by1));
     return frags;
 }
 
-struct Tally { int grp, leaf, tested, setup, tiny, recs, fallback, classified, cells; };
+// Plane p of the tile frustum, n.(q - m_w) >= 0 with q = X - P_ego (unit normals, offset -n.m_w
+// plus near / far), and for p >= 2 the same side plane in camera space.
+template <class S>
+__device__ __forceinline__ void tile_planes(S& s, int p, const Cam& c, const TileCtx& t) {
+    const float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
+    float nx, ny, nz, off = 0.f, sx = 0.f, sy = 0.f, sz = 0.f;
+    const float Rx = c.rx, Ry = c.ry, Dx = c.dx, Dy = c.dy, Dz = c.dz, Fx = c.fx_, Fy = c.fy_, Fz = c.fz_;
+    switch (p) {
+        case 0: nx = Fx; ny = Fy; nz = Fz; off = -t.near_z * 0.999f; break;                                       // z >= near
+        case 1: nx = -Fx; ny = -Fy; nz = -Fz; off = t.far_z * 1.001f; break;                                      // z <= far
+        case 2: nx = c.focx * Rx - l * Fx; ny = c.focx * Ry - l * Fy; nz = -l * Fz; sx = c.focx; sz = -l; break;  // x f >= z l
+        case 3: nx = r * Fx - c.focx * Rx; ny = r * Fy - c.focx * Ry; nz = r * Fz; sx = -c.focx; sz = r; break;   // x f <= z r
+        case 4: nx = c.focy * Dx - u * Fx; ny = c.focy * Dy - u * Fy; nz = c.focy * Dz - u * Fz; sy = c.focy; sz = -u; break;
+        default: nx = d * Fx - c.focy * Dx; ny = d * Fy - c.focy * Dy; nz = d * Fz - c.focy * Dz; sy = -c.focy; sz = d; break;
+    }
+    const float inv = rsqrtf(nx * nx + ny * ny + nz * nz);
+    nx *= inv; ny *= inv; nz *= inv;
+    s.plane[p][0] = nx; s.plane[p][1] = ny; s.plane[p][2] = nz;
+    s.plane[p][3] = off - (nx * c.mwx + ny * c.mwy + nz * c.mwz);
+    if (p >= 2) {
+        const float is = rsqrtf(sx * sx + sy * sy + sz * sz);
+        s.side[p - 2][0] = sx * is; s.side[p - 2][1] = sy * is; s.side[p - 2][2] = sz * is; s.side[p - 2][3] = 0.f;
+    }
+}
+
+// Which faces of another agent's box can reach the tile: 0 if its bounding sphere misses the
+// frustum, else the faces that can face the camera (all six near the near plane or inside the box).
+template <class S>
+__device__ __forceinline__ uint32_t box_faces(const S& s, const Cam& c, const TileCtx& t, const AgentGeom& g) {
+    const float hh = 0.5f * g.h;
+    const V3 ctr = rotate_to_camera(c, sub(sub(g.x, c.px), c.mwx), sub(sub(g.y, c.py), c.mwy), sub(hh, c.mwz));
+    const float rad = sqrtf(g.hl * g.hl + g.hw * g.hw + hh * hh) * 1.0001f + 1e-4f;
+    bool vis = (ctr.z + rad >= t.near_z * 0.999f) && (ctr.z - rad <= t.far_z * 1.001f);
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+        vis = vis && (s.side[p][0] * ctr.x + s.side[p][1] * ctr.y + s.side[p][2] * ctr.z >= -rad);
+    if (!vis) return 0u;
+    uint32_t faces = 0x3fu;
+    if (ctr.z - rad > t.near_z * 1.01f) {
+        const float dx = sub(c.mwx, sub(g.x, c.px)), dy = sub(c.mwy, sub(g.y, c.py));
+        const float u = g.c * dx + g.s * dy, v = g.c * dy - g.s * dx;
+        const float eps = 1e-4f * (1.f + fabsf(dx) + fabsf(dy));
+        faces = 0u;
+        if (u < -g.hl + eps) faces |= 1u;          // rear
+        if (u > g.hl - eps) faces |= 2u;           // front
+        if (v < -g.hw + eps) faces |= 4u;          // right
+        if (v > g.hw - eps) faces |= 8u;           // left
+        if (c.mwz < eps) faces |= 16u;             // bottom
+        if (c.mwz > g.h - eps) faces |= 32u;       // top
+    }
+    return faces;
+}
+
+// Work counters of a thread; the production kernel is compiled with NoTally, where they vanish.
+struct Tally { int grp, leaf, tested, setup, tiny, recs, fallback, classified, cells, jobs, coop; };
+struct NoCount {
+    __device__ __forceinline__ NoCount& operator++() { return *this; }
+    __device__ __forceinline__ NoCount& operator=(int) { return *this; }
+};
+struct NoTally { NoCount grp, leaf, tested, setup, tiny, recs, fallback, classified, cells, jobs, coop; };
 
 // Phase 2b body: set a surviving primitive up, rasterize it (tiny) or leave a record.
+template <class TL>
 __device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
-                                           const V3 Pn, uint32_t key_lo, uint32_t box, int rec_cap, Tally& n) {
+                                           const V3 Pn, uint32_t key_lo, uint32_t box, int rec_cap, TL& n) {
     PrimEq q;
     if (!prim_equations(V, quad, flags, Pn, q)) return;
     ++n.setup;
@@ -142,11 +205,12 @@ __device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const 
     } else {
         ++n.tiny;
     }
-    raster_in_thread(s, t, q, key_lo, box);
+    raster_in_thread(s, s.touched, t, q, key_lo, box);
 }
 
 // Candidate `i` of the round: a primitive of a visible leaf or a box-face item, in camera space.
-__device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderParams& P, int i, int nl, int e, uint32_t n_map_tris,
+template <class S>
+__device__ __forceinline__ bool fetch_candidate(const S& s, const RenderParams& P, int i, int nl, int e, uint32_t n_map_tris,
                                                 V3 (&V)[4], V3& Pn, uint32_t& key_lo, uint32_t& flags, bool want_plane) {
     const Cam& c = s.cam;
     if (i < nl * LEAF_PRIMS) {
@@ -176,7 +240,8 @@ __device__ __forceinline__ bool fetch_candidate(const TileSmem& s, const RenderP
 // loads and stores -- in phase 3 the rows of a cell belong to exactly one warp.  `need`: the edges
 // that still have to be tested on this cell (0: the cell is known to be covered and in depth
 // range; the range test rides on the edge tests).  Returns whether any lane produced a fragment.
-__device__ __forceinline__ bool raster_cell(TileSmem& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, int xx, int yy,
+template <class S>
+__device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, int xx, int yy,
                                             uint32_t need, int lane) {
     const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
     const float rx0 = s.ray_x[x], rx1 = s.ray_x[x + 1], ry = s.ray_y[y];
@@ -211,12 +276,14 @@ __device__ __forceinline__ bool raster_cell(TileSmem& s, const TileCtx& t, const
 // Phase 3: every warp walks all records but rasterizes only the bands (4 pixel rows) it owns --
 // band b belongs to warp b % NW -- so keys are updated without atomics and the bands of a large
 // primitive are shared out evenly.
-__device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool classify, Tally& n) {
+template <class S, class TL>
+__device__ __forceinline__ void raster_records(S& s, const float4* rec, uint32_t* touched_out, const TileCtx& t, int n_rec, bool classify, TL& n) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     unsigned long long touched = 0ull;     // 8x8 blocks
     for (int p = 0; p < n_rec; ++p) {
-        const float4* r = &s.rec[p * (REC / 4)];
+        const float4* r = &rec[p * (REC / 4)];
         const uint32_t bw = __float_as_uint(r[4].x);
+        if (bw >> 28) continue;                  // rasterized by its own thread, or degenerate
         const int bx0 = bw & 63, by0 = (bw >> 6) & 63, bx1 = (bw >> 12) & 63, by1 = (bw >> 18) & 63;
         // first band of this warp at or after the box's first band
         const int band0 = by0 >> 2, band1 = by1 >> 2;
@@ -229,7 +296,7 @@ __device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool cl
         q.nz[0] = r2.x; q.nz[1] = r2.y; q.nz[2] = r2.z; q.nz[3] = r2.w;
         q.wx = r3.x; q.wy = r3.y; q.wz = r3.z;
         const uint32_t key_lo = __float_as_uint(r3.w);
-        q.tl = bw >> 24;
+        q.tl = (bw >> 24) & 15u;
         if (classify && (bx1 - bx0 + 1) * (by1 - by0 + 1) >= CLASSIFY_MIN_PIXELS) {
             // (b) lanes 0..15 classify this warp's 16 cells: reject / partly covered / inside
             if (warp == 0) ++n.classified;
@@ -270,17 +337,19 @@ __device__ void raster_records(TileSmem& s, const TileCtx& t, int n_rec, bool cl
                 }
         }
     }
-    if (lane == 0 && touched) mark_touched(s, touched);
+    if (lane == 0 && touched) mark_touched(touched_out, touched);
 }
 
-// (d) keys -> class / depth images.
-__device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderParams& P, size_t view, int k, bool ego_active) {
+// (d) keys -> class / depth images.  `touched`: the 8x8 blocks that may hold a fragment; with
+// `clear`, the keys that were read are reset to "no fragment" for the next tile.
+template <class S>
+__device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderParams& P, size_t view, int k, bool ego_active,
+                                           unsigned long long touched, bool clear) {
     const size_t img = (size_t)P.H * P.W;
     uint8_t* oc = P.out_class + view * img;
     uint16_t* od = P.out_depth + view * img;
     float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
     const bool vec_ok = (P.W % 16 == 0) && o32 == nullptr;
-    const unsigned long long touched = ((unsigned long long)s.touched[1] << 32) | s.touched[0];
     const int segs_per_row = (t.tw + 15) >> 4;
     const int n_seg = t.th * segs_per_row;
     for (int seg = threadIdx.x; seg < n_seg; seg += NTHREADS) {
@@ -304,7 +373,9 @@ __device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderPara
             } else {
 #pragma unroll
                 for (int j = 0; j < 16; j += 2) {
-                    const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(&s.key[key_index(xs + j, y)]);
+                    ulonglong2* kp = reinterpret_cast<ulonglong2*>(&s.key[key_index(xs + j, y)]);
+                    const ulonglong2 kk = *kp;
+                    if (clear) *kp = make_ulonglong2(0ull, 0ull);
                     const float z0 = kk.x ? fast_rcp(__uint_as_float((uint32_t)(kk.x >> 32))) : bg_z;
                     const float z1 = kk.y ? fast_rcp(__uint_as_float((uint32_t)(kk.y >> 32))) : bg_z;
                     const uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bg_cls, c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bg_cls;
@@ -319,6 +390,7 @@ __device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderPara
         } else {
             for (int j = 0; j < 16 && xs + j < t.tw; ++j) {
                 const unsigned long long key = empty ? 0ull : s.key[key_index(xs + j, y)];
+                if (clear && !empty) s.key[key_index(xs + j, y)] = 0ull;
                 const float z = key ? fast_rcp(__uint_as_float((uint32_t)(key >> 32))) : bg_z;
                 oc[o + j] = (uint8_t)(key ? (uint32_t)(key & 0xff) : bg_cls);
                 od[o + j] = __half_as_ushort(__float2half_rn(z));
@@ -328,35 +400,56 @@ __device__ void store_tile(const TileSmem& s, const TileCtx& t, const RenderPara
     }
 }
 
-__global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    TileSmem& s = *reinterpret_cast<TileSmem*>(smem_raw);
-    const int tiles = P.tiles_x * P.tiles_y;
+// One unit of work: a tile of a view.
+struct Job {
+    int tile, k, a, e;
+    size_t view;
+    TileCtx t;
+};
+
+// Job `id` of the launch: tiles of a view are consecutive, views follow P.view_first.
+__device__ __forceinline__ Job decode_job(const RenderParams& P, unsigned id) {
+    const unsigned tiles = (unsigned)(P.tiles_x * P.tiles_y);
+    const unsigned vrel = id / tiles;
+    const unsigned long long v = (unsigned long long)P.view_first + vrel;
+    Job j;
+    j.tile = (int)(id - vrel * tiles);
+    j.view = (size_t)v;
+    const unsigned va = (unsigned)(v / (unsigned)P.K);        // E * A * K < 2^31 (checked by the launcher)
+    j.k = (int)((unsigned)v - va * (unsigned)P.K);
+    j.e = (int)(va / (unsigned)P.A);
+    j.a = (int)(va - (unsigned)j.e * (unsigned)P.A);
+    j.t.x0 = (j.tile % P.tiles_x) * TILE; j.t.y0 = (j.tile / P.tiles_x) * TILE;
+    j.t.tw = min(TILE, P.W - j.t.x0); j.t.th = min(TILE, P.H - j.t.y0);
+    j.t.w_near = P.w_near; j.t.w_far = P.w_far; j.t.near_z = P.near_z; j.t.far_z = P.far_z;
+    return j;
+}
+
+// Ray coordinates of tile column / row i (threads 0..63 of a pass call this with i = 0..63).
+// Columns / rows past the image edge (ragged tiles) continue the same formula, so the tables
+// stay monotone for the cell classification.
+template <class S>
+__device__ __forceinline__ void load_rays(S& s, const RenderParams& P, const Job& j, int i) {
+    const CamConst& ck = P.cam[j.k];
+    s.ray_x[i] = (j.t.x0 + i < P.W) ? __ldg(P.rig.ray_x + (size_t)j.k * P.W + j.t.x0 + i)
+                                    : __fdiv_rn(sub(add((float)(j.t.x0 + i), 0.5f), 0.5f * (float)P.W), ck.fx);
+    s.ray_y[i] = (j.t.y0 + i < P.H) ? __ldg(P.rig.ray_y + (size_t)j.k * P.H + j.t.y0 + i)
+                                    : __fdiv_rn(sub(add((float)(j.t.y0 + i), 0.5f), 0.5f * (float)P.H), ck.fy);
+}
+
+// A whole tile rendered by the CTA in barrier-separated phases with per-round lists: any number of
+// groups, boxes, survivors and records.  The fused kernel uses it for the tiles whose lists do
+// not fit its per-warp front end.
+template <class TL>
+__device__ __forceinline__ void cooperative_job(TileSmem& s, const RenderParams& P, unsigned job_id, TL& n) {
+    const Job job = decode_job(P, job_id);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool classify = !(P.debug_flags & 1);
     const int rec_cap = (P.debug_flags & 2) ? 2 : RCAP;
     const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave after phase `stop` (image incomplete)
-    Tally n = {0, 0, 0, 0, 0, 0, 0, 0, 0};
-    // grid: x = tile + tiles * camera, y = agent, z = env; a 1-D grid (gridDim.y == 0 is impossible,
-    // so "linear" is flagged by P.linear) serves view sub-ranges
-    int tile, k, a, e;
-    if (P.linear) {
-        const unsigned job = blockIdx.x;
-        const unsigned v = (unsigned)P.view_first + job / (unsigned)tiles;
-        tile = (int)(job % (unsigned)tiles);
-        k = (int)(v % (unsigned)P.K);
-        a = (int)((v / (unsigned)P.K) % (unsigned)P.A);
-        e = (int)(v / ((unsigned)P.K * (unsigned)P.A));
-    } else {
-        k = (int)(blockIdx.x / (unsigned)tiles);
-        tile = (int)(blockIdx.x - (unsigned)k * (unsigned)tiles);
-        a = (int)blockIdx.y; e = (int)blockIdx.z;
-    }
-    const size_t view = ((size_t)e * P.A + a) * P.K + k;
-    TileCtx t;
-    t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
-    t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
-    t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
+    const int k = job.k, a = job.a, e = job.e;
+    const size_t view = job.view;
+    const TileCtx t = job.t;
     const bool ego_active = P.agents[(size_t)e * P.A + a].active != 0;
     // issued now so that their latency overlaps the prologue: the map of this environment, the
     // group box this lane tests first, and the background of the two rows this thread stores
@@ -374,37 +467,10 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             s.n_rec = 0; s.n_leaf = 0; s.n_face = 0; s.n_surv = 0;
             s.touched[0] = 0u; s.touched[1] = 0u;
         } else {
-            // frustum planes n.(q - m_w) >= 0 with q = X - P_ego; unit normals, offset -n.m_w (+ near/far)
-            const int p = threadIdx.x;
-            const float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
-            float nx, ny, nz, off = 0.f, sx = 0.f, sy = 0.f, sz = 0.f;
-            const float Rx = c.rx, Ry = c.ry, Dx = c.dx, Dy = c.dy, Dz = c.dz, Fx = c.fx_, Fy = c.fy_, Fz = c.fz_;
-            switch (p) {
-                case 0: nx = Fx; ny = Fy; nz = Fz; off = -P.near_z * 0.999f; break;                                       // z >= near
-                case 1: nx = -Fx; ny = -Fy; nz = -Fz; off = P.far_z * 1.001f; break;                                      // z <= far
-                case 2: nx = c.focx * Rx - l * Fx; ny = c.focx * Ry - l * Fy; nz = -l * Fz; sx = c.focx; sz = -l; break;  // x f >= z l
-                case 3: nx = r * Fx - c.focx * Rx; ny = r * Fy - c.focx * Ry; nz = r * Fz; sx = -c.focx; sz = r; break;   // x f <= z r
-                case 4: nx = c.focy * Dx - u * Fx; ny = c.focy * Dy - u * Fy; nz = c.focy * Dz - u * Fz; sy = c.focy; sz = -u; break;
-                default: nx = d * Fx - c.focy * Dx; ny = d * Fy - c.focy * Dy; nz = d * Fz - c.focy * Dz; sy = -c.focy; sz = d; break;
-            }
-            const float inv = rsqrtf(nx * nx + ny * ny + nz * nz);
-            nx *= inv; ny *= inv; nz *= inv;
-            s.plane[p][0] = nx; s.plane[p][1] = ny; s.plane[p][2] = nz;
-            s.plane[p][3] = off - (nx * c.mwx + ny * c.mwy + nz * c.mwz);
-            if (p >= 2) {
-                const float is = rsqrtf(sx * sx + sy * sy + sz * sz);
-                s.side[p - 2][0] = sx * is; s.side[p - 2][1] = sy * is; s.side[p - 2][2] = sz * is; s.side[p - 2][3] = 0.f;
-            }
+            tile_planes(s, threadIdx.x, c, t);
         }
     } else if (threadIdx.x >= 64) {
-        // columns / rows past the image edge (ragged tiles) continue the same formula, so the
-        // tables stay monotone for the cell classification
-        const int i = threadIdx.x - 64;
-        const CamConst& ck = P.cam[k];
-        s.ray_x[i] = (t.x0 + i < P.W) ? __ldg(P.rig.ray_x + (size_t)k * P.W + t.x0 + i)
-                                      : __fdiv_rn(sub(add((float)(t.x0 + i), 0.5f), 0.5f * (float)P.W), ck.fx);
-        s.ray_y[i] = (t.y0 + i < P.H) ? __ldg(P.rig.ray_y + (size_t)k * P.H + t.y0 + i)
-                                      : __fdiv_rn(sub(add((float)(t.y0 + i), 0.5f), 0.5f * (float)P.H), ck.fy);
+        load_rays(s, P, job, threadIdx.x - 64);
     }
 #pragma unroll
     for (int i = 0; i < TILE * TILE / 2 / NTHREADS; ++i)
@@ -445,29 +511,8 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
                 if (b == a) continue;
                 const AgentGeom g = P.agents[(size_t)e * P.A + b];
                 if (!g.active) continue;
-                const float hh = 0.5f * g.h;
-                const V3 ctr = rotate_to_camera(c, sub(sub(g.x, c.px), c.mwx), sub(sub(g.y, c.py), c.mwy), sub(hh, c.mwz));
-                const float rad = sqrtf(g.hl * g.hl + g.hw * g.hw + hh * hh) * 1.0001f + 1e-4f;
-                bool vis = (ctr.z + rad >= t.near_z * 0.999f) && (ctr.z - rad <= t.far_z * 1.001f);
-#pragma unroll
-                for (int p = 0; p < 4; ++p)
-                    vis = vis && (s.side[p][0] * ctr.x + s.side[p][1] * ctr.y + s.side[p][2] * ctr.z >= -rad);
-                if (!vis) continue;
-                // the camera position in the box frame decides which faces can face the camera;
-                // near the near plane (or inside the box) every face is kept
-                uint32_t faces = 0x3fu;
-                if (ctr.z - rad > t.near_z * 1.01f) {
-                    const float dx = sub(c.mwx, sub(g.x, c.px)), dy = sub(c.mwy, sub(g.y, c.py));
-                    const float u = g.c * dx + g.s * dy, v = g.c * dy - g.s * dx;
-                    const float eps = 1e-4f * (1.f + fabsf(dx) + fabsf(dy));
-                    faces = 0u;
-                    if (u < -g.hl + eps) faces |= 1u;          // rear
-                    if (u > g.hl - eps) faces |= 2u;           // front
-                    if (v < -g.hw + eps) faces |= 4u;          // right
-                    if (v > g.hw - eps) faces |= 8u;           // left
-                    if (c.mwz < eps) faces |= 16u;             // bottom
-                    if (c.mwz > g.h - eps) faces |= 32u;       // top
-                }
+                uint32_t faces = box_faces(s, c, t, g);
+                if (!faces) continue;
                 int slot = atomicAdd(&s.n_face, __popc(faces));
                 for (; faces; faces &= faces - 1) s.face[slot++] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
             }
@@ -511,52 +556,331 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             if (round + 1 < n_rounds) {
                 // the lists are reused by the next round; records are rasterized now if they might overflow
                 const int n_rec = min(s.n_rec, rec_cap);
-                if (n_rec > rec_cap / 2) raster_records(s, t, n_rec, classify, n);
+                if (n_rec > rec_cap / 2) raster_records(s, s.rec, s.touched, t, n_rec, classify, n);
                 __syncthreads();
                 if (threadIdx.x == 0) { s.n_leaf = 0; s.n_face = 0; s.n_surv = 0; if (n_rec > rec_cap / 2) s.n_rec = 0; }
                 __syncthreads();
             }
         }
         // ---- phase 3 (b)+(c): one warp per record
-        if (stop == 0 || stop > 5) raster_records(s, t, min(s.n_rec, rec_cap), classify, n);
+        if (stop == 0 || stop > 5) raster_records(s, s.rec, s.touched, t, min(s.n_rec, rec_cap), classify, n);
         if (stop == 5 && threadIdx.x == 0) { s.touched[0] = 0xffffffffu; s.touched[1] = 0xffffffffu; }
         __syncthreads();
     }
     // ---- phase 4 (d)
-    store_tile(s, t, P, view, k, ego_active);
-    if (P.counters) {
-        const int vals[9] = {n.grp, n.leaf, n.tested, n.setup, n.tiny, n.recs, n.fallback, n.classified, n.cells};
+    store_tile(s, t, P, view, k, ego_active, ((unsigned long long)s.touched[1] << 32) | s.touched[0], false);
+    if (threadIdx.x == 0) { ++n.jobs; ++n.coop; }
+}
+
+// Adds the CTA's tallies to the optional counters: [0] tiles, [1..9] group tests, leaf tests,
+// candidates tested, set up, rasterized by their thread, records, record-list overflows, records
+// classified per cell, cells visited, [10] tiles rendered by cooperative_job.
+__device__ __forceinline__ void flush_counters(const RenderParams&, const NoTally&) {}
+__device__ __forceinline__ void flush_counters(const RenderParams& P, const Tally& n) {
+    const int lane = threadIdx.x & 31;
+    const int vals[11] = {n.jobs, n.grp, n.leaf, n.tested, n.setup, n.tiny, n.recs, n.fallback, n.classified, n.cells, n.coop};
 #pragma unroll
-        for (int i = 0; i < 9; ++i) {
-            // classified / cells are counted by every lane of a warp alike
-            const int v = (i >= 7 && lane != 0) ? 0 : vals[i];
-            const int sum = __reduce_add_sync(0xffffffffu, v);
-            if (lane == 0 && sum) atomicAdd(&P.counters[1 + i], (unsigned long long)sum);
-        }
-        if (threadIdx.x == 0) atomicAdd(&P.counters[0], 1ull);
+    for (int i = 0; i < 11; ++i) {
+        // classified / cells are counted by every lane of a warp alike
+        const int v = ((i == 8 || i == 9) && lane != 0) ? 0 : vals[i];
+        const int sum = __reduce_add_sync(0xffffffffu, v);
+        if (lane == 0 && sum) atomicAdd(&P.counters[i], (unsigned long long)sum);
     }
 }
 
-static_assert(sizeof(TileSmem) <= 44 * 1024, "TileSmem must leave room for 5 CTAs per SM (228 KB, 1 KB reserved per CTA)");
-size_t render_smem_bytes() { return sizeof(TileSmem); }
+// ---------------------------------------------------------------------------------------------
+// Fused kernel: a CTA takes NW consecutive tiles.
+//
+//   front   warp w culls tile w on its own (hierarchy, boxes, candidate tests), with warp-level
+//           synchronisation only and its lists in the (still unused) key buffer; the survivors
+//           of the NW tiles then get consecutive ranges of one record pool and are set up, one
+//           lane per survivor.  Dense passes, no CTA barrier inside.
+//   back    tile after tile, by the whole CTA: primitives of <= TINY_MAX_PIXELS pixels by one
+//           thread each (atomic max), the others by band-owning warps (raster_records), then the
+//           store, which also resets the keys it read.
+//   rest    tiles whose lists or records did not fit go through cooperative_job afterwards.
+// ---------------------------------------------------------------------------------------------
+constexpr int POOL = 144;         // records shared by the NW tiles of a CTA
+constexpr int W_LEAF = 256;       // per-warp front-end lists (they live in the key buffer, 8 KB per warp)
+constexpr int W_FACE = 384;
+constexpr int W_SURV = 256;
+constexpr uint32_t REC_TINY = 1u << 28, REC_DEAD = 1u << 29;   // flags in the box word of a record
+
+struct __align__(16) FrontLists {
+    uint2 surv[W_SURV];                       // (candidate, pixel box)
+    uint32_t leaf[W_LEAF];                    // first primitive << 4 | count
+    uint32_t face[W_FACE];                    // agent << 3 | face
+    float plane[6][4];
+    float side[4][4];
+    Cam cam;
+    int n_face, pad[3];
+};
+
+struct __align__(16) FusedSmem {
+    union {
+        unsigned long long key[TILE * TILE];  // back end
+        FrontLists fl[NW];                    // front end
+    };
+    float4 pool[POOL * REC / 4];
+    float ray_x[TILE], ray_y[TILE];
+    uint32_t touched[NW][2];
+    int n_surv[NW];                           // survivors of tile w; -1: lists overflowed, -2: no such tile
+};
+static_assert(sizeof(FrontLists) * NW <= sizeof(unsigned long long) * TILE * TILE, "front-end lists must fit the key buffer");
+static_assert(sizeof(FusedSmem) <= 44 * 1024 && sizeof(TileSmem) <= 44 * 1024,
+              "shared memory must leave room for 5 CTAs per SM (228 KB, 1 KB reserved per CTA)");
+constexpr size_t RENDER_SMEM = sizeof(FusedSmem) > sizeof(TileSmem) ? sizeof(FusedSmem) : sizeof(TileSmem);
+
+__device__ __forceinline__ void write_record(float4* r, const PrimEq& q, uint32_t key_lo, uint32_t box, uint32_t extra) {
+    const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    r[0] = make_float4(q.nx[0], q.nx[1], q.nx[2], q.nx[3]);
+    r[1] = make_float4(q.ny[0], q.ny[1], q.ny[2], q.ny[3]);
+    r[2] = make_float4(q.nz[0], q.nz[1], q.nz[2], q.nz[3]);
+    r[3] = make_float4(q.wx, q.wy, q.wz, __uint_as_float(key_lo));
+    // the pixel box needs 6 bits per coordinate; the top-left bits and the flags ride along
+    r[4].x = __uint_as_float(bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24) | extra);
+}
+
+__device__ __forceinline__ void read_record(const float4* r, PrimEq& q, uint32_t& key_lo) {
+    const float4 r0 = r[0], r1 = r[1], r2 = r[2], r3 = r[3];
+    q.nx[0] = r0.x; q.nx[1] = r0.y; q.nx[2] = r0.z; q.nx[3] = r0.w;
+    q.ny[0] = r1.x; q.ny[1] = r1.y; q.ny[2] = r1.z; q.ny[3] = r1.w;
+    q.nz[0] = r2.x; q.nz[1] = r2.y; q.nz[2] = r2.z; q.nz[3] = r2.w;
+    q.wx = r3.x; q.wy = r3.y; q.wz = r3.z;
+    key_lo = __float_as_uint(r3.w);
+}
+
+// Front end of one tile by one warp: fills f.leaf / f.face / f.surv.  Returns the number of
+// survivors, or -1 if a list overflowed (the tile then goes to cooperative_job).
+template <class TL>
+__device__ __forceinline__ int front_cull(FrontLists& f, const RenderParams& P, const Job& job, const MapInfo& mi,
+                                          int lane, int& nl_out, TL& n) {
+    const TileCtx& t = job.t;
+    if (lane < 7) {
+        Cam c;
+        load_camera(c, P.cams[job.view], P.cam[job.k], P.W, P.H);
+        if (lane == 6) { f.cam = c; f.n_face = 0; }
+        else tile_planes(f, lane, c, t);
+    }
+    __syncwarp();
+    const Cam& c = f.cam;
+    // ---- hierarchy: 32 groups per pass, a visible group's leaves one per lane
+    int n_leaf = 0;
+    for (uint32_t g0 = mi.group_begin; g0 < mi.group_end; g0 += 32) {
+        const uint32_t g = g0 + lane;
+        bool vis = false;
+        Node gn;
+        gn.first = 0; gn.count = 0;
+        if (g < mi.group_end) { gn = P.groups[g]; vis = box_visible(f, gn); ++n.grp; }
+        for (unsigned gm = __ballot_sync(0xffffffffu, vis); gm; gm &= gm - 1) {
+            const int src = __ffs(gm) - 1;
+            const uint32_t first = __shfl_sync(0xffffffffu, gn.first, src);
+            const uint32_t cnt = __shfl_sync(0xffffffffu, gn.count, src);
+            bool lvis = false;
+            Node lf;
+            lf.first = 0; lf.count = 0;
+            if (lane < (int)cnt) { lf = P.leaves[first + lane]; lvis = box_visible(f, lf); ++n.leaf; }
+            const unsigned lm = __ballot_sync(0xffffffffu, lvis);
+            if (lvis) {
+                const int slot = n_leaf + __popc(lm & ((1u << lane) - 1u));
+                if (slot < W_LEAF) f.leaf[slot] = (lf.first << 4) | lf.count;
+            }
+            n_leaf += __popc(lm);
+        }
+    }
+    // ---- other agents' boxes
+    for (int b0 = 0; b0 < P.A; b0 += 32) {
+        const int b = b0 + lane;
+        uint32_t faces = 0u;
+        if (b < P.A && b != job.a) {
+            const AgentGeom g = P.agents[(size_t)job.e * P.A + b];
+            if (g.active) faces = box_faces(f, c, t, g);
+        }
+        if (faces) {
+            int slot = atomicAdd(&f.n_face, __popc(faces));
+            for (; faces; faces &= faces - 1, ++slot)
+                if (slot < W_FACE) f.face[slot] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
+        }
+    }
+    __syncwarp();
+    const int n_face = f.n_face;
+    if (n_leaf > W_LEAF || n_face > W_FACE) return -1;
+    nl_out = n_leaf;
+    // ---- candidates: camera space, pixel box; survivors are compacted
+    const int n_items = n_leaf * LEAF_PRIMS + n_face;
+    int n_surv = 0;
+    for (int i0 = 0; i0 < n_items; i0 += 32) {
+        const int i = i0 + lane;
+        V3 V[4], Pn;
+        uint32_t key_lo, flags, box = 0;
+        bool keep = false;
+        if (i < n_items && fetch_candidate(f, P, i, n_leaf, job.e, mi.n_tris, V, Pn, key_lo, flags, false)) {
+            ++n.tested;
+            keep = pixel_box(c, t, V, box);
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (keep) {
+            const int slot = n_surv + __popc(m & ((1u << lane) - 1u));
+            if (slot < W_SURV) f.surv[slot] = make_uint2((uint32_t)i, box);
+        }
+        n_surv += __popc(m);
+    }
+    __syncwarp();
+    return n_surv > W_SURV ? -1 : n_surv;
+}
+
+// Set-up of a tile's survivors by its warp: survivor i becomes record i of `rec`.
+template <class TL>
+__device__ __forceinline__ void front_setup(const FrontLists& f, float4* rec, const RenderParams& P, const Job& job,
+                                            const MapInfo& mi, int nl, int ns, int lane, TL& n) {
+    for (int i = lane; i < ns; i += 32) {
+        const uint2 sv = f.surv[i];
+        V3 V[4], Pn;
+        uint32_t key_lo, flags;
+        fetch_candidate(f, P, (int)sv.x, nl, job.e, mi.n_tris, V, Pn, key_lo, flags, true);
+        PrimEq q;
+        float4* r = rec + i * (REC / 4);
+        if (!prim_equations(V, flags & 1u, flags, Pn, q)) { r[4].x = __uint_as_float(REC_DEAD); continue; }
+        ++n.setup;
+        const uint32_t box = sv.y;
+        const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+        const bool tiny = (bx1 - bx0 + 1) * (by1 - by0 + 1) <= TINY_MAX_PIXELS;
+        if (tiny) ++n.tiny; else ++n.recs;
+        write_record(r, q, key_lo, box, tiny ? REC_TINY : 0u);
+    }
+}
+
+// Back end of one tile by the CTA; the keys are all "no fragment" on entry and on exit.
+template <class TL>
+__device__ __forceinline__ void back_job(FusedSmem& s, const RenderParams& P, const Job& job, bool ego_active,
+                                         const float4* rec, int n_rec, uint32_t* touched, bool classify, int stop, TL& n) {
+    const TileCtx& t = job.t;
+    for (int i = threadIdx.x; i < n_rec; i += NTHREADS) {
+        const float4* r = rec + i * (REC / 4);
+        const uint32_t bw = __float_as_uint(r[4].x);
+        if (bw & REC_TINY) {
+            PrimEq q;
+            uint32_t key_lo;
+            read_record(r, q, key_lo);
+            q.tl = (bw >> 24) & 15u;
+            const uint32_t box = (bw & 63u) | (((bw >> 6) & 63u) << 8) | (((bw >> 12) & 63u) << 16) | (((bw >> 18) & 63u) << 24);
+            raster_in_thread(s, touched, t, q, key_lo, box);
+        }
+    }
+    __syncthreads();
+    if (stop == 0 || stop > 5) raster_records(s, rec, touched, t, n_rec, classify, n);
+    if (stop == 5 && threadIdx.x == 0) { touched[0] = 0xffffffffu; touched[1] = 0xffffffffu; }
+    __syncthreads();
+    // the cell raster of a ragged tile may leave keys past the image edge, which the store never
+    // visits: such a tile clears the whole buffer instead of the keys it read
+    const bool ragged = t.tw < TILE || t.th < TILE;
+    store_tile(s, t, P, job.view, job.k, ego_active, ((unsigned long long)touched[1] << 32) | touched[0], !ragged);
+    if (ragged) {
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < TILE * TILE / 2 / NTHREADS; ++i)
+            reinterpret_cast<ulonglong2*>(s.key)[i * NTHREADS + threadIdx.x] = make_ulonglong2(0ull, 0ull);
+    }
+}
+
+template <class TL>
+__global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    FusedSmem& s = *reinterpret_cast<FusedSmem*>(smem_raw);
+    TileSmem& cs = *reinterpret_cast<TileSmem*>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned first = blockIdx.x * (unsigned)NW, n_jobs = P.n_jobs;
+    TL n = {};
+    const bool classify = !(P.debug_flags & 1);
+    const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave work out (image incomplete)
+    // test aids: a pool of 2 records sends nearly every tile to cooperative_job, one of 40 mixes both paths
+    const int pool_cap = (P.debug_flags & 2) ? 2 : (P.debug_flags & 8) ? 40 : POOL;
+    if (threadIdx.x < 2 * NW) (&s.touched[0][0])[threadIdx.x] = 0u;
+
+    // ---- front end: warp w culls tile first + w
+    const bool valid = first + warp < n_jobs;
+    Job job;
+    MapInfo mi;
+    int nl = 0, ns = -2;
+    if (valid) {
+        job = decode_job(P, first + warp);
+        mi = P.env_maps[job.e];
+        ns = 0;
+        if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
+        else if (P.agents[(size_t)job.e * P.A + job.a].active != 0 && stop != 1) ns = front_cull(s.fl[warp], P, job, mi, lane, nl, n);
+    }
+    if (lane == 0) s.n_surv[warp] = ns;
+    __syncthreads();
+    // every thread lays the record pool out alike: tiles in order, a tile that does not fit is left
+    // out.  One byte per tile: first record, and count (0xff: to cooperative_job, 0xfe: no such tile)
+    uint32_t bases = 0u, cnts = 0u;
+    {
+        int off = 0;
+#pragma unroll
+        for (int j = 0; j < NW; ++j) {
+            const int c = s.n_surv[j];
+            bases |= (uint32_t)off << (8 * j);
+            if (c >= 0 && off + c <= pool_cap) { cnts |= (uint32_t)c << (8 * j); off += c; }
+            else cnts |= ((c == -2) ? 0xfeu : 0xffu) << (8 * j);
+        }
+    }
+    {
+        const int my_base = (int)((bases >> (8 * warp)) & 0xffu), my_cnt = (int)((cnts >> (8 * warp)) & 0xffu);
+        if (my_cnt == 0xff) { n.grp = 0; n.leaf = 0; n.tested = 0; }       // counted again by cooperative_job
+        else if (my_cnt != 0xfe && my_cnt > 0) front_setup(s.fl[warp], s.pool + my_base * (REC / 4), P, job, mi, nl, my_cnt, lane, n);
+    }
+    __syncthreads();
+    // ---- back end: the lists are dead, their memory becomes the key buffer
+#pragma unroll
+    for (int i = 0; i < TILE * TILE / 2 / NTHREADS; ++i)
+        reinterpret_cast<ulonglong2*>(s.key)[i * NTHREADS + threadIdx.x] = make_ulonglong2(0ull, 0ull);
+    bool rays_loaded = false;
+#pragma unroll 1
+    for (int j = 0; j < NW; ++j) {
+        const int cj = (int)((cnts >> (8 * j)) & 0xffu);
+        if (cj >= 0xfe) continue;                   // uniform over the CTA
+        const Job jb = decode_job(P, first + j);
+        const bool ego_active = P.agents[(size_t)jb.e * P.A + jb.a].active != 0;
+        if (!rays_loaded) {
+            if (threadIdx.x < TILE) load_rays(s, P, jb, threadIdx.x);
+            rays_loaded = true;
+            __syncthreads();
+        }
+        back_job(s, P, jb, ego_active, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, s.touched[j], classify, stop, n);
+        if (threadIdx.x == 0) ++n.jobs;
+        // the ray tables of the next tile of the pool: nothing reads them between here and the barrier
+        int nx = -1;
+        for (int j2 = NW - 1; j2 > j; --j2) if (((cnts >> (8 * j2)) & 0xffu) < 0xfeu) nx = j2;
+        if (nx >= 0 && threadIdx.x < TILE) load_rays(s, P, decode_job(P, first + nx), threadIdx.x);
+        __syncthreads();
+    }
+    // ---- the rest: tiles that did not fit
+#pragma unroll 1
+    for (int j = 0; j < NW; ++j)
+        if (((cnts >> (8 * j)) & 0xffu) == 0xffu) {
+            cooperative_job(cs, P, first + j, n);
+            __syncthreads();
+        }
+    flush_counters(P, n);
+}
+
+size_t render_smem_bytes() { return RENDER_SMEM; }
 
 cudaError_t configure_render_kernel() {
-    return cudaFuncSetAttribute(render_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+    cudaError_t err = cudaFuncSetAttribute(render_kernel<NoTally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(render_kernel<Tally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
 }
 
 cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cudaStream_t stream) {
     RenderParams P = P0;
-    const long long tiles = (long long)P.tiles_x * P.tiles_y;
-    const bool whole = P.view_first == 0 && n_views == (long long)P.E * P.A * P.K;
-    if (whole && tiles * P.K <= 0x7fffffffLL && P.A <= 65535 && P.E <= 65535) {
-        P.linear = 0;
-        render_kernel<<<dim3((unsigned)(tiles * P.K), (unsigned)P.A, (unsigned)P.E), NTHREADS, sizeof(TileSmem), stream>>>(P);
-    } else {
-        const long long blocks = n_views * tiles;
-        if (blocks > 0x7fffffffLL || (long long)P.E * P.A * P.K > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-        P.linear = 1;
-        render_kernel<<<(unsigned)blocks, NTHREADS, sizeof(TileSmem), stream>>>(P);
-    }
+    const long long jobs = n_views * P.tiles_x * P.tiles_y;
+    if (jobs > 0x7fffffffLL || (long long)P.E * P.A * P.K > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (jobs <= 0) return cudaSuccess;
+    P.n_jobs = (uint32_t)jobs;
+    const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
+    if (P.counters) render_kernel<Tally><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
+    else render_kernel<NoTally><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     return cudaGetLastError();
 }
 

@@ -91,7 +91,7 @@ struct RenderParams {
     float* out_depth32;             // optional
     unsigned long long* counters;   // optional [16]
     int32_t debug_flags;            // bit 0: no per-cell trivial accept/reject, bit 1: record list of 2 entries (forces the overflow path)
-    int32_t linear;                 // 1: 1-D grid over a view sub-range, 0: grid (tile+camera, agent, env); set by the launcher
+    uint32_t n_jobs;                // tiles to render in this launch (views x tiles per view); set by the launcher
     long long view_first;           // render views [view_first, view_first + gridDim / tiles)
     CamConst cam[MAX_CAMS];
 };

@@ -145,7 +145,7 @@ def test_production_kernel_equals_exhaustive_kernel(gu, cfg, E):
         if count < V:
             assert (a[0][count:] == 255).all()          # views outside the range are left untouched
         # switching the kernel's shortcuts off / forcing its overflow path must not change the image
-        for flags in (1, 2, 3):
+        for flags in (1, 2, 3, 4, 8, 9):
             c = g.render(brute=False, view_first=0, view_count=count, debug_flags=flags)
             assert (a[0][:count] == c[0][:count]).all() and (a[2][:count] == c[2][:count]).all()
     finally:
