@@ -68,6 +68,7 @@ struct pic_scene {
     pic::Prim* d_prims = nullptr;
     pic::AgentGeom* d_agents = nullptr;
     pic::ViewCam* d_cams = nullptr;   // [E*A*K]
+    uint32_t* d_overflow = nullptr;   // [1 + E*A*K*tiles] tiles handed from the fused to the cooperative render kernel
     float* d_tables = nullptr;        // per-camera ray and background tables, K*(W+3H) words
     float* d_state = nullptr;       // [E*A*4]
     float* d_dims = nullptr;        // [E*A*3]
@@ -106,7 +107,7 @@ struct DeviceGuard {
 
 void free_scene(pic_scene* s) {
     cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
-    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
+    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
     if (s->ev) {
@@ -132,6 +133,7 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.env_map = s->d_env_map; P.env_maps = s->d_env_maps; P.maps = s->d_maps; P.groups = s->d_groups; P.leaves = s->d_leaves; P.prims = s->d_prims;
     P.agents = s->d_agents;
     P.cams = s->d_cams;
+    P.overflow = s->d_overflow;
     P.rig.ray_x = s->d_tables;
     P.rig.ray_y = P.rig.ray_x + (size_t)s->K * s->W;
     P.rig.bg_z = P.rig.ray_y + (size_t)s->K * s->H;
@@ -236,6 +238,7 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_prims, sizeof(pic::Prim) * np);
     dmalloc((void**)&s->d_agents, sizeof(pic::AgentGeom) * n_agents);
     dmalloc((void**)&s->d_cams, sizeof(pic::ViewCam) * n_agents * d->K);
+    dmalloc((void**)&s->d_overflow, sizeof(uint32_t) * (1 + (size_t)n_agents * d->K * ((d->W + pic::TILE - 1) / pic::TILE) * ((d->H + pic::TILE - 1) / pic::TILE)));
     dmalloc((void**)&s->d_tables, sizeof(float) * (size_t)d->K * ((size_t)d->W + 3 * (size_t)d->H));
     dmalloc((void**)&s->d_state, sizeof(float) * 4 * n_agents);
     dmalloc((void**)&s->d_dims, sizeof(float) * 3 * n_agents);

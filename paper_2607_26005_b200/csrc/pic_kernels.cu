@@ -71,8 +71,9 @@ __global__ void agent_kernel(int n, const float* __restrict__ poses, float* stat
 
 // Per-camera tables: ray coordinates of every pixel column / row and the background of every row.
 __global__ void rig_kernel(const __grid_constant__ RigParams R, float* __restrict__ ray_x, float* __restrict__ ray_y,
-                           float* __restrict__ bg_z, uint32_t* __restrict__ bg_cls) {
+                           float* __restrict__ bg_z, uint32_t* __restrict__ bg_cls, uint32_t* overflow) {
     const int k = blockIdx.x;
+    if (overflow && k == 0 && threadIdx.x == 0) overflow[0] = 0u;   // the render kernels' list of left-out tiles starts empty (absent for callers that do not use them)
     const CamConst c = R.cam[k];
     const float cx = 0.5f * (float)R.W, cy = 0.5f * (float)R.H;
     for (int u = threadIdx.x; u < R.W; u += blockDim.x)
@@ -211,7 +212,7 @@ cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses
     float* ray_y = ray_x + (size_t)P.K * P.W;
     float* bg_z = ray_y + (size_t)P.K * P.H;
     uint32_t* bg_cls = reinterpret_cast<uint32_t*>(bg_z + (size_t)P.K * P.H);
-    rig_kernel<<<P.K, 256, 0, stream>>>(R, ray_x, ray_y, bg_z, bg_cls);
+    rig_kernel<<<P.K, 256, 0, stream>>>(R, ray_x, ray_y, bg_z, bg_cls, P.overflow);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess || n_agents <= 0) return err;
     agent_kernel<<<(n_agents + 127) / 128, 128, 0, stream>>>(n_agents, poses, state, actions, dims, active, agents_out,

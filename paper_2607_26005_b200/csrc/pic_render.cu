@@ -41,6 +41,7 @@ constexpr int FACECAP = 6 * BOX_ROUND;
 constexpr int SCAP = 128;         // candidates that survive the pixel-box test, per round
 constexpr int TINY_MAX_PIXELS = 4;         // pixel centres in the box of a primitive rasterized by its own thread
 constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large classify cells before rasterizing
+constexpr int CLASSIFY_MIN_STRIP = 96;     // the same for the part of a box inside a 16-row strip
 
 struct __align__(16) TileSmem {
     unsigned long long key[TILE * TILE];      // 32 KB, 16-byte chunks XOR-swizzled by row (key_index)
@@ -344,7 +345,7 @@ __device__ __forceinline__ void raster_records(S& s, const float4* rec, uint32_t
 // `clear`, the keys that were read are reset to "no fragment" for the next tile.
 template <class S>
 __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderParams& P, size_t view, int k, bool ego_active,
-                                           unsigned long long touched, bool clear) {
+                                           unsigned long long touched, bool clear, int tid = threadIdx.x, int nthr = NTHREADS) {
     const size_t img = (size_t)P.H * P.W;
     uint8_t* oc = P.out_class + view * img;
     uint16_t* od = P.out_depth + view * img;
@@ -352,7 +353,7 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
     const bool vec_ok = (P.W % 16 == 0) && o32 == nullptr;
     const int segs_per_row = (t.tw + 15) >> 4;
     const int n_seg = t.th * segs_per_row;
-    for (int seg = threadIdx.x; seg < n_seg; seg += NTHREADS) {
+    for (int seg = tid; seg < n_seg; seg += nthr) {
         const int y = (segs_per_row == 4) ? (seg >> 2) : seg / segs_per_row;
         const int xs = (seg - y * segs_per_row) * 16;
         uint32_t bg_cls = P.cls_sky;
@@ -600,10 +601,13 @@ __device__ __forceinline__ void flush_counters(const RenderParams& P, const Tall
 //           store, which also resets the keys it read.
 //   rest    tiles whose lists or records did not fit go through cooperative_job afterwards.
 // ---------------------------------------------------------------------------------------------
-constexpr int POOL = 144;         // records shared by the NW tiles of a CTA
+constexpr int POOL = 136;         // records shared by the NW tiles of a CTA
+constexpr int STRIP = 16;         // pixel rows a warp rasterizes at a time
+constexpr int STRIP_KEYS = TILE * STRIP;
 constexpr int W_LEAF = 256;       // per-warp front-end lists (they live in the key buffer, 8 KB per warp)
 constexpr int W_FACE = 384;
 constexpr int W_SURV = 256;
+constexpr long long COOP_GRID = 148 * 5;   // CTAs of the cooperative kernel: one wave
 constexpr uint32_t REC_TINY = 1u << 28, REC_DEAD = 1u << 29;   // flags in the box word of a record
 
 struct __align__(16) FrontLists {
@@ -617,18 +621,21 @@ struct __align__(16) FrontLists {
 };
 
 struct __align__(16) FusedSmem {
-    union {
-        unsigned long long key[TILE * TILE];  // back end
-        FrontLists fl[NW];                    // front end
-    };
+    unsigned long long key[NW][STRIP_KEYS];   // warp w's strip of keys; during the front end, its FrontLists
     float4 pool[POOL * REC / 4];
-    float ray_x[TILE], ray_y[TILE];
-    uint32_t touched[NW][2];
+    float ray_x[NW][TILE], ray_y[NW][STRIP];  // ray tables of the strip a warp works on
     int n_surv[NW];                           // survivors of tile w; -1: lists overflowed, -2: no such tile
+    int next_task, pad[3];
 };
-static_assert(sizeof(FrontLists) * NW <= sizeof(unsigned long long) * TILE * TILE, "front-end lists must fit the key buffer");
+static_assert(sizeof(FrontLists) <= sizeof(unsigned long long) * STRIP_KEYS, "front-end lists must fit a warp's key strip");
 static_assert(sizeof(FusedSmem) <= 44 * 1024 && sizeof(TileSmem) <= 44 * 1024,
               "shared memory must leave room for 5 CTAs per SM (228 KB, 1 KB reserved per CTA)");
+// What the raster and store templates need of a warp's strip: rows are counted from the strip's first.
+struct StripView {
+    unsigned long long* key;
+    const float* ray_x;
+    const float* ray_y;
+};
 constexpr size_t RENDER_SMEM = sizeof(FusedSmem) > sizeof(TileSmem) ? sizeof(FusedSmem) : sizeof(TileSmem);
 
 __device__ __forceinline__ void write_record(float4* r, const PrimEq& q, uint32_t key_lo, uint32_t box, uint32_t extra) {
@@ -750,36 +757,105 @@ __device__ __forceinline__ void front_setup(const FrontLists& f, float4* rec, co
     }
 }
 
-// Back end of one tile by the CTA; the keys are all "no fragment" on entry and on exit.
+// Back end of one strip (rows ys .. ys + STRIP - 1 of the tile) by one warp; the strip's keys are
+// all "no fragment" on entry and on exit.
 template <class TL>
-__device__ __forceinline__ void back_job(FusedSmem& s, const RenderParams& P, const Job& job, bool ego_active,
-                                         const float4* rec, int n_rec, uint32_t* touched, bool classify, int stop, TL& n) {
+__device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, const Job& job, bool ego_active, int ys,
+                                           const float4* rec, int n_rec, bool classify, int stop, int lane, TL& n) {
     const TileCtx& t = job.t;
-    for (int i = threadIdx.x; i < n_rec; i += NTHREADS) {
+    const int rows = min(STRIP, t.th - ys);
+    uint32_t touched = 0u;                       // 8x8 blocks of the strip: bit (row >> 3) * 8 + (column >> 3)
+    // ---- primitives of a few pixels: a lane each, atomic max
+    for (int i = lane; i < n_rec; i += 32) {
         const float4* r = rec + i * (REC / 4);
         const uint32_t bw = __float_as_uint(r[4].x);
-        if (bw & REC_TINY) {
+        if (!(bw & REC_TINY)) continue;
+        const int bx0 = bw & 63, bx1 = (bw >> 12) & 63;
+        const int y0 = max((int)((bw >> 6) & 63), ys) - ys, y1 = min((int)((bw >> 18) & 63), ys + STRIP - 1) - ys;
+        if (y0 > y1) continue;
+        PrimEq q;
+        uint32_t key_lo;
+        read_record(r, q, key_lo);
+        q.tl = (bw >> 24) & 15u;
+        bool any = false;
+        for (int y = y0; y <= y1; ++y) {
+            const float ry = s.ray_y[y];
+            for (int x = bx0; x <= bx1; ++x) {
+                const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
+                if (wb) { put_fragment(s, x, y, wb, key_lo); any = true; }
+            }
+        }
+        if (any) touched |= (uint32_t)block_mask(bx0, y0, bx1, y1);
+    }
+    __syncwarp();
+    // ---- the others: the warp walks the records that reach the strip, a lane per pixel pair
+    if (stop == 0 || stop > 5) {
+        for (int p = 0; p < n_rec; ++p) {
+            const float4* r = &rec[p * (REC / 4)];
+            const uint32_t bw = __float_as_uint(r[4].x);
+            if (bw >> 28) continue;                  // rasterized above, or degenerate
+            const int by0 = (bw >> 6) & 63, by1 = (bw >> 18) & 63;
+            if (by1 < ys || by0 >= ys + STRIP) continue;
+            const int bx0 = bw & 63, bx1 = (bw >> 12) & 63;
+            const int ly0 = max(by0, ys) - ys, ly1 = min(by1, ys + STRIP - 1) - ys;
             PrimEq q;
             uint32_t key_lo;
             read_record(r, q, key_lo);
             q.tl = (bw >> 24) & 15u;
-            const uint32_t box = (bw & 63u) | (((bw >> 6) & 63u) << 8) | (((bw >> 12) & 63u) << 16) | (((bw >> 18) & 63u) << 24);
-            raster_in_thread(s, touched, t, q, key_lo, box);
+            if (classify && (bx1 - bx0 + 1) * (ly1 - ly0 + 1) >= CLASSIFY_MIN_STRIP) {
+                // lanes 0..15 classify the strip's 16 x 4 pixel cells: reject / partly covered / inside
+                ++n.classified;
+                const int xa = (lane & 3) * 16, xb = xa + 15, ya = ((lane >> 2) & 3) * 4, yb = ya + 3;
+                bool reject = lane >= 16 || xb < bx0 || xa > bx1 || yb < ly0 || ya > ly1;
+                uint32_t need = 0u;
+                if (!reject) {
+                    const float rxa = s.ray_x[xa], rxb = s.ray_x[xb], rya = s.ray_y[ya], ryb = s.ray_y[yb];   // rxa < rxb, rya < ryb
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        // fma is monotone in each argument, so the cell's extreme values are at its corners
+                        const float ta = fm(q.ny[e], rya, q.nz[e]), tb = fm(q.ny[e], ryb, q.nz[e]);
+                        const float emax = fm(q.nx[e], q.nx[e] >= 0.f ? rxb : rxa, fmaxf(ta, tb));
+                        const float emin = fm(q.nx[e], q.nx[e] >= 0.f ? rxa : rxb, fminf(ta, tb));
+                        reject = reject || (emax < 0.f);
+                        if (!(emin > 0.f)) need |= 1u << e;
+                    }
+                    const float wa = fm(q.wy, rya, q.wz), wb = fm(q.wy, ryb, q.wz);
+                    const float wmax = fm(q.wx, q.wx >= 0.f ? rxb : rxa, fmaxf(wa, wb));
+                    const float wmin = fm(q.wx, q.wx >= 0.f ? rxa : rxb, fminf(wa, wb));
+                    reject = reject || (wmax < t.w_far) || (wmin > t.w_near);
+                    // the depth range test rides on the edge tests: if it is still needed, so is one edge
+                    if (need == 0u && !((wmin >= t.w_far) && (wmax <= t.w_near))) need = 1u;
+                }
+                for (unsigned m = __ballot_sync(0xffffffffu, !reject); m; m &= m - 1) {
+                    const int cell = __ffs(m) - 1;
+                    const int xx = (cell & 3) * 16, yy = (cell >> 2) * 4;
+                    const uint32_t need_c = __shfl_sync(0xffffffffu, need, cell);
+                    ++n.cells;
+                    if (raster_cell(s, t, q, key_lo, xx, yy, need_c, lane)) touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
+                }
+            } else {
+                for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
+                    for (int xx = bx0 & ~15; xx <= bx1; xx += 16) {
+                        ++n.cells;
+                        if (raster_cell(s, t, q, key_lo, xx, yy, 0xFu, lane)) touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
+                    }
+            }
         }
     }
-    __syncthreads();
-    if (stop == 0 || stop > 5) raster_records(s, rec, touched, t, n_rec, classify, n);
-    if (stop == 5 && threadIdx.x == 0) { touched[0] = 0xffffffffu; touched[1] = 0xffffffffu; }
-    __syncthreads();
-    // the cell raster of a ragged tile may leave keys past the image edge, which the store never
-    // visits: such a tile clears the whole buffer instead of the keys it read
-    const bool ragged = t.tw < TILE || t.th < TILE;
-    store_tile(s, t, P, job.view, job.k, ego_active, ((unsigned long long)touched[1] << 32) | touched[0], !ragged);
+    touched = __reduce_or_sync(0xffffffffu, touched);
+    if (stop == 5) touched = 0xffffu;
+    // ---- store; a ragged strip may hold keys past the image edge, which the store never visits:
+    // it clears the whole strip instead of the keys it read
+    TileCtx ts = t;
+    ts.y0 = t.y0 + ys; ts.th = rows;
+    const bool ragged = t.tw < TILE || rows < STRIP;
+    store_tile(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32);
+    __syncwarp();
     if (ragged) {
-        __syncthreads();
 #pragma unroll
-        for (int i = 0; i < TILE * TILE / 2 / NTHREADS; ++i)
-            reinterpret_cast<ulonglong2*>(s.key)[i * NTHREADS + threadIdx.x] = make_ulonglong2(0ull, 0ull);
+        for (int i = 0; i < STRIP_KEYS / 2 / 32; ++i)
+            reinterpret_cast<ulonglong2*>(s.key)[i * 32 + lane] = make_ulonglong2(0ull, 0ull);
+        __syncwarp();
     }
 }
 
@@ -787,7 +863,6 @@ template <class TL>
 __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     FusedSmem& s = *reinterpret_cast<FusedSmem*>(smem_raw);
-    TileSmem& cs = *reinterpret_cast<TileSmem*>(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned first = blockIdx.x * (unsigned)NW, n_jobs = P.n_jobs;
     TL n = {};
@@ -795,7 +870,8 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave work out (image incomplete)
     // test aids: a pool of 2 records sends nearly every tile to cooperative_job, one of 40 mixes both paths
     const int pool_cap = (P.debug_flags & 2) ? 2 : (P.debug_flags & 8) ? 40 : POOL;
-    if (threadIdx.x < 2 * NW) (&s.touched[0][0])[threadIdx.x] = 0u;
+    if (threadIdx.x == 0) s.next_task = 0;
+    FrontLists& fl = *reinterpret_cast<FrontLists*>(s.key[warp]);
 
     // ---- front end: warp w culls tile first + w
     const bool valid = first + warp < n_jobs;
@@ -807,7 +883,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         mi = P.env_maps[job.e];
         ns = 0;
         if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
-        else if (P.agents[(size_t)job.e * P.A + job.a].active != 0 && stop != 1) ns = front_cull(s.fl[warp], P, job, mi, lane, nl, n);
+        else if (P.agents[(size_t)job.e * P.A + job.a].active != 0 && stop != 1) ns = front_cull(fl, P, job, mi, lane, nl, n);
     }
     if (lane == 0) s.n_surv[warp] = ns;
     __syncthreads();
@@ -827,40 +903,63 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     {
         const int my_base = (int)((bases >> (8 * warp)) & 0xffu), my_cnt = (int)((cnts >> (8 * warp)) & 0xffu);
         if (my_cnt == 0xff) { n.grp = 0; n.leaf = 0; n.tested = 0; }       // counted again by cooperative_job
-        else if (my_cnt != 0xfe && my_cnt > 0) front_setup(s.fl[warp], s.pool + my_base * (REC / 4), P, job, mi, nl, my_cnt, lane, n);
+        else if (my_cnt != 0xfe && my_cnt > 0) front_setup(fl, s.pool + my_base * (REC / 4), P, job, mi, nl, my_cnt, lane, n);
     }
     __syncthreads();
-    // ---- back end: the lists are dead, their memory becomes the key buffer
+    // ---- back end: the NW tiles' strips are tasks that the warps draw from a counter; a warp's
+    // lists are dead, their memory becomes its strip of keys
 #pragma unroll
-    for (int i = 0; i < TILE * TILE / 2 / NTHREADS; ++i)
-        reinterpret_cast<ulonglong2*>(s.key)[i * NTHREADS + threadIdx.x] = make_ulonglong2(0ull, 0ull);
-    bool rays_loaded = false;
+    for (int i = 0; i < STRIP_KEYS / 2 / 32; ++i)
+        reinterpret_cast<ulonglong2*>(s.key[warp])[i * 32 + lane] = make_ulonglong2(0ull, 0ull);
+    __syncwarp();
+    StripView sv;
+    sv.key = s.key[warp]; sv.ray_x = s.ray_x[warp]; sv.ray_y = s.ray_y[warp];
+    constexpr int STRIPS = TILE / STRIP;
 #pragma unroll 1
-    for (int j = 0; j < NW; ++j) {
+    for (;;) {
+        int task = 0;
+        if (lane == 0) task = atomicAdd(&s.next_task, 1);
+        task = __shfl_sync(0xffffffffu, task, 0);
+        if (task >= NW * STRIPS) break;
+        const int j = task / STRIPS, ys = (task % STRIPS) * STRIP;
         const int cj = (int)((cnts >> (8 * j)) & 0xffu);
-        if (cj >= 0xfe) continue;                   // uniform over the CTA
+        if (cj >= 0xfe) continue;
         const Job jb = decode_job(P, first + j);
+        if (ys >= jb.t.th) continue;
         const bool ego_active = P.agents[(size_t)jb.e * P.A + jb.a].active != 0;
-        if (!rays_loaded) {
-            if (threadIdx.x < TILE) load_rays(s, P, jb, threadIdx.x);
-            rays_loaded = true;
-            __syncthreads();
+        {   // ray tables of the strip (columns / rows past the image edge continue the formula)
+            const CamConst& ck = P.cam[jb.k];
+#pragma unroll
+            for (int i = lane; i < TILE; i += 32)
+                s.ray_x[warp][i] = (jb.t.x0 + i < P.W) ? __ldg(P.rig.ray_x + (size_t)jb.k * P.W + jb.t.x0 + i)
+                                                      : __fdiv_rn(sub(add((float)(jb.t.x0 + i), 0.5f), 0.5f * (float)P.W), ck.fx);
+            if (lane < STRIP) {
+                const int y = jb.t.y0 + ys + lane;
+                s.ray_y[warp][lane] = (y < P.H) ? __ldg(P.rig.ray_y + (size_t)jb.k * P.H + y)
+                                                : __fdiv_rn(sub(add((float)y, 0.5f), 0.5f * (float)P.H), ck.fy);
+            }
         }
-        back_job(s, P, jb, ego_active, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, s.touched[j], classify, stop, n);
-        if (threadIdx.x == 0) ++n.jobs;
-        // the ray tables of the next tile of the pool: nothing reads them between here and the barrier
-        int nx = -1;
-        for (int j2 = NW - 1; j2 > j; --j2) if (((cnts >> (8 * j2)) & 0xffu) < 0xfeu) nx = j2;
-        if (nx >= 0 && threadIdx.x < TILE) load_rays(s, P, decode_job(P, first + nx), threadIdx.x);
+        __syncwarp();
+        back_strip(sv, P, jb, ego_active, ys, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, classify, stop, lane, n);
+        if (lane == 0 && ys == 0) ++n.jobs;
+    }
+    // ---- the rest: tiles that did not fit are left to the cooperative kernel
+    if (threadIdx.x < NW && ((cnts >> (8 * threadIdx.x)) & 0xffu) == 0xffu)
+        P.overflow[1u + atomicAdd(&P.overflow[0], 1u)] = first + threadIdx.x;
+    flush_counters(P, n);
+}
+
+// The tiles the fused kernel left out, a CTA at a time.
+template <class TL>
+__global__ void __launch_bounds__(NTHREADS, 5) cooperative_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TileSmem& cs = *reinterpret_cast<TileSmem*>(smem_raw);
+    TL n = {};
+    const unsigned count = __ldcg(&P.overflow[0]);
+    for (unsigned i = blockIdx.x; i < count; i += gridDim.x) {
+        cooperative_job(cs, P, __ldcg(&P.overflow[1u + i]), n);
         __syncthreads();
     }
-    // ---- the rest: tiles that did not fit
-#pragma unroll 1
-    for (int j = 0; j < NW; ++j)
-        if (((cnts >> (8 * j)) & 0xffu) == 0xffu) {
-            cooperative_job(cs, P, first + j, n);
-            __syncthreads();
-        }
     flush_counters(P, n);
 }
 
@@ -869,7 +968,11 @@ size_t render_smem_bytes() { return RENDER_SMEM; }
 cudaError_t configure_render_kernel() {
     cudaError_t err = cudaFuncSetAttribute(render_kernel<NoTally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
     if (err != cudaSuccess) return err;
-    return cudaFuncSetAttribute(render_kernel<Tally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    err = cudaFuncSetAttribute(render_kernel<Tally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    if (err != cudaSuccess) return err;
+    err = cudaFuncSetAttribute(cooperative_kernel<NoTally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(cooperative_kernel<Tally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
 }
 
 cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cudaStream_t stream) {
@@ -881,6 +984,12 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cuda
     const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
     if (P.counters) render_kernel<Tally><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     else render_kernel<NoTally><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    // the tiles left out (their number is only known on the device): a fixed grid walks the list
+    const unsigned cgrid = (unsigned)(jobs < COOP_GRID ? jobs : COOP_GRID);
+    if (P.counters) cooperative_kernel<Tally><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    else cooperative_kernel<NoTally><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
     return cudaGetLastError();
 }
 

@@ -90,6 +90,7 @@ struct RenderParams {
     uint16_t* out_depth;
     float* out_depth32;             // optional
     unsigned long long* counters;   // optional [16]
+    uint32_t* overflow;             // [1 + tiles of all views]: count, then the tiles left to the cooperative kernel
     int32_t debug_flags;            // bit 0: no per-cell trivial accept/reject, bit 1: record list of 2 entries (forces the overflow path)
     uint32_t n_jobs;                // tiles to render in this launch (views x tiles per view); set by the launcher
     long long view_first;           // render views [view_first, view_first + gridDim / tiles)

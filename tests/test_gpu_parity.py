@@ -179,7 +179,8 @@ def test_counters_are_plausible(gu):
         assert cnt[0] == V
         # tiles, group tests, leaf tests, primitives tested, set up, rasterized by their thread, records,
         # record-list overflows, records classified per cell, cells visited
-        assert 0 < cnt[4] <= cnt[3] and cnt[5] + cnt[6] + cnt[7] == cnt[4] and cnt[7] == 0 and cnt[8] <= cnt[6] <= cnt[9]
+        # (a record may be classified once per 16-row strip it reaches)
+        assert 0 < cnt[4] <= cnt[3] and cnt[5] + cnt[6] + cnt[7] == cnt[4] and cnt[7] == 0 and cnt[8] <= 4 * cnt[6] and cnt[6] <= cnt[9]
         print("counters per view:", (cnt / V).round(1).tolist())
     finally:
         g.close()
