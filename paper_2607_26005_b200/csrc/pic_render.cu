@@ -601,7 +601,7 @@ __device__ __forceinline__ void flush_counters(const RenderParams& P, const Tall
 //           store, which also resets the keys it read.
 //   rest    tiles whose lists or records did not fit go through cooperative_job afterwards.
 // ---------------------------------------------------------------------------------------------
-constexpr int POOL = 136;         // records shared by the NW tiles of a CTA
+constexpr int POOL = 132;         // records shared by the NW tiles of a CTA
 constexpr int STRIP = 16;         // pixel rows a warp rasterizes at a time
 constexpr int STRIP_KEYS = TILE * STRIP;
 constexpr int W_LEAF = 256;       // per-warp front-end lists (they live in the key buffer, 8 KB per warp)
@@ -625,7 +625,9 @@ struct __align__(16) FusedSmem {
     float4 pool[POOL * REC / 4];
     float ray_x[NW][TILE], ray_y[NW][STRIP];  // ray tables of the strip a warp works on
     int n_surv[NW];                           // survivors of tile w; -1: lists overflowed, -2: no such tile
-    int next_task, pad[3];
+    int next_task;
+    int tile_active[NW];                      // is the ego agent of tile w active
+    Job tile_job[NW];                         // tile w, decoded by its warp
 };
 static_assert(sizeof(FrontLists) <= sizeof(unsigned long long) * STRIP_KEYS, "front-end lists must fit a warp's key strip");
 static_assert(sizeof(FusedSmem) <= 44 * 1024 && sizeof(TileSmem) <= 44 * 1024,
@@ -881,9 +883,11 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     if (valid) {
         job = decode_job(P, first + warp);
         mi = P.env_maps[job.e];
+        const bool ego_active = P.agents[(size_t)job.e * P.A + job.a].active != 0;
+        if (lane == 0) { s.tile_job[warp] = job; s.tile_active[warp] = ego_active; }
         ns = 0;
         if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
-        else if (P.agents[(size_t)job.e * P.A + job.a].active != 0 && stop != 1) ns = front_cull(fl, P, job, mi, lane, nl, n);
+        else if (ego_active && stop != 1) ns = front_cull(fl, P, job, mi, lane, nl, n);
     }
     if (lane == 0) s.n_surv[warp] = ns;
     __syncthreads();
@@ -924,9 +928,9 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         const int j = task / STRIPS, ys = (task % STRIPS) * STRIP;
         const int cj = (int)((cnts >> (8 * j)) & 0xffu);
         if (cj >= 0xfe) continue;
-        const Job jb = decode_job(P, first + j);
+        const Job jb = s.tile_job[j];
         if (ys >= jb.t.th) continue;
-        const bool ego_active = P.agents[(size_t)jb.e * P.A + jb.a].active != 0;
+        const bool ego_active = s.tile_active[j] != 0;
         {   // ray tables of the strip (columns / rows past the image edge continue the formula)
             const CamConst& ck = P.cam[jb.k];
 #pragma unroll
