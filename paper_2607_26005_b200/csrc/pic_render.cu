@@ -767,37 +767,44 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
     const TileCtx& t = job.t;
     const int rows = min(STRIP, t.th - ys);
     uint32_t touched = 0u;                       // 8x8 blocks of the strip: bit (row >> 3) * 8 + (column >> 3)
-    // ---- primitives of a few pixels: a lane each, atomic max
-    for (int i = lane; i < n_rec; i += 32) {
-        const float4* r = rec + i * (REC / 4);
-        const uint32_t bw = __float_as_uint(r[4].x);
-        if (!(bw & REC_TINY)) continue;
-        const int bx0 = bw & 63, bx1 = (bw >> 12) & 63;
-        const int y0 = max((int)((bw >> 6) & 63), ys) - ys, y1 = min((int)((bw >> 18) & 63), ys + STRIP - 1) - ys;
-        if (y0 > y1) continue;
-        PrimEq q;
-        uint32_t key_lo;
-        read_record(r, q, key_lo);
-        q.tl = (bw >> 24) & 15u;
-        bool any = false;
-        for (int y = y0; y <= y1; ++y) {
-            const float ry = s.ray_y[y];
-            for (int x = bx0; x <= bx1; ++x) {
-                const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
-                if (wb) { put_fragment(s, x, y, wb, key_lo); any = true; }
+    // Records are looked at 32 at a time, a lane each: which reach the strip?  Those of a few
+    // pixels are rasterized by their lane (atomic max); the warp then walks the other hits
+    // together, a lane per pixel pair.
+    for (int base = 0; base < n_rec; base += 32) {
+        uint32_t bw_lane = 0u;
+        bool hit = false;
+        if (base + lane < n_rec) {
+            const float4* r = rec + (base + lane) * (REC / 4);
+            bw_lane = __float_as_uint(r[4].x);
+            const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
+            hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + STRIP;
+            if (hit && (bw_lane & REC_TINY)) {
+                hit = false;
+                const int bx0 = bw_lane & 63, bx1 = (bw_lane >> 12) & 63;
+                const int y0 = max(by0, ys) - ys, y1 = min(by1, ys + STRIP - 1) - ys;
+                PrimEq q;
+                uint32_t key_lo;
+                read_record(r, q, key_lo);
+                q.tl = (bw_lane >> 24) & 15u;
+                bool any = false;
+                for (int y = y0; y <= y1; ++y) {
+                    const float ry = s.ray_y[y];
+                    for (int x = bx0; x <= bx1; ++x) {
+                        const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
+                        if (wb) { put_fragment(s, x, y, wb, key_lo); any = true; }
+                    }
+                }
+                if (any) touched |= (uint32_t)block_mask(bx0, y0, bx1, y1);
             }
         }
-        if (any) touched |= (uint32_t)block_mask(bx0, y0, bx1, y1);
-    }
-    __syncwarp();
-    // ---- the others: the warp walks the records that reach the strip, a lane per pixel pair
-    if (stop == 0 || stop > 5) {
-        for (int p = 0; p < n_rec; ++p) {
-            const float4* r = &rec[p * (REC / 4)];
-            const uint32_t bw = __float_as_uint(r[4].x);
-            if (bw >> 28) continue;                  // rasterized above, or degenerate
+        __syncwarp();
+        unsigned hits = __ballot_sync(0xffffffffu, hit);
+        if (!(stop == 0 || stop > 5)) hits = 0u;
+        for (; hits; hits &= hits - 1) {
+            const int src = __ffs(hits) - 1;
+            const uint32_t bw = __shfl_sync(0xffffffffu, bw_lane, src);
+            const float4* r = &rec[(base + src) * (REC / 4)];
             const int by0 = (bw >> 6) & 63, by1 = (bw >> 18) & 63;
-            if (by1 < ys || by0 >= ys + STRIP) continue;
             const int bx0 = bw & 63, bx1 = (bw >> 12) & 63;
             const int ly0 = max(by0, ys) - ys, ly1 = min(by1, ys + STRIP - 1) - ys;
             PrimEq q;
@@ -843,6 +850,7 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
                     }
             }
         }
+        __syncwarp();
     }
     touched = __reduce_or_sync(0xffffffffu, touched);
     if (stop == 5) touched = 0xffffu;
