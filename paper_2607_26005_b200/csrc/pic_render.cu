@@ -1,31 +1,40 @@
-// Production render kernel of the batched egocentric rasterizer (sm_100a).
+// Production render kernels of the batched egocentric rasterizer (sm_100a).
 //
-// One CTA of 128 threads renders one tile (up to 64 x 64 pixels) of one view.  The z-buffer lives
-// in shared memory as one 64-bit key per pixel,
+// The z-buffer lives in shared memory as one 64-bit key per pixel,
 //     key = float_bits(1/z) << 32 | (0xFFFFFF - primitive index) << 8 | class,
 // so "nearest fragment wins, exact ties go to the lower index" is an unsigned max that does not
 // depend on the order in which primitives arrive; 0 means "no fragment" (background).
 //
-// Phases, each ended by one CTA barrier:
-//   1  (a) cull     every warp tests the map's group boxes against the tile frustum, then takes
-//                   its share of the visible groups and tests their leaf boxes; visible leaves
-//                   are compacted into a list with warp ballots.  Other agents' boxes are culled as
-//                   spheres; only their camera-facing faces become items.
-//   2a (a) cull     one thread per candidate (8 per visible leaf, 1 per face item): camera-space
-//                   vertices and pixel box; candidates whose box holds no pixel centre of the tile
-//                   stop here, the survivors are compacted again.
-//   2b (c) set-up   one thread per survivor: 3-4 edge functions + 1/z plane.  Primitives whose
-//                   pixel box holds <= 4 pixel centres are rasterized at once by their thread
-//                   (atomic max); the others leave a 17-word record.
-//   3  (b)+(c)      bands of 4 pixel rows belong to warp (band mod 4); every warp walks the records
-//                   and rasterizes its own bands, a lane per pixel pair, plain loads and stores.
-//                   Primitives covering many pixels first classify the warp's 16 x 4 pixel cells
-//                   (trivial reject / trivial accept from the same float32 edge functions).
-//   4  (d) store    keys -> class u8 + depth binary16; a thread converts 16 pixels and issues
-//                   128-bit stores; 8 x 8 blocks no primitive touched are written without reading keys.
+// A unit of work is a tile: up to 64 x 64 pixels of one view.  Two kernels share the work.
+//
+// render_kernel (the fused kernel).  A CTA of 4 warps takes 4 consecutive tiles.
+//   front   (a) cull, (c) set-up -- one warp per tile, warp-level synchronisation only.  The warp
+//           tests the map's group boxes and the leaf boxes of the visible groups against the tile
+//           frustum (a lane per box), culls the other agents' boxes as spheres and keeps their
+//           camera-facing faces, then tests the candidates 32 at a time (camera-space vertices,
+//           pixel box) and compacts the survivors with ballots.  Its lists live in the key buffer,
+//           which is idle until the back end starts.  After one CTA barrier the survivors of the 4
+//           tiles get consecutive ranges of a shared record pool and are set up, a lane per
+//           survivor: 3-4 edge functions + 1/z plane in a 17-word record.
+//   back    (b) raster, (c), (d) store -- after a second CTA barrier the 16 strips of 16 pixel rows
+//           (4 per tile) are tasks that the warps draw from a counter.  A warp owns one strip of
+//           keys (8 KB).  Per strip it looks at the tile's records 32 at a time (a lane each: does
+//           the box reach the strip?), rasterizes primitives of <= 4 pixels from their lane with
+//           atomic max, then walks the other hits together: a lane per pixel pair of a 16 x 4
+//           pixel cell, plain loads and stores; boxes of >= 96 pixels first classify the strip's
+//           16 cells (trivial reject / trivial accept / which edges still need testing) from the
+//           same float32 edge functions.  The store converts keys to class u8 + depth binary16
+//           with 128-bit stores, resets the keys it read, and writes 8 x 8 blocks that nothing
+//           touched without reading keys.
+//   Tiles whose lists overflow, or whose records do not fit the pool beside their fellows', are
+//   appended to a list in device memory.
+//
+// cooperative_kernel.  One wave of CTAs walks that list; a whole CTA renders a tile in
+// barrier-separated phases with per-round lists (any number of groups, boxes, survivors and
+// records): the general path, and the one the fused kernel is checked against in the tests.
 //
 // Cameras (one 64-byte record per view) and per-camera ray / background tables are prepared by
-// the agent and rig kernels, so the prologue is a few loads.
+// the agent and rig kernels, so the prologues are a few loads.
 #include "pic_device.cuh"
 
 namespace pic {
@@ -354,8 +363,12 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
     const int segs_per_row = (t.tw + 15) >> 4;
     const int n_seg = t.th * segs_per_row;
     for (int seg = tid; seg < n_seg; seg += nthr) {
-        const int y = (segs_per_row == 4) ? (seg >> 2) : seg / segs_per_row;
-        const int xs = (seg - y * segs_per_row) * 16;
+        // full-width tiles with a multiple of 8 rows: eight consecutive threads take eight consecutive
+        // rows of one 16-pixel column strip, so that their 16-byte key accesses fall in different
+        // banks (the swizzle is by row); a warp still covers 8 rows x 64 pixels of the image
+        const bool by_rows = segs_per_row == 4 && (t.th & 7) == 0;
+        const int y = by_rows ? ((seg & 7) | ((seg >> 5) << 3)) : seg / segs_per_row;
+        const int xs = by_rows ? ((seg >> 3) & 3) * 16 : (seg - y * segs_per_row) * 16;
         uint32_t bg_cls = P.cls_sky;
         float bg_z = P.far_z;
         if (ego_active) { bg_cls = __ldg(P.rig.bg_cls + (size_t)k * P.H + t.y0 + y); bg_z = __ldg(P.rig.bg_z + (size_t)k * P.H + t.y0 + y); }
