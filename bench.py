@@ -32,9 +32,9 @@ if ROOT not in sys.path:
 CFG = 2                       # scene of the stepping workload
 ALU_LANES_PER_SM = 128        # FP32 lanes per SM
 FALLBACK_HBM_GBS = 6650.0
-# DRAM traffic of one render-kernel launch per view, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 16-env launch / its views); None = not captured.
-NCU_DRAM_BYTES_PER_VIEW = 9306
+# DRAM traffic of one launch of the fused render kernel per view, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 64-env launch / its views); None = not captured.
+NCU_DRAM_BYTES_PER_VIEW = 8644
 
 
 def _affinity_cores() -> int:
@@ -294,7 +294,9 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
                     "frac": ach / (alu_peak / 1e12), "peak_kind": "derived: SMs x 128 lanes x max SM clock"}
         roof.update({
             "traffic": None if NCU_DRAM_BYTES_PER_VIEW is None else NCU_DRAM_BYTES_PER_VIEW * s.E * s.A * s.K,
-            "kernel": "render_kernel", "kernel_ms": k_ms, "kernel_launches_timed": int(len(kt)),
+            # kernel_ms: the library's event pair around its render launches (the fused kernel and the
+            # short cooperative kernel for the tiles it leaves out), i.e. all the render work of a step
+            "kernel": "render_kernel (+ cooperative_kernel)", "kernel_ms": k_ms, "kernel_launches_timed": int(len(kt)),
             "algorithmic_bytes": alg_bytes, "t_hbm_ms": 1e3 * t_hbm, "t_alu_ms": 1e3 * t_alu,
             "alg_lane_ops_per_view": float(n_alg_view), "write_only_fill_gbs": fill_gbs})
         line = {
@@ -310,7 +312,7 @@ def run_cuda(args, rank: int, world: int, local_rank: int) -> None:
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "agent-steps/s", "h2d_bytes_per_step": 25 * s.E * s.A,
                     "d2h_bytes_per_step": 3 * px, "steps": n_e2e, "entry": "pic_render_host, pinned host buffers"},
-            "gpu_launches": 3 * args.steps,
+            "gpu_launches": 4 * args.steps,       # rig, agent, fused render and cooperative render kernels per step
             "roofline": roof,
             "cpu_baseline": {"value": cpu_value, "unit": "agent-steps/s", "cores": min(cores, 64), "kind": "oracle",
                              "sample": f"{len(or_views)} seeded views of this workload in {t_or:.1f} s"},

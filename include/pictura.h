@@ -146,15 +146,20 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *                         depth the binary16 image was rounded from.
  *   PIC_OPT_COUNTERS      value = dev u64* [16] (as uintptr) or 0: accumulate work counters (tiles,
  *                         group tests, leaf tests, primitives tested, set up, rasterized by their
- *                         thread, records, record-list overflows, records classified per cell, cells visited).
+ *                         thread, records, record-list overflows, records classified per cell (once
+ *                         per 16-row strip they reach), cells visited, tiles rendered by the
+ *                         cooperative kernel).
  *   PIC_OPT_VIEW_FIRST,   render only views [first, first + count) (flat index (e*A + a)*K + k);
  *   PIC_OPT_VIEW_COUNT    count 0 = through the last view.  Other views' pixels are left untouched.
  *   PIC_OPT_DEBUG_FLAGS   bit 0: rasterize large primitives without the per-cell trivial
- *                         accept/reject; bit 1: shrink the per-tile record list to 2 entries so that
- *                         the overflow path runs.  Both leave the images unchanged (tests rely on it).
- *                         Bits 4-7: leave the render kernel after phase n = 1..3 (profiling aid;
- *                         the images are then incomplete).
- *   PIC_OPT_TIMING        1: bracket every render-kernel launch with CUDA events on its stream
+ *                         accept/reject; bit 1: shrink the fused kernel's record pool and the
+ *                         cooperative kernel's record list to 2 entries so that the overflow paths
+ *                         run; bit 2: send every tile to the cooperative kernel; bit 3: shrink the
+ *                         record pool to 40 so that both kernels share the tiles.  All leave the
+ *                         images unchanged (tests rely on it).  Bits 4-7: profiling aid, leaves work
+ *                         out (1: no culling, 4: no record raster, 5: as 4 with every pixel
+ *                         converted); the images are then incomplete.
+ *   PIC_OPT_TIMING        1: bracket the render kernels of every call with CUDA events on its stream
  *                         (up to 1024 launches between two pic_get_kernel_times calls); 0: off.
  *                         Turning it on creates the events (allocates), so do it outside timed code.
  */
