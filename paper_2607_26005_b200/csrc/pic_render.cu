@@ -362,13 +362,14 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
     const bool vec_ok = (P.W % 16 == 0) && o32 == nullptr;
     const int segs_per_row = (t.tw + 15) >> 4;
     const int n_seg = t.th * segs_per_row;
+    // full-width tiles with a multiple of 8 rows: eight consecutive threads take eight consecutive
+    // rows of one 16-pixel column strip, so that their 16-byte key accesses fall in different
+    // banks (the swizzle is by row); a warp still covers 8 rows x 64 pixels of the image
+    const bool by_rows = segs_per_row == 4 && (t.th & 7) == 0;
     for (int seg = tid; seg < n_seg; seg += nthr) {
-        // full-width tiles with a multiple of 8 rows: eight consecutive threads take eight consecutive
-        // rows of one 16-pixel column strip, so that their 16-byte key accesses fall in different
-        // banks (the swizzle is by row); a warp still covers 8 rows x 64 pixels of the image
-        const bool by_rows = segs_per_row == 4 && (t.th & 7) == 0;
-        const int y = by_rows ? ((seg & 7) | ((seg >> 5) << 3)) : seg / segs_per_row;
-        const int xs = by_rows ? ((seg >> 3) & 3) * 16 : (seg - y * segs_per_row) * 16;
+        int y, xs;
+        if (by_rows) { y = (seg & 7) | ((seg >> 5) << 3); xs = ((seg >> 3) & 3) * 16; }
+        else { y = seg / segs_per_row; xs = (seg - y * segs_per_row) * 16; }
         uint32_t bg_cls = P.cls_sky;
         float bg_z = P.far_z;
         if (ego_active) { bg_cls = __ldg(P.rig.bg_cls + (size_t)k * P.H + t.y0 + y); bg_z = __ldg(P.rig.bg_z + (size_t)k * P.H + t.y0 + y); }
@@ -952,7 +953,12 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         const Job jb = s.tile_job[j];
         if (ys >= jb.t.th) continue;
         const bool ego_active = s.tile_active[j] != 0;
-        {   // ray tables of the strip (columns / rows past the image edge continue the formula)
+        if (jb.t.tw == TILE && ys + STRIP <= jb.t.th) {     // ray tables of the strip
+            const float* rx = P.rig.ray_x + (size_t)jb.k * P.W + jb.t.x0;
+            s.ray_x[warp][lane] = __ldg(rx + lane);
+            s.ray_x[warp][lane + 32] = __ldg(rx + lane + 32);
+            if (lane < STRIP) s.ray_y[warp][lane] = __ldg(P.rig.ray_y + (size_t)jb.k * P.H + jb.t.y0 + ys + lane);
+        } else {                                            // ragged: columns / rows past the image edge continue the formula
             const CamConst& ck = P.cam[jb.k];
 #pragma unroll
             for (int i = lane; i < TILE; i += 32)
