@@ -157,7 +157,9 @@ __device__ __forceinline__ uint32_t fragment(const PrimEq& q, float rx, float ry
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         float e = fm(q.nx[i], rx, fm(q.ny[i], ry, q.nz[i]));
-        in = in && (e > 0.f || (e == 0.f && ((q.tl >> i) & 1u)));
+        // e > 0 || (e == 0 && the edge owns its zeros) as one comparison: nothing lies between the
+        // smallest negative subnormal and zero, and neither fma nor the comparison flushes subnormals
+        in = in && (e > __int_as_float(((q.tl >> i) & 1u) ? (int)0x80000001u : 0));
     }
     float w = fm(q.wx, rx, fm(q.wy, ry, q.wz));
     in = in && (w >= w_far) && (w <= w_near);

@@ -264,9 +264,11 @@ __device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq
             if ((need >> e) & 1u) {          // warp-uniform: edges known to be positive on the whole cell are skipped
                 const float te = fm(q.ny[e], ry, q.nz[e]);
                 const float e0 = fm(q.nx[e], rx0, te), e1 = fm(q.nx[e], rx1, te);
-                const bool own = (q.tl >> e) & 1u;
-                in0 = in0 && (e0 > 0.f || (e0 == 0.f && own));
-                in1 = in1 && (e1 > 0.f || (e1 == 0.f && own));
+                // e > 0 || (e == 0 && own) as one comparison: nothing lies between the smallest
+                // negative subnormal and zero, and neither fma nor the comparison flushes subnormals
+                const float thr = __int_as_float(((q.tl >> e) & 1u) ? (int)0x80000001u : 0);
+                in0 = in0 && (e0 > thr);
+                in1 = in1 && (e1 > thr);
             }
         }
         in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
