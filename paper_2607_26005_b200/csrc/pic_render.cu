@@ -21,7 +21,7 @@
 //           keys (8 KB).  Per strip it looks at the tile's records 32 at a time (a lane each: does
 //           the box reach the strip?), rasterizes primitives of <= 4 pixels from their lane with
 //           atomic max, then walks the other hits together: a lane per pixel pair of a 16 x 4
-//           pixel cell, plain loads and stores; boxes of >= 96 pixels first classify the strip's
+//           pixel cell, plain loads and stores; boxes of >= 256 pixels first classify the strip's
 //           16 cells (trivial reject / trivial accept / which edges still need testing) from the
 //           same float32 edge functions.  The store converts keys to class u8 + depth binary16
 //           with 128-bit stores, resets the keys it read, and writes 8 x 8 blocks that nothing
@@ -50,7 +50,7 @@ constexpr int FACECAP = 6 * BOX_ROUND;
 constexpr int SCAP = 128;         // candidates that survive the pixel-box test, per round
 constexpr int TINY_MAX_PIXELS = 4;         // pixel centres in the box of a primitive rasterized by its own thread
 constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large classify cells before rasterizing
-constexpr int CLASSIFY_MIN_STRIP = 96;     // the same for the part of a box inside a 16-row strip
+constexpr int CLASSIFY_MIN_STRIP = 256;    // the same for the part of a box inside a 16-row strip
 
 struct __align__(16) TileSmem {
     unsigned long long key[TILE * TILE];      // 32 KB, 16-byte chunks XOR-swizzled by row (key_index)
