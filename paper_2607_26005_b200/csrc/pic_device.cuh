@@ -180,7 +180,8 @@ __device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const 
     float zmin = V[0].z, zmax = V[0].z;
 #pragma unroll
     for (int i = 1; i < n; ++i) { zmin = fminf(zmin, V[i].z); zmax = fmaxf(zmax, V[i].z); }
-    if (!(zmax >= t.near_z * 0.9999f) || !(zmin <= t.far_z * 1.0001f)) return false;
+    // (written without early exits: the lanes of a warp rarely agree, so exits save nothing)
+    bool ok = (zmax >= t.near_z * 0.9999f) && (zmin <= t.far_z * 1.0001f);
     int bx0 = 0, by0 = 0, bx1 = t.tw - 1, by1 = t.th - 1;
     if (zmin >= t.near_z * ZPROJ_FRAC) {
         float sx0 = 3e38f, sx1 = -3e38f, sy0 = 3e38f, sy1 = -3e38f;
@@ -194,11 +195,10 @@ __device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const 
         const float m = 0.00390625f;
         float fx0 = ceilf(sx0 - 0.5f - m) - (float)t.x0, fx1 = floorf(sx1 - 0.5f + m) - (float)t.x0;
         float fy0 = ceilf(sy0 - 0.5f - m) - (float)t.y0, fy1 = floorf(sy1 - 0.5f + m) - (float)t.y0;
-        if (!(fx0 <= fx1) || !(fy0 <= fy1)) return false;
-        if (fx1 < 0.f || fy1 < 0.f || fx0 > (float)(t.tw - 1) || fy0 > (float)(t.th - 1)) return false;
+        ok = ok && (fx0 <= fx1) && (fy0 <= fy1) && (fx1 >= 0.f) && (fy1 >= 0.f) && (fx0 <= (float)(t.tw - 1)) && (fy0 <= (float)(t.th - 1));
         bx0 = (int)fmaxf(fx0, 0.f); by0 = (int)fmaxf(fy0, 0.f);
         bx1 = (int)fminf(fx1, (float)(t.tw - 1)); by1 = (int)fminf(fy1, (float)(t.th - 1));
-    } else {
+    } else if (ok) {
         // frustum side planes through the camera centre, valid for any sign of z
         float l = (float)t.x0 - c.cx, r = (float)(t.x0 + t.tw) - c.cx, u = (float)t.y0 - c.cy, d = (float)(t.y0 + t.th) - c.cy;
         bool ol = true, orr = true, ou = true, od = true;
@@ -210,10 +210,10 @@ __device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const 
             ou = ou && (Y < mul(Z, u) - 1e-4f * (fabsf(Y) + fabsf(mul(Z, u))));
             od = od && (Y > mul(Z, d) + 1e-4f * (fabsf(Y) + fabsf(mul(Z, d))));
         }
-        if (ol || orr || ou || od) return false;
+        ok = !(ol || orr || ou || od);
     }
     packed = (uint32_t)bx0 | ((uint32_t)by0 << 8) | ((uint32_t)bx1 << 16) | ((uint32_t)by1 << 24);
-    return true;
+    return ok;
 }
 
 
