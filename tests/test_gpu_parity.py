@@ -182,6 +182,12 @@ def test_counters_are_plausible(gu):
         # (a record may be classified once per 16-row strip it reaches)
         assert 0 < cnt[4] <= cnt[3] and cnt[5] + cnt[6] + cnt[7] == cnt[4] and cnt[7] == 0 and cnt[8] <= 4 * cnt[6] and cnt[6] <= cnt[9]
         print("counters per view:", (cnt / V).round(1).tolist())
+        # [10]: tiles the fused kernel left to the cooperative kernel -- a few at most here, all of
+        # them when the test aid asks for it, and the work counts of both routes agree
+        assert cnt[10] <= 0.2 * V
+        *_, cnt_coop = g.render(counters=True, debug_flags=4)
+        assert cnt_coop[0] == V and cnt_coop[10] == V
+        assert cnt_coop[4] == cnt[4] and cnt_coop[3] == cnt[3]
     finally:
         g.close()
 
