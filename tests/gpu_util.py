@@ -66,6 +66,9 @@ def check_against_oracle(scene, view_ids=None, gpu: CudaRun = None, **kw):
         gpu = CudaRun(scene)
     try:
         cls, d16, d32 = gpu.render()
+        # without the float32 depth image the kernels take their vector-store paths: same images
+        cls_v, d16_v, _ = gpu.render(depth32=False)
+        assert (cls_v == cls).all() and (d16_v.view(np.uint16) == d16.view(np.uint16)).all()
         if view_ids is None:
             view_ids = np.arange(scene.E * scene.A * scene.K)
         view_ids = np.asarray(view_ids, dtype=np.int64)
