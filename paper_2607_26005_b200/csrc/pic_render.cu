@@ -190,7 +190,7 @@ struct NoCount {
 };
 struct NoTally { NoCount grp, leaf, tested, setup, tiny, recs, fallback, classified, cells, jobs, coop; };
 
-// Phase 2b body: set a surviving primitive up, rasterize it (tiny) or leave a record.
+// Cooperative kernel, phase 2b body: set a surviving primitive up, rasterize it (tiny) or leave a record.
 template <class TL>
 __device__ __forceinline__ void setup_prim(TileSmem& s, const TileCtx& t, const V3 (&V)[4], bool quad, uint32_t flags,
                                            const V3 Pn, uint32_t key_lo, uint32_t box, int rec_cap, TL& n) {
@@ -247,7 +247,8 @@ __device__ __forceinline__ bool fetch_candidate(const S& s, const RenderParams& 
 }
 
 // One 16 x 4 cell at (xx, yy): every lane tests its two pixels and updates their keys with plain
-// loads and stores -- in phase 3 the rows of a cell belong to exactly one warp.  `need`: the edges
+// loads and stores -- the rows of a cell belong to exactly one warp (its strip in the fused kernel,
+// its bands in the cooperative kernel).  `need`: the edges
 // that still have to be tested on this cell (0: the cell is known to be covered and in depth
 // range; the range test rides on the edge tests).  Returns whether any lane produced a fragment.
 template <class S>
@@ -285,7 +286,7 @@ __device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq
     return __any_sync(0xffffffffu, in0 || in1);
 }
 
-// Phase 3: every warp walks all records but rasterizes only the bands (4 pixel rows) it owns --
+// Cooperative kernel, phase 3: every warp walks all records but rasterizes only the bands (4 pixel rows) it owns --
 // band b belongs to warp b % NW -- so keys are updated without atomics and the bands of a large
 // primitive are shared out evenly.
 template <class S, class TL>
@@ -455,8 +456,7 @@ __device__ __forceinline__ void load_rays(S& s, const RenderParams& P, const Job
 }
 
 // A whole tile rendered by the CTA in barrier-separated phases with per-round lists: any number of
-// groups, boxes, survivors and records.  The fused kernel uses it for the tiles whose lists do
-// not fit its per-warp front end.
+// groups, boxes, survivors and records.  It serves the tiles that the fused kernel leaves out.
 template <class TL>
 __device__ __forceinline__ void cooperative_job(TileSmem& s, const RenderParams& P, unsigned job_id, TL& n) {
     const Job job = decode_job(P, job_id);
@@ -606,16 +606,15 @@ __device__ __forceinline__ void flush_counters(const RenderParams& P, const Tall
 }
 
 // ---------------------------------------------------------------------------------------------
-// Fused kernel: a CTA takes NW consecutive tiles.
+// Fused kernel: a CTA takes NW consecutive tiles (see the head of this file).
 //
 //   front   warp w culls tile w on its own (hierarchy, boxes, candidate tests), with warp-level
-//           synchronisation only and its lists in the (still unused) key buffer; the survivors
-//           of the NW tiles then get consecutive ranges of one record pool and are set up, one
-//           lane per survivor.  Dense passes, no CTA barrier inside.
-//   back    tile after tile, by the whole CTA: primitives of <= TINY_MAX_PIXELS pixels by one
-//           thread each (atomic max), the others by band-owning warps (raster_records), then the
-//           store, which also resets the keys it read.
-//   rest    tiles whose lists or records did not fit go through cooperative_job afterwards.
+//           synchronisation only and its lists in its (still unused) strip of keys; after a CTA
+//           barrier the survivors of the NW tiles get consecutive ranges of one record pool and
+//           are set up, one lane per survivor.  Dense passes.
+//   back    after a second CTA barrier, 16-row strips are tasks drawn from a counter: a warp
+//           rasterizes a strip of some tile into its own strip of keys and stores it (back_strip).
+//   rest    tiles whose lists or records did not fit are appended to the cooperative kernel's list.
 // ---------------------------------------------------------------------------------------------
 constexpr int POOL = 132;         // records shared by the NW tiles of a CTA
 constexpr int STRIP = 16;         // pixel rows a warp rasterizes at a time
@@ -676,7 +675,7 @@ __device__ __forceinline__ void read_record(const float4* r, PrimEq& q, uint32_t
 }
 
 // Front end of one tile by one warp: fills f.leaf / f.face / f.surv.  Returns the number of
-// survivors, or -1 if a list overflowed (the tile then goes to cooperative_job).
+// survivors, or -1 if a list overflowed (the tile then goes to the cooperative kernel).
 template <class TL>
 __device__ __forceinline__ int front_cull(FrontLists& f, const RenderParams& P, const Job& job, const MapInfo& mi,
                                           int lane, int& nl_out, TL& n) {
