@@ -275,13 +275,14 @@ __device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq
         in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
         in1 = in1 && (w1 >= t.w_far) && (w1 <= t.w_near);
     }
-    if (in0 || in1) {
+    {
         ulonglong2* kp = reinterpret_cast<ulonglong2*>(&s.key[key_index(x, y)]);
         ulonglong2 kk = *kp;
         const unsigned long long k0 = make_key(__float_as_uint(w0), key_lo), k1 = make_key(__float_as_uint(w1), key_lo);
-        if (in0 && k0 > kk.x) kk.x = k0;
-        if (in1 && k1 > kk.y) kk.y = k1;
-        *kp = kk;
+        const bool up0 = in0 && k0 > kk.x, up1 = in1 && k1 > kk.y;
+        if (up0) kk.x = k0;
+        if (up1) kk.y = k1;
+        if (up0 || up1) *kp = kk;
     }
     return __any_sync(0xffffffffu, in0 || in1);
 }
