@@ -49,6 +49,7 @@ constexpr int BOX_ROUND = 64;     // boxes examined per round
 constexpr int FACECAP = 6 * BOX_ROUND;
 constexpr int SCAP = 128;         // candidates that survive the pixel-box test, per round
 constexpr int TINY_MAX_PIXELS = 4;         // pixel centres in the box of a primitive rasterized by its own thread
+static_assert(TINY_MAX_PIXELS == 4, "the strip back end enumerates the pixels of such a box for at most 4");
 constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large classify cells before rasterizing
 constexpr int CLASSIFY_MIN_STRIP = 256;    // the same for the part of a box inside a 16-row strip
 
@@ -110,7 +111,7 @@ template <class S>
 __device__ __forceinline__ void put_fragment(S& s, int x, int y, uint32_t wbits, uint32_t key_lo) {
     const unsigned long long k = make_key(wbits, key_lo);
     unsigned long long* addr = &s.key[key_index(x, y)];
-    if (k > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, k);
+    atomicMax(addr, k);
 }
 
 // Rasterize a primitive from one thread: loop over its pixel box, atomic max per fragment.
@@ -802,11 +803,14 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
                 uint32_t key_lo;
                 read_record(r, q, key_lo);
                 q.tl = (bw_lane >> 24) & 15u;
+                // at most TINY_MAX_PIXELS pixels: one column (w == 1), two columns, or one row
+                const int w = bx1 - bx0 + 1, npx = w * (y1 - y0 + 1);
                 bool any = false;
-                for (int y = y0; y <= y1; ++y) {
-                    const float ry = s.ray_y[y];
-                    for (int x = bx0; x <= bx1; ++x) {
-                        const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
+#pragma unroll
+                for (int px = 0; px < TINY_MAX_PIXELS; ++px) {
+                    if (px < npx) {
+                        const int x = bx0 + (w == 1 ? 0 : w == 2 ? (px & 1) : px), y = y0 + (w == 1 ? px : w == 2 ? (px >> 1) : 0);
+                        const uint32_t wb = fragment(q, s.ray_x[x], s.ray_y[y], t.w_near, t.w_far);
                         if (wb) { put_fragment(s, x, y, wb, key_lo); any = true; }
                     }
                 }
