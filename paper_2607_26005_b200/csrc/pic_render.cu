@@ -247,13 +247,21 @@ __device__ __forceinline__ bool fetch_candidate(const S& s, const RenderParams& 
     return true;
 }
 
+// The top-left rule "e > 0 || (e == 0 && the edge owns its zeros)" as one comparison e > thr:
+// thr is 0 or the smallest negative subnormal -- nothing lies between the two, and neither fma nor
+// the comparison flushes subnormals.
+__device__ __forceinline__ void edge_thresholds(uint32_t tl, float (&thr)[4]) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) thr[e] = __int_as_float(((tl >> e) & 1u) ? (int)0x80000001u : 0);
+}
+
 // One 16 x 4 cell at (xx, yy): every lane tests its two pixels and updates their keys with plain
 // loads and stores -- the rows of a cell belong to exactly one warp (its strip in the fused kernel,
 // its bands in the cooperative kernel).  `need`: the edges
 // that still have to be tested on this cell (0: the cell is known to be covered and in depth
 // range; the range test rides on the edge tests).  Returns whether any lane produced a fragment.
 template <class S>
-__device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq& q, uint32_t key_lo, int xx, int yy,
+__device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq& q, const float (&thr)[4], uint32_t key_lo, int xx, int yy,
                                             uint32_t need, int lane) {
     const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
     const float rx0 = s.ray_x[x], rx1 = s.ray_x[x + 1], ry = s.ray_y[y];
@@ -266,11 +274,8 @@ __device__ __forceinline__ bool raster_cell(S& s, const TileCtx& t, const PrimEq
             if ((need >> e) & 1u) {          // warp-uniform: edges known to be positive on the whole cell are skipped
                 const float te = fm(q.ny[e], ry, q.nz[e]);
                 const float e0 = fm(q.nx[e], rx0, te), e1 = fm(q.nx[e], rx1, te);
-                // e > 0 || (e == 0 && own) as one comparison: nothing lies between the smallest
-                // negative subnormal and zero, and neither fma nor the comparison flushes subnormals
-                const float thr = __int_as_float(((q.tl >> e) & 1u) ? (int)0x80000001u : 0);
-                in0 = in0 && (e0 > thr);
-                in1 = in1 && (e1 > thr);
+                in0 = in0 && (e0 > thr[e]);
+                in1 = in1 && (e1 > thr[e]);
             }
         }
         in0 = in0 && (w0 >= t.w_far) && (w0 <= t.w_near);
@@ -312,6 +317,8 @@ __device__ __forceinline__ void raster_records(S& s, const float4* rec, uint32_t
         q.wx = r3.x; q.wy = r3.y; q.wz = r3.z;
         const uint32_t key_lo = __float_as_uint(r3.w);
         q.tl = (bw >> 24) & 15u;
+        float thr[4];
+        edge_thresholds(q.tl, thr);
         if (classify && (bx1 - bx0 + 1) * (by1 - by0 + 1) >= CLASSIFY_MIN_PIXELS) {
             // (b) lanes 0..15 classify this warp's 16 cells: reject / partly covered / inside
             if (warp == 0) ++n.classified;
@@ -342,13 +349,13 @@ __device__ __forceinline__ void raster_records(S& s, const float4* rec, uint32_t
                 const int xx = (cell & 3) * 16, yy = ((cell >> 2) * NW + warp) * 4;
                 const uint32_t need_c = __shfl_sync(0xffffffffu, need, cell);
                 ++n.cells;
-                if (raster_cell(s, t, q, key_lo, xx, yy, need_c, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
+                if (raster_cell(s, t, q, thr, key_lo, xx, yy, need_c, lane)) touched |= 3ull << ((yy >> 3) * 8 + (xx >> 3));
             }
         } else {
             for (int band = first; band <= band1; band += NW)
                 for (int xx = bx0 & ~15; xx <= bx1; xx += 16) {
                     ++n.cells;
-                    if (raster_cell(s, t, q, key_lo, xx, band * 4, 0xFu, lane)) touched |= 3ull << ((band >> 1) * 8 + (xx >> 3));
+                    if (raster_cell(s, t, q, thr, key_lo, xx, band * 4, 0xFu, lane)) touched |= 3ull << ((band >> 1) * 8 + (xx >> 3));
                 }
         }
     }
@@ -831,6 +838,8 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
             uint32_t key_lo;
             read_record(r, q, key_lo);
             q.tl = (bw >> 24) & 15u;
+            float thr[4];
+            edge_thresholds(q.tl, thr);
             if (classify && (bx1 - bx0 + 1) * (ly1 - ly0 + 1) >= CLASSIFY_MIN_STRIP) {
                 // lanes 0..15 classify the strip's 16 x 4 pixel cells: reject / partly covered / inside
                 ++n.classified;
@@ -860,13 +869,13 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
                     const int xx = (cell & 3) * 16, yy = (cell >> 2) * 4;
                     const uint32_t need_c = __shfl_sync(0xffffffffu, need, cell);
                     ++n.cells;
-                    if (raster_cell(s, t, q, key_lo, xx, yy, need_c, lane)) touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
+                    if (raster_cell(s, t, q, thr, key_lo, xx, yy, need_c, lane)) touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
                 }
             } else {
                 for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
                     for (int xx = bx0 & ~15; xx <= bx1; xx += 16) {
                         ++n.cells;
-                        if (raster_cell(s, t, q, key_lo, xx, yy, 0xFu, lane)) touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
+                        if (raster_cell(s, t, q, thr, key_lo, xx, yy, 0xFu, lane)) touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
                     }
             }
         }
