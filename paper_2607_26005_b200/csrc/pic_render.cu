@@ -364,20 +364,22 @@ __device__ __forceinline__ void raster_records(S& s, const float4* rec, uint32_t
 
 // (d) keys -> class / depth images.  `touched`: the 8x8 blocks that may hold a fragment; with
 // `clear`, the keys that were read are reset to "no fragment" for the next tile.
-template <class S>
+// FULL: the caller guarantees full tiles of an image whose rows allow 128-bit stores and no float32
+// depth image, so that only the vector path is compiled in.
+template <bool FULL = false, class S>
 __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderParams& P, size_t view, int k, bool ego_active,
                                            unsigned long long touched, bool clear, int tid = threadIdx.x, int nthr = NTHREADS) {
     const size_t img = (size_t)P.H * P.W;
     uint8_t* oc = P.out_class + view * img;
     uint16_t* od = P.out_depth + view * img;
     float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
-    const bool vec_ok = (P.W % 16 == 0) && o32 == nullptr;
+    const bool vec_ok = FULL || ((P.W % 16 == 0) && o32 == nullptr);
     const int segs_per_row = (t.tw + 15) >> 4;
     const int n_seg = t.th * segs_per_row;
     // full-width tiles with a multiple of 8 rows: eight consecutive threads take eight consecutive
     // rows of one 16-pixel column strip, so that their 16-byte key accesses fall in different
     // banks (the swizzle is by row); a warp still covers 8 rows x 64 pixels of the image
-    const bool by_rows = segs_per_row == 4 && (t.th & 7) == 0;
+    const bool by_rows = FULL || (segs_per_row == 4 && (t.th & 7) == 0);
     for (int seg = tid; seg < n_seg; seg += nthr) {
         int y, xs;
         if (by_rows) { y = (seg & 7) | ((seg >> 5) << 3); xs = ((seg >> 3) & 3) * 16; }
@@ -387,7 +389,7 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
         if (ego_active) { bg_cls = __ldg(P.rig.bg_cls + (size_t)k * P.H + t.y0 + y); bg_z = __ldg(P.rig.bg_z + (size_t)k * P.H + t.y0 + y); }
         const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + xs;
         const bool empty = ((touched >> ((y >> 3) * 8 + (xs >> 3))) & 3ull) == 0ull;   // both blocks of the segment
-        if (vec_ok && xs + 16 <= t.tw) {
+        if (FULL || (vec_ok && xs + 16 <= t.tw)) {
             uint32_t cw[4], dw[8];
             if (empty) {
                 const uint32_t c4 = bg_cls * 0x01010101u;
@@ -785,11 +787,11 @@ __device__ __forceinline__ void front_setup(const FrontLists& f, float4* rec, co
 
 // Back end of one strip (rows ys .. ys + STRIP - 1 of the tile) by one warp; the strip's keys are
 // all "no fragment" on entry and on exit.
-template <class TL>
+template <bool FULL, class TL>
 __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, const Job& job, bool ego_active, int ys,
                                            const float4* rec, int n_rec, bool classify, int stop, int lane, TL& n) {
     const TileCtx& t = job.t;
-    const int rows = min(STRIP, t.th - ys);
+    const int rows = FULL ? STRIP : min(STRIP, t.th - ys);
     uint32_t touched = 0u;                       // 8x8 blocks of the strip: bit (row >> 3) * 8 + (column >> 3)
     // Records are looked at 32 at a time, a lane each: which reach the strip?  Those of a few
     // pixels are rasterized by their lane (atomic max); the warp then walks the other hits
@@ -887,8 +889,8 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
     // it clears the whole strip instead of the keys it read
     TileCtx ts = t;
     ts.y0 = t.y0 + ys; ts.th = rows;
-    const bool ragged = t.tw < TILE || rows < STRIP;
-    store_tile(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32);
+    const bool ragged = !FULL && (t.tw < TILE || rows < STRIP);
+    store_tile<FULL>(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32);
     __syncwarp();
     if (ragged) {
 #pragma unroll
@@ -898,7 +900,9 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
     }
 }
 
-template <class TL>
+// FULL: every tile is 64 x 64, rows allow 128-bit stores, no float32 depth image (the launcher
+// checks) -- the instantiation the workloads run, without the code for ragged tiles.
+template <class TL, bool FULL>
 __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     FusedSmem& s = *reinterpret_cast<FusedSmem*>(smem_raw);
@@ -966,9 +970,9 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         const int cj = (int)((cnts >> (8 * j)) & 0xffu);
         if (cj >= 0xfe) continue;
         const Job jb = s.tile_job[j];
-        if (ys >= jb.t.th) continue;
+        if (!FULL && ys >= jb.t.th) continue;
         const bool ego_active = s.tile_active[j] != 0;
-        if (jb.t.tw == TILE && ys + STRIP <= jb.t.th) {     // ray tables of the strip
+        if (FULL || (jb.t.tw == TILE && ys + STRIP <= jb.t.th)) {     // ray tables of the strip
             const float* rx = P.rig.ray_x + (size_t)jb.k * P.W + jb.t.x0;
             s.ray_x[warp][lane] = __ldg(rx + lane);
             s.ray_x[warp][lane + 32] = __ldg(rx + lane + 32);
@@ -986,7 +990,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             }
         }
         __syncwarp();
-        back_strip(sv, P, jb, ego_active, ys, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, classify, stop, lane, n);
+        back_strip<FULL>(sv, P, jb, ego_active, ys, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, classify, stop, lane, n);
         if (lane == 0 && ys == 0) ++n.jobs;
     }
     // ---- the rest: tiles that did not fit are left to the cooperative kernel
@@ -1012,9 +1016,11 @@ __global__ void __launch_bounds__(NTHREADS, 5) cooperative_kernel(const __grid_c
 size_t render_smem_bytes() { return RENDER_SMEM; }
 
 cudaError_t configure_render_kernel() {
-    cudaError_t err = cudaFuncSetAttribute(render_kernel<NoTally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    cudaError_t err = cudaFuncSetAttribute(render_kernel<NoTally, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
     if (err != cudaSuccess) return err;
-    err = cudaFuncSetAttribute(render_kernel<Tally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    err = cudaFuncSetAttribute(render_kernel<NoTally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    if (err != cudaSuccess) return err;
+    err = cudaFuncSetAttribute(render_kernel<Tally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
     if (err != cudaSuccess) return err;
     err = cudaFuncSetAttribute(cooperative_kernel<NoTally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
     if (err != cudaSuccess) return err;
@@ -1028,8 +1034,10 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cuda
     if (jobs <= 0) return cudaSuccess;
     P.n_jobs = (uint32_t)jobs;
     const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
-    if (P.counters) render_kernel<Tally><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
-    else render_kernel<NoTally><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
+    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr;
+    if (P.counters) render_kernel<Tally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
+    else if (full) render_kernel<NoTally, true><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
+    else render_kernel<NoTally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     // the tiles left out (their number is only known on the device): a fixed grid walks the list
