@@ -34,7 +34,7 @@ ALU_LANES_PER_SM = 128        # FP32 lanes per SM
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the fused render kernel per view, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 64-env launch / its views); None = not captured.
-NCU_DRAM_BYTES_PER_VIEW = 8658
+NCU_DRAM_BYTES_PER_VIEW = 8634
 
 
 def _affinity_cores() -> int:
