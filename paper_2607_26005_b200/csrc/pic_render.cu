@@ -912,7 +912,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     const bool classify = !(P.debug_flags & 1);
     const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave work out (image incomplete)
     // test aids: a pool of 2 records sends nearly every tile to cooperative_job, one of 40 mixes both paths
-    const int pool_cap = (P.debug_flags & 2) ? 2 : (P.debug_flags & 8) ? 40 : POOL;
+    const int pool_cap = FULL ? POOL : (P.debug_flags & 2) ? 2 : (P.debug_flags & 8) ? 40 : POOL;   // (FULL is launched without debug flags)
     if (threadIdx.x == 0) s.next_task = 0;
     FrontLists& fl = *reinterpret_cast<FrontLists*>(s.key[warp]);
 
@@ -1034,7 +1034,7 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cuda
     if (jobs <= 0) return cudaSuccess;
     P.n_jobs = (uint32_t)jobs;
     const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
-    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr;
+    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr && P.debug_flags == 0;
     if (P.counters) render_kernel<Tally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     else if (full) render_kernel<NoTally, true><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     else render_kernel<NoTally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
