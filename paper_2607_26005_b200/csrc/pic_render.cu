@@ -468,7 +468,7 @@ __device__ __forceinline__ void load_rays(S& s, const RenderParams& P, const Job
 
 // A whole tile rendered by the CTA in barrier-separated phases with per-round lists: any number of
 // groups, boxes, survivors and records.  It serves the tiles that the fused kernel leaves out.
-template <class TL>
+template <class TL, bool FULL>
 __device__ __forceinline__ void cooperative_job(TileSmem& s, const RenderParams& P, unsigned job_id, TL& n) {
     const Job job = decode_job(P, job_id);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -596,7 +596,7 @@ __device__ __forceinline__ void cooperative_job(TileSmem& s, const RenderParams&
         __syncthreads();
     }
     // ---- phase 4 (d)
-    store_tile(s, t, P, view, k, ego_active, ((unsigned long long)s.touched[1] << 32) | s.touched[0], false);
+    store_tile<FULL>(s, t, P, view, k, ego_active, ((unsigned long long)s.touched[1] << 32) | s.touched[0], false);
     if (threadIdx.x == 0) { ++n.jobs; ++n.coop; }
 }
 
@@ -1000,14 +1000,14 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
 }
 
 // The tiles the fused kernel left out, a CTA at a time.
-template <class TL>
+template <class TL, bool FULL>
 __global__ void __launch_bounds__(NTHREADS, 5) cooperative_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileSmem& cs = *reinterpret_cast<TileSmem*>(smem_raw);
     TL n = {};
     const unsigned count = __ldcg(&P.overflow[0]);
     for (unsigned i = blockIdx.x; i < count; i += gridDim.x) {
-        cooperative_job(cs, P, __ldcg(&P.overflow[1u + i]), n);
+        cooperative_job<TL, FULL>(cs, P, __ldcg(&P.overflow[1u + i]), n);
         __syncthreads();
     }
     flush_counters(P, n);
@@ -1022,9 +1022,11 @@ cudaError_t configure_render_kernel() {
     if (err != cudaSuccess) return err;
     err = cudaFuncSetAttribute(render_kernel<Tally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
     if (err != cudaSuccess) return err;
-    err = cudaFuncSetAttribute(cooperative_kernel<NoTally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+    err = cudaFuncSetAttribute(cooperative_kernel<NoTally, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
     if (err != cudaSuccess) return err;
-    return cudaFuncSetAttribute(cooperative_kernel<Tally>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+    err = cudaFuncSetAttribute(cooperative_kernel<NoTally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(cooperative_kernel<Tally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
 }
 
 cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cudaStream_t stream) {
@@ -1042,8 +1044,9 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cuda
     if (err != cudaSuccess) return err;
     // the tiles left out (their number is only known on the device): a fixed grid walks the list
     const unsigned cgrid = (unsigned)(jobs < COOP_GRID ? jobs : COOP_GRID);
-    if (P.counters) cooperative_kernel<Tally><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
-    else cooperative_kernel<NoTally><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    if (P.counters) cooperative_kernel<Tally, false><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    else if (full) cooperative_kernel<NoTally, true><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    else cooperative_kernel<NoTally, false><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
     return cudaGetLastError();
 }
 
