@@ -70,13 +70,16 @@ def assert_same_as_exhaustive(prod, brute, sl=slice(None)):
     assert (np.abs(a - b) <= 5e-7 * b).all(), "depths differ between the production and the exhaustive kernel"
 
 
-def random_scene(seed: int):
+def random_scene(seed: int, full_tiles: bool = False):
     """A seeded random scene for fuzzing: triangle soups far from the origin with planar quad pairs
     and a degenerate triangle, random rigs (mounts, yaw, pitch up to 0.5 rad, unequal focal lengths),
-    random image sizes incl. ragged ones, random near/far, inactive agents."""
+    random image sizes incl. ragged ones (`full_tiles`: multiples of 64 only, the sizes that take the
+    kernels' full-tile instantiations), random near/far, inactive agents."""
     car = (4.5, 1.9, 1.5)
     rng = np.random.default_rng(seed)
     H = int(rng.choice([16, 36, 54, 64, 70, 128])); W = int(rng.choice([16, 48, 64, 96, 100, 160]))
+    if full_tiles:
+        H = 64 * (1 + seed % 2); W = 64 * (1 + (seed // 2) % 3)
     K = int(rng.integers(1, 5)); A = int(rng.integers(1, 7)); E = int(rng.integers(1, 3))
     n = int(rng.integers(0, 150))
     scale = float(rng.choice([3.0, 10.0, 40.0]))
