@@ -16,7 +16,8 @@ cudaError_t configure_kernels();
 cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses, float* state, const float* actions,
                          const float* dims, const uint8_t* active, AgentGeom* agents_out, ViewCam* cams_out,
                          float* tables, uint32_t* status, float dt, float wheelbase, float v_max, cudaStream_t stream);
-cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, cudaStream_t stream);
+cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, int sm_count, cudaStream_t stream);
+size_t survivor_bytes_per_tile();
 }  // namespace pic
 
 namespace {
@@ -68,7 +69,9 @@ struct pic_scene {
     pic::Prim* d_prims = nullptr;
     pic::AgentGeom* d_agents = nullptr;
     pic::ViewCam* d_cams = nullptr;   // [E*A*K]
-    uint32_t* d_overflow = nullptr;   // [1 + E*A*K*tiles] tiles handed from the fused to the cooperative render kernel
+    uint32_t* d_overflow = nullptr;   // [1 + E*A*K*tiles] tiles handed from the render kernel to the cooperative kernel
+    uint2* d_surv = nullptr;          // per tile: survivors of the cull kernel, read by the render kernel
+    int sm_count = 0;
     float* d_tables = nullptr;        // per-camera ray and background tables, K*(W+3H) words
     float* d_state = nullptr;       // [E*A*4]
     float* d_dims = nullptr;        // [E*A*3]
@@ -107,7 +110,7 @@ struct DeviceGuard {
 
 void free_scene(pic_scene* s) {
     cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
-    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
+    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_surv); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
     if (s->ev) {
@@ -134,6 +137,7 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.agents = s->d_agents;
     P.cams = s->d_cams;
     P.overflow = s->d_overflow;
+    P.surv = s->d_surv;
     P.rig.ray_x = s->d_tables;
     P.rig.ray_y = P.rig.ray_x + (size_t)s->K * s->W;
     P.rig.bg_z = P.rig.ray_y + (size_t)s->K * s->H;
@@ -213,6 +217,7 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     s->near_z = d->near_z; s->far_z = d->far_z; s->M = d->num_maps;
     s->cls_agent = d->agent_class; s->cls_sky = d->sky_class; s->cls_ground = d->ground_class;
     s->device = d->device;
+    s->sm_count = prop.multiProcessorCount;
 
     size_t np, nl, ng, nm;
     const pic::Prim* prims = pic::hierarchy_prims(hh, &np);
@@ -239,6 +244,7 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_agents, sizeof(pic::AgentGeom) * n_agents);
     dmalloc((void**)&s->d_cams, sizeof(pic::ViewCam) * n_agents * d->K);
     dmalloc((void**)&s->d_overflow, sizeof(uint32_t) * (1 + (size_t)n_agents * d->K * ((d->W + pic::TILE - 1) / pic::TILE) * ((d->H + pic::TILE - 1) / pic::TILE)));
+    dmalloc((void**)&s->d_surv, pic::survivor_bytes_per_tile() * (size_t)n_agents * d->K * ((d->W + pic::TILE - 1) / pic::TILE) * ((d->H + pic::TILE - 1) / pic::TILE));
     dmalloc((void**)&s->d_tables, sizeof(float) * (size_t)d->K * ((size_t)d->W + 3 * (size_t)d->H));
     dmalloc((void**)&s->d_state, sizeof(float) * 4 * n_agents);
     dmalloc((void**)&s->d_dims, sizeof(float) * 3 * n_agents);
@@ -369,7 +375,7 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
     P.view_first = s->view_first;
     const bool timed = s->timing && s->n_timed < kMaxTimed;
     if (timed) CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed], stream));
-    CUDA_TRY(pic::launch_render(P, count, s->brute, stream));
+    CUDA_TRY(pic::launch_render(P, count, s->brute, s->sm_count, stream));
     if (timed) { CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed + 1], stream)); ++s->n_timed; }
     return PIC_OK;
 }

@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(BRUTE_THREADS) render_brute_kernel(const __gri
 // ------------------------------------------------------------------------------------------------
 size_t render_smem_bytes();                       // pic_render.cu
 cudaError_t configure_render_kernel();            // pic_render.cu
-cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, cudaStream_t stream);
+cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, int sm_count, cudaStream_t stream);
 
 size_t max_smem_bytes() { return render_smem_bytes() > sizeof(BruteSmem) ? render_smem_bytes() : sizeof(BruteSmem); }
 
@@ -220,9 +220,9 @@ cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses
     return cudaGetLastError();
 }
 
-cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, cudaStream_t stream) {
+cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, int sm_count, cudaStream_t stream) {
     if (n_views <= 0) return cudaSuccess;
-    if (!brute) return launch_render_kernel(P, n_views, stream);
+    if (!brute) return launch_render_kernel(P, n_views, sm_count, stream);
     const long long blocks = n_views * P.tiles_x * P.tiles_y;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     render_brute_kernel<<<(unsigned)blocks, BRUTE_THREADS, sizeof(BruteSmem), stream>>>(P);

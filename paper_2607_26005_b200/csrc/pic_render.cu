@@ -39,6 +39,15 @@
 
 namespace pic {
 
+// Profiling aid, compiled in only with -DPIC_PROFILE (never in the shipped library): bits 4-7 of the
+// debug flags leave work out so that the cost of a phase can be timed by difference.  The images
+// are then incomplete.
+#ifdef PIC_PROFILE
+#define PIC_STOP(P) (((P).debug_flags >> 4) & 15)
+#else
+#define PIC_STOP(P) 0
+#endif
+
 constexpr int NTHREADS = 128;
 constexpr int NW = NTHREADS / 32;
 constexpr int RCAP = 64;          // records (primitives rasterized by a warp) per tile
@@ -67,10 +76,21 @@ struct __align__(16) TileSmem {
     uint32_t touched[2];                      // 8x8 blocks that may hold a fragment (rows 0-3, rows 4-7)
 };
 
-// Keys are stored so that a 16 x 4 cell (raster) and 16-pixel row segments (store) spread over
-// all banks: the 16-byte chunk holding pixels (2c, 2c+1) of row y sits at chunk c ^ (y & 7).
+// Keys are stored so that both access patterns spread over all banks.  A 16-byte chunk holds pixels
+// (2c, 2c+1) of row y; its low three index bits are XORed with (y & 1) << 2 | (c >> 3).  Raster: a
+// 16 x 4 cell is read a row (8 chunks of one 16-pixel column block) per quarter warp.  Store: 32
+// consecutive lanes take 32 consecutive 16-pixel segments (two rows x four column blocks per quarter
+// warp) and read chunk i of their segment together.
 __device__ __forceinline__ int key_index(int x, int y) {
-    return (y << 6) | ((((x >> 1) ^ (y & 7)) << 1) | (x & 1));
+    const int c = x >> 1;
+    return (y << 6) | (((c ^ (((y & 1) << 2) | (c >> 3))) << 1) | (x & 1));
+}
+
+// 256-bit store (sm_100): a lane's 16 depth values land in one fully written 32-byte sector.
+__device__ __forceinline__ void store_256(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+                 "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
 }
 
 // Bit mask of the 8x8 blocks touched by a pixel box (inclusive).
@@ -189,6 +209,8 @@ struct NoCount {
     __device__ __forceinline__ NoCount& operator++() { return *this; }
     __device__ __forceinline__ NoCount& operator=(int) { return *this; }
 };
+__device__ __forceinline__ int tally_value(int v) { return v; }
+__device__ __forceinline__ int tally_value(const NoCount&) { return 0; }
 struct NoTally { NoCount grp, leaf, tested, setup, tiny, recs, fallback, classified, cells, jobs, coop; };
 
 // Cooperative kernel, phase 2b body: set a surviving primitive up, rasterize it (tiny) or leave a record.
@@ -374,16 +396,13 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
     uint16_t* od = P.out_depth + view * img;
     float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
     const bool vec_ok = FULL || ((P.W % 16 == 0) && o32 == nullptr);
-    const int segs_per_row = (t.tw + 15) >> 4;
+    const int segs_per_row = FULL ? TILE / 16 : (t.tw + 15) >> 4;
     const int n_seg = t.th * segs_per_row;
-    // full-width tiles with a multiple of 8 rows: eight consecutive threads take eight consecutive
-    // rows of one 16-pixel column strip, so that their 16-byte key accesses fall in different
-    // banks (the swizzle is by row); a warp still covers 8 rows x 64 pixels of the image
-    const bool by_rows = FULL || (segs_per_row == 4 && (t.th & 7) == 0);
+    // consecutive threads take consecutive 16-pixel segments of a row, then the next row: a warp's
+    // class stores cover 512 contiguous bytes of a 64-pixel-wide image, its depth stores 1 KB
     for (int seg = tid; seg < n_seg; seg += nthr) {
-        int y, xs;
-        if (by_rows) { y = (seg & 7) | ((seg >> 5) << 3); xs = ((seg >> 3) & 3) * 16; }
-        else { y = seg / segs_per_row; xs = (seg - y * segs_per_row) * 16; }
+        const int y = FULL ? seg >> 2 : seg / segs_per_row;
+        const int xs = (seg - y * segs_per_row) * 16;
         uint32_t bg_cls = P.cls_sky;
         float bg_z = P.far_z;
         if (ego_active) { bg_cls = __ldg(P.rig.bg_cls + (size_t)k * P.H + t.y0 + y); bg_z = __ldg(P.rig.bg_z + (size_t)k * P.H + t.y0 + y); }
@@ -413,9 +432,16 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
                     if ((j & 3) == 0) cw[j >> 2] = c0 | (c1 << 8); else cw[j >> 2] |= (c0 << 16) | (c1 << 24);
                 }
             }
+#ifdef PIC_PROFILE
+            if (PIC_STOP(P) == 6 && !(P.debug_flags & 0x10000)) continue;
+#endif
             *reinterpret_cast<uint4*>(oc + o) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-            *reinterpret_cast<uint4*>(od + o) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
-            *reinterpret_cast<uint4*>(od + o + 8) = make_uint4(dw[4], dw[5], dw[6], dw[7]);
+            if (FULL) {
+                store_256(od + o, dw);
+            } else {
+                *reinterpret_cast<uint4*>(od + o) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
+                *reinterpret_cast<uint4*>(od + o + 8) = make_uint4(dw[4], dw[5], dw[6], dw[7]);
+            }
         } else {
             for (int j = 0; j < 16 && xs + j < t.tw; ++j) {
                 const unsigned long long key = empty ? 0ull : s.key[key_index(xs + j, y)];
@@ -474,7 +500,7 @@ __device__ __forceinline__ void cooperative_job(TileSmem& s, const RenderParams&
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool classify = !(P.debug_flags & 1);
     const int rec_cap = (P.debug_flags & 2) ? 2 : RCAP;
-    const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave after phase `stop` (image incomplete)
+    const int stop = PIC_STOP(P);
     const int k = job.k, a = job.a, e = job.e;
     const size_t view = job.view;
     const TileCtx t = job.t;
@@ -627,17 +653,17 @@ __device__ __forceinline__ void flush_counters(const RenderParams& P, const Tall
 //           rasterizes a strip of some tile into its own strip of keys and stores it (back_strip).
 //   rest    tiles whose lists or records did not fit are appended to the cooperative kernel's list.
 // ---------------------------------------------------------------------------------------------
-constexpr int POOL = 132;         // records shared by the NW tiles of a CTA
+constexpr int POOL = 128;         // records shared by the NW tiles of a CTA
 constexpr int STRIP = 16;         // pixel rows a warp rasterizes at a time
 constexpr int STRIP_KEYS = TILE * STRIP;
 constexpr int W_LEAF = 256;       // per-warp front-end lists (they live in the key buffer, 8 KB per warp)
 constexpr int W_FACE = 384;
-constexpr int W_SURV = 256;
-constexpr long long COOP_GRID = 148 * 5;   // CTAs of the cooperative kernel: one wave
+constexpr int SURV_STRIDE = 128;  // uint2 per tile in the survivor buffer: a 16-byte head (count; work counts), then the list
+constexpr int W_SURV = SURV_STRIDE - 2;
+constexpr uint32_t SURV_FACE = 0x80000000u;   // survivor id: primitive index, or SURV_FACE | agent << 3 | face
 constexpr uint32_t REC_TINY = 1u << 28, REC_DEAD = 1u << 29;   // flags in the box word of a record
 
 struct __align__(16) FrontLists {
-    uint2 surv[W_SURV];                       // (candidate, pixel box)
     uint32_t leaf[W_LEAF];                    // first primitive << 4 | count
     uint32_t face[W_FACE];                    // agent << 3 | face
     float plane[6][4];
@@ -654,8 +680,8 @@ struct __align__(16) FusedSmem {
     int next_task;
     int tile_active[NW];                      // is the ego agent of tile w active
     Job tile_job[NW];                         // tile w, decoded by its warp
+    Cam cam[NW];                              // its camera
 };
-static_assert(sizeof(FrontLists) <= sizeof(unsigned long long) * STRIP_KEYS, "front-end lists must fit a warp's key strip");
 static_assert(sizeof(FusedSmem) <= 44 * 1024 && sizeof(TileSmem) <= 44 * 1024,
               "shared memory must leave room for 5 CTAs per SM (228 KB, 1 KB reserved per CTA)");
 // What the raster and store templates need of a warp's strip: rows are counted from the strip's first.
@@ -664,7 +690,7 @@ struct StripView {
     const float* ray_x;
     const float* ray_y;
 };
-constexpr size_t RENDER_SMEM = sizeof(FusedSmem) > sizeof(TileSmem) ? sizeof(FusedSmem) : sizeof(TileSmem);
+constexpr size_t RENDER_SMEM_BASE = sizeof(FusedSmem) > sizeof(TileSmem) ? sizeof(FusedSmem) : sizeof(TileSmem);
 
 __device__ __forceinline__ void write_record(float4* r, const PrimEq& q, uint32_t key_lo, uint32_t box, uint32_t extra) {
     const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
@@ -685,12 +711,56 @@ __device__ __forceinline__ void read_record(const float4* r, PrimEq& q, uint32_t
     key_lo = __float_as_uint(r3.w);
 }
 
+// Box test against planes held in registers (see box_visible).
+__device__ __forceinline__ bool box_visible_reg(const float4 (&pl)[6], float px, float py, const Node& b) {
+    const float ax = sub(b.lo[0], px), bx = sub(b.hi[0], px);
+    const float ay = sub(b.lo[1], py), by = sub(b.hi[1], py);
+    const float cx = 0.5f * (ax + bx), cy = 0.5f * (ay + by), cz = 0.5f * (b.lo[2] + b.hi[2]);
+    const float hx = 0.5f * (bx - ax), hy = 0.5f * (by - ay), hz = 0.5f * (b.hi[2] - b.lo[2]);
+    const float slack = 1e-3f + 4e-6f * (fabsf(cx) + fabsf(cy) + fabsf(cz) + hx + hy + hz);
+    bool vis = true;
+#pragma unroll
+    for (int p = 0; p < 6; ++p) {
+        const float dist = pl[p].x * cx + pl[p].y * cy + pl[p].z * cz + pl[p].w;
+        const float reach = fabsf(pl[p].x) * hx + fabsf(pl[p].y) * hy + fabsf(pl[p].z) * hz;
+        vis = vis && (dist + reach >= -slack);
+    }
+    return vis;
+}
+
+__device__ __forceinline__ Node load_node(const Node* p) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    Node nd;
+    nd.lo[0] = a.x; nd.lo[1] = a.y; nd.lo[2] = a.z; nd.first = __float_as_uint(a.w);
+    nd.hi[0] = b.x; nd.hi[1] = b.y; nd.hi[2] = b.z; nd.count = __float_as_uint(b.w);
+    return nd;
+}
+
+__device__ __forceinline__ AgentGeom load_agent(const AgentGeom* p) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    AgentGeom g;
+    g.x = a.x; g.y = a.y; g.c = a.z; g.s = a.w; g.hl = b.x; g.hw = b.y; g.h = b.z; g.active = __float_as_uint(b.w);
+    return g;
+}
+
 // Front end of one tile by one warp: fills f.leaf / f.face / f.surv.  Returns the number of
 // survivors, or -1 if a list overflowed (the tile then goes to the cooperative kernel).
+// Loads that do not depend on one another are issued together (the first group boxes and the
+// first agents before the camera is even set up; the leaf boxes of three visible groups, two
+// candidates per lane), so that a pass waits for memory once.
 template <class TL>
-__device__ __forceinline__ int front_cull(FrontLists& f, const RenderParams& P, const Job& job, const MapInfo& mi,
-                                          int lane, int& nl_out, TL& n) {
+__device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ surv, const RenderParams& P, const Job& job,
+                                          const MapInfo& mi, int lane, TL& n) {
+    const int stop = PIC_STOP(P);
     const TileCtx& t = job.t;
+    Node gn0;
+    gn0.first = 0; gn0.count = 0;
+    if (mi.group_begin + lane < mi.group_end) gn0 = load_node(P.groups + mi.group_begin + lane);
+    const AgentGeom* env_agents = P.agents + (size_t)job.e * P.A;
+    AgentGeom ag0, ag1;
+    ag0.active = 0u; ag1.active = 0u;
+    if (lane < P.A) ag0 = load_agent(env_agents + lane);
+    if (lane + 32 < P.A) ag1 = load_agent(env_agents + lane + 32);
     if (lane < 7) {
         Cam c;
         load_camera(c, P.cams[job.view], P.cam[job.k], P.W, P.H);
@@ -698,81 +768,170 @@ __device__ __forceinline__ int front_cull(FrontLists& f, const RenderParams& P, 
         else tile_planes(f, lane, c, t);
     }
     __syncwarp();
+    if (stop == 11) return 0;
     const Cam& c = f.cam;
-    // ---- hierarchy: 32 groups per pass, a visible group's leaves one per lane
+    float4 pl[6];
+#pragma unroll
+    for (int p = 0; p < 6; ++p) pl[p] = *reinterpret_cast<const float4*>(f.plane[p]);
+    const float epx = c.px, epy = c.py;
+    // ---- hierarchy: 32 groups per pass; the leaves of three visible groups at a time, one per lane
     int n_leaf = 0;
     for (uint32_t g0 = mi.group_begin; g0 < mi.group_end; g0 += 32) {
         const uint32_t g = g0 + lane;
         bool vis = false;
         Node gn;
         gn.first = 0; gn.count = 0;
-        if (g < mi.group_end) { gn = P.groups[g]; vis = box_visible(f, gn); ++n.grp; }
-        for (unsigned gm = __ballot_sync(0xffffffffu, vis); gm; gm &= gm - 1) {
-            const int src = __ffs(gm) - 1;
-            const uint32_t first = __shfl_sync(0xffffffffu, gn.first, src);
-            const uint32_t cnt = __shfl_sync(0xffffffffu, gn.count, src);
-            bool lvis = false;
-            Node lf;
-            lf.first = 0; lf.count = 0;
-            if (lane < (int)cnt) { lf = P.leaves[first + lane]; lvis = box_visible(f, lf); ++n.leaf; }
-            const unsigned lm = __ballot_sync(0xffffffffu, lvis);
-            if (lvis) {
-                const int slot = n_leaf + __popc(lm & ((1u << lane) - 1u));
-                if (slot < W_LEAF) f.leaf[slot] = (lf.first << 4) | lf.count;
+        if (g < mi.group_end) { gn = (g0 == mi.group_begin) ? gn0 : load_node(P.groups + g); vis = box_visible_reg(pl, epx, epy, gn); ++n.grp; }
+        unsigned gm = __ballot_sync(0xffffffffu, vis);
+        while (gm) {
+            Node lf[3];
+            bool lvis[3];
+#pragma unroll
+            for (int u = 0; u < 3; ++u) {
+                const int src = gm ? __ffs(gm) - 1 : 0;
+                const bool have = gm != 0u;
+                gm &= gm - 1;
+                const uint32_t first = __shfl_sync(0xffffffffu, gn.first, src);
+                const uint32_t cnt = have ? __shfl_sync(0xffffffffu, gn.count, src) : 0u;
+                lvis[u] = lane < (int)cnt;
+                lf[u].first = 0; lf[u].count = 0;
+                if (lvis[u]) lf[u] = load_node(P.leaves + first + lane);
             }
-            n_leaf += __popc(lm);
+#pragma unroll
+            for (int u = 0; u < 3; ++u) {
+                if (lvis[u]) { lvis[u] = box_visible_reg(pl, epx, epy, lf[u]); ++n.leaf; }
+                const unsigned lm = __ballot_sync(0xffffffffu, lvis[u]);
+                if (lvis[u]) {
+                    const int slot = n_leaf + __popc(lm & ((1u << lane) - 1u));
+                    if (slot < W_LEAF) f.leaf[slot] = (lf[u].first << 4) | lf[u].count;
+                }
+                n_leaf += __popc(lm);
+            }
         }
     }
-    // ---- other agents' boxes
-    for (int b0 = 0; b0 < P.A; b0 += 32) {
-        const int b = b0 + lane;
-        uint32_t faces = 0u;
-        if (b < P.A && b != job.a) {
-            const AgentGeom g = P.agents[(size_t)job.e * P.A + b];
-            if (g.active) faces = box_faces(f, c, t, g);
+    if (stop == 12) return 0;
+    // ---- other agents' boxes, two per lane at a time
+    for (int b0 = 0; b0 < P.A; b0 += 64) {
+        if (b0 > 0) {
+            ag0.active = 0u; ag1.active = 0u;
+            if (b0 + lane < P.A) ag0 = load_agent(env_agents + b0 + lane);
+            if (b0 + lane + 32 < P.A) ag1 = load_agent(env_agents + b0 + lane + 32);
         }
-        if (faces) {
-            int slot = atomicAdd(&f.n_face, __popc(faces));
-            for (; faces; faces &= faces - 1, ++slot)
-                if (slot < W_FACE) f.face[slot] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const AgentGeom& g = u ? ag1 : ag0;
+            const int b = b0 + lane + 32 * u;
+            uint32_t faces = 0u;
+            if (b < P.A && b != job.a && g.active) faces = box_faces(f, c, t, g);
+            if (faces) {
+                int slot = atomicAdd(&f.n_face, __popc(faces));
+                for (; faces; faces &= faces - 1, ++slot)
+                    if (slot < W_FACE) f.face[slot] = ((uint32_t)b << 3) | (uint32_t)(__ffs(faces) - 1);
+            }
         }
     }
     __syncwarp();
     const int n_face = f.n_face;
     if (n_leaf > W_LEAF || n_face > W_FACE) return -1;
-    nl_out = n_leaf;
-    // ---- candidates: camera space, pixel box; survivors are compacted
-    const int n_items = n_leaf * LEAF_PRIMS + n_face;
+    if (stop == 13) return 0;
+    // ---- candidates: camera space, pixel box; survivors are compacted.  Map primitives two per
+    // lane at a time, then the box faces.
+    const int n_prim_items = n_leaf * LEAF_PRIMS;
     int n_surv = 0;
-    for (int i0 = 0; i0 < n_items; i0 += 32) {
+    for (int i0 = 0; i0 < n_prim_items; i0 += 64) {
+        float v[2][12];
+        bool have[2];
+        uint32_t id[2] = {0u, 0u};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + 32 * u + lane;
+            have[u] = false;
+            if (i < n_prim_items) {
+                const uint32_t lf = f.leaf[i / LEAF_PRIMS];
+                const uint32_t j = i % LEAF_PRIMS;
+                if (j < (lf & 15u)) {
+                    have[u] = true;
+                    uint32_t key_lo, flags;
+                    id[u] = (lf >> 4) + j;
+                    load_prim(P.prims + id[u], v[u], key_lo, flags);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            uint32_t box = 0;
+            bool keep = false;
+            if (have[u]) {
+                V3 V[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[u][3 * q], v[u][3 * q + 1], v[u][3 * q + 2]);
+                ++n.tested;
+                keep = pixel_box(c, t, V, box);
+            }
+            const unsigned m = __ballot_sync(0xffffffffu, keep);
+            if (keep) {
+                const int slot = n_surv + __popc(m & ((1u << lane) - 1u));
+                if (slot < W_SURV) surv[slot] = make_uint2(id[u], box);
+            }
+            n_surv += __popc(m);
+        }
+    }
+    for (int i0 = 0; i0 < n_face; i0 += 32) {
         const int i = i0 + lane;
-        V3 V[4], Pn;
-        uint32_t key_lo, flags, box = 0;
+        uint32_t box = 0, it = 0;
         bool keep = false;
-        if (i < n_items && fetch_candidate(f, P, i, n_leaf, job.e, mi.n_tris, V, Pn, key_lo, flags, false)) {
+        if (i < n_face) {
+            it = f.face[i];
+            const AgentGeom g = load_agent(env_agents + (it >> 3));
+            const uint32_t corners = face_corners((int)(it & 7u));
+            V3 V[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
             ++n.tested;
             keep = pixel_box(c, t, V, box);
         }
         const unsigned m = __ballot_sync(0xffffffffu, keep);
         if (keep) {
             const int slot = n_surv + __popc(m & ((1u << lane) - 1u));
-            if (slot < W_SURV) f.surv[slot] = make_uint2((uint32_t)i, box);
+            if (slot < W_SURV) surv[slot] = make_uint2(SURV_FACE | it, box);
         }
         n_surv += __popc(m);
     }
     __syncwarp();
+    if (stop == 14) return 0;
     return n_surv > W_SURV ? -1 : n_surv;
 }
 
-// Set-up of a tile's survivors by its warp: survivor i becomes record i of `rec`.
+// Survivor `id` in camera space with its plane normal.
+__device__ __forceinline__ void fetch_survivor(const Cam& c, const RenderParams& P, uint32_t id, int e, uint32_t n_map_tris,
+                                               V3 (&V)[4], V3& Pn, uint32_t& key_lo, uint32_t& flags) {
+    if (!(id & SURV_FACE)) {
+        float v[12];
+        load_prim(P.prims + id, v, key_lo, flags);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
+        Pn = plane_normal_world(c, v, flags & 1u);
+    } else {
+        const int b = (int)((id & ~SURV_FACE) >> 3), f = (int)(id & 7u);
+        const AgentGeom g = P.agents[(size_t)e * P.A + b];
+        const uint32_t corners = face_corners(f);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
+        key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+        flags = face_flags(corners);
+        Pn = plane_normal(V, true);
+    }
+}
+
+// Set-up of a tile's survivors (the cull kernel's list) by its warp: survivor i becomes record i of `rec`.
 template <class TL>
-__device__ __forceinline__ void front_setup(const FrontLists& f, float4* rec, const RenderParams& P, const Job& job,
-                                            const MapInfo& mi, int nl, int ns, int lane, TL& n) {
+__device__ __forceinline__ void front_setup(const Cam& c, const uint2* __restrict__ surv, float4* rec, const RenderParams& P,
+                                            const Job& job, const MapInfo& mi, int ns, int lane, TL& n) {
     for (int i = lane; i < ns; i += 32) {
-        const uint2 sv = f.surv[i];
+        const uint2 sv = __ldcg(surv + i);
         V3 V[4], Pn;
         uint32_t key_lo, flags;
-        fetch_candidate(f, P, (int)sv.x, nl, job.e, mi.n_tris, V, Pn, key_lo, flags, true);
+        fetch_survivor(c, P, sv.x, job.e, mi.n_tris, V, Pn, key_lo, flags);
         PrimEq q;
         float4* r = rec + i * (REC / 4);
         if (!prim_equations(V, flags & 1u, flags, Pn, q)) { r[4].x = __uint_as_float(REC_DEAD); continue; }
@@ -804,6 +963,7 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
             bw_lane = __float_as_uint(r[4].x);
             const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
             hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + STRIP;
+            if (hit && (bw_lane & REC_TINY) && stop == 7) hit = false;
             if (hit && (bw_lane & REC_TINY)) {
                 hit = false;
                 const int bx0 = bw_lane & 63, bx1 = (bw_lane >> 12) & 63;
@@ -890,7 +1050,7 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
     TileCtx ts = t;
     ts.y0 = t.y0 + ys; ts.th = rows;
     const bool ragged = !FULL && (t.tw < TILE || rows < STRIP);
-    store_tile<FULL>(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32);
+    if (stop != 8) store_tile<FULL>(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32);
     __syncwarp();
     if (ragged) {
 #pragma unroll
@@ -900,8 +1060,39 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
     }
 }
 
-// FULL: every tile is 64 x 64, rows allow 128-bit stores, no float32 depth image (the launcher
-// checks) -- the instantiation the workloads run, without the code for ragged tiles.
+// Cull kernel: a warp per tile walks the hierarchy and the other agents' boxes, tests the candidates
+// and leaves the tile's survivors (id, pixel box) in device memory: a 16-byte head (count, or -1 if a
+// list overflowed; with counters, the tile's group / leaf / candidate tests), then the list.  No
+// CTA-wide synchronisation.  The lists are small (about 250 bytes per view on the benchmark
+// workload) and are read back by the render kernel that follows on the stream.
+struct __align__(16) CullSmem {
+    FrontLists lists[NW];
+};
+
+template <class TL>
+__global__ void __launch_bounds__(NTHREADS, 5) cull_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    CullSmem& s = *reinterpret_cast<CullSmem*>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned id = blockIdx.x * (unsigned)NW + warp;
+    if (id >= P.n_jobs) return;
+    TL n = {};
+    const int stop = PIC_STOP(P);
+    const Job job = decode_job(P, id);
+    const MapInfo mi = P.env_maps[job.e];
+    const bool ego_active = P.agents[(size_t)job.e * P.A + job.a].active != 0;
+    uint2* blk = P.surv + (size_t)id * SURV_STRIDE;
+    int ns = 0;
+    if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
+    else if (ego_active && stop != 1 && !(stop >= 8 && stop <= 10)) ns = front_cull(s.lists[warp], blk + 2, P, job, mi, lane, n);
+    // (the work counts are summed over the warp's lanes; without counters they are constants)
+    const uint32_t c_grp = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.grp)), c_leaf = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.leaf)),
+                   c_tested = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.tested));
+    if (lane == 0) *reinterpret_cast<uint4*>(blk) = make_uint4((uint32_t)ns, c_grp, c_leaf, c_tested);
+}
+
+// Render kernel.  FULL: every tile is 64 x 64, rows allow 128-bit stores, no float32 depth image (the
+// launcher checks) -- the instantiation the workloads run, without the code for ragged tiles.
 template <class TL, bool FULL>
 __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -910,25 +1101,29 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     const unsigned first = blockIdx.x * (unsigned)NW, n_jobs = P.n_jobs;
     TL n = {};
     const bool classify = !(P.debug_flags & 1);
-    const int stop = (P.debug_flags >> 4) & 15;     // profiling aid: leave work out (image incomplete)
+    const int stop = PIC_STOP(P);
     // test aids: a pool of 2 records sends nearly every tile to cooperative_job, one of 40 mixes both paths
-    const int pool_cap = FULL ? POOL : (P.debug_flags & 2) ? 2 : (P.debug_flags & 8) ? 40 : POOL;   // (FULL is launched without debug flags)
+    const int pool_cap = FULL ? POOL : (P.debug_flags & 2) ? 2 : (P.debug_flags & 8) ? 40 : POOL;   // (FULL is launched without these flags)
     if (threadIdx.x == 0) s.next_task = 0;
-    FrontLists& fl = *reinterpret_cast<FrontLists*>(s.key[warp]);
 
-    // ---- front end: warp w culls tile first + w
+    // ---- the cull kernel's survivors of tile first + w
     const bool valid = first + warp < n_jobs;
     Job job;
     MapInfo mi;
-    int nl = 0, ns = -2;
+    const uint2* blk = P.surv + (size_t)(first + warp) * SURV_STRIDE;
+    int ns = -2;
     if (valid) {
+        const uint4 head = __ldcg(reinterpret_cast<const uint4*>(blk));
         job = decode_job(P, first + warp);
         mi = P.env_maps[job.e];
         const bool ego_active = P.agents[(size_t)job.e * P.A + job.a].active != 0;
-        if (lane == 0) { s.tile_job[warp] = job; s.tile_active[warp] = ego_active; }
-        ns = 0;
-        if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
-        else if (ego_active && stop != 1) ns = front_cull(fl, P, job, mi, lane, nl, n);
+        if (lane == 0) {
+            s.tile_job[warp] = job; s.tile_active[warp] = ego_active;
+            load_camera(s.cam[warp], P.cams[job.view], P.cam[job.k], P.W, P.H);
+        }
+        ns = (int)head.x;
+        if (ns > W_SURV) ns = -1;
+        if (lane == 0) { n.grp = (int)head.y; n.leaf = (int)head.z; n.tested = (int)head.w; }
     }
     if (lane == 0) s.n_surv[warp] = ns;
     __syncthreads();
@@ -948,15 +1143,18 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     {
         const int my_base = (int)((bases >> (8 * warp)) & 0xffu), my_cnt = (int)((cnts >> (8 * warp)) & 0xffu);
         if (my_cnt == 0xff) { n.grp = 0; n.leaf = 0; n.tested = 0; }       // counted again by cooperative_job
-        else if (my_cnt != 0xfe && my_cnt > 0) front_setup(fl, s.pool + my_base * (REC / 4), P, job, mi, nl, my_cnt, lane, n);
+        else if (my_cnt != 0xfe && my_cnt > 0 && stop != 14) front_setup(s.cam[warp], blk + 2, s.pool + my_base * (REC / 4), P, job, mi, my_cnt, lane, n);
     }
     __syncthreads();
     // ---- back end: the NW tiles' strips are tasks that the warps draw from a counter; a warp's
     // lists are dead, their memory becomes its strip of keys
+    if (stop != 9) {
 #pragma unroll
-    for (int i = 0; i < STRIP_KEYS / 2 / 32; ++i)
-        reinterpret_cast<ulonglong2*>(s.key[warp])[i * 32 + lane] = make_ulonglong2(0ull, 0ull);
+        for (int i = 0; i < STRIP_KEYS / 2 / 32; ++i)
+            reinterpret_cast<ulonglong2*>(s.key[warp])[i * 32 + lane] = make_ulonglong2(0ull, 0ull);
+    }
     __syncwarp();
+    if (stop == 10) return;
     StripView sv;
     sv.key = s.key[warp]; sv.ray_x = s.ray_x[warp]; sv.ray_y = s.ray_y[warp];
     constexpr int STRIPS = TILE / STRIP;
@@ -1013,6 +1211,16 @@ __global__ void __launch_bounds__(NTHREADS, 5) cooperative_kernel(const __grid_c
     flush_counters(P, n);
 }
 
+#ifdef PIC_PROFILE
+}  // namespace pic
+#include <cstdlib>
+namespace pic {
+// profiling aid: extra dynamic shared memory per CTA lowers the number of resident CTAs per SM
+static size_t smem_pad() { const char* e = getenv("PIC_SMEM_PAD"); return e ? (size_t)atoi(e) : 0; }
+#define RENDER_SMEM (RENDER_SMEM_BASE + smem_pad())
+#else
+#define RENDER_SMEM RENDER_SMEM_BASE
+#endif
 size_t render_smem_bytes() { return RENDER_SMEM; }
 
 cudaError_t configure_render_kernel() {
@@ -1029,21 +1237,31 @@ cudaError_t configure_render_kernel() {
     return cudaFuncSetAttribute(cooperative_kernel<Tally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
 }
 
-cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, cudaStream_t stream) {
+size_t survivor_bytes_per_tile() { return sizeof(uint2) * SURV_STRIDE; }
+
+cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int sm_count, cudaStream_t stream) {
     RenderParams P = P0;
     const long long jobs = n_views * P.tiles_x * P.tiles_y;
     if (jobs > 0x7fffffffLL || (long long)P.E * P.A * P.K > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     if (jobs <= 0) return cudaSuccess;
     P.n_jobs = (uint32_t)jobs;
     const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
-    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr && P.debug_flags == 0;
+    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr && (P.debug_flags & 15) == 0 &&
+                      (reinterpret_cast<uintptr_t>(P.out_depth) & 31u) == 0;   // 256-bit depth stores
+    // (a) cull: survivors per tile
+    if (P.counters) cull_kernel<Tally><<<grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    else cull_kernel<NoTally><<<grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    // (b)-(d) set-up, raster, store
     if (P.counters) render_kernel<Tally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     else if (full) render_kernel<NoTally, true><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     else render_kernel<NoTally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
-    cudaError_t err = cudaGetLastError();
+    err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    // the tiles left out (their number is only known on the device): a fixed grid walks the list
-    const unsigned cgrid = (unsigned)(jobs < COOP_GRID ? jobs : COOP_GRID);
+    // the tiles left out (their number is only known on the device): one wave of CTAs walks the list
+    const long long wave = (long long)(sm_count > 0 ? sm_count : 148) * 5;
+    const unsigned cgrid = (unsigned)(jobs < wave ? jobs : wave);
     if (P.counters) cooperative_kernel<Tally, false><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
     else if (full) cooperative_kernel<NoTally, true><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
     else cooperative_kernel<NoTally, false><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);

@@ -1,6 +1,7 @@
 // Device/host data layout of the rasterizer library (internal).
 #pragma once
 #include <stdint.h>
+#include <vector_types.h>
 
 namespace pic {
 
@@ -91,6 +92,7 @@ struct RenderParams {
     float* out_depth32;             // optional
     unsigned long long* counters;   // optional [16]
     uint32_t* overflow;             // [1 + tiles of all views]: count, then the tiles left to the cooperative kernel
+    uint2* surv;                    // per tile: the cull kernel's survivors (head + list), read by the render kernel
     int32_t debug_flags;            // bit 0: no per-cell trivial accept/reject, bit 1: record pool / list of 2 entries, bit 2: cooperative kernel only, bit 3: pool of 40, bits 4-7: profiling stop
     uint32_t n_jobs;                // tiles to render in this launch (views x tiles per view); set by the launcher
     long long view_first;           // render views [view_first, view_first + gridDim / tiles)
