@@ -658,10 +658,16 @@ constexpr int STRIP = 16;         // pixel rows a warp rasterizes at a time
 constexpr int STRIP_KEYS = TILE * STRIP;
 constexpr int W_LEAF = 256;       // per-warp front-end lists (they live in the key buffer, 8 KB per warp)
 constexpr int W_FACE = 384;
-constexpr int SURV_STRIDE = 128;  // uint2 per tile in the survivor buffer: a 16-byte head (count; work counts), then the list
+// Survivor buffer, SURV_STRIDE uint2 per tile: a 16-byte head (counts; work counts), then W_SURV
+// entries (id, pixel box).  Survivors whose pixel box holds more than TINY_MAX_PIXELS pixel centres
+// fill the list from the front, the others from the back; head.x = front count | back count << 16,
+// or all ones if a list overflowed.
+constexpr int SURV_STRIDE = 128;
 constexpr int W_SURV = SURV_STRIDE - 2;
+constexpr uint32_t SURV_OVERFLOW = 0xffffffffu;
 constexpr uint32_t SURV_FACE = 0x80000000u;   // survivor id: primitive index, or SURV_FACE | agent << 3 | face
 constexpr uint32_t REC_TINY = 1u << 28, REC_DEAD = 1u << 29;   // flags in the box word of a record
+constexpr uint32_t REC_INRANGE = 1u << 30;   // every covered pixel is within [near, far]: no per-pixel range test
 
 struct __align__(16) FrontLists {
     uint32_t leaf[W_LEAF];                    // first primitive << 4 | count
@@ -743,8 +749,26 @@ __device__ __forceinline__ AgentGeom load_agent(const AgentGeom* p) {
     return g;
 }
 
-// Front end of one tile by one warp: fills f.leaf / f.face / f.surv.  Returns the number of
-// survivors, or -1 if a list overflowed (the tile then goes to the cooperative kernel).
+__device__ __forceinline__ bool tiny_box(uint32_t box) {
+    const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    return (bx1 - bx0 + 1) * (by1 - by0 + 1) <= TINY_MAX_PIXELS;
+}
+
+// Warp-wide append to the two-ended survivor list (see SURV_STRIDE).
+__device__ __forceinline__ void append_survivor(uint2* __restrict__ surv, bool keep, uint32_t id, uint32_t box, int& n_big, int& n_tiny, int lane) {
+    const bool tiny = keep && tiny_box(box), big = keep && !tiny;
+    const unsigned mb = __ballot_sync(0xffffffffu, big), mt = __ballot_sync(0xffffffffu, tiny);
+    const unsigned below = (1u << lane) - 1u;
+    // (a slot is written only while front and back have not met; the caller checks the total)
+    if (big) { const int slot = n_big + __popc(mb & below); if (slot + n_tiny < W_SURV) surv[slot] = make_uint2(id, box); }
+    if (tiny) { const int slot = n_tiny + __popc(mt & below); if (slot + n_big + __popc(mb) < W_SURV) surv[W_SURV - 1 - slot] = make_uint2(id, box); }
+    n_big += __popc(mb);
+    n_tiny += __popc(mt);
+}
+
+// Front end of one tile by one warp: fills f.leaf / f.face and the survivor list.  Returns the
+// survivor counts (front | back << 16), or -1 if a list overflowed (the tile then goes to the
+// cooperative kernel).
 // Loads that do not depend on one another are issued together (the first group boxes and the
 // first agents before the camera is even set up; the leaf boxes of three visible groups, two
 // candidates per lane), so that a pass waits for memory once.
@@ -837,7 +861,7 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
     // ---- candidates: camera space, pixel box; survivors are compacted.  Map primitives two per
     // lane at a time, then the box faces.
     const int n_prim_items = n_leaf * LEAF_PRIMS;
-    int n_surv = 0;
+    int n_big = 0, n_tiny = 0;
     for (int i0 = 0; i0 < n_prim_items; i0 += 64) {
         float v[2][12];
         bool have[2];
@@ -868,12 +892,7 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
                 ++n.tested;
                 keep = pixel_box(c, t, V, box);
             }
-            const unsigned m = __ballot_sync(0xffffffffu, keep);
-            if (keep) {
-                const int slot = n_surv + __popc(m & ((1u << lane) - 1u));
-                if (slot < W_SURV) surv[slot] = make_uint2(id[u], box);
-            }
-            n_surv += __popc(m);
+            append_survivor(surv, keep, id[u], box, n_big, n_tiny, lane);
         }
     }
     for (int i0 = 0; i0 < n_face; i0 += 32) {
@@ -890,16 +909,11 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
             ++n.tested;
             keep = pixel_box(c, t, V, box);
         }
-        const unsigned m = __ballot_sync(0xffffffffu, keep);
-        if (keep) {
-            const int slot = n_surv + __popc(m & ((1u << lane) - 1u));
-            if (slot < W_SURV) surv[slot] = make_uint2(SURV_FACE | it, box);
-        }
-        n_surv += __popc(m);
+        append_survivor(surv, keep, SURV_FACE | it, box, n_big, n_tiny, lane);
     }
     __syncwarp();
     if (stop == 14) return 0;
-    return n_surv > W_SURV ? -1 : n_surv;
+    return n_big + n_tiny > W_SURV ? -1 : (n_big | (n_tiny << 16));
 }
 
 // Survivor `id` in camera space with its plane normal.
@@ -923,12 +937,19 @@ __device__ __forceinline__ void fetch_survivor(const Cam& c, const RenderParams&
     }
 }
 
+// A covered pixel's depth lies between the vertices' depths; with a margin far above the rounding
+// of the 1/z plane, vertices well inside [near, far] make the per-pixel range test redundant.
+__device__ __forceinline__ bool record_in_range(const V3 (&V)[4], const RenderParams& P) {
+    const float zlo = fminf(fminf(V[0].z, V[1].z), fminf(V[2].z, V[3].z)), zhi = fmaxf(fmaxf(V[0].z, V[1].z), fmaxf(V[2].z, V[3].z));
+    return zlo >= P.near_z * 1.001f && zhi <= P.far_z * 0.999f;
+}
+
 // Set-up of a tile's survivors (the cull kernel's list) by its warp: survivor i becomes record i of `rec`.
 template <class TL>
 __device__ __forceinline__ void front_setup(const Cam& c, const uint2* __restrict__ surv, float4* rec, const RenderParams& P,
-                                            const Job& job, const MapInfo& mi, int ns, int lane, TL& n) {
+                                            const Job& job, const MapInfo& mi, int ns, int n_big, int lane, TL& n) {
     for (int i = lane; i < ns; i += 32) {
-        const uint2 sv = __ldcg(surv + i);
+        const uint2 sv = __ldcg(surv + (i < n_big ? i : W_SURV - 1 - (i - n_big)));
         V3 V[4], Pn;
         uint32_t key_lo, flags;
         fetch_survivor(c, P, sv.x, job.e, mi.n_tris, V, Pn, key_lo, flags);
@@ -940,7 +961,7 @@ __device__ __forceinline__ void front_setup(const Cam& c, const uint2* __restric
         const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
         const bool tiny = (bx1 - bx0 + 1) * (by1 - by0 + 1) <= TINY_MAX_PIXELS;
         if (tiny) ++n.tiny; else ++n.recs;
-        write_record(r, q, key_lo, box, tiny ? REC_TINY : 0u);
+        write_record(r, q, key_lo, box, (tiny ? REC_TINY : 0u) | (record_in_range(V, P) ? REC_INRANGE : 0u));
     }
 }
 
@@ -1069,8 +1090,14 @@ struct __align__(16) CullSmem {
     FrontLists lists[NW];
 };
 
+#ifndef PIC_CULL_CTAS
+#define PIC_CULL_CTAS 5
+#endif
+#ifndef PIC_RENDER_CTAS
+#define PIC_RENDER_CTAS 5
+#endif
 template <class TL>
-__global__ void __launch_bounds__(NTHREADS, 5) cull_kernel(const __grid_constant__ RenderParams P) {
+__global__ void __launch_bounds__(NTHREADS, PIC_CULL_CTAS) cull_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     CullSmem& s = *reinterpret_cast<CullSmem*>(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1097,6 +1124,7 @@ template <class TL, bool FULL>
 __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     FusedSmem& s = *reinterpret_cast<FusedSmem*>(smem_raw);
+    if (PIC_STOP(P) == 15) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned first = blockIdx.x * (unsigned)NW, n_jobs = P.n_jobs;
     TL n = {};
@@ -1111,7 +1139,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     Job job;
     MapInfo mi;
     const uint2* blk = P.surv + (size_t)(first + warp) * SURV_STRIDE;
-    int ns = -2;
+    int ns = -2, n_big = 0;
     if (valid) {
         const uint4 head = __ldcg(reinterpret_cast<const uint4*>(blk));
         job = decode_job(P, first + warp);
@@ -1121,8 +1149,8 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             s.tile_job[warp] = job; s.tile_active[warp] = ego_active;
             load_camera(s.cam[warp], P.cams[job.view], P.cam[job.k], P.W, P.H);
         }
-        ns = (int)head.x;
-        if (ns > W_SURV) ns = -1;
+        n_big = (int)(head.x & 0xffffu);
+        ns = head.x == SURV_OVERFLOW ? -1 : n_big + (int)(head.x >> 16);
         if (lane == 0) { n.grp = (int)head.y; n.leaf = (int)head.z; n.tested = (int)head.w; }
     }
     if (lane == 0) s.n_surv[warp] = ns;
@@ -1143,7 +1171,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     {
         const int my_base = (int)((bases >> (8 * warp)) & 0xffu), my_cnt = (int)((cnts >> (8 * warp)) & 0xffu);
         if (my_cnt == 0xff) { n.grp = 0; n.leaf = 0; n.tested = 0; }       // counted again by cooperative_job
-        else if (my_cnt != 0xfe && my_cnt > 0 && stop != 14) front_setup(s.cam[warp], blk + 2, s.pool + my_base * (REC / 4), P, job, mi, my_cnt, lane, n);
+        else if (my_cnt != 0xfe && my_cnt > 0 && stop != 14) front_setup(s.cam[warp], blk + 2, s.pool + my_base * (REC / 4), P, job, mi, my_cnt, n_big, lane, n);
     }
     __syncthreads();
     // ---- back end: the NW tiles' strips are tasks that the warps draw from a counter; a warp's
@@ -1197,6 +1225,328 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
     flush_counters(P, n);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Render kernel for images made of full 64 x 64 tiles whose rows allow vector stores (every
+// benchmark workload).  Like render_kernel, with less bookkeeping: ray tables of the four tiles are
+// loaded once, per-tile constants are a 16-byte record, the background rows a lane stores are
+// fetched before the strip is rasterized.  The record pool is handed out in rounds: tiles that do
+// not fit beside their fellows are set up and rasterized in a further round of the same CTA (their
+// survivors are already in device memory), so only a tile whose own survivors exceed the pool, or
+// whose cull lists overflowed, is left to the cooperative kernel.
+// ---------------------------------------------------------------------------------------------
+#ifndef PIC_FSTRIP
+#define PIC_FSTRIP 16
+#endif
+#ifndef PIC_FPOOL
+#define PIC_FPOOL 118
+#endif
+constexpr int FPOOL = PIC_FPOOL;     // records shared by the four tiles of a CTA
+constexpr int FSTRIP = PIC_FSTRIP;   // pixel rows of a strip: 16 or 8
+constexpr int FSTRIP_KEYS = TILE * FSTRIP;
+constexpr int FSTRIPS = TILE / FSTRIP;
+static_assert(FSTRIP == 16 || FSTRIP == 8, "strips of 16 or 8 rows");
+
+struct __align__(16) TileRef {
+    size_t pixel0;       // offset of the tile's first pixel in the output images
+    int bg_row0;         // first row of the tile in the per-camera background tables
+    int active;          // is the ego agent active
+};
+
+struct __align__(16) FullSmem {
+    unsigned long long key[NW][FSTRIP_KEYS];  // warp w's strip of keys
+    float4 pool[FPOOL * REC / 4];
+    float ray_x[NW][TILE], ray_y[NW][TILE];   // ray tables of tile w
+    Cam cam[NW];
+    TileRef tile[NW];
+    int n_surv[NW];
+    int next_task;
+};
+static_assert(sizeof(FullSmem) <= 44 * 1024, "shared memory must leave room for 5 CTAs per SM");
+
+// The 16 x 4 cell of strip_cell's comment, for the full-tile kernel: `kbase` and `lsw` are the
+// lane's share of the key address (row lane >> 3, chunk lane & 7, swizzle), `range` says whether
+// the depth range still has to be tested (warp-uniform), keys are written with one predicated
+// 64-bit store per pixel; the caller marks the touched blocks.
+__device__ __forceinline__ void strip_cell(unsigned long long* key, const float* ray_x, const float* ray_y, const PrimEq& q,
+                                           const float (&thr)[4], uint32_t key_lo, float w_near, float w_far, int xx, int yy,
+                                           uint32_t need, bool range, int kbase, int lsw, int lane) {
+    const float2 rx = *reinterpret_cast<const float2*>(ray_x + xx + (lane & 7) * 2);
+    const float ry = ray_y[yy + (lane >> 3)];
+    const float wt = fm(q.wy, ry, q.wz);
+    const float w0 = fm(q.wx, rx.x, wt), w1 = fm(q.wx, rx.y, wt);
+    bool in0 = true, in1 = true;
+    if (need) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if ((need >> e) & 1u) {          // warp-uniform: edges known to be positive on the whole cell are skipped
+                const float te = fm(q.ny[e], ry, q.nz[e]);
+                const float e0 = fm(q.nx[e], rx.x, te), e1 = fm(q.nx[e], rx.y, te);
+                in0 = in0 && (e0 > thr[e]);
+                in1 = in1 && (e1 > thr[e]);
+            }
+        }
+        if (range) {
+            in0 = in0 && (w0 >= w_far) && (w0 <= w_near);
+            in1 = in1 && (w1 >= w_far) && (w1 <= w_near);
+        }
+    }
+    const int cb = xx >> 4;
+    unsigned long long* kp = key + (kbase + (yy << 6) + (cb << 4) + ((lsw ^ cb) << 1));
+    const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(kp);
+    const unsigned long long k0 = make_key(__float_as_uint(w0), key_lo), k1 = make_key(__float_as_uint(w1), key_lo);
+    if (in0 && k0 > kk.x) kp[0] = k0;
+    if (in1 && k1 > kk.y) kp[1] = k1;
+}
+
+// Strip -> class / depth images, 16 pixels per lane and pass (see store_tile); resets the keys it reads.
+__device__ __forceinline__ void store_strip_full(unsigned long long* key, uint8_t* oc, uint16_t* od, int W, uint32_t touched,
+                                                 const uint32_t (&bgc)[2], const float (&bgz)[2], int lane) {
+#pragma unroll
+    for (int it = 0; it < FSTRIP / 8; ++it) {
+        const int y = it * 8 + (lane >> 2), xs = (lane & 3) * 16;
+        const size_t o = (size_t)y * W + xs;
+        uint32_t cw[4], dw[8];
+        if (((touched >> (it * 8 + (xs >> 3))) & 3u) == 0u) {       // both 8 x 8 blocks of the segment are background
+            const uint32_t c4 = bgc[it] * 0x01010101u;
+            const __half2 h = __floats2half2_rn(bgz[it], bgz[it]);
+            const uint32_t d2 = *reinterpret_cast<const uint32_t*>(&h);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) cw[j] = c4;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) dw[j] = d2;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+                ulonglong2* kp = reinterpret_cast<ulonglong2*>(&key[key_index(xs + j, y)]);
+                const ulonglong2 kk = *kp;
+                *kp = make_ulonglong2(0ull, 0ull);
+                const float z0 = kk.x ? fast_rcp(__uint_as_float((uint32_t)(kk.x >> 32))) : bgz[it];
+                const float z1 = kk.y ? fast_rcp(__uint_as_float((uint32_t)(kk.y >> 32))) : bgz[it];
+                const uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bgc[it], c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bgc[it];
+                const __half2 h = __floats2half2_rn(z0, z1);
+                dw[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                if ((j & 3) == 0) cw[j >> 2] = c0 | (c1 << 8); else cw[j >> 2] |= (c0 << 16) | (c1 << 24);
+            }
+        }
+#ifdef PIC_PROFILE
+        if (touched & 0x80000000u) continue;       // profiling: no global stores
+#endif
+        *reinterpret_cast<uint4*>(oc + o) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+        store_256(od + o, dw);
+    }
+}
+
+// One strip (rows ys .. of the tile) by one warp: the tile's fragments that fall into it, then
+// the records that reach it, cell by cell.  Returns the touched 8 x 8 blocks.
+__device__ __forceinline__ uint32_t raster_strip_full(StripView& s, const float4* rec, int n_rec, int ys, float w_near, float w_far,
+                                                      int stop, int lane) {
+    uint32_t touched = 0u;                       // bit (row >> 3) * 8 + (column >> 3)
+    const int kbase = (lane >> 3) << 6, lsw = (lane & 7) ^ (((lane >> 3) & 1) << 2);   // see strip_cell
+    for (int base = 0; base < n_rec; base += 32) {
+        uint32_t bw_lane = 0u;
+        bool hit = false;
+        if (base + lane < n_rec) {
+            const float4* r = rec + (base + lane) * (REC / 4);
+            bw_lane = __float_as_uint(r[4].x);
+            const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
+            hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + FSTRIP;
+            if (hit && (bw_lane & REC_TINY)) {           // a few pixels: rasterized by this lane (atomic max)
+                hit = false;
+                const int bx0 = bw_lane & 63, bx1 = (bw_lane >> 12) & 63;
+                const int y0 = max(by0, ys) - ys, y1 = min(by1, ys + FSTRIP - 1) - ys;
+                PrimEq q;
+                uint32_t key_lo;
+                read_record(r, q, key_lo);
+                q.tl = (bw_lane >> 24) & 15u;
+                // at most TINY_MAX_PIXELS pixels: one column (w == 1), two columns, or one row
+                const int w = bx1 - bx0 + 1, npx = (stop == 7) ? 0 : w * (y1 - y0 + 1);
+                bool any = false;
+#pragma unroll
+                for (int px = 0; px < TINY_MAX_PIXELS; ++px) {
+                    if (px < npx) {
+                        const int x = bx0 + (w == 1 ? 0 : w == 2 ? (px & 1) : px), y = y0 + (w == 1 ? px : w == 2 ? (px >> 1) : 0);
+                        const uint32_t wb = fragment(q, s.ray_x[x], s.ray_y[y], w_near, w_far);
+                        if (wb) { put_fragment(s, x, y, wb, key_lo); any = true; }
+                    }
+                }
+                if (any) touched |= (uint32_t)block_mask(bx0, y0, bx1, y1);
+            }
+        }
+        __syncwarp();
+        unsigned hits = __ballot_sync(0xffffffffu, hit);
+        if (!(stop == 0 || stop == 2 || stop == 3 || stop > 5)) hits = 0u;
+        for (; hits; hits &= hits - 1) {
+            const int src = __ffs(hits) - 1;
+            const uint32_t bw = __shfl_sync(0xffffffffu, bw_lane, src);
+            const float4* r = &rec[(base + src) * (REC / 4)];
+            const int by0 = (bw >> 6) & 63, by1 = (bw >> 18) & 63;
+            const int bx0 = bw & 63, bx1 = (bw >> 12) & 63;
+            const int ly0 = max(by0, ys) - ys, ly1 = min(by1, ys + FSTRIP - 1) - ys;
+            PrimEq q;
+            uint32_t key_lo;
+            read_record(r, q, key_lo);
+            q.tl = (bw >> 24) & 15u;
+            float thr[4];
+            edge_thresholds(q.tl, thr);
+            const bool range = !(bw & REC_INRANGE);
+            if (stop != 3 && (bx1 - bx0 + 1) * (ly1 - ly0 + 1) >= CLASSIFY_MIN_STRIP * FSTRIP / 16) {
+                // a lane per 16 x 4 pixel cell of the strip classifies it: reject / partly covered / inside
+                const int xa = (lane & 3) * 16, xb = xa + 15, ya = ((lane >> 2) & 3) * 4, yb = ya + 3;
+                bool reject = lane >= FSTRIP || xb < bx0 || xa > bx1 || yb < ly0 || ya > ly1;
+                uint32_t need = 0u;
+                if (!reject) {
+                    const float rxa = s.ray_x[xa], rxb = s.ray_x[xb], rya = s.ray_y[ya], ryb = s.ray_y[yb];   // rxa < rxb, rya < ryb
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        // fma is monotone in each argument, so the cell's extreme values are at its corners
+                        const float ta = fm(q.ny[e], rya, q.nz[e]), tb = fm(q.ny[e], ryb, q.nz[e]);
+                        const float emax = fm(q.nx[e], q.nx[e] >= 0.f ? rxb : rxa, fmaxf(ta, tb));
+                        const float emin = fm(q.nx[e], q.nx[e] >= 0.f ? rxa : rxb, fminf(ta, tb));
+                        reject = reject || (emax < 0.f);
+                        if (!(emin > 0.f)) need |= 1u << e;
+                    }
+                    const float wa = fm(q.wy, rya, q.wz), wb = fm(q.wy, ryb, q.wz);
+                    const float wmax = fm(q.wx, q.wx >= 0.f ? rxb : rxa, fmaxf(wa, wb));
+                    const float wmin = fm(q.wx, q.wx >= 0.f ? rxa : rxb, fminf(wa, wb));
+                    reject = reject || (wmax < w_far) || (wmin > w_near);
+                    // the depth range test rides on the edge tests: if it is still needed, so is one edge
+                    if (need == 0u && !((wmin >= w_far) && (wmax <= w_near))) need = 1u;
+                }
+                for (unsigned m = __ballot_sync(0xffffffffu, !reject); m; m &= m - 1) {
+                    const int cell = __ffs(m) - 1;
+                    const int xx = (cell & 3) * 16, yy = (cell >> 2) * 4;
+                    const uint32_t need_c = __shfl_sync(0xffffffffu, need, cell);
+                    if (stop != 2 && stop != 3) strip_cell(s.key, s.ray_x, s.ray_y, q, thr, key_lo, w_near, w_far, xx, yy, need_c, true, kbase, lsw, lane);
+                    touched |= 3u << ((yy >> 3) * 8 + (xx >> 3));
+                }
+            } else {
+                for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
+                    for (int xx = bx0 & ~15; xx <= bx1; xx += 16)
+                        if (stop != 2 && stop != 3) strip_cell(s.key, s.ray_x, s.ray_y, q, thr, key_lo, w_near, w_far, xx, yy, 0xFu, range, kbase, lsw, lane);
+                touched |= (uint32_t)block_mask(bx0, ly0, bx1, ly1);
+            }
+        }
+        __syncwarp();
+    }
+    return __reduce_or_sync(0xffffffffu, touched);
+}
+
+__global__ void __launch_bounds__(NTHREADS, PIC_RENDER_CTAS) render_full_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    FullSmem& s = *reinterpret_cast<FullSmem*>(smem_raw);
+    const int stop = PIC_STOP(P);
+    if (stop == 15) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned id = blockIdx.x * (unsigned)NW + warp;
+    const bool valid = id < P.n_jobs;
+    // ---- the cull kernel's survivors of tile first + w, and everything that does not depend on them
+    const uint2* blk = P.surv + (size_t)id * SURV_STRIDE;
+    int ns = -2, n_big = 0;
+    uint2 sv0 = make_uint2(0u, 0u);
+    Job job;
+    uint32_t n_map_tris = 0u;
+    if (valid) {
+        const uint4 head = __ldcg(reinterpret_cast<const uint4*>(blk));
+        job = decode_job(P, id);
+        n_map_tris = __ldg(&P.env_maps[job.e].n_tris);
+        const bool ego_active = __ldg(&P.agents[(size_t)job.e * P.A + job.a].active) != 0u;
+        const float* rx = P.rig.ray_x + (size_t)job.k * P.W + job.t.x0;
+        const float* ry = P.rig.ray_y + (size_t)job.k * P.H + job.t.y0;
+        s.ray_x[warp][lane] = __ldg(rx + lane); s.ray_x[warp][lane + 32] = __ldg(rx + lane + 32);
+        s.ray_y[warp][lane] = __ldg(ry + lane); s.ray_y[warp][lane + 32] = __ldg(ry + lane + 32);
+        if (lane == 0) {
+            load_camera(s.cam[warp], P.cams[job.view], P.cam[job.k], P.W, P.H);
+            TileRef tr;
+            tr.pixel0 = job.view * ((size_t)P.H * P.W) + (size_t)job.t.y0 * P.W + job.t.x0;
+            tr.bg_row0 = job.k * P.H + job.t.y0;
+            tr.active = ego_active ? 1 : 0;
+            s.tile[warp] = tr;
+        }
+        n_big = (int)(head.x & 0xffffu);
+        ns = head.x == SURV_OVERFLOW ? -1 : n_big + (int)(head.x >> 16);
+        if (ns > FPOOL) ns = -1;                            // more survivors than the whole pool
+        // the first survivor of this lane (front list, then back list); the others are fetched in the set-up loop
+        if (lane < ns) sv0 = __ldcg(blk + 2 + (lane < n_big ? lane : W_SURV - 1 - (lane - n_big)));
+    }
+    if (lane == 0) s.n_surv[warp] = ns;
+#pragma unroll
+    for (int i = 0; i < FSTRIP_KEYS / 2 / 32; ++i)
+        reinterpret_cast<ulonglong2*>(s.key[warp])[i * 32 + lane] = make_ulonglong2(0ull, 0ull);
+    __syncthreads();
+    StripView sv;
+    sv.key = s.key[warp];
+    // Rounds: every thread lays the record pool out alike -- the tiles not yet rendered, in order,
+    // as long as they fit.  One byte per tile: first record, and count (0xff: not in this round).
+    uint32_t done = 0u;                                      // bit j: tile j is rendered, absent, or left to the cooperative kernel
+#pragma unroll
+    for (int j = 0; j < NW; ++j)
+        if (s.n_surv[j] < 0) done |= 1u << j;
+#pragma unroll 1
+    while (done != (1u << NW) - 1u) {
+        uint32_t bases = 0u, cnts = 0u, now = 0u;
+        {
+            int off = 0;
+#pragma unroll
+            for (int j = 0; j < NW; ++j) {
+                const int c = s.n_surv[j];
+                bases |= (uint32_t)off << (8 * j);
+                if (!((done >> j) & 1u) && off + c <= FPOOL) { cnts |= (uint32_t)c << (8 * j); off += c; now |= 1u << j; }
+                else cnts |= 0xffu << (8 * j);
+            }
+        }
+        // ---- set-up by the tile's warp: survivor i becomes record i
+        if ((now >> warp) & 1u) {
+            const int my_base = (int)((bases >> (8 * warp)) & 0xffu);
+            const int my_cnt = (stop == 14) ? 0 : ns;
+            for (int i = lane; i < my_cnt; i += 32) {
+                const uint2 svi = (i < 32) ? sv0 : __ldcg(blk + 2 + (i < n_big ? i : W_SURV - 1 - (i - n_big)));
+                V3 V[4], Pn;
+                uint32_t key_lo, flags;
+                fetch_survivor(s.cam[warp], P, svi.x, job.e, n_map_tris, V, Pn, key_lo, flags);
+                PrimEq q;
+                float4* r = s.pool + (my_base + i) * (REC / 4);
+                if (!prim_equations(V, flags & 1u, flags, Pn, q)) { r[4].x = __uint_as_float(REC_DEAD); continue; }
+                write_record(r, q, key_lo, svi.y, (tiny_box(svi.y) ? REC_TINY : 0u) | (record_in_range(V, P) ? REC_INRANGE : 0u));
+            }
+        }
+        if (threadIdx.x == 0) s.next_task = 0;
+        __syncthreads();
+        if (stop == 10) return;
+        // ---- the strips of this round's tiles are tasks that the warps draw from a counter
+#pragma unroll 1
+        for (;;) {
+            int task = 0;
+            if (lane == 0) task = atomicAdd(&s.next_task, 1);
+            task = __shfl_sync(0xffffffffu, task, 0);
+            if (task >= NW * FSTRIPS) break;
+            const int j = task / FSTRIPS, ys = (task % FSTRIPS) * FSTRIP;
+            const int cj = (int)((cnts >> (8 * j)) & 0xffu);
+            if (cj == 0xff) continue;
+            const TileRef tr = s.tile[j];
+            uint32_t bgc[2] = {P.cls_sky, P.cls_sky};
+            float bgz[2] = {P.far_z, P.far_z};
+            if (tr.active) {                                 // background of the rows this lane stores
+                const uint32_t* bg_cls = P.rig.bg_cls + tr.bg_row0 + ys + (lane >> 2);
+                const float* bg_z = P.rig.bg_z + tr.bg_row0 + ys + (lane >> 2);
+                bgc[0] = __ldg(bg_cls); bgz[0] = __ldg(bg_z);
+                if (FSTRIP == 16) { bgc[1] = __ldg(bg_cls + 8); bgz[1] = __ldg(bg_z + 8); }
+            }
+            sv.ray_x = s.ray_x[j]; sv.ray_y = s.ray_y[j] + ys;
+            uint32_t touched = raster_strip_full(sv, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), (stop == 14) ? 0 : cj, ys, P.w_near, P.w_far, stop, lane);
+            if (stop == 5) touched = 0xffffu;
+            if (stop == 6) touched |= 0x80000000u;
+            const size_t o = tr.pixel0 + (size_t)ys * P.W;
+            if (stop != 8) store_strip_full(sv.key, P.out_class + o, P.out_depth + o, P.W, touched, bgc, bgz, lane);
+            __syncwarp();
+        }
+        done |= now;
+        if (done != (1u << NW) - 1u) __syncthreads();        // the pool is reused by the next round
+    }
+    // ---- the rest: tiles with too many survivors, or whose cull lists overflowed, are left to the cooperative kernel
+    if (threadIdx.x < NW && s.n_surv[threadIdx.x] == -1)
+        P.overflow[1u + atomicAdd(&P.overflow[0], 1u)] = blockIdx.x * (unsigned)NW + threadIdx.x;
+}
+
 // The tiles the fused kernel left out, a CTA at a time.
 template <class TL, bool FULL>
 __global__ void __launch_bounds__(NTHREADS, 5) cooperative_kernel(const __grid_constant__ RenderParams P) {
@@ -1221,10 +1571,11 @@ static size_t smem_pad() { const char* e = getenv("PIC_SMEM_PAD"); return e ? (s
 #else
 #define RENDER_SMEM RENDER_SMEM_BASE
 #endif
+#define FULL_SMEM (sizeof(FullSmem) + (RENDER_SMEM - RENDER_SMEM_BASE))
 size_t render_smem_bytes() { return RENDER_SMEM; }
 
 cudaError_t configure_render_kernel() {
-    cudaError_t err = cudaFuncSetAttribute(render_kernel<NoTally, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
+    cudaError_t err = cudaFuncSetAttribute(render_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FULL_SMEM);
     if (err != cudaSuccess) return err;
     err = cudaFuncSetAttribute(render_kernel<NoTally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RENDER_SMEM);
     if (err != cudaSuccess) return err;
@@ -1255,7 +1606,7 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int 
     if (err != cudaSuccess) return err;
     // (b)-(d) set-up, raster, store
     if (P.counters) render_kernel<Tally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
-    else if (full) render_kernel<NoTally, true><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
+    else if (full) render_full_kernel<<<grid, NTHREADS, FULL_SMEM, stream>>>(P);
     else render_kernel<NoTally, false><<<grid, NTHREADS, RENDER_SMEM, stream>>>(P);
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
