@@ -30,6 +30,14 @@
  * caller's buffer.  Unless stated otherwise calls are asynchronous on the given CUDA stream
  * (a cudaStream_t passed as void*; NULL is the default stream) and allocate nothing.
  *
+ * One stream at a time per scene: every pic_render / pic_step / pic_set_state of a scene writes
+ * the scene's own per-call buffers (agent geometry, per-view cameras, per-camera tables, the
+ * survivor lists handed from the cull kernel to the render kernel, the list of left-out tiles,
+ * timing events), and options are plain fields read when a call is issued.  Calls on one scene
+ * must therefore be issued from one host thread at a time and be ordered on the device -- the
+ * same stream, or streams ordered with events; two calls of one scene that overlap on the GPU
+ * race silently.  Different scenes are independent.
+ *
  * Errors: every call returns a pic_status; nothing throws, aborts or traps.  pic_last_error()
  * returns a thread-local description of the last failure.  Device-detected conditions are
  * accumulated in sticky flags read by pic_get_status().
@@ -56,7 +64,9 @@ typedef enum {
 } pic_status;
 
 /* Sticky device flags returned by pic_get_status. */
-#define PIC_FLAG_NONFINITE_POSE 0x1u /* a pose, size or action was NaN/Inf; that agent's output is unspecified */
+#define PIC_FLAG_NONFINITE_POSE 0x1u /* a pose, size or action was NaN/Inf (or a step overflowed): that agent is treated as
+                                        inactive for the call -- its images are sky, nobody sees it -- and pic_step leaves
+                                        its state as it was */
 
 /* One pinhole camera of the rig, in the agent frame (x forward, y left, z up). */
 typedef struct {
@@ -75,6 +85,8 @@ typedef struct {
     const int64_t* map_tri_offset; /* host [M+1], non-decreasing, [0] == 0                       */
     const float* tri_xyz;          /* host [N,3,3] f32 world coordinates, N = map_tri_offset[M] */
     const uint8_t* tri_class;      /* host [N] class id of each triangle                         */
+                                   /* (both arrays must be HOST memory in this build: the hierarchy is built on
+                                      the host; device pointers are not accepted)                              */
     uint8_t agent_class;           /* class written for agent boxes                              */
     uint8_t sky_class;             /* background above the horizon                               */
     uint8_t ground_class;          /* background below the horizon                               */
@@ -156,9 +168,7 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *                         cooperative kernel's record list to 2 entries so that the overflow paths
  *                         run; bit 2: send every tile to the cooperative kernel; bit 3: shrink the
  *                         record pool to 40 so that both kernels share the tiles.  All leave the
- *                         images unchanged (tests rely on it).  Bits 4-7: profiling aid, leaves work
- *                         out (1: no culling, 4: no record raster, 5: as 4 with every pixel
- *                         converted); the images are then incomplete.
+ *                         images unchanged (tests rely on it); other bits are ignored.
  *   PIC_OPT_TIMING        1: bracket the render kernels of every call with CUDA events on its stream
  *                         (up to 1024 launches between two pic_get_kernel_times calls); 0: off.
  *                         Turning it on creates the events (allocates), so do it outside timed code.
@@ -208,7 +218,9 @@ pic_status pic_map_stats(const pic_scene_desc* desc, int64_t out[8]);
  * The call itself uses no cudaMalloc/cudaFree and no allocating library routine.
  *
  * Limits (PIC_ERR_CAPACITY beyond them): E*A <= PIC_STATIC_MAX_AGENTS, E*A*K <= PIC_STATIC_MAX_VIEWS,
- * H, W <= PIC_STATIC_MAX_SIDE, n_tris <= PIC_STATIC_MAX_TRIS, K <= 16.
+ * H, W <= PIC_STATIC_MAX_SIDE, n_tris <= PIC_STATIC_MAX_TRIS, K <= 16, and, because every primitive
+ * is tested against every pixel of every view by one launch that cannot be interrupted,
+ * (n_tris + 6*A) * E*A*K*H*W <= PIC_STATIC_MAX_WORK (a few tenths of a second on a B200).
  *
  *   tri_xyz    dev f32 [n_tris,3,3], tri_class dev u8 [n_tris]   (may be NULL when n_tris == 0)
  *   poses, dims, active, rig, out_class, out_depth: as in pic_render (outputs need no alignment)
@@ -217,12 +229,16 @@ pic_status pic_map_stats(const pic_scene_desc* desc, int64_t out[8]);
  * stream capture.  All calls on a device share the one array and it keeps the previous call's
  * contents: the call clears what must start at zero itself, but two calls whose kernels overlap
  * on the GPU (different streams, or several host threads) race on it -- serialise them.
- * A non-finite pose or size makes that agent inactive (its images are sky), as in pic_render.
+ * A non-finite pose or size makes that agent inactive (its images are sky), as in pic_render, and
+ * sets PIC_FLAG_NONFINITE_POSE in a sticky word inside the same array; pic_static_status
+ * synchronises `cuda_stream`, copies that word to *flags (host) and clears it -- it allocates
+ * nothing either, and reports 0 on a device where pic_render_static has not run yet.
  */
 #define PIC_STATIC_MAX_AGENTS 1024
 #define PIC_STATIC_MAX_VIEWS 4096
 #define PIC_STATIC_MAX_SIDE 512
 #define PIC_STATIC_MAX_TRIS 65536
+#define PIC_STATIC_MAX_WORK 274877906944.0 /* 2^38 primitive-pixel tests */
 typedef struct {
     uint32_t size;                 /* = sizeof(pic_static_desc)                                  */
     int32_t E, A, K, H, W;
@@ -233,6 +249,7 @@ typedef struct {
 pic_status pic_render_static(const pic_static_desc* desc, const float* tri_xyz, const uint8_t* tri_class,
                              const float* poses, const float* dims, const uint8_t* active, const pic_camera* rig,
                              uint8_t* out_class, uint16_t* out_depth, void* cuda_stream);
+pic_status pic_static_status(uint32_t* flags, void* cuda_stream);
 
 /* Thread-local, never NULL; valid until the next failing call on this thread. */
 const char* pic_last_error(void);

@@ -21,7 +21,7 @@ OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static",
+           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status",
            "pic_last_error", "pic_version"]
 
 
@@ -77,6 +77,7 @@ def load(path: Optional[str] = None):
     lib.pic_get_kernel_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int32, C.POINTER(C.c_int32)]
     lib.pic_map_stats.argtypes = [C.POINTER(pic_scene_desc), C.POINTER(C.c_int64)]
     lib.pic_render_static.argtypes = [C.POINTER(pic_static_desc), vp, vp, vp, vp, vp, C.POINTER(pic_camera), vp, vp, vp]
+    lib.pic_static_status.argtypes = [C.POINTER(C.c_uint32), vp]
     for name in EXPORTS:
         getattr(lib, name).restype = C.c_int
     lib.pic_last_error.restype = C.c_char_p
@@ -164,6 +165,14 @@ def render_static(E: int, A: int, K: int, H: int, W: int, near: float, far: floa
         _rig_array(rig), _dev_ptr(out_class, torch.uint8, npx), _dev_ptr(out_depth, torch.float16, npx),
         _stream_ptr(stream)))
     return out_class, out_depth
+
+
+def static_status(stream=None) -> int:
+    """pic_static_status: read and clear the sticky flags of pic_render_static on the current device."""
+    lib = load()
+    flags = C.c_uint32(0)
+    _check(lib, lib.pic_static_status(C.byref(flags), _stream_ptr(stream)))
+    return int(flags.value)
 
 
 class Scene:

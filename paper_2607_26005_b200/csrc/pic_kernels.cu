@@ -1,16 +1,10 @@
 // Agent kernel, rig-table kernel, exhaustive cross-check kernel and host-side launchers.
 //
-// The exhaustive kernel tests every primitive of the map and every face of every other agent's
-// box against every pixel of a 64 x 64 tile (one CTA per tile, a thread per primitive, a
-// shared-memory atomic max per fragment): no hierarchy, no frustum or pixel-box culling, no
-// size classes.  It shares only the per-primitive arithmetic of pic_device.cuh (and the per-call
-// camera and ray tables) with the production kernel in pic_render.cu, so comparing the two
-// images bit for bit checks everything the production kernel adds.
-#include "pic_device.cuh"
+// The exhaustive kernel (see pic_exhaustive.cuh) is the cross-check of the production kernels in
+// pic_render.cu.
+#include "pic_exhaustive.cuh"
 
 namespace pic {
-
-constexpr int BRUTE_THREADS = 128;
 
 struct RigParams {
     int32_t K, W, H;
@@ -42,8 +36,15 @@ __global__ void agent_kernel(int n, const float* __restrict__ poses, float* stat
             const float ny = fm(mul(v, s), dt, y);
             const float nth = fm(mul(__fdiv_rn(v, wheelbase), tanf(steer)), dt, th);
             const float nv = fminf(fmaxf(fm(acc, dt, v), 0.f), v_max);
-            x = nx; y = ny; th = nth; v = nv;
-            state[4 * i] = x; state[4 * i + 1] = y; state[4 * i + 2] = th; state[4 * i + 3] = v;
+            if (isfinite(acc) && isfinite(steer) && isfinite(nx) && isfinite(ny) && isfinite(nth) && isfinite(nv)) {
+                x = nx; y = ny; th = nth; v = nv;
+                state[4 * i] = x; state[4 * i + 1] = y; state[4 * i + 2] = th; state[4 * i + 3] = v;
+            } else {
+                // a non-finite action (or a step that overflows) is flagged, leaves the agent's
+                // state as it was and takes the agent out of this step's images
+                atomicOr(status, 1u);
+                act = false;
+            }
         }
     } else {
         x = poses[3 * i]; y = poses[3 * i + 1]; th = poses[3 * i + 2];
@@ -89,96 +90,24 @@ __global__ void rig_kernel(const __grid_constant__ RigParams R, float* __restric
 }
 
 // ------------------------------------------------------------------------------------------------
-// exhaustive kernel
+// exhaustive kernel: the scene's preprocessed primitives through the shared exhaustive tile renderer
 // ------------------------------------------------------------------------------------------------
-struct __align__(16) BruteSmem {
-    unsigned long long key[TILE * TILE];      // key = bits(1/z) << 32 | (0xFFFFFF - index) << 8 | class; 0 = background
-    float ray_x[TILE], ray_y[TILE];
-    Cam cam;
-};
-
-__global__ void __launch_bounds__(BRUTE_THREADS) render_brute_kernel(const __grid_constant__ RenderParams P) {
+__global__ void __launch_bounds__(EXH_THREADS) render_brute_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    BruteSmem& s = *reinterpret_cast<BruteSmem*>(smem_raw);
-    const int tiles = P.tiles_x * P.tiles_y;
-    const long long job = blockIdx.x;
-    const size_t view = (size_t)(P.view_first + job / tiles);
-    const int tile = (int)(job % tiles);
-    const int k = (int)(view % P.K);
-    const int a = (int)((view / P.K) % P.A);
-    const int e = (int)(view / ((size_t)P.K * P.A));
-    TileCtx t;
-    t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
-    t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
-    t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
-    const AgentGeom ego = P.agents[(size_t)e * P.A + a];
-    if (threadIdx.x == 0) load_camera(s.cam, P.cams[view], P.cam[k], P.W, P.H);
-    for (int i = threadIdx.x; i < TILE * TILE; i += BRUTE_THREADS) s.key[i] = 0ull;
-    if (threadIdx.x < TILE) {
-        const int i = threadIdx.x;
-        s.ray_x[i] = (t.x0 + i < P.W) ? P.rig.ray_x[(size_t)k * P.W + t.x0 + i] : 0.f;
-        s.ray_y[i] = (t.y0 + i < P.H) ? P.rig.ray_y[(size_t)k * P.H + t.y0 + i] : 0.f;
-    }
-    __syncthreads();
-    const Cam& c = s.cam;
-    if (ego.active) {
-        const MapInfo mi = P.maps[P.env_map[e]];
-        const uint32_t n_map = mi.prim_end - mi.prim_begin;
-        const uint32_t n_items = n_map + 6u * (uint32_t)P.A;
-        for (uint32_t i = threadIdx.x; i < n_items; i += BRUTE_THREADS) {
-            V3 V[4], Pn; bool quad; uint32_t flags, key_lo;
-            if (i < n_map) {
-                float v[12];
-                load_prim(P.prims + mi.prim_begin + i, v, key_lo, flags);
-                quad = flags & 1u;
+    ExhaustiveSmem& s = *reinterpret_cast<ExhaustiveSmem*>(smem_raw);
+    const unsigned tiles = (unsigned)(P.tiles_x * P.tiles_y);
+    const int e = (int)(((size_t)P.view_first + blockIdx.x / tiles) / ((size_t)P.K * P.A));
+    const MapInfo mi = P.maps[P.env_map[e]];
+    const Prim* prims = P.prims + mi.prim_begin;
+    exhaustive_tile(s, P, blockIdx.x, mi.prim_end - mi.prim_begin, mi.n_tris,
+                    [prims](uint32_t i, const Cam& c, V3 (&V)[4], V3& Pn, bool& quad, uint32_t& flags, uint32_t& key_lo) {
+                        float v[12];
+                        load_prim(prims + i, v, key_lo, flags);
+                        quad = flags & 1u;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
-                Pn = plane_normal_world(c, v, quad);
-            } else {
-                const uint32_t j = i - n_map;
-                const int b = (int)(j / 6u), f = (int)(j % 6u);
-                if (b == a) continue;
-                const AgentGeom g = P.agents[(size_t)e * P.A + b];
-                if (!g.active) continue;
-                const uint32_t corners = face_corners(f);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
-                quad = true; flags = face_flags(corners);
-                key_lo = ((0xFFFFFFu - (mi.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
-                Pn = plane_normal(V, true);
-            }
-            PrimEq q;
-            if (!prim_equations(V, quad, flags, Pn, q)) continue;
-            for (int y = 0; y < t.th; ++y) {
-                const float ry = s.ray_y[y];
-                for (int x = 0; x < t.tw; ++x) {
-                    const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
-                    if (wb) {
-                        const unsigned long long key = make_key(wb, key_lo);
-                        unsigned long long* addr = &s.key[y * TILE + x];
-                        if (key > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, key);
-                    }
-                }
-            }
-        }
-    }
-    __syncthreads();
-    // keys -> images (scalar stores; this kernel is a cross-check, not a fast path)
-    const size_t img = (size_t)P.H * P.W;
-    uint8_t* oc = P.out_class + view * img;
-    uint16_t* od = P.out_depth + view * img;
-    float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
-    for (int i = threadIdx.x; i < t.th * t.tw; i += BRUTE_THREADS) {
-        const int y = i / t.tw, x = i % t.tw;
-        uint32_t cls = P.cls_sky; float z = P.far_z;
-        if (ego.active) { cls = P.rig.bg_cls[(size_t)k * P.H + t.y0 + y]; z = P.rig.bg_z[(size_t)k * P.H + t.y0 + y]; }
-        const unsigned long long key = s.key[y * TILE + x];
-        if (key) { cls = (uint32_t)(key & 0xff); z = fast_rcp(__uint_as_float((uint32_t)(key >> 32))); }
-        const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + x;
-        oc[o] = (uint8_t)cls;
-        od[o] = __half_as_ushort(__float2half_rn(z));
-        if (o32) o32[o] = z;
-    }
+                        for (int j = 0; j < 4; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
+                        Pn = plane_normal_world(c, v, quad);
+                    });
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -188,12 +117,12 @@ size_t render_smem_bytes();                       // pic_render.cu
 cudaError_t configure_render_kernel();            // pic_render.cu
 cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, int sm_count, cudaStream_t stream);
 
-size_t max_smem_bytes() { return render_smem_bytes() > sizeof(BruteSmem) ? render_smem_bytes() : sizeof(BruteSmem); }
+size_t max_smem_bytes() { return render_smem_bytes() > sizeof(ExhaustiveSmem) ? render_smem_bytes() : sizeof(ExhaustiveSmem); }
 
 cudaError_t configure_kernels() {
     cudaError_t err = configure_render_kernel();
     if (err != cudaSuccess) return err;
-    return cudaFuncSetAttribute(render_brute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BruteSmem));
+    return cudaFuncSetAttribute(render_brute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ExhaustiveSmem));
 }
 
 static RigParams rig_params(const RenderParams& P) {
@@ -225,7 +154,7 @@ cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, 
     if (!brute) return launch_render_kernel(P, n_views, sm_count, stream);
     const long long blocks = n_views * P.tiles_x * P.tiles_y;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    render_brute_kernel<<<(unsigned)blocks, BRUTE_THREADS, sizeof(BruteSmem), stream>>>(P);
+    render_brute_kernel<<<(unsigned)blocks, EXH_THREADS, sizeof(ExhaustiveSmem), stream>>>(P);
     return cudaGetLastError();
 }
 

@@ -60,7 +60,10 @@ constexpr int SCAP = 128;         // candidates that survive the pixel-box test,
 constexpr int TINY_MAX_PIXELS = 4;         // pixel centres in the box of a primitive rasterized by its own thread
 static_assert(TINY_MAX_PIXELS == 4, "the strip back end enumerates the pixels of such a box for at most 4");
 constexpr int CLASSIFY_MIN_PIXELS = 192;   // pixel boxes at least this large classify cells before rasterizing
-constexpr int CLASSIFY_MIN_STRIP = 256;    // the same for the part of a box inside a 16-row strip
+#ifndef PIC_CLASSIFY_MIN
+#define PIC_CLASSIFY_MIN 256
+#endif
+constexpr int CLASSIFY_MIN_STRIP = PIC_CLASSIFY_MIN;    // the same for the part of a box inside a 16-row strip
 
 struct __align__(16) TileSmem {
     unsigned long long key[TILE * TILE];      // 32 KB, 16-byte chunks XOR-swizzled by row (key_index)

@@ -17,7 +17,7 @@
 #include <mutex>
 
 #include "../../include/pictura.h"
-#include "pic_device.cuh"
+#include "pic_exhaustive.cuh"
 
 namespace pic {
 cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses, float* state, const float* actions,
@@ -34,7 +34,6 @@ constexpr int kMaxAgents = PIC_STATIC_MAX_AGENTS;
 constexpr int kMaxViews = PIC_STATIC_MAX_VIEWS;
 constexpr int kMaxSide = PIC_STATIC_MAX_SIDE;
 constexpr int kMaxDevices = 64;
-constexpr int kThreads = 128;
 
 // scratch layout (bytes)
 constexpr size_t kOffAgents = 0;
@@ -57,110 +56,37 @@ struct StaticParams {
     uint32_t n_tris;
 };
 
-struct __align__(16) StaticSmem {
-    unsigned long long key[TILE * TILE];
-    float ray_x[TILE], ray_y[TILE];
-    Cam cam;
-};
-
 __device__ __forceinline__ bool lex_less(float ax, float ay, float az, float bx, float by, float bz) {
     if (ax != bx) return ax < bx;
     if (ay != by) return ay < by;
     return az < bz;
 }
 
-// Variant of the exhaustive kernel that reads the caller's raw triangles: every triangle and every
-// face of every other agent's box against every pixel of a 64 x 64 tile.
-__global__ void __launch_bounds__(kThreads) render_static_kernel(const __grid_constant__ StaticParams S) {
+// The exhaustive tile renderer over the caller's raw triangles.
+__global__ void __launch_bounds__(EXH_THREADS) render_static_kernel(const __grid_constant__ StaticParams S) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    StaticSmem& s = *reinterpret_cast<StaticSmem*>(smem_raw);
-    const RenderParams& P = S.P;
-    const unsigned tiles = (unsigned)(P.tiles_x * P.tiles_y);
-    const unsigned job = blockIdx.x;
-    const unsigned view = job / tiles;
-    const int tile = (int)(job % tiles);
-    const int k = (int)(view % (unsigned)P.K);
-    const int a = (int)((view / (unsigned)P.K) % (unsigned)P.A);
-    const int e = (int)(view / ((unsigned)P.K * (unsigned)P.A));
-    TileCtx t;
-    t.x0 = (tile % P.tiles_x) * TILE; t.y0 = (tile / P.tiles_x) * TILE;
-    t.tw = min(TILE, P.W - t.x0); t.th = min(TILE, P.H - t.y0);
-    t.w_near = P.w_near; t.w_far = P.w_far; t.near_z = P.near_z; t.far_z = P.far_z;
-    const AgentGeom ego = P.agents[(size_t)e * P.A + a];
-    if (threadIdx.x == 0) load_camera(s.cam, P.cams[view], P.cam[k], P.W, P.H);
-    for (int i = threadIdx.x; i < TILE * TILE; i += kThreads) s.key[i] = 0ull;
-    if (threadIdx.x < TILE) {
-        const int i = threadIdx.x;
-        s.ray_x[i] = (t.x0 + i < P.W) ? P.rig.ray_x[(size_t)k * P.W + t.x0 + i] : 0.f;
-        s.ray_y[i] = (t.y0 + i < P.H) ? P.rig.ray_y[(size_t)k * P.H + t.y0 + i] : 0.f;
-    }
-    __syncthreads();
-    const Cam& c = s.cam;
-    if (ego.active) {
-        const uint32_t n_items = S.n_tris + 6u * (uint32_t)P.A;
-        for (uint32_t i = threadIdx.x; i < n_items; i += kThreads) {
-            V3 V[4], Pn; bool quad; uint32_t flags, key_lo;
-            if (i < S.n_tris) {
-                const float* p = S.tri_xyz + 9 * (size_t)i;
-                float v[9];
+    ExhaustiveSmem& s = *reinterpret_cast<ExhaustiveSmem*>(smem_raw);
+    const float* tri_xyz = S.tri_xyz;
+    const uint8_t* tri_class = S.tri_class;
+    exhaustive_tile(s, S.P, blockIdx.x, S.n_tris, S.n_tris,
+                    [tri_xyz, tri_class](uint32_t i, const Cam& c, V3 (&V)[4], V3& Pn, bool& quad, uint32_t& flags, uint32_t& key_lo) {
+                        const float* p = tri_xyz + 9 * (size_t)i;
+                        float v[9];
 #pragma unroll
-                for (int j = 0; j < 9; ++j) v[j] = __ldg(p + j);
+                        for (int j = 0; j < 9; ++j) v[j] = __ldg(p + j);
 #pragma unroll
-                for (int j = 0; j < 3; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
-                V[3] = V[2];
-                {
-                    const float v12[12] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], v[8], v[6], v[7], v[8]};
-                    Pn = plane_normal_world(c, v12, false);
-                }
-                quad = false;
-                flags = 0u;
-                // an edge shared by two triangles is evaluated in the same direction by both
-                if (!lex_less(v[0], v[1], v[2], v[3], v[4], v[5])) flags |= 1u << 4;
-                if (!lex_less(v[3], v[4], v[5], v[6], v[7], v[8])) flags |= 1u << 5;
-                if (!lex_less(v[6], v[7], v[8], v[0], v[1], v[2])) flags |= 1u << 6;
-                key_lo = ((0xFFFFFFu - i) << 8) | __ldg(S.tri_class + i);
-            } else {
-                const uint32_t j = i - S.n_tris;
-                const int b = (int)(j / 6u), f = (int)(j % 6u);
-                if (b == a) continue;
-                const AgentGeom g = P.agents[(size_t)e * P.A + b];
-                if (!g.active) continue;
-                const uint32_t corners = face_corners(f);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
-                quad = true; flags = face_flags(corners);
-                key_lo = ((0xFFFFFFu - (S.n_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
-                Pn = plane_normal(V, true);
-            }
-            PrimEq q;
-            if (!prim_equations(V, quad, flags, Pn, q)) continue;
-            for (int y = 0; y < t.th; ++y) {
-                const float ry = s.ray_y[y];
-                for (int x = 0; x < t.tw; ++x) {
-                    const uint32_t wb = fragment(q, s.ray_x[x], ry, t.w_near, t.w_far);
-                    if (wb) {
-                        const unsigned long long key = make_key(wb, key_lo);
-                        unsigned long long* addr = &s.key[y * TILE + x];
-                        if (key > *reinterpret_cast<volatile unsigned long long*>(addr)) atomicMax(addr, key);
-                    }
-                }
-            }
-        }
-    }
-    __syncthreads();
-    const size_t img = (size_t)P.H * P.W;
-    uint8_t* oc = P.out_class + view * img;
-    uint16_t* od = P.out_depth + view * img;
-    for (int i = threadIdx.x; i < t.th * t.tw; i += kThreads) {
-        const int y = i / t.tw, x = i % t.tw;
-        uint32_t cls = P.cls_sky; float z = P.far_z;
-        if (ego.active) { cls = P.rig.bg_cls[(size_t)k * P.H + t.y0 + y]; z = P.rig.bg_z[(size_t)k * P.H + t.y0 + y]; }
-        const unsigned long long key = s.key[y * TILE + x];
-        if (key) { cls = (uint32_t)(key & 0xff); z = fast_rcp(__uint_as_float((uint32_t)(key >> 32))); }
-        const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + x;
-        oc[o] = (uint8_t)cls;
-        od[o] = __half_as_ushort(__float2half_rn(z));
-    }
+                        for (int j = 0; j < 3; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
+                        V[3] = V[2];
+                        const float v12[12] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], v[8], v[6], v[7], v[8]};
+                        Pn = plane_normal_world(c, v12, false);
+                        quad = false;
+                        flags = 0u;
+                        // an edge shared by two triangles is evaluated in the same direction by both
+                        if (!lex_less(v[0], v[1], v[2], v[3], v[4], v[5])) flags |= 1u << 4;
+                        if (!lex_less(v[3], v[4], v[5], v[6], v[7], v[8])) flags |= 1u << 5;
+                        if (!lex_less(v[6], v[7], v[8], v[0], v[1], v[2])) flags |= 1u << 6;
+                        key_lo = ((0xFFFFFFu - i) << 8) | __ldg(tri_class + i);
+                    });
 }
 
 pic_status fail(pic_status st, const char* fmt, ...) {
@@ -189,6 +115,14 @@ extern "C" pic_status pic_render_static(const pic_static_desc* d, const float* t
     if (d->H > kMaxSide || d->W > kMaxSide)
         return fail(PIC_ERR_CAPACITY, "pic_render_static renders images up to %d x %d, got %d x %d", kMaxSide, kMaxSide, d->H, d->W);
     if (d->n_tris > PIC_STATIC_MAX_TRIS) return fail(PIC_ERR_CAPACITY, "pic_render_static reads at most %d triangles, got %d", PIC_STATIC_MAX_TRIS, d->n_tris);
+    {
+        // every primitive is tested against every pixel of every view: bound the product, so that a
+        // request at all the limits at once cannot occupy the GPU for hours
+        const double work = ((double)d->n_tris + 6.0 * d->A) * (double)d->E * d->A * d->K * (double)d->H * d->W;
+        if (work > (double)PIC_STATIC_MAX_WORK)
+            return fail(PIC_ERR_CAPACITY, "pic_render_static: (n_tris + 6A) * E*A*K*H*W = %.3g primitive-pixel tests, at most %.3g", work,
+                        (double)PIC_STATIC_MAX_WORK);
+    }
     if (!(d->near_z > 0.f) || !(d->far_z > d->near_z) || !std::isfinite(d->far_z)) return fail(PIC_ERR_INVALID_ARG, "need 0 < near_z < far_z < inf");
     if (!poses || !dims || !rig || !out_class || !out_depth) return fail(PIC_ERR_INVALID_ARG, "a required pointer is NULL");
     if (d->n_tris > 0 && (!tri_xyz || !tri_class)) return fail(PIC_ERR_INVALID_ARG, "triangle arrays are NULL");
@@ -210,7 +144,7 @@ extern "C" pic_status pic_render_static(const pic_static_desc* d, const float* t
             void* p = nullptr;
             ce = cudaGetSymbolAddress(&p, g_static_scratch);
             if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(ce));
-            ce = cudaFuncSetAttribute(render_static_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StaticSmem));
+            ce = cudaFuncSetAttribute(render_static_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ExhaustiveSmem));
             if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ce));
             g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
         }
@@ -242,14 +176,34 @@ extern "C" pic_status pic_render_static(const pic_static_desc* d, const float* t
         o.fx = rig[k].fx; o.fy = rig[k].fy;
     }
     S.tri_xyz = tri_xyz; S.tri_class = tri_class; S.n_tris = (uint32_t)d->n_tris;
-    // the array keeps whatever the previous call left: the status word must start at zero
-    ce = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
-    if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(ce));
+    // (the status word is sticky across calls, like a scene's: pic_static_status reads and clears it)
     ce = pic::launch_setup(P, d->E * d->A, poses, nullptr, nullptr, dims, active, agents, cams, tables, status, 0.f, 1.f, 0.f, stream);
     if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "set-up kernels: %s", cudaGetErrorString(ce));
     const unsigned blocks = (unsigned)(d->E * d->A * d->K * P.tiles_x * P.tiles_y);
-    render_static_kernel<<<blocks, kThreads, sizeof(StaticSmem), stream>>>(S);
+    render_static_kernel<<<blocks, EXH_THREADS, sizeof(ExhaustiveSmem), stream>>>(S);
     ce = cudaGetLastError();
     if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "render_static_kernel: %s", cudaGetErrorString(ce));
+    return PIC_OK;
+}
+
+extern "C" pic_status pic_static_status(uint32_t* flags, void* cuda_stream) {
+    if (!flags) return fail(PIC_ERR_INVALID_ARG, "flags is NULL");
+    *flags = 0u;
+    int dev = -1;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(ce));
+    if (dev < 0 || dev >= kMaxDevices) return fail(PIC_ERR_INVALID_ARG, "device ordinal %d not supported", dev);
+    unsigned char* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        scratch = g_scratch_ptr[dev];
+    }
+    if (!scratch) return PIC_OK;                  // pic_render_static has not run on this device
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t* status = reinterpret_cast<uint32_t*>(scratch + kOffStatus);
+    ce = cudaMemcpyAsync(flags, status, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+    if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "reading the status word: %s", cudaGetErrorString(ce));
     return PIC_OK;
 }

@@ -264,6 +264,22 @@ def test_error_codes(gu):
         assert g.scene.status() & pic.FLAG_NONFINITE_POSE
         assert g.scene.status() == 0
         assert (cls.cpu().numpy() == 0).all()          # that agent is treated as inactive: sky
+        # a non-finite action (or a step that overflows) is flagged as well; the agent keeps its state and
+        # is drawn as sky for that step, and a finite action afterwards moves it again
+        state0 = torch.tensor([[[1.0, 2.0, 0.3, 5.0]]], dtype=torch.float32, device=g.dev)
+        g.scene.set_state(state0, g.dims)
+        for bad in ((float("nan"), 0.0), (0.0, float("nan")), (float("inf"), 0.0), (0.0, float("inf"))):
+            act = torch.tensor([[list(bad)]], dtype=torch.float32, device=g.dev)
+            cls.fill_(7)
+            g.scene.step(act, s.rig, cls, dep)
+            assert g.scene.status() & pic.FLAG_NONFINITE_POSE
+            assert torch.equal(g.scene.get_state(), state0)
+            assert (cls.cpu().numpy() == 0).all()
+        g.scene.step(torch.zeros((1, 1, 2), dtype=torch.float32, device=g.dev), s.rig, cls, dep)
+        assert g.scene.status() == 0
+        moved = g.scene.get_state().cpu().numpy()[0, 0]
+        assert abs(moved[0] - (1.0 + 5.0 * np.cos(0.3) * 0.1)) < 1e-5 and moved[3] == 5.0
+        assert (cls.cpu().numpy()[..., 8:, :] == 1).all()      # an empty scene below the horizon: ground
     finally:
         g.close()
 
