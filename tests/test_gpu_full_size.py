@@ -21,7 +21,11 @@ def gu():
     return gpu_util
 
 
-def _sample_and_check(gu, s, n_oracle, n_brute, seed):
+def _sample_and_check(gu, s, n_oracle, n_brute, seed, env0_views=None):
+    """Full-size run in the launch configuration the benchmark times (no float32 depth image: the full-tile
+    kernels), compared with the oracle on `n_oracle` seeded views plus every view of environment 0; the same
+    views once more with the float32 depth image (the general kernels) at the literal 1e-4 depth tolerance; and a
+    window of `n_brute` views against the exhaustive kernel."""
     import oracle
     g = gu.CudaRun(s)
     try:
@@ -29,9 +33,19 @@ def _sample_and_check(gu, s, n_oracle, n_brute, seed):
         cls, d16, _ = g.render(depth32=False)
         assert (cls != 255).all()                              # every view was written
         rng = np.random.default_rng(seed)
-        views = np.sort(rng.choice(V, size=n_oracle, replace=False))
+        views = np.union1d(rng.choice(V, size=n_oracle, replace=False), np.arange(s.A * s.K if env0_views is None else env0_views))
         ref = oracle.render(s, views)
-        st = compare_images(ref.cls, ref.depth, ref.flag, cls[views], None, d16[views], ref_kappa=ref.kappa)
+        # the comparisons below are given no conditioning numbers: the depth tolerance tested on the benchmark
+        # workloads is the literal 1e-4 everywhere, also on the handful of pixels whose winning plane grazes the
+        # camera centre (mask bit 16, counted here)
+        grazing = int(((ref.flag & 16) != 0).sum())
+        assert grazing <= 1e-4 * ref.flag.size
+        st = compare_images(ref.cls, ref.depth, ref.flag, cls[views], None, d16[views])
+        cls32, d16b, d32 = g.render(depth32=True)
+        assert (cls32 == cls).all() and (d16b.view(np.uint16) == d16.view(np.uint16)).all()
+        compare_images(ref.cls, ref.depth, ref.flag, cls32[views], d32[views], d16b[views])
+        del cls32, d16b, d32
+        st["views"] = int(len(views)); st["grazing_pixels"] = grazing
         first = int(rng.integers(0, V - n_brute))
         a = g.render(view_first=first, view_count=n_brute)
         b = g.render(brute=True, view_first=first, view_count=n_brute)
@@ -43,18 +57,40 @@ def _sample_and_check(gu, s, n_oracle, n_brute, seed):
 
 
 def test_config1_full(gu):
-    st = _sample_and_check(gu, make_config(1), n_oracle=96, n_brute=1024, seed=1)
+    st = _sample_and_check(gu, make_config(1), n_oracle=512, n_brute=1024, seed=1)
+    assert st["views"] >= 512 + 100
     print("cfg1 full", st)
 
 
 def test_config2_full(gu):
-    st = _sample_and_check(gu, make_config(2), n_oracle=96, n_brute=1024, seed=2)
+    st = _sample_and_check(gu, make_config(2), n_oracle=512, n_brute=1024, seed=2)
+    assert st["views"] >= 512 + 200
     print("cfg2 full", st)
 
 
 def test_config3_full(gu):
-    st = _sample_and_check(gu, make_config(3), n_oracle=12, n_brute=48, seed=3)
+    # (the oracle needs 0.8 s per 128 x 256 view of this 37 504-triangle map: 64 seeded views plus the 16 views
+    # of environment 0's first four agents, not all 256 views of environment 0)
+    st = _sample_and_check(gu, make_config(3), n_oracle=64, n_brute=48, seed=3, env0_views=16)
+    assert st["views"] >= 64
     print("cfg3 full", st)
+
+
+def _camera_inside_a_box(s, state, view):
+    """Is the camera of `view` inside (or within 5 cm of) the box of another active agent of its environment?"""
+    e, a, k = view // (s.A * s.K), (view // s.K) % s.A, view % s.K
+    x, y, th = (float(t) for t in state[e, a, :3])
+    mx, my, mz = (float(t) for t in s.rig[k, :3])
+    cx, cy = x + np.cos(th) * mx - np.sin(th) * my, y + np.sin(th) * mx + np.cos(th) * my
+    for b in range(s.A):
+        if b == a or not s.active[e, b]:
+            continue
+        bx, by, bth = (float(t) for t in state[e, b, :3])
+        dx, dy = cx - bx, cy - by
+        u, v = np.cos(bth) * dx + np.sin(bth) * dy, -np.sin(bth) * dx + np.cos(bth) * dy
+        if abs(u) <= 0.5 * s.dims[e, b, 0] + 0.05 and abs(v) <= 0.5 * s.dims[e, b, 1] + 0.05 and mz <= s.dims[e, b, 2] + 0.05:
+            return True
+    return False
 
 
 def test_config4_full_hundred_steps(gu):
@@ -69,17 +105,26 @@ def test_config4_full_hundred_steps(gu):
         rng = np.random.default_rng(4)
         agents = np.sort(rng.choice(s.E * s.A, size=256, replace=False))
         st64 = s.state().astype(np.float64).reshape(-1, 4)[agents]
+        n_inside = 0
         for step in range(1, 101):
             act = make_actions(4, step, s.E, s.A)
             g.scene.step(torch.from_numpy(act).to(dev), s.rig, cls, dep)
             st64 = oracle.step(st64, act.reshape(-1, 2)[agents], None, DT, WHEELBASE, V_MAX)
             if step in (1, 50, 100):
                 got = g.scene.get_state().cpu().numpy()
-                views = np.sort(rng.choice(s.E * s.A * s.K, size=16, replace=False))
+                views = np.sort(rng.choice(s.E * s.A * s.K, size=128, replace=False))
                 ref = oracle.render(s, views, poses=got[..., :3])
                 c = cls.cpu().numpy().reshape(-1, s.H, s.W)[views]
                 d = dep.cpu().numpy().reshape(-1, s.H, s.W)[views]
-                compare_images(ref.cls, ref.depth, ref.flag, c, None, None)
+                # The protocol has no collision handling, so after some steps a few agents overlap.  A camera
+                # that sits inside another agent's box looks at that box's bottom face from above, which is
+                # coplanar with the road: a whole surface of exact depth ties between two classes.  Those
+                # views are held to "every mismatch on a flagged pixel" only; all the others to the full rule.
+                inside = np.array([_camera_inside_a_box(s, got, int(v)) for v in views])
+                compare_images(ref.cls[~inside], ref.depth[~inside], ref.flag[~inside], c[~inside], None, None)
+                if inside.any():
+                    compare_images(ref.cls[inside], ref.depth[inside], ref.flag[inside], c[inside], None, None, max_mismatch_frac=1.0)
+                n_inside += int(inside.sum())
                 ok = (c == ref.cls) & (ref.flag == 0)
                 ulp = np.abs(d.view(np.uint16).astype(np.int32) - ref.depth.astype(np.float16).view(np.uint16).astype(np.int32))
                 assert (ulp[ok] <= 1).all()
@@ -88,6 +133,7 @@ def test_config4_full_hundred_steps(gu):
                 assert np.abs((sub[:, 2] - st64[:, 2] + np.pi) % (2 * np.pi) - np.pi).max() <= 1e-5 * max(1.0, np.abs(st64[:, 2]).max())
                 assert np.abs(sub[:, 3] - st64[:, 3]).max() <= 1e-4
         assert g.scene.status() == 0
+        assert n_inside <= 12, "more than a handful of the 384 sampled cameras sit inside another agent's box"
     finally:
         g.close()
 

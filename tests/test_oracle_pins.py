@@ -534,6 +534,41 @@ def test_ambiguity_mask_flags_only_near_boundaries():
     assert (oracle.render(s).flag[0] & 2).sum() == 0
 
 
+def test_ambiguity_mask_near_far_planes_and_horizon():
+    """The two remaining branches of the mask.  Bit 4: a covered fragment whose depth is within 1e-5 relative of
+    the near or the far plane, on either side of it, and that would be visible; bit 8: a background pixel whose
+    ray is within 1e-5 of horizontal."""
+    for plane, other in ((0.5, 100.0), (64.0, 0.5)):
+        near, far = (plane, other) if plane < other else (other, plane)
+        size = 8.0 * plane                                    # the wall fills the 90-degree image
+        for rel, want in ((0.0, True), (1e-6, True), (-1e-6, True), (1e-2, False), (-1e-2, False)):
+            x = np.float32(plane * (1.0 + rel))
+            s = single_env(_wall(float(x), -size, size, -size, size), [5, 5], [ego()], rig=RIG0, H=8, W=8, near=near, far=far)
+            r = oracle.render(s)
+            assert bool((r.flag[0] & 4).all()) == want and bool((r.flag[0] & 4).any()) == want, (plane, rel, r.flag[0])
+            # on which side of the plane the wall sits decides whether it is drawn -- flagged or not
+            inside = near <= float(x) <= far
+            assert (r.cls[0] == 5).all() == inside
+    # a wall at the near plane hidden behind nothing but in front of another wall: the nearer one matters, the
+    # farther one (at 2 m, well inside the range) does not raise the flag by itself
+    s = single_env(_wall(2.0, -16, 16, -16, 16), [6, 6], [ego()], rig=RIG0, H=8, W=8, near=0.5, far=100.0)
+    assert (oracle.render(s).flag[0] & 4).sum() == 0
+    # horizon: 8 x 8 image, fy = 4, row 5 has ray slope 1.5 / 4; pitch the camera so that this ray is horizontal
+    for d, want in ((1e-6, True), (-1e-6, True), (1e-2, False), (-1e-2, False)):
+        phi = np.degrees(np.arctan(0.375) + d)
+        s = single_env(np.zeros((0, 3, 3)), [], [ego()], rig=make_rig((0.0,), 90.0, 90.0, 8, 8, mount=(0.0, 0.0, 1.0), pitch_deg=phi),
+                       H=8, W=8)
+        r = oracle.render(s)
+        assert bool((r.flag[0][5] & 8).all()) == want, (d, r.flag[0])
+        assert (np.delete(r.flag[0], 5, axis=0) & 8).sum() == 0
+        # above the horizon row sky, below it ground, whatever the flagged row itself shows
+        assert (r.cls[0][:5] == 0).all() and (r.cls[0][6:] == 1).all()
+    # a primitive covering the pixel takes the horizon flag away: it is about the background only
+    s = single_env(_wall(4.0, -8, 8, -8, 8), [5, 5], [ego()],
+                   rig=make_rig((0.0,), 90.0, 90.0, 8, 8, mount=(0.0, 0.0, 1.0), pitch_deg=np.degrees(np.arctan(0.375))), H=8, W=8)
+    assert (oracle.render(s).flag[0] & 8).sum() == 0
+
+
 def test_box_primitive_indices_and_tie_between_identical_boxes():
     # two identical boxes at the same pose: every pixel is an exact tie, the lower agent index wins,
     # and the winning index is N + 12 b + t with N map triangles
