@@ -163,6 +163,11 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *                         cooperative kernel).
  *   PIC_OPT_VIEW_FIRST,   render only views [first, first + count) (flat index (e*A + a)*K + k);
  *   PIC_OPT_VIEW_COUNT    count 0 = through the last view.  Other views' pixels are left untouched.
+ *   PIC_OPT_OUT_RELATIVE  1: out_class / out_depth (and the PIC_OPT_DEPTH32 image) hold only the rendered
+ *                         views, the first rendered view at offset 0 -- so a batch can be streamed in
+ *                         passes through buffers of count*H*W pixels (the paper's renderer likewise
+ *                         streams a batch in passes bounded by free memory, App. "Renderer memory
+ *                         usage"); 0: the images are indexed by absolute view.
  *   PIC_OPT_DEBUG_FLAGS   bit 0: rasterize large primitives without the per-cell trivial
  *                         accept/reject; bit 1: shrink the fused kernel's record pool and the
  *                         cooperative kernel's record list to 2 entries so that the overflow paths
@@ -180,6 +185,7 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
 #define PIC_OPT_VIEW_COUNT 5
 #define PIC_OPT_TIMING 6
 #define PIC_OPT_DEBUG_FLAGS 7
+#define PIC_OPT_OUT_RELATIVE 8
 pic_status pic_scene_set_option(pic_scene* scene, int32_t option, uint64_t value);
 
 /*
@@ -250,6 +256,21 @@ pic_status pic_render_static(const pic_static_desc* desc, const float* tri_xyz, 
                              const float* poses, const float* dims, const uint8_t* active, const pic_camera* rig,
                              uint8_t* out_class, uint16_t* out_depth, void* cuda_stream);
 pic_status pic_static_status(uint32_t* flags, void* cuda_stream);
+
+/*
+ * Measurement aids (the paper has no counterpart): the two microbenchmarks that give a roofline its
+ * denominators on the machine at hand.  Both run on the CURRENT device, asynchronously on
+ * `cuda_stream`, allocate nothing, and are timed by the caller (CUDA events around the call).
+ *   pic_probe_fill   writes `bytes` bytes at dst (dev, 16-byte aligned, bytes % 16 == 0) with 128-bit
+ *                    stores from 32 CTAs per multiprocessor: the write-only stream the image store
+ *                    competes with.
+ *   pic_probe_ffma   runs a register-only loop of `iters` x 8 independent fused multiply-adds per
+ *                    thread on 8 CTAs of 256 threads per multiprocessor; out (dev) must hold 2048 floats
+ *                    per multiprocessor (out_floats is checked), *fma_count (host) receives the number of
+ *                    per-lane multiply-adds the launch executes.
+ */
+pic_status pic_probe_fill(void* dst, uint64_t bytes, void* cuda_stream);
+pic_status pic_probe_ffma(float* out, uint64_t out_floats, int32_t iters, uint64_t* fma_count, void* cuda_stream);
 
 /* Thread-local, never NULL; valid until the next failing call on this thread. */
 const char* pic_last_error(void);

@@ -17,11 +17,11 @@ from . import build as _build
 PIC_OK = 0
 STATUS_NAMES = {0: "PIC_OK", 1: "PIC_ERR_INVALID_ARG", 2: "PIC_ERR_SHAPE", 3: "PIC_ERR_OOM", 4: "PIC_ERR_CUDA",
                 5: "PIC_ERR_CAPACITY", 6: "PIC_ERR_NONFINITE"}
-OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_TIMING, OPT_DEBUG_FLAGS = 1, 2, 3, 4, 5, 6, 7
+OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_TIMING, OPT_DEBUG_FLAGS, OPT_OUT_RELATIVE = 1, 2, 3, 4, 5, 6, 7, 8
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status",
+           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
            "pic_last_error", "pic_version"]
 
 
@@ -78,6 +78,8 @@ def load(path: Optional[str] = None):
     lib.pic_map_stats.argtypes = [C.POINTER(pic_scene_desc), C.POINTER(C.c_int64)]
     lib.pic_render_static.argtypes = [C.POINTER(pic_static_desc), vp, vp, vp, vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     lib.pic_static_status.argtypes = [C.POINTER(C.c_uint32), vp]
+    lib.pic_probe_fill.argtypes = [vp, C.c_uint64, vp]
+    lib.pic_probe_ffma.argtypes = [vp, C.c_uint64, C.c_int32, C.POINTER(C.c_uint64), vp]
     for name in EXPORTS:
         getattr(lib, name).restype = C.c_int
     lib.pic_last_error.restype = C.c_char_p
@@ -167,6 +169,23 @@ def render_static(E: int, A: int, K: int, H: int, W: int, near: float, far: floa
     return out_class, out_depth
 
 
+def probe_fill(dst, stream=None) -> int:
+    """pic_probe_fill on a CUDA tensor (write-only stream, 128-bit stores); returns the bytes written."""
+    lib = load()
+    nbytes = dst.numel() * dst.element_size()
+    _check(lib, lib.pic_probe_fill(C.c_void_p(dst.data_ptr()), nbytes, _stream_ptr(stream)))
+    return nbytes
+
+
+def probe_ffma(out, iters: int, stream=None) -> int:
+    """pic_probe_ffma (register-only FFMA loop); `out` is a float32 CUDA tensor; returns the per-lane FMA count."""
+    import torch
+    lib = load()
+    n = C.c_uint64(0)
+    _check(lib, lib.pic_probe_ffma(_dev_ptr(out, torch.float32, out.numel()), out.numel(), int(iters), C.byref(n), _stream_ptr(stream)))
+    return int(n.value)
+
+
 def static_status(stream=None) -> int:
     """pic_static_status: read and clear the sticky flags of pic_render_static on the current device."""
     lib = load()
@@ -235,6 +254,38 @@ class Scene:
             _dev_ptr(active, torch.uint8, n) if active is not None else None, _rig_array(rig),
             _dev_ptr(out_class, torch.uint8, npx), _dev_ptr(out_depth, torch.float16, npx), _stream_ptr(stream)))
         return out_class, out_depth
+
+    def render_in_passes(self, poses, dims, rig, consume, max_bytes: int, active=None, stream=None) -> int:
+        """Render all views in passes whose output fits `max_bytes` (class + depth bytes), into one pair of
+        pass-sized buffers that is reused: after each pass `consume(first_view, n_views, class_u8, depth_f16)` is
+        called with views of the buffers (shape [n_views, H, W]); the device is synchronised before it runs, and
+        the next pass overwrites the buffers.  Returns the number of passes.  Argument marshalling only: every
+        pass is one pic_render call with PIC_OPT_VIEW_FIRST / VIEW_COUNT / OUT_RELATIVE set."""
+        import torch
+        total = self.n_agents * self.K
+        per_view = 3 * self.H * self.W
+        n_pass_views = max(1, min(total, int(max_bytes) // per_view))
+        out_c = torch.empty((n_pass_views, self.H, self.W), dtype=torch.uint8, device=self.device)
+        out_d = torch.empty((n_pass_views, self.H, self.W), dtype=torch.float16, device=self.device)
+        n, passes = self.n_agents, 0
+        try:
+            self.set_option(OPT_OUT_RELATIVE, 1)
+            for first in range(0, total, n_pass_views):
+                cnt = min(n_pass_views, total - first)
+                self.set_option(OPT_VIEW_FIRST, first)
+                self.set_option(OPT_VIEW_COUNT, cnt)
+                _check(self._lib, self._lib.pic_render(
+                    self._h, _dev_ptr(poses, torch.float32, 3 * n), _dev_ptr(dims, torch.float32, 3 * n),
+                    _dev_ptr(active, torch.uint8, n) if active is not None else None, _rig_array(rig),
+                    out_c.data_ptr(), out_d.data_ptr(), _stream_ptr(stream)))
+                torch.cuda.synchronize(self.device)
+                consume(first, cnt, out_c[:cnt], out_d[:cnt])
+                passes += 1
+        finally:
+            self.set_option(OPT_VIEW_FIRST, 0)
+            self.set_option(OPT_VIEW_COUNT, 0)
+            self.set_option(OPT_OUT_RELATIVE, 0)
+        return passes
 
     def render_host(self, poses: np.ndarray, dims: np.ndarray, rig, out_class: np.ndarray, out_depth: np.ndarray,
                     active: Optional[np.ndarray] = None, stream=None):

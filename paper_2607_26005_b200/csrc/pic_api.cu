@@ -90,6 +90,7 @@ struct pic_scene {
     unsigned long long* counters = nullptr;
     long long view_first = 0, view_count = 0;
     int debug_flags = 0;
+    bool out_relative = false;
     bool timing = false;
     cudaEvent_t* ev = nullptr;      // 2 * kMaxTimed events
     int n_timed = 0;
@@ -342,6 +343,7 @@ pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
             s->view_first = (long long)value; return PIC_OK;
         case PIC_OPT_VIEW_COUNT: s->view_count = (long long)value; return PIC_OK;
         case PIC_OPT_DEBUG_FLAGS: s->debug_flags = (int)value; return PIC_OK;
+        case PIC_OPT_OUT_RELATIVE: s->out_relative = value != 0; return PIC_OK;
         case PIC_OPT_TIMING: {
             if (value && !s->ev) {
                 DeviceGuard guard(s->device);
@@ -373,6 +375,13 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
     long long count = total - s->view_first;
     if (s->view_count > 0 && s->view_count < count) count = s->view_count;
     P.view_first = s->view_first;
+    if (s->out_relative) {
+        // the caller's buffers start at the first rendered view: shift the bases so that the kernels'
+        // absolute view indexing lands there (never dereferenced below view_first)
+        const size_t off = (size_t)s->view_first * s->H * s->W;
+        P.out_class -= off; P.out_depth -= off;
+        if (P.out_depth32) P.out_depth32 -= off;
+    }
     const bool timed = s->timing && s->n_timed < kMaxTimed;
     if (timed) CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed], stream));
     CUDA_TRY(pic::launch_render(P, count, s->brute, s->sm_count, stream));

@@ -359,6 +359,62 @@ def make_config(cfg: int, E: Optional[int] = None, A: Optional[int] = None, env_
                            dict(min=int(counts.min()), max=int(counts.max()), mean=float(counts.mean()))))
 
 
+# ----------------------------------------------------------------------------------------------
+# the paper's own workload shape: its four-camera rig at 16:9, variable agent counts, ego chunks
+# ----------------------------------------------------------------------------------------------
+# Table "Camera rig": per-camera mounts (ego frame, metres) and yaws; one 1545 px focal length on a
+# 1920 x 1080 sensor, rendered at 96 x 54 by default (32 x 18 ... 384 x 216 in the resolution sweep).
+PAPER_RIG_MOUNTS = ((1.66, -0.01, 1.49, 0.0), (1.63, 0.12, 1.48, 55.0), (1.62, -0.16, 1.49, -55.0), (-0.47, 0.02, 1.43, 180.0))
+PAPER_FOCAL_PX, PAPER_SENSOR_W, PAPER_SENSOR_H = 1545.0, 1920, 1080
+PAPER_SEED = 7000
+
+
+def make_paper_rig(W: int = 96, H: int = 54) -> np.ndarray:
+    """The paper's rig at render size W x H: front, front-left (+55 deg), front-right (-55 deg), back.  The four
+    cameras have different mounts, so they do not share an origin."""
+    rig = np.zeros((4, 7), dtype=np.float32)
+    for k, (x, y, z, yaw) in enumerate(PAPER_RIG_MOUNTS):
+        rig[k] = (x, y, z, np.deg2rad(yaw), 0.0, PAPER_FOCAL_PX * W / PAPER_SENSOR_W, PAPER_FOCAL_PX * H / PAPER_SENSOR_H)
+    return rig
+
+
+def make_paper_workload(W: int = 96, H: int = 54, egos: int = 2048, slots: int = 120, E: Optional[int] = None,
+                        far: float = 100.0, env_offset: int = 0) -> Scene:
+    """One chunk of about `egos` egos in the paper's shape (Appendix, hyper-parameter table and Sec. "Renderer
+    memory usage"): map instances with a number of agents drawn from U{1, slots} each -- A = slots agent slots
+    per environment, the surplus marked inactive -- rendered by the four-camera rig at 16:9.  Environments are
+    added until the active agents reach `egos` (or exactly E environments if E is given).  Maps are the
+    8 x 8 grids with curved connectors of workload 2 (stand-ins for the town maps); agents sit on road
+    centre-lines.  Seeds: PAPER_SEED + env for maps, PAPER_SEED + 500000 + env for agents."""
+    maps: List[GridMap] = []
+    poses_l, dims_l, active_l = [], [], []
+    n_active, e = 0, 0
+    while (E is None and n_active < egos) or (E is not None and e < E):
+        gm = grid_map(PAPER_SEED + env_offset + e, 8, 100.0, 10.0, True, 0)
+        rng = np.random.default_rng(PAPER_SEED + 500000 + env_offset + e)
+        n = int(rng.integers(1, slots + 1))
+        if E is None:
+            n = min(n, egos - n_active)
+        pos, yaw = _agents_on_centrelines(rng, gm, slots)
+        p = np.zeros((slots, 3), np.float32)
+        p[:, :2] = pos
+        p[:, 2] = yaw
+        a = np.zeros(slots, np.uint8)
+        a[:n] = 1
+        maps.append(gm); poses_l.append(p); dims_l.append(_dims(rng, slots, 0.1)); active_l.append(a)
+        n_active += n
+        e += 1
+    n_env = len(maps)
+    counts = np.array([m.tri_xyz.shape[0] for m in maps], dtype=np.int64)
+    return Scene(name=f"paper{W}x{H}", E=n_env, A=slots, K=4, H=H, W=W, near=0.5, far=far, num_maps=n_env,
+                 env_map_id=np.arange(n_env, dtype=np.int32), map_tri_offset=np.concatenate([[0], np.cumsum(counts)]).astype(np.int64),
+                 tri_xyz=np.concatenate([m.tri_xyz for m in maps]).astype(np.float32),
+                 tri_class=np.concatenate([m.tri_class for m in maps]).astype(np.uint8),
+                 poses=np.stack(poses_l).astype(np.float32), dims=np.stack(dims_l).astype(np.float32),
+                 active=np.stack(active_l), rig=make_paper_rig(W, H), speed=np.zeros((n_env, slots), np.float32),
+                 meta=dict(active_agents=int(n_active)))
+
+
 def make_actions(cfg: int, step: int, E: int, A: int) -> np.ndarray:
     """Actions of one step, f32 [E,A,2]: accel ~ U[-3,2] m/s^2, steer ~ U[-0.3,0.3] rad."""
     rng = np.random.default_rng(1000 * cfg + 900000 + step)
