@@ -163,6 +163,15 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
  *                         cooperative kernel).
  *   PIC_OPT_VIEW_FIRST,   render only views [first, first + count) (flat index (e*A + a)*K + k);
  *   PIC_OPT_VIEW_COUNT    count 0 = through the last view.  Other views' pixels are left untouched.
+ *   PIC_OPT_OCCLUSION     value = dev u32* [E,A,K,A,2] (as uintptr) or 0: per view and per OTHER agent b of the
+ *                         environment, [0] the pixels of the image won by b's box ("visible") and [1] the
+ *                         pixels at which b's box drawn alone (no map, no other agent) leaves a fragment
+ *                         within [near, far] ("unoccluded"); 100 * (1 - visible / unoccluded) is the road
+ *                         user's occlusion percentage as the renderer sees it (Sec. 5.2, counterfactual
+ *                         probes; the paper gives no formula, this is the reading taken).  Entries of the
+ *                         ego itself and of inactive agents are 0; the entries of the rendered views are
+ *                         overwritten, indexed by absolute view.  Costs an extra pass over the agents' boxes
+ *                         and selects the general kernels.
  *   PIC_OPT_OUT_RELATIVE  1: out_class / out_depth (and the PIC_OPT_DEPTH32 image) hold only the rendered
  *                         views, the first rendered view at offset 0 -- so a batch can be streamed in
  *                         passes through buffers of count*H*W pixels (the paper's renderer likewise
@@ -186,6 +195,7 @@ pic_status pic_get_status(pic_scene* scene, uint32_t* flags, void* cuda_stream);
 #define PIC_OPT_TIMING 6
 #define PIC_OPT_DEBUG_FLAGS 7
 #define PIC_OPT_OUT_RELATIVE 8
+#define PIC_OPT_OCCLUSION 9
 pic_status pic_scene_set_option(pic_scene* scene, int32_t option, uint64_t value);
 
 /*

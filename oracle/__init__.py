@@ -5,5 +5,6 @@ tests, the smoke check and the benchmark's CPU-baseline leg may import this pack
 package never does, and this package never imports the product.
 """
 from .wrapper import build, render, step, f64_to_f16_bits, max_threads, OracleResult
+from .occlusion import occlusion_counts
 
-__all__ = ["build", "render", "step", "f64_to_f16_bits", "max_threads", "OracleResult"]
+__all__ = ["build", "render", "step", "f64_to_f16_bits", "max_threads", "OracleResult", "occlusion_counts"]

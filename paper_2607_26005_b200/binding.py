@@ -17,7 +17,7 @@ from . import build as _build
 PIC_OK = 0
 STATUS_NAMES = {0: "PIC_OK", 1: "PIC_ERR_INVALID_ARG", 2: "PIC_ERR_SHAPE", 3: "PIC_ERR_OOM", 4: "PIC_ERR_CUDA",
                 5: "PIC_ERR_CAPACITY", 6: "PIC_ERR_NONFINITE"}
-OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_TIMING, OPT_DEBUG_FLAGS, OPT_OUT_RELATIVE = 1, 2, 3, 4, 5, 6, 7, 8
+OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_TIMING, OPT_DEBUG_FLAGS, OPT_OUT_RELATIVE, OPT_OCCLUSION = 1, 2, 3, 4, 5, 6, 7, 8, 9
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",

@@ -88,6 +88,7 @@ struct pic_scene {
     bool brute = false;
     float* depth32 = nullptr;
     unsigned long long* counters = nullptr;
+    uint32_t* occlusion = nullptr;
     long long view_first = 0, view_count = 0;
     int debug_flags = 0;
     bool out_relative = false;
@@ -143,7 +144,7 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.rig.ray_y = P.rig.ray_x + (size_t)s->K * s->W;
     P.rig.bg_z = P.rig.ray_y + (size_t)s->K * s->H;
     P.rig.bg_cls = reinterpret_cast<const uint32_t*>(P.rig.bg_z + (size_t)s->K * s->H);
-    P.out_class = out_class; P.out_depth = out_depth; P.out_depth32 = s->depth32; P.counters = s->counters;
+    P.out_class = out_class; P.out_depth = out_depth; P.out_depth32 = s->depth32; P.counters = s->counters; P.occlusion = s->occlusion;
     P.view_first = 0;
     P.debug_flags = s->debug_flags;
     for (int k = 0; k < s->K; ++k) {
@@ -338,6 +339,7 @@ pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
         case PIC_OPT_BRUTE_FORCE: s->brute = value != 0; return PIC_OK;
         case PIC_OPT_DEPTH32: s->depth32 = reinterpret_cast<float*>(static_cast<uintptr_t>(value)); return PIC_OK;
         case PIC_OPT_COUNTERS: s->counters = reinterpret_cast<unsigned long long*>(static_cast<uintptr_t>(value)); return PIC_OK;
+        case PIC_OPT_OCCLUSION: s->occlusion = reinterpret_cast<uint32_t*>(static_cast<uintptr_t>(value)); return PIC_OK;
         case PIC_OPT_VIEW_FIRST:
             if (value >= (uint64_t)s->E * s->A * s->K) return fail(PIC_ERR_INVALID_ARG, "first view out of range");
             s->view_first = (long long)value; return PIC_OK;
@@ -382,6 +384,8 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
         P.out_class -= off; P.out_depth -= off;
         if (P.out_depth32) P.out_depth32 -= off;
     }
+    if (P.occlusion)    // the counts of the rendered views start at zero
+        CUDA_TRY(cudaMemsetAsync(P.occlusion + (size_t)s->view_first * s->A * 2, 0, sizeof(uint32_t) * 2 * (size_t)count * s->A, stream));
     const bool timed = s->timing && s->n_timed < kMaxTimed;
     if (timed) CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed], stream));
     CUDA_TRY(pic::launch_render(P, count, s->brute, s->sm_count, stream));

@@ -166,6 +166,13 @@ __device__ __forceinline__ uint32_t fragment(const PrimEq& q, float rx, float ry
     return in ? __float_as_uint(w) : 0u;
 }
 
+// Counts a pixel won by a box face for its agent: the low key word holds 0xFFFFFF - primitive index,
+// box primitives start at n_map_tris, 12 per agent.
+__device__ __forceinline__ void count_visible(uint32_t* occ_view, unsigned long long key, uint32_t n_map_tris) {
+    const uint32_t index = 0xFFFFFFu - ((uint32_t)key >> 8);
+    if (key != 0ull && index >= n_map_tris) atomicAdd(occ_view + 2u * ((index - n_map_tris) / 12u), 1u);
+}
+
 __device__ __forceinline__ unsigned long long make_key(uint32_t wbits, uint32_t key_lo) {
     return ((unsigned long long)wbits << 32) | key_lo;
 }

@@ -91,6 +91,7 @@ __device__ __forceinline__ void exhaustive_tile(ExhaustiveSmem& s, const RenderP
         uint32_t cls = P.cls_sky; float z = P.far_z;
         if (ego.active) { cls = P.rig.bg_cls[(size_t)k * P.H + t.y0 + y]; z = P.rig.bg_z[(size_t)k * P.H + t.y0 + y]; }
         const unsigned long long key = s.key[y * TILE + x];
+        if (P.occlusion) count_visible(P.occlusion + view * (size_t)P.A * 2u, key, n_map_tris);
         if (key) { cls = (uint32_t)(key & 0xff); z = fast_rcp(__uint_as_float((uint32_t)(key >> 32))); }
         const size_t o = (size_t)(t.y0 + y) * P.W + t.x0 + x;
         oc[o] = (uint8_t)cls;

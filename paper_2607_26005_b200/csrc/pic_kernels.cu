@@ -116,6 +116,7 @@ __global__ void __launch_bounds__(EXH_THREADS) render_brute_kernel(const __grid_
 size_t render_smem_bytes();                       // pic_render.cu
 cudaError_t configure_render_kernel();            // pic_render.cu
 cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, int sm_count, cudaStream_t stream);
+cudaError_t launch_coverage_kernel(const RenderParams& P, long long n_views, cudaStream_t stream);
 
 size_t max_smem_bytes() { return render_smem_bytes() > sizeof(ExhaustiveSmem) ? render_smem_bytes() : sizeof(ExhaustiveSmem); }
 
@@ -155,7 +156,8 @@ cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, 
     const long long blocks = n_views * P.tiles_x * P.tiles_y;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     render_brute_kernel<<<(unsigned)blocks, EXH_THREADS, sizeof(ExhaustiveSmem), stream>>>(P);
-    return cudaGetLastError();
+    const cudaError_t err = cudaGetLastError();
+    return err != cudaSuccess ? err : launch_coverage_kernel(P, n_views, stream);
 }
 
 }  // namespace pic

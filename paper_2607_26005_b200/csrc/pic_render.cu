@@ -393,8 +393,10 @@ __device__ __forceinline__ void raster_records(S& s, const float4* rec, uint32_t
 // depth image, so that only the vector path is compiled in.
 template <bool FULL = false, class S>
 __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderParams& P, size_t view, int k, bool ego_active,
-                                           unsigned long long touched, bool clear, int tid = threadIdx.x, int nthr = NTHREADS) {
+                                           unsigned long long touched, bool clear, int tid = threadIdx.x, int nthr = NTHREADS,
+                                           uint32_t n_map_tris = 0u) {
     const size_t img = (size_t)P.H * P.W;
+    uint32_t* occ = (!FULL && P.occlusion) ? P.occlusion + view * (size_t)P.A * 2u : nullptr;   // visible-pixel counts of this view
     uint8_t* oc = P.out_class + view * img;
     uint16_t* od = P.out_depth + view * img;
     float* o32 = P.out_depth32 ? P.out_depth32 + view * img : nullptr;
@@ -427,6 +429,7 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
                     ulonglong2* kp = reinterpret_cast<ulonglong2*>(&s.key[key_index(xs + j, y)]);
                     const ulonglong2 kk = *kp;
                     if (clear) *kp = make_ulonglong2(0ull, 0ull);
+                    if (occ) { count_visible(occ, kk.x, n_map_tris); count_visible(occ, kk.y, n_map_tris); }
                     const float z0 = kk.x ? fast_rcp(__uint_as_float((uint32_t)(kk.x >> 32))) : bg_z;
                     const float z1 = kk.y ? fast_rcp(__uint_as_float((uint32_t)(kk.y >> 32))) : bg_z;
                     const uint32_t c0 = kk.x ? (uint32_t)(kk.x & 0xff) : bg_cls, c1 = kk.y ? (uint32_t)(kk.y & 0xff) : bg_cls;
@@ -449,6 +452,7 @@ __device__ __forceinline__ void store_tile(S& s, const TileCtx& t, const RenderP
             for (int j = 0; j < 16 && xs + j < t.tw; ++j) {
                 const unsigned long long key = empty ? 0ull : s.key[key_index(xs + j, y)];
                 if (clear && !empty) s.key[key_index(xs + j, y)] = 0ull;
+                if (occ) count_visible(occ, key, n_map_tris);
                 const float z = key ? fast_rcp(__uint_as_float((uint32_t)(key >> 32))) : bg_z;
                 oc[o + j] = (uint8_t)(key ? (uint32_t)(key & 0xff) : bg_cls);
                 od[o + j] = __half_as_ushort(__float2half_rn(z));
@@ -625,7 +629,7 @@ __device__ __forceinline__ void cooperative_job(TileSmem& s, const RenderParams&
         __syncthreads();
     }
     // ---- phase 4 (d)
-    store_tile<FULL>(s, t, P, view, k, ego_active, ((unsigned long long)s.touched[1] << 32) | s.touched[0], false);
+    store_tile<FULL>(s, t, P, view, k, ego_active, ((unsigned long long)s.touched[1] << 32) | s.touched[0], false, threadIdx.x, NTHREADS, mi.n_tris);
     if (threadIdx.x == 0) { ++n.jobs; ++n.coop; }
 }
 
@@ -688,6 +692,7 @@ struct __align__(16) FusedSmem {
     int n_surv[NW];                           // survivors of tile w; -1: lists overflowed, -2: no such tile
     int next_task;
     int tile_active[NW];                      // is the ego agent of tile w active
+    uint32_t tile_ntris[NW];                  // triangles of its environment's map as given (box primitive indices start there)
     Job tile_job[NW];                         // tile w, decoded by its warp
     Cam cam[NW];                              // its camera
 };
@@ -972,7 +977,7 @@ __device__ __forceinline__ void front_setup(const Cam& c, const uint2* __restric
 // all "no fragment" on entry and on exit.
 template <bool FULL, class TL>
 __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, const Job& job, bool ego_active, int ys,
-                                           const float4* rec, int n_rec, bool classify, int stop, int lane, TL& n) {
+                                           const float4* rec, int n_rec, bool classify, int stop, int lane, uint32_t n_map_tris, TL& n) {
     const TileCtx& t = job.t;
     const int rows = FULL ? STRIP : min(STRIP, t.th - ys);
     uint32_t touched = 0u;                       // 8x8 blocks of the strip: bit (row >> 3) * 8 + (column >> 3)
@@ -1074,7 +1079,7 @@ __device__ __forceinline__ void back_strip(StripView& s, const RenderParams& P, 
     TileCtx ts = t;
     ts.y0 = t.y0 + ys; ts.th = rows;
     const bool ragged = !FULL && (t.tw < TILE || rows < STRIP);
-    if (stop != 8) store_tile<FULL>(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32);
+    if (stop != 8) store_tile<FULL>(s, ts, P, job.view, job.k, ego_active, (unsigned long long)touched, !ragged, lane, 32, n_map_tris);
     __syncwarp();
     if (ragged) {
 #pragma unroll
@@ -1096,6 +1101,10 @@ struct __align__(16) CullSmem {
 #ifndef PIC_CULL_CTAS
 #define PIC_CULL_CTAS 5
 #endif
+#ifndef PIC_CULL_ROUNDS
+#define PIC_CULL_ROUNDS 1
+#endif
+constexpr int CULL_ROUNDS = PIC_CULL_ROUNDS;   // rounds of NW tiles per CTA of the cull kernel
 #ifndef PIC_RENDER_CTAS
 #define PIC_RENDER_CTAS 5
 #endif
@@ -1104,21 +1113,27 @@ __global__ void __launch_bounds__(NTHREADS, PIC_CULL_CTAS) cull_kernel(const __g
     extern __shared__ __align__(16) unsigned char smem_raw[];
     CullSmem& s = *reinterpret_cast<CullSmem*>(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned id = blockIdx.x * (unsigned)NW + warp;
-    if (id >= P.n_jobs) return;
-    TL n = {};
     const int stop = PIC_STOP(P);
-    const Job job = decode_job(P, id);
-    const MapInfo mi = P.env_maps[job.e];
-    const bool ego_active = P.agents[(size_t)job.e * P.A + job.a].active != 0;
-    uint2* blk = P.surv + (size_t)id * SURV_STRIDE;
-    int ns = 0;
-    if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
-    else if (ego_active && stop != 1 && !(stop >= 8 && stop <= 10)) ns = front_cull(s.lists[warp], blk + 2, P, job, mi, lane, n);
-    // (the work counts are summed over the warp's lanes; without counters they are constants)
-    const uint32_t c_grp = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.grp)), c_leaf = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.leaf)),
-                   c_tested = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.tested));
-    if (lane == 0) *reinterpret_cast<uint4*>(blk) = make_uint4((uint32_t)ns, c_grp, c_leaf, c_tested);
+    // a CTA takes CULL_ROUNDS x NW consecutive tiles, NW at a time: consecutive tiles belong to the
+    // same or to neighbouring agents, so the map data a round pulls in serves the next from L1
+#pragma unroll 1
+    for (int round = 0; round < CULL_ROUNDS; ++round) {
+        const unsigned id = (blockIdx.x * (unsigned)CULL_ROUNDS + round) * (unsigned)NW + warp;
+        if (id >= P.n_jobs) return;
+        TL n = {};
+        const Job job = decode_job(P, id);
+        const MapInfo mi = P.env_maps[job.e];
+        const bool ego_active = P.agents[(size_t)job.e * P.A + job.a].active != 0;
+        uint2* blk = P.surv + (size_t)id * SURV_STRIDE;
+        int ns = 0;
+        if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
+        else if (ego_active && stop != 1 && !(stop >= 8 && stop <= 10)) ns = front_cull(s.lists[warp], blk + 2, P, job, mi, lane, n);
+        // (the work counts are summed over the warp's lanes; without counters they are constants)
+        const uint32_t c_grp = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.grp)), c_leaf = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.leaf)),
+                       c_tested = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.tested));
+        if (lane == 0) *reinterpret_cast<uint4*>(blk) = make_uint4((uint32_t)ns, c_grp, c_leaf, c_tested);
+        __syncwarp();
+    }
 }
 
 // Render kernel.  FULL: every tile is 64 x 64, rows allow 128-bit stores, no float32 depth image (the
@@ -1149,7 +1164,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
         mi = P.env_maps[job.e];
         const bool ego_active = P.agents[(size_t)job.e * P.A + job.a].active != 0;
         if (lane == 0) {
-            s.tile_job[warp] = job; s.tile_active[warp] = ego_active;
+            s.tile_job[warp] = job; s.tile_active[warp] = ego_active; s.tile_ntris[warp] = mi.n_tris;
             load_camera(s.cam[warp], P.cams[job.view], P.cam[job.k], P.W, P.H);
         }
         n_big = (int)(head.x & 0xffffu);
@@ -1219,7 +1234,7 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
             }
         }
         __syncwarp();
-        back_strip<FULL>(sv, P, jb, ego_active, ys, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, classify, stop, lane, n);
+        back_strip<FULL>(sv, P, jb, ego_active, ys, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), cj, classify, stop, lane, s.tile_ntris[j], n);
         if (lane == 0 && ys == 0) ++n.jobs;
     }
     // ---- the rest: tiles that did not fit are left to the cooperative kernel
@@ -1591,6 +1606,71 @@ cudaError_t configure_render_kernel() {
     return cudaFuncSetAttribute(cooperative_kernel<Tally, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileSmem));
 }
 
+// ---------------------------------------------------------------------------------------------
+// Coverage kernel (only with the occlusion option): for every tile and every other active agent,
+// the pixels at which that agent's box, drawn alone, leaves a kept fragment.  A warp per tile;
+// per agent, the six faces are rasterized into a bit mask of the tile (a lane per pixel of a face's
+// pixel box), the set bits are counted and added to the view's count.  The arithmetic that decides
+// a pixel is the production kernels' (pic_device.cuh).
+// ---------------------------------------------------------------------------------------------
+struct __align__(16) CoverWarp {
+    float plane[6][4];
+    float side[4][4];
+    Cam cam;
+    uint32_t mask[TILE * TILE / 32];
+    float ray_x[TILE], ray_y[TILE];
+};
+
+__global__ void __launch_bounds__(NTHREADS) coverage_kernel(const __grid_constant__ RenderParams P) {
+    __shared__ CoverWarp sm[NW];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned id = blockIdx.x * (unsigned)NW + warp;
+    if (id >= P.n_jobs) return;
+    CoverWarp& s = sm[warp];
+    const Job job = decode_job(P, id);
+    const TileCtx& t = job.t;
+    const AgentGeom* env_agents = P.agents + (size_t)job.e * P.A;
+    if (!env_agents[job.a].active) return;
+    if (lane < 7) {
+        Cam c;
+        load_camera(c, P.cams[job.view], P.cam[job.k], P.W, P.H);
+        if (lane == 6) s.cam = c;
+        else tile_planes(s, lane, c, t);
+    }
+    for (int i = lane; i < TILE; i += 32) load_rays(s, P, job, i);
+    for (int i = lane; i < TILE * TILE / 32; i += 32) s.mask[i] = 0u;
+    __syncwarp();
+    const Cam& c = s.cam;
+    uint32_t* occ = P.occlusion + job.view * (size_t)P.A * 2u;
+    for (int b = 0; b < P.A; ++b) {
+        if (b == job.a) continue;
+        const AgentGeom g = env_agents[b];
+        if (!g.active || !box_faces(s, c, t, g)) continue;        // its bounding sphere misses the tile's frustum
+        for (int f = 0; f < 6; ++f) {
+            const uint32_t corners = face_corners(f);
+            V3 V[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
+            uint32_t box;
+            if (!pixel_box(c, t, V, box)) continue;
+            PrimEq q;
+            if (!prim_equations(V, true, face_flags(corners), plane_normal(V, true), q)) continue;
+            const int bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+            const int w = bx1 - bx0 + 1, npx = w * (by1 - by0 + 1);
+            for (int i = lane; i < npx; i += 32) {
+                const int x = bx0 + i % w, y = by0 + i / w;
+                if (fragment(q, s.ray_x[x], s.ray_y[y], t.w_near, t.w_far)) atomicOr(&s.mask[y * (TILE / 32) + (x >> 5)], 1u << (x & 31));
+            }
+        }
+        __syncwarp();
+        uint32_t cnt = 0u;
+        for (int i = lane; i < TILE * TILE / 32; i += 32) { cnt += __popc(s.mask[i]); s.mask[i] = 0u; }
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (lane == 0 && cnt) atomicAdd(occ + 2 * b + 1, cnt);
+        __syncwarp();
+    }
+}
+
 size_t survivor_bytes_per_tile() { return sizeof(uint2) * SURV_STRIDE; }
 
 cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int sm_count, cudaStream_t stream) {
@@ -1600,11 +1680,12 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int 
     if (jobs <= 0) return cudaSuccess;
     P.n_jobs = (uint32_t)jobs;
     const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
-    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr && (P.debug_flags & 15) == 0 &&
+    const bool full = P.W % TILE == 0 && P.H % TILE == 0 && P.out_depth32 == nullptr && P.occlusion == nullptr && (P.debug_flags & 15) == 0 &&
                       (reinterpret_cast<uintptr_t>(P.out_depth) & 31u) == 0;   // 256-bit depth stores
     // (a) cull: survivors per tile
-    if (P.counters) cull_kernel<Tally><<<grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
-    else cull_kernel<NoTally><<<grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    const unsigned cull_grid = (unsigned)((jobs + NW * CULL_ROUNDS - 1) / (NW * CULL_ROUNDS));
+    if (P.counters) cull_kernel<Tally><<<cull_grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    else cull_kernel<NoTally><<<cull_grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     // (b)-(d) set-up, raster, store
@@ -1619,6 +1700,20 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int 
     if (P.counters) cooperative_kernel<Tally, false><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
     else if (full) cooperative_kernel<NoTally, true><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
     else cooperative_kernel<NoTally, false><<<cgrid, NTHREADS, sizeof(TileSmem), stream>>>(P);
+    err = cudaGetLastError();
+    if (err != cudaSuccess || !P.occlusion) return err;
+    coverage_kernel<<<grid, NTHREADS, 0, stream>>>(P);
+    return cudaGetLastError();
+}
+
+// The coverage pass alone (after the exhaustive kernel, which counts the visible pixels itself).
+cudaError_t launch_coverage_kernel(const RenderParams& P0, long long n_views, cudaStream_t stream) {
+    RenderParams P = P0;
+    const long long jobs = n_views * P.tiles_x * P.tiles_y;
+    if (jobs <= 0 || !P.occlusion) return cudaSuccess;
+    if (jobs > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    P.n_jobs = (uint32_t)jobs;
+    coverage_kernel<<<(unsigned)((jobs + NW - 1) / NW), NTHREADS, 0, stream>>>(P);
     return cudaGetLastError();
 }
 

@@ -620,3 +620,44 @@ def test_grazing_plane_flag():
     # and none of the benchmark workloads' pixels are (camera 1.5 m above the roads)
     r = oracle.render(make_config(0))
     assert (r.flag & 16).sum() == 0
+
+
+# ------------------------------------------------------------------------------------------------
+# occlusion counts (visible pixels of a road user / pixels its box would cover alone)
+# ------------------------------------------------------------------------------------------------
+def test_occlusion_counts_closed_forms():
+    """Worked by hand on the one-box scene (camera 1.5 m high at the ego's box front, 64 x 64, fx = fy = 32): a car
+    of the nominal size 12.5 m ahead shows its rear face 8 m in front of the camera as the rectangle rows 32..37 x
+    columns 28..35 = 48 pixels; its other faces project inside that rectangle."""
+    car = ego(12.5, 0.0, 0.0)
+    # alone: fully visible
+    s = single_env(np.zeros((0, 3, 3)), [], [ego(), car])
+    vis, un, sv, su = oracle.occlusion_counts(s, [0])
+    assert vis[0].tolist() == [0, 48] and un[0].tolist() == [0, 48]
+    # behind a wall that spans the whole image: fully hidden, but still 48 pixels when alone
+    wall6 = [[(6.0, -40, -5), (6.0, 40, -5), (6.0, 40, 30)], [(6.0, -40, -5), (6.0, 40, 30), (6.0, -40, 30)]]
+    s = single_env(wall6, [5, 5], [ego(), car])
+    vis, un, *_ = oracle.occlusion_counts(s, [0])
+    assert vis[0, 1] == 0 and un[0, 1] == 48
+    # a wall 3.75 m ahead of the camera (x = 6) that ends at y = 0: at depth 3.75 its edge projects to the image
+    # centre u = 32, and y > 0 is the left half -- columns 28..31 of the car are hidden, 32..35 stay: 4 x 6 = 24
+    half = [[(6.0, 0.0, -5), (6.0, 40, -5), (6.0, 40, 30)], [(6.0, 0.0, -5), (6.0, 40, 30), (6.0, 0.0, 30)]]
+    s = single_env(half, [5, 5], [ego(), car])
+    r = oracle.render(s, [0])
+    assert (r.cls[0][32:38, 28:32] == 5).all() and (r.cls[0][32:38, 32:36] == 4).all()
+    vis, un, sv, su = oracle.occlusion_counts(s, [0])
+    assert vis[0, 1] == 24 and un[0, 1] == 48
+    # a second car right behind the first (20 m ahead): it projects to a smaller rectangle inside the first
+    # one's footprint (rear face at 15.5 m: rows 32..34, half-width 0.95 * 32 / 15.5 = 1.96 px -> columns 30..33),
+    # so all of it is hidden; the first car is untouched.  The ego itself and an inactive car count nothing.
+    s = single_env(np.zeros((0, 3, 3)), [], [ego(), car, ego(20.0, 0.0, 0.0), ego(30.0, 20.0, 0.0)], active=[1, 1, 1, 0])
+    vis, un, *_ = oracle.occlusion_counts(s, [0])
+    assert vis[0].tolist() == [0, 48, 0, 0] and un[0, 1] == 48 and un[0, 2] == 3 * 4 and un[0, 0] == 0 and un[0, 3] == 0
+    # the counts of all road users add up to the vehicle-class pixels of the image
+    s = make_config(2, E=1)
+    views = [0, 5, 130, 255]
+    vis, un, sv, su = oracle.occlusion_counts(s, views)
+    r = oracle.render(s, views)
+    assert (vis.sum(1) == (r.cls == 4).reshape(len(views), -1).sum(1)).all()
+    assert (vis <= un + sv).all() and (un[vis > 0] > 0).all()
+    assert ((un > 0).sum(1) >= (vis > 0).sum(1)).all() and (un > vis).any()     # heavy occlusion: somebody is partly hidden
