@@ -1256,13 +1256,39 @@ __global__ void __launch_bounds__(NTHREADS, 5) render_kernel(const __grid_consta
 #define PIC_FSTRIP 16
 #endif
 #ifndef PIC_FPOOL
-#define PIC_FPOOL 118
+#define PIC_FPOOL 144
 #endif
 constexpr int FPOOL = PIC_FPOOL;     // records shared by the four tiles of a CTA
 constexpr int FSTRIP = PIC_FSTRIP;   // pixel rows of a strip: 16 or 8
 constexpr int FSTRIP_KEYS = TILE * FSTRIP;
 constexpr int FSTRIPS = TILE / FSTRIP;
 static_assert(FSTRIP == 16 || FSTRIP == 8, "strips of 16 or 8 rows");
+
+// The record pool of the full-tile kernel, one array per 16-byte part of a record: 17 words per
+// record instead of the 20 of an array of padded records, so more records fit beside the keys.
+struct __align__(16) RecordPool {
+    float4 nx[FPOOL], ny[FPOOL], nz[FPOOL];   // edge functions E_i = nx[i] rx + ny[i] ry + nz[i]
+    float4 w[FPOOL];                          // 1/z plane wx, wy, wz; key low word
+    uint32_t box[FPOOL];                      // pixel box (6 bits per coordinate), top-left bits, flags
+};
+
+__device__ __forceinline__ void write_record(RecordPool& pool, int slot, const PrimEq& q, uint32_t key_lo, uint32_t box, uint32_t extra) {
+    const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+    pool.nx[slot] = make_float4(q.nx[0], q.nx[1], q.nx[2], q.nx[3]);
+    pool.ny[slot] = make_float4(q.ny[0], q.ny[1], q.ny[2], q.ny[3]);
+    pool.nz[slot] = make_float4(q.nz[0], q.nz[1], q.nz[2], q.nz[3]);
+    pool.w[slot] = make_float4(q.wx, q.wy, q.wz, __uint_as_float(key_lo));
+    pool.box[slot] = bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24) | extra;
+}
+
+__device__ __forceinline__ void read_record(const RecordPool& pool, int slot, PrimEq& q, uint32_t& key_lo) {
+    const float4 r0 = pool.nx[slot], r1 = pool.ny[slot], r2 = pool.nz[slot], r3 = pool.w[slot];
+    q.nx[0] = r0.x; q.nx[1] = r0.y; q.nx[2] = r0.z; q.nx[3] = r0.w;
+    q.ny[0] = r1.x; q.ny[1] = r1.y; q.ny[2] = r1.z; q.ny[3] = r1.w;
+    q.nz[0] = r2.x; q.nz[1] = r2.y; q.nz[2] = r2.z; q.nz[3] = r2.w;
+    q.wx = r3.x; q.wy = r3.y; q.wz = r3.z;
+    key_lo = __float_as_uint(r3.w);
+}
 
 struct __align__(16) TileRef {
     size_t pixel0;       // offset of the tile's first pixel in the output images
@@ -1272,7 +1298,7 @@ struct __align__(16) TileRef {
 
 struct __align__(16) FullSmem {
     unsigned long long key[NW][FSTRIP_KEYS];  // warp w's strip of keys
-    float4 pool[FPOOL * REC / 4];
+    RecordPool pool;
     float ray_x[NW][TILE], ray_y[NW][TILE];   // ray tables of tile w
     Cam cam[NW];
     TileRef tile[NW];
@@ -1356,16 +1382,16 @@ __device__ __forceinline__ void store_strip_full(unsigned long long* key, uint8_
 
 // One strip (rows ys .. of the tile) by one warp: the tile's fragments that fall into it, then
 // the records that reach it, cell by cell.  Returns the touched 8 x 8 blocks.
-__device__ __forceinline__ uint32_t raster_strip_full(StripView& s, const float4* rec, int n_rec, int ys, float w_near, float w_far,
-                                                      int stop, int lane) {
+__device__ __forceinline__ uint32_t raster_strip_full(StripView& s, const RecordPool& pool, int first, int n_rec, int ys, float w_near,
+                                                      float w_far, int stop, int lane) {
     uint32_t touched = 0u;                       // bit (row >> 3) * 8 + (column >> 3)
     const int kbase = (lane >> 3) << 6, lsw = (lane & 7) ^ (((lane >> 3) & 1) << 2);   // see strip_cell
     for (int base = 0; base < n_rec; base += 32) {
         uint32_t bw_lane = 0u;
         bool hit = false;
         if (base + lane < n_rec) {
-            const float4* r = rec + (base + lane) * (REC / 4);
-            bw_lane = __float_as_uint(r[4].x);
+            const int slot = first + base + lane;
+            bw_lane = pool.box[slot];
             const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
             hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + FSTRIP;
             if (hit && (bw_lane & REC_TINY)) {           // a few pixels: rasterized by this lane (atomic max)
@@ -1374,7 +1400,7 @@ __device__ __forceinline__ uint32_t raster_strip_full(StripView& s, const float4
                 const int y0 = max(by0, ys) - ys, y1 = min(by1, ys + FSTRIP - 1) - ys;
                 PrimEq q;
                 uint32_t key_lo;
-                read_record(r, q, key_lo);
+                read_record(pool, slot, q, key_lo);
                 q.tl = (bw_lane >> 24) & 15u;
                 // at most TINY_MAX_PIXELS pixels: one column (w == 1), two columns, or one row
                 const int w = bx1 - bx0 + 1, npx = (stop == 7) ? 0 : w * (y1 - y0 + 1);
@@ -1396,13 +1422,12 @@ __device__ __forceinline__ uint32_t raster_strip_full(StripView& s, const float4
         for (; hits; hits &= hits - 1) {
             const int src = __ffs(hits) - 1;
             const uint32_t bw = __shfl_sync(0xffffffffu, bw_lane, src);
-            const float4* r = &rec[(base + src) * (REC / 4)];
             const int by0 = (bw >> 6) & 63, by1 = (bw >> 18) & 63;
             const int bx0 = bw & 63, bx1 = (bw >> 12) & 63;
             const int ly0 = max(by0, ys) - ys, ly1 = min(by1, ys + FSTRIP - 1) - ys;
             PrimEq q;
             uint32_t key_lo;
-            read_record(r, q, key_lo);
+            read_record(pool, first + base + src, q, key_lo);
             q.tl = (bw >> 24) & 15u;
             float thr[4];
             edge_thresholds(q.tl, thr);
@@ -1522,9 +1547,8 @@ __global__ void __launch_bounds__(NTHREADS, PIC_RENDER_CTAS) render_full_kernel(
                 uint32_t key_lo, flags;
                 fetch_survivor(s.cam[warp], P, svi.x, job.e, n_map_tris, V, Pn, key_lo, flags);
                 PrimEq q;
-                float4* r = s.pool + (my_base + i) * (REC / 4);
-                if (!prim_equations(V, flags & 1u, flags, Pn, q)) { r[4].x = __uint_as_float(REC_DEAD); continue; }
-                write_record(r, q, key_lo, svi.y, (tiny_box(svi.y) ? REC_TINY : 0u) | (record_in_range(V, P) ? REC_INRANGE : 0u));
+                if (!prim_equations(V, flags & 1u, flags, Pn, q)) { s.pool.box[my_base + i] = REC_DEAD; continue; }
+                write_record(s.pool, my_base + i, q, key_lo, svi.y, (tiny_box(svi.y) ? REC_TINY : 0u) | (record_in_range(V, P) ? REC_INRANGE : 0u));
             }
         }
         if (threadIdx.x == 0) s.next_task = 0;
@@ -1550,7 +1574,7 @@ __global__ void __launch_bounds__(NTHREADS, PIC_RENDER_CTAS) render_full_kernel(
                 if (FSTRIP == 16) { bgc[1] = __ldg(bg_cls + 8); bgz[1] = __ldg(bg_z + 8); }
             }
             sv.ray_x = s.ray_x[j]; sv.ray_y = s.ray_y[j] + ys;
-            uint32_t touched = raster_strip_full(sv, s.pool + ((bases >> (8 * j)) & 0xffu) * (REC / 4), (stop == 14) ? 0 : cj, ys, P.w_near, P.w_far, stop, lane);
+            uint32_t touched = raster_strip_full(sv, s.pool, (int)((bases >> (8 * j)) & 0xffu), (stop == 14) ? 0 : cj, ys, P.w_near, P.w_far, stop, lane);
             if (stop == 5) touched = 0xffffu;
             if (stop == 6) touched |= 0x80000000u;
             const size_t o = tr.pixel0 + (size_t)ys * P.W;
