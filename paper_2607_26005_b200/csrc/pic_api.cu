@@ -67,6 +67,9 @@ struct pic_scene {
     pic::Node* d_groups = nullptr;
     pic::Node* d_leaves = nullptr;
     pic::Prim* d_prims = nullptr;
+    uint32_t* d_cell_start = nullptr;
+    pic::Prim* d_grid_prims = nullptr;
+    pic::Node* d_large_leaves = nullptr;
     pic::AgentGeom* d_agents = nullptr;
     pic::ViewCam* d_cams = nullptr;   // [E*A*K]
     uint32_t* d_overflow = nullptr;   // [1 + E*A*K*tiles] tiles handed from the render kernel to the cooperative kernel
@@ -111,7 +114,7 @@ struct DeviceGuard {
 };
 
 void free_scene(pic_scene* s) {
-    cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims);
+    cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims); cudaFree(s->d_cell_start); cudaFree(s->d_grid_prims); cudaFree(s->d_large_leaves);
     cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_surv); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
@@ -136,6 +139,7 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.w_near = 1.0f / s->near_z; P.w_far = 1.0f / s->far_z;
     P.cls_agent = s->cls_agent; P.cls_sky = s->cls_sky; P.cls_ground = s->cls_ground;
     P.env_map = s->d_env_map; P.env_maps = s->d_env_maps; P.maps = s->d_maps; P.groups = s->d_groups; P.leaves = s->d_leaves; P.prims = s->d_prims;
+    P.cell_start = s->d_cell_start; P.grid_prims = s->d_grid_prims; P.large_leaves = s->d_large_leaves;
     P.agents = s->d_agents;
     P.cams = s->d_cams;
     P.overflow = s->d_overflow;
@@ -226,6 +230,10 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     const pic::Node* leaves = pic::hierarchy_leaves(hh, &nl);
     const pic::Node* groups = pic::hierarchy_groups(hh, &ng);
     const pic::MapInfo* maps = pic::hierarchy_maps(hh, &nm);
+    size_t ncs, ngp, nll;
+    const uint32_t* cell_start = pic::hierarchy_cell_start(hh, &ncs);
+    const pic::Prim* grid_prims = pic::hierarchy_grid_prims(hh, &ngp);
+    const pic::Node* large_leaves = pic::hierarchy_large_leaves(hh, &nll);
     s->n_prims = np; s->n_leaves = nl; s->n_groups = ng;
     const size_t n_agents = (size_t)d->E * d->A;
     int32_t* env_map = new (std::nothrow) int32_t[d->E];
@@ -243,6 +251,9 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_groups, sizeof(pic::Node) * ng);
     dmalloc((void**)&s->d_leaves, sizeof(pic::Node) * nl);
     dmalloc((void**)&s->d_prims, sizeof(pic::Prim) * np);
+    dmalloc((void**)&s->d_cell_start, sizeof(uint32_t) * ncs);
+    dmalloc((void**)&s->d_grid_prims, sizeof(pic::Prim) * ngp);
+    dmalloc((void**)&s->d_large_leaves, sizeof(pic::Node) * nll);
     dmalloc((void**)&s->d_agents, sizeof(pic::AgentGeom) * n_agents);
     dmalloc((void**)&s->d_cams, sizeof(pic::ViewCam) * n_agents * d->K);
     dmalloc((void**)&s->d_overflow, sizeof(uint32_t) * (1 + (size_t)n_agents * d->K * ((d->W + pic::TILE - 1) / pic::TILE) * ((d->H + pic::TILE - 1) / pic::TILE)));
@@ -266,6 +277,9 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     upload(s->d_groups, groups, sizeof(pic::Node) * ng);
     upload(s->d_leaves, leaves, sizeof(pic::Node) * nl);
     upload(s->d_prims, prims, sizeof(pic::Prim) * np);
+    upload(s->d_cell_start, cell_start, sizeof(uint32_t) * ncs);
+    upload(s->d_grid_prims, grid_prims, sizeof(pic::Prim) * ngp);
+    upload(s->d_large_leaves, large_leaves, sizeof(pic::Node) * nll);
     if (ce == cudaSuccess) ce = cudaMemset(s->d_status, 0, sizeof(uint32_t));
     if (ce == cudaSuccess) ce = cudaMemset(s->d_state, 0, sizeof(float) * 4 * n_agents);
     if (ce == cudaSuccess) ce = cudaMemset(s->d_dims, 0, sizeof(float) * 3 * n_agents);

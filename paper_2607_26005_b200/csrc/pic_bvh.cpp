@@ -6,6 +6,15 @@
 // grouped by GROUP_LEAVES.  Primitives much longer than the average get leaves of their own, so
 // that one long road quad does not inflate the box of its neighbouring lane markings.  The renderer tests group boxes, then
 // leaf boxes, then primitives against each view frustum.
+//
+// The cull kernel uses a second, flatter structure over the same primitives: a uniform grid on
+// the ground plane.  A primitive whose box (xy) has a half-diagonal of at most half a cell is
+// "small" and is listed under the cell that holds the centre of its box; a second copy of the
+// primitives is stored in that order, cell after cell, row-major, so the small primitives of a run
+// of cells of one grid row are one contiguous range of it (the large ones follow, leaf by leaf).
+// A view then needs one range per grid row that its frustum's footprint (widened by the largest
+// half-diagonal of a small primitive) crosses.  The few primitives too large for a cell (long road
+// quads) are kept in leaves of LARGE_LEAF_PRIMS with boxes, tested one by one.
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
@@ -21,6 +30,9 @@ struct HostHierarchy {
     std::vector<Node> leaves;
     std::vector<Node> groups;
     std::vector<MapInfo> maps;
+    std::vector<uint32_t> cell_start;
+    std::vector<Prim> grid_prims;             // the same primitives once more, in grid order
+    std::vector<Node> large_leaves;
 };
 
 namespace {
@@ -93,6 +105,83 @@ void box_of_prim(const Prim& p, float lo[3], float hi[3]) {
             lo[c] = std::min(lo[c], p.v[3 * k + c]);
             hi[c] = std::max(hi[c], p.v[3 * k + c]);
         }
+}
+
+// The uniform grid and the large-primitive leaves of one map (primitives mi.prim_begin .. mi.prim_end of h.prims).
+void build_grid(HostHierarchy& h, MapInfo& mi) {
+    const size_t p0 = mi.prim_begin, np = mi.prim_end - mi.prim_begin;
+    std::vector<float> cx(np), cy(np), half(np);
+    float x0 = 0.f, y0 = 0.f, x1 = 0.f, y1 = 0.f;
+    for (size_t i = 0; i < np; ++i) {
+        float lo[3], hi[3];
+        box_of_prim(h.prims[p0 + i], lo, hi);
+        cx[i] = 0.5f * (lo[0] + hi[0]); cy[i] = 0.5f * (lo[1] + hi[1]);
+        // (rounded up a little: the margin derived from it must not fall short)
+        half[i] = 0.5f * (float)std::sqrt((double)(hi[0] - lo[0]) * (hi[0] - lo[0]) + (double)(hi[1] - lo[1]) * (hi[1] - lo[1])) * 1.0001f + 1e-6f;
+        if (i == 0 || cx[i] < x0) x0 = cx[i];
+        if (i == 0 || cx[i] > x1) x1 = cx[i];
+        if (i == 0 || cy[i] < y0) y0 = cy[i];
+        if (i == 0 || cy[i] > y1) y1 = cy[i];
+    }
+    // cell size: about one primitive per cell, at most 1024 x 1024 cells
+    const double ex = std::max((double)x1 - x0, 1e-3), ey = std::max((double)y1 - y0, 1e-3);
+    double cell = std::sqrt(ex * ey / (double)std::max<size_t>(np, 1));
+    cell = std::max(cell, std::max(ex, ey) / 1024.0);
+    cell = std::max(cell, 1e-3);
+    const uint32_t nx = (uint32_t)std::min(1024.0, std::floor(ex / cell) + 1.0), ny = (uint32_t)std::min(1024.0, std::floor(ey / cell) + 1.0);
+    mi.gx0 = x0; mi.gy0 = y0; mi.cell = (float)cell; mi.inv_cell = (float)(1.0 / cell); mi.nx = nx; mi.ny = ny;
+    mi.cell_begin = (uint32_t)h.cell_start.size();
+    // small primitives by cell; the cell of a centre is computed exactly as the kernel computes the cells
+    // of a range (same float32 expression), so a centre can never fall outside the range that covers it
+    std::vector<uint32_t> cell_of(np, 0xffffffffu);
+    std::vector<uint32_t> count((size_t)nx * ny + 1, 0u);
+    float margin = 0.f;
+    std::vector<Item> large;
+    for (size_t i = 0; i < np; ++i) {
+        if (half[i] <= 0.5f * mi.cell) {
+            const float fx = std::floor((cx[i] - mi.gx0) * mi.inv_cell), fy = std::floor((cy[i] - mi.gy0) * mi.inv_cell);
+            const uint32_t ix = (uint32_t)std::min((float)(nx - 1), std::max(0.f, fx)), iy = (uint32_t)std::min((float)(ny - 1), std::max(0.f, fy));
+            cell_of[i] = iy * nx + ix;
+            ++count[cell_of[i] + 1];
+            margin = std::max(margin, half[i]);
+        } else {
+            uint64_t code = 0;
+            const double ext = std::max(ex, ey);
+            code |= spread21((uint64_t)std::min(2097151.0, std::max(0.0, (cx[i] - x0) / ext * 2097152.0)));
+            code |= spread21((uint64_t)std::min(2097151.0, std::max(0.0, (cy[i] - y0) / ext * 2097152.0))) << 1;
+            large.push_back({code, (uint32_t)i});
+        }
+    }
+    // a float32 centre and the kernel's float32 range arithmetic differ by rounding: widen the margin
+    mi.margin = margin * 1.0001f + 1e-4f * (1.f + std::fabs(x0) + std::fabs(y0) + (float)std::max(ex, ey));
+    for (size_t c = 0; c < (size_t)nx * ny; ++c) count[c + 1] += count[c];
+    const size_t base = h.grid_prims.size();
+    h.grid_prims.resize(base + count[(size_t)nx * ny]);
+    {
+        std::vector<uint32_t> fill(count.begin(), count.end() - 1);
+        for (size_t i = 0; i < np; ++i)
+            if (cell_of[i] != 0xffffffffu) h.grid_prims[base + fill[cell_of[i]]++] = h.prims[p0 + i];
+    }
+    for (size_t c = 0; c <= (size_t)nx * ny; ++c) h.cell_start.push_back((uint32_t)(base + count[c]));
+    // large primitives: Morton order, leaves of LARGE_LEAF_PRIMS
+    std::sort(large.begin(), large.end(), [](const Item& a, const Item& b) { return a.code != b.code ? a.code < b.code : a.id < b.id; });
+    mi.large_begin = (uint32_t)h.large_leaves.size();
+    for (size_t i = 0; i < large.size(); i += LARGE_LEAF_PRIMS) {
+        Node leaf;
+        leaf.first = (uint32_t)h.grid_prims.size();
+        leaf.count = (uint32_t)std::min<size_t>(LARGE_LEAF_PRIMS, large.size() - i);
+        for (uint32_t k = 0; k < leaf.count; ++k) {
+            float lo[3], hi[3];
+            box_of_prim(h.prims[p0 + large[i + k].id], lo, hi);
+            for (int c = 0; c < 3; ++c) {
+                leaf.lo[c] = (k == 0) ? lo[c] : std::min(leaf.lo[c], lo[c]);
+                leaf.hi[c] = (k == 0) ? hi[c] : std::max(leaf.hi[c], hi[c]);
+            }
+            h.grid_prims.push_back(h.prims[p0 + large[i + k].id]);
+        }
+        h.large_leaves.push_back(leaf);
+    }
+    mi.large_end = (uint32_t)h.large_leaves.size();
 }
 
 }  // namespace
@@ -211,6 +300,7 @@ HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const fl
             h->groups.push_back(g);
         }
         mi.group_end = (uint32_t)h->groups.size();
+        build_grid(*h, mi);
         if (h->prims.size() >= (1ull << 28)) {
             std::snprintf(err, err_len, "more than 2^28 primitives in one scene");
             delete h;
@@ -225,5 +315,8 @@ const Prim* hierarchy_prims(const HostHierarchy* h, size_t* n) { *n = h->prims.s
 const Node* hierarchy_leaves(const HostHierarchy* h, size_t* n) { *n = h->leaves.size(); return h->leaves.data(); }
 const Node* hierarchy_groups(const HostHierarchy* h, size_t* n) { *n = h->groups.size(); return h->groups.data(); }
 const MapInfo* hierarchy_maps(const HostHierarchy* h, size_t* n) { *n = h->maps.size(); return h->maps.data(); }
+const uint32_t* hierarchy_cell_start(const HostHierarchy* h, size_t* n) { *n = h->cell_start.size(); return h->cell_start.data(); }
+const Prim* hierarchy_grid_prims(const HostHierarchy* h, size_t* n) { *n = h->grid_prims.size(); return h->grid_prims.data(); }
+const Node* hierarchy_large_leaves(const HostHierarchy* h, size_t* n) { *n = h->large_leaves.size(); return h->large_leaves.data(); }
 
 }  // namespace pic

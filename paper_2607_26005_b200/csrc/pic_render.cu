@@ -35,6 +35,8 @@
 //
 // Cameras (one 64-byte record per view) and per-camera ray / background tables are prepared by
 // the agent and rig kernels, so the prologues are a few loads.
+#include <cstddef>
+
 #include "pic_device.cuh"
 
 namespace pic {
@@ -663,8 +665,7 @@ __device__ __forceinline__ void flush_counters(const RenderParams& P, const Tall
 constexpr int POOL = 128;         // records shared by the NW tiles of a CTA
 constexpr int STRIP = 16;         // pixel rows a warp rasterizes at a time
 constexpr int STRIP_KEYS = TILE * STRIP;
-constexpr int W_LEAF = 256;       // per-warp front-end lists (they live in the key buffer, 8 KB per warp)
-constexpr int W_FACE = 384;
+constexpr int W_FACE = 384;        // box-face items of a tile in the cull kernel
 // Survivor buffer, SURV_STRIDE uint2 per tile: a 16-byte head (counts; work counts), then W_SURV
 // entries (id, pixel box).  Survivors whose pixel box holds more than TINY_MAX_PIXELS pixel centres
 // fill the list from the front, the others from the back; head.x = front count | back count << 16,
@@ -672,18 +673,24 @@ constexpr int W_FACE = 384;
 constexpr int SURV_STRIDE = 128;
 constexpr int W_SURV = SURV_STRIDE - 2;
 constexpr uint32_t SURV_OVERFLOW = 0xffffffffu;
-constexpr uint32_t SURV_FACE = 0x80000000u;   // survivor id: primitive index, or SURV_FACE | agent << 3 | face
+constexpr uint32_t SURV_FACE = 0x80000000u;   // survivor id: index into grid_prims, or SURV_FACE | agent << 3 | face
 constexpr uint32_t REC_TINY = 1u << 28, REC_DEAD = 1u << 29;   // flags in the box word of a record
 constexpr uint32_t REC_INRANGE = 1u << 30;   // every covered pixel is within [near, far]: no per-pixel range test
 
+constexpr int W_LARGE = 64;       // visible leaves of the large-primitive list
 struct __align__(16) FrontLists {
-    uint32_t leaf[W_LEAF];                    // first primitive << 4 | count
-    uint32_t face[W_FACE];                    // agent << 3 | face
-    float plane[6][4];
+    float plane[6][4];                        // (read as float4: kept first, 16-byte aligned)
     float side[4][4];
     Cam cam;
-    int n_face, pad[3];
+    float seg[10][6];                         // footprint segments: x, y, dx, dy, 1 / dy, unused
+    float pt[5][2];                           // footprint corners (ego-relative xy): apex, four far corners
+    uint32_t face[W_FACE];                    // agent << 3 | face
+    uint32_t lleaf[W_LARGE];                  // visible large-primitive leaves: first << 3 | count
+    uint32_t row_first[32];                   // grid rows of a pass: first entry of the row's range in cell_prims
+    uint32_t row_off[33];                     //   and the number of candidates before the row (the total at [32])
+    int n_face;
 };
+static_assert(offsetof(FrontLists, plane) % 16 == 0 && offsetof(FrontLists, side) % 16 == 0, "planes are read with 128-bit loads");
 
 struct __align__(16) FusedSmem {
     unsigned long long key[NW][STRIP_KEYS];   // warp w's strip of keys; during the front end, its FrontLists
@@ -774,21 +781,25 @@ __device__ __forceinline__ void append_survivor(uint2* __restrict__ surv, bool k
     n_tiny += __popc(mt);
 }
 
-// Front end of one tile by one warp: fills f.leaf / f.face and the survivor list.  Returns the
-// survivor counts (front | back << 16), or -1 if a list overflowed (the tile then goes to the
-// cooperative kernel).
-// Loads that do not depend on one another are issued together (the first group boxes and the
-// first agents before the camera is even set up; the leaf boxes of three visible groups, two
-// candidates per lane), so that a pass waits for memory once.
+// Front end of one tile by one warp: fills the survivor list.  Returns the survivor counts
+// (front | back << 16), or -1 if a list overflowed (the tile then goes to the cooperative kernel).
+//
+// Map primitives come from the uniform grid: the footprint of the tile's frustum on the ground
+// plane is the convex hull of the apex and the four far corners; for every grid row the footprint
+// (widened by the map's margin) crosses, the small primitives of the cells it covers are one
+// contiguous range of cell_prims.  The ranges of up to 32 rows are laid end to end and tested two
+// candidates per lane at a time (camera space, pixel box).  The large primitives are found through
+// their leaves (a lane per leaf box against the six frustum planes), the other agents' boxes as
+// bounding spheres.  Loads that do not depend on one another are issued together.
 template <class TL>
 __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ surv, const RenderParams& P, const Job& job,
                                           const MapInfo& mi, int lane, TL& n) {
     const int stop = PIC_STOP(P);
     const TileCtx& t = job.t;
-    Node gn0;
-    gn0.first = 0; gn0.count = 0;
-    if (mi.group_begin + lane < mi.group_end) gn0 = load_node(P.groups + mi.group_begin + lane);
     const AgentGeom* env_agents = P.agents + (size_t)job.e * P.A;
+    Node ln0;
+    ln0.first = 0; ln0.count = 0;
+    if (mi.large_begin + lane < mi.large_end) ln0 = load_node(P.large_leaves + mi.large_begin + lane);
     AgentGeom ag0, ag1;
     ag0.active = 0u; ag1.active = 0u;
     if (lane < P.A) ag0 = load_agent(env_agents + lane);
@@ -798,50 +809,85 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
         load_camera(c, P.cams[job.view], P.cam[job.k], P.W, P.H);
         if (lane == 6) { f.cam = c; f.n_face = 0; }
         else tile_planes(f, lane, c, t);
+        if (lane < 5) {
+            // footprint corner `lane`: the apex, or a corner of the tile's frustum at depth far (a little beyond)
+            const float F = lane ? t.far_z * 1.001f : 0.f;
+            const float xc = ((float)((lane & 1) ? t.x0 + t.tw : t.x0) - c.cx) / c.focx * F;
+            const float yc = ((float)((lane & 2) ? t.y0 + t.th : t.y0) - c.cy) / c.focy * F;
+            f.pt[lane][0] = c.mwx + c.rx * xc + c.dx * yc + c.fx_ * F;
+            f.pt[lane][1] = c.mwy + c.ry * xc + c.dy * yc + c.fy_ * F;
+        }
+    }
+    __syncwarp();
+    if (lane < 10) {
+        // segment between two of the five corners (every pair: the hull's edges are among them, the others lie inside it)
+        const int i = lane < 4 ? 0 : lane < 7 ? 1 : lane < 9 ? 2 : 3, j = lane < 4 ? lane + 1 : lane < 7 ? lane - 2 : lane < 9 ? lane - 4 : 4;
+        const float px = f.pt[i][0], py = f.pt[i][1], dx = f.pt[j][0] - px, dy = f.pt[j][1] - py;
+        f.seg[lane][0] = px; f.seg[lane][1] = py; f.seg[lane][2] = dx; f.seg[lane][3] = dy;
+        f.seg[lane][4] = dy != 0.f ? 1.f / dy : 0.f; f.seg[lane][5] = 0.f;
     }
     __syncwarp();
     if (stop == 11) return 0;
     const Cam& c = f.cam;
-    float4 pl[6];
+    int n_big = 0, n_tiny = 0;
+    // ---- the grid rows crossed by the widened footprint; the range of a row's cells in grid_prims
+    const float margin = mi.margin, gx0 = sub(mi.gx0, c.px), gy0 = sub(mi.gy0, c.py);
+    float ylo = f.pt[0][1], yhi = ylo;
 #pragma unroll
-    for (int p = 0; p < 6; ++p) pl[p] = *reinterpret_cast<const float4*>(f.plane[p]);
-    const float epx = c.px, epy = c.py;
-    // ---- hierarchy: 32 groups per pass; the leaves of three visible groups at a time, one per lane
-    int n_leaf = 0;
-    for (uint32_t g0 = mi.group_begin; g0 < mi.group_end; g0 += 32) {
-        const uint32_t g = g0 + lane;
-        bool vis = false;
-        Node gn;
-        gn.first = 0; gn.count = 0;
-        if (g < mi.group_end) { gn = (g0 == mi.group_begin) ? gn0 : load_node(P.groups + g); vis = box_visible_reg(pl, epx, epy, gn); ++n.grp; }
-        unsigned gm = __ballot_sync(0xffffffffu, vis);
-        while (gm) {
-            Node lf[3];
-            bool lvis[3];
+    for (int k = 1; k < 5; ++k) { ylo = fminf(ylo, f.pt[k][1]); yhi = fmaxf(yhi, f.pt[k][1]); }
+    const float fr0 = floorf((ylo - margin - gy0) * mi.inv_cell), fr1 = floorf((yhi + margin - gy0) * mi.inv_cell);
+    const int row_lo = (int)fmaxf(fr0, 0.f), row_hi = (int)fminf(fr1, (float)mi.ny - 1.f);     // (empty if the footprint misses the grid)
+    auto row_range = [&](int row, uint32_t& first, uint32_t& cnt) {
+        first = 0u; cnt = 0u;
+        if (row > row_hi) return;
+        ++n.grp;
+        const float blo = gy0 + (float)row * mi.cell - margin, bhi = blo + mi.cell + 2.f * margin;
+        float xlo = 3e38f, xhi = -3e38f;
 #pragma unroll
-            for (int u = 0; u < 3; ++u) {
-                const int src = gm ? __ffs(gm) - 1 : 0;
-                const bool have = gm != 0u;
-                gm &= gm - 1;
-                const uint32_t first = __shfl_sync(0xffffffffu, gn.first, src);
-                const uint32_t cnt = have ? __shfl_sync(0xffffffffu, gn.count, src) : 0u;
-                lvis[u] = lane < (int)cnt;
-                lf[u].first = 0; lf[u].count = 0;
-                if (lvis[u]) lf[u] = load_node(P.leaves + first + lane);
-            }
-#pragma unroll
-            for (int u = 0; u < 3; ++u) {
-                if (lvis[u]) { lvis[u] = box_visible_reg(pl, epx, epy, lf[u]); ++n.leaf; }
-                const unsigned lm = __ballot_sync(0xffffffffu, lvis[u]);
-                if (lvis[u]) {
-                    const int slot = n_leaf + __popc(lm & ((1u << lane) - 1u));
-                    if (slot < W_LEAF) f.leaf[slot] = (lf[u].first << 4) | lf[u].count;
-                }
-                n_leaf += __popc(lm);
+        for (int k = 0; k < 10; ++k) {
+            const float px = f.seg[k][0], py = f.seg[k][1], dx = f.seg[k][2], dy = f.seg[k][3], idy = f.seg[k][4];
+            const float ya = fminf(py, py + dy), yb = fmaxf(py, py + dy);
+            if (yb >= blo && ya <= bhi) {
+                const float ta = (blo - py) * idy, tb = (bhi - py) * idy;
+                const float t0 = dy != 0.f ? fminf(fmaxf(fminf(ta, tb), 0.f), 1.f) : 0.f, t1 = dy != 0.f ? fminf(fmaxf(fmaxf(ta, tb), 0.f), 1.f) : 1.f;
+                const float xa = px + t0 * dx, xb = px + t1 * dx;
+                xlo = fminf(xlo, fminf(xa, xb)); xhi = fmaxf(xhi, fmaxf(xa, xb));
             }
         }
+        if (xlo <= xhi) {
+            const float fx0 = floorf((xlo - margin - gx0) * mi.inv_cell), fx1 = floorf((xhi + margin - gx0) * mi.inv_cell);
+            if (fx1 >= 0.f && fx0 <= (float)mi.nx - 1.f) {
+                const uint32_t ix0 = (uint32_t)fmaxf(fx0, 0.f), ix1 = (uint32_t)fminf(fx1, (float)mi.nx - 1.f);
+                const uint32_t* cs = P.cell_start + mi.cell_begin + (uint32_t)row * mi.nx;
+                first = __ldg(cs + ix0);
+                cnt = __ldg(cs + ix1 + 1) - first;
+            }
+        }
+    };
+    // the first 32 rows' ranges are requested now; the boxes below are tested while the loads are under way
+    uint32_t first0, cnt0;
+    row_range(row_lo + lane, first0, cnt0);
+    // ---- the large primitives' leaves: a lane per leaf box against the six frustum planes
+    int n_ll = 0;
+    {
+        float4 pl[6];
+#pragma unroll
+        for (int p = 0; p < 6; ++p) pl[p] = *reinterpret_cast<const float4*>(f.plane[p]);
+        for (uint32_t l0 = mi.large_begin; l0 < mi.large_end; l0 += 32) {
+            const uint32_t l = l0 + lane;
+            bool vis = false;
+            Node ln;
+            ln.first = 0; ln.count = 0;
+            if (l < mi.large_end) { ln = (l0 == mi.large_begin) ? ln0 : load_node(P.large_leaves + l); vis = box_visible_reg(pl, c.px, c.py, ln); ++n.leaf; }
+            const unsigned m = __ballot_sync(0xffffffffu, vis);
+            if (vis) {
+                const int slot = n_ll + __popc(m & ((1u << lane) - 1u));
+                if (slot < W_LARGE) f.lleaf[slot] = (ln.first << 3) | ln.count;
+            }
+            n_ll += __popc(m);
+        }
+        if (n_ll > W_LARGE) return -1;
     }
-    if (stop == 12) return 0;
     // ---- other agents' boxes, two per lane at a time
     for (int b0 = 0; b0 < P.A; b0 += 64) {
         if (b0 > 0) {
@@ -862,47 +908,83 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
             }
         }
     }
-    __syncwarp();
-    const int n_face = f.n_face;
-    if (n_leaf > W_LEAF || n_face > W_FACE) return -1;
-    if (stop == 13) return 0;
-    // ---- candidates: camera space, pixel box; survivors are compacted.  Map primitives two per
-    // lane at a time, then the box faces.
-    const int n_prim_items = n_leaf * LEAF_PRIMS;
-    int n_big = 0, n_tiny = 0;
-    for (int i0 = 0; i0 < n_prim_items; i0 += 64) {
-        float v[2][12];
-        bool have[2];
-        uint32_t id[2] = {0u, 0u};
+    if (stop == 12) return 0;
+    // ---- candidates of the grid rows, 32 rows per pass: camera space, pixel box; survivors are compacted
+    for (int r0 = row_lo; r0 <= row_hi; r0 += 32) {
+        uint32_t first = first0, cnt = cnt0;
+        if (r0 != row_lo) row_range(r0 + lane, first, cnt);
+        uint32_t incl = cnt;
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int i = i0 + 32 * u + lane;
-            have[u] = false;
-            if (i < n_prim_items) {
-                const uint32_t lf = f.leaf[i / LEAF_PRIMS];
-                const uint32_t j = i % LEAF_PRIMS;
-                if (j < (lf & 15u)) {
-                    have[u] = true;
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        const int total = (int)__shfl_sync(0xffffffffu, incl, 31);
+        __syncwarp();
+        f.row_first[lane] = first;
+        f.row_off[lane] = incl - cnt;
+        if (lane == 31) f.row_off[32] = incl;
+        __syncwarp();
+        for (int i0 = 0; i0 < total; i0 += 64) {         // two candidates per lane at a time
+            float v[2][12];
+            bool have[2];
+            uint32_t id[2] = {0u, 0u};
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int i = i0 + 32 * u + lane;
+                have[u] = i < total;
+                if (have[u]) {
+                    int r = 0;
+#pragma unroll
+                    for (int st = 16; st; st >>= 1)
+                        if (f.row_off[r + st] <= (uint32_t)i) r += st;
+                    id[u] = f.row_first[r] + ((uint32_t)i - f.row_off[r]);
                     uint32_t key_lo, flags;
-                    id[u] = (lf >> 4) + j;
-                    load_prim(P.prims + id[u], v[u], key_lo, flags);
+                    load_prim(P.grid_prims + id[u], v[u], key_lo, flags);
                 }
             }
-        }
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            uint32_t box = 0;
-            bool keep = false;
-            if (have[u]) {
+            for (int u = 0; u < 2; ++u) {
+                uint32_t box = 0;
+                bool keep = false;
+                if (have[u]) {
+                    V3 V[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[u][3 * q], v[u][3 * q + 1], v[u][3 * q + 2]);
+                    ++n.tested;
+                    keep = pixel_box(c, t, V, box);
+                }
+                append_survivor(surv, keep, id[u], box, n_big, n_tiny, lane);
+            }
+        }
+    }
+    // ---- the primitives of the visible large leaves
+    __syncwarp();
+    for (int i0 = 0; i0 < n_ll * LARGE_LEAF_PRIMS; i0 += 32) {
+        const int i = i0 + lane;
+        uint32_t box = 0, id = 0;
+        bool keep = false;
+        if (i < n_ll * LARGE_LEAF_PRIMS) {
+            const uint32_t lf = f.lleaf[i / LARGE_LEAF_PRIMS];
+            const uint32_t j = i % LARGE_LEAF_PRIMS;
+            if (j < (lf & 7u)) {
+                id = (lf >> 3) + j;
+                float v[12];
+                uint32_t key_lo, flags;
+                load_prim(P.grid_prims + id, v, key_lo, flags);
                 V3 V[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[u][3 * q], v[u][3 * q + 1], v[u][3 * q + 2]);
+                for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
                 ++n.tested;
                 keep = pixel_box(c, t, V, box);
             }
-            append_survivor(surv, keep, id[u], box, n_big, n_tiny, lane);
         }
+        append_survivor(surv, keep, id, box, n_big, n_tiny, lane);
     }
+    __syncwarp();
+    const int n_face = f.n_face;
+    if (n_face > W_FACE) return -1;
+    if (stop == 13) return 0;
     for (int i0 = 0; i0 < n_face; i0 += 32) {
         const int i = i0 + lane;
         uint32_t box = 0, it = 0;
@@ -929,7 +1011,7 @@ __device__ __forceinline__ void fetch_survivor(const Cam& c, const RenderParams&
                                                V3 (&V)[4], V3& Pn, uint32_t& key_lo, uint32_t& flags) {
     if (!(id & SURV_FACE)) {
         float v[12];
-        load_prim(P.prims + id, v, key_lo, flags);
+        load_prim(P.grid_prims + id, v, key_lo, flags);
 #pragma unroll
         for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
         Pn = plane_normal_world(c, v, flags & 1u);
@@ -1099,7 +1181,7 @@ struct __align__(16) CullSmem {
 };
 
 #ifndef PIC_CULL_CTAS
-#define PIC_CULL_CTAS 5
+#define PIC_CULL_CTAS 6
 #endif
 #ifndef PIC_CULL_ROUNDS
 #define PIC_CULL_ROUNDS 1

@@ -10,6 +10,7 @@ constexpr int MAX_CAMS = 16;    // cameras per rig
 constexpr int LEAF_PRIMS = 8;   // primitives per leaf (8 threads per leaf in the cull pass)
 constexpr int LONG_LEAF_PRIMS = 8;   // long primitives get leaves of their own so the others' boxes stay tight
 constexpr int GROUP_LEAVES = 32;     // leaves per group (one per lane)
+constexpr int LARGE_LEAF_PRIMS = 4;  // primitives per leaf of the large-primitive list
 
 // Map primitive in hierarchy order: a triangle, or a planar convex quad fused from two consecutive
 // triangles of the input that share an edge (same class).  64 bytes, read as four 128-bit loads.
@@ -35,8 +36,16 @@ struct MapInfo {
     uint32_t n_tris;                   // triangles of the map as given (box indices start here)
     uint32_t prim_begin;               // first primitive (used by the exhaustive kernel)
     uint32_t prim_end;
-    uint32_t pad[3];
+    // uniform grid over the map's ground-plane extent (the cull kernel's structure, see pic_bvh.cpp)
+    uint32_t cell_begin;               // first entry of this map in the cell-start array (nx * ny + 1 entries)
+    uint32_t nx, ny;                   // cells per row, rows
+    float gx0, gy0;                    // corner of cell (0, 0)
+    float cell, inv_cell;              // cell size, its reciprocal
+    float margin;                      // no small primitive reaches farther than this from the centre of its box (xy)
+    uint32_t large_begin, large_end;   // range in the large-primitive leaves
+    uint32_t pad;
 };
+static_assert(sizeof(MapInfo) == 64, "MapInfo must be 64 bytes");
 
 // Per-agent geometry written once per render by the agent kernel; 32 bytes.
 struct AgentGeom {
@@ -84,6 +93,9 @@ struct RenderParams {
     const Node* groups;
     const Node* leaves;
     const Prim* prims;
+    const uint32_t* cell_start;     // grid: per map nx * ny + 1 offsets into grid_prims
+    const Prim* grid_prims;         // the primitives in grid order: small ones cell by cell (row-major), then the large ones leaf by leaf
+    const Node* large_leaves;       // boxes over up to LARGE_LEAF_PRIMS consecutive large primitives of grid_prims
     const AgentGeom* agents;
     const ViewCam* cams;            // [E*A*K]
     RigTables rig;
@@ -109,5 +121,8 @@ const Prim* hierarchy_prims(const HostHierarchy*, size_t* n);
 const Node* hierarchy_leaves(const HostHierarchy*, size_t* n);
 const Node* hierarchy_groups(const HostHierarchy*, size_t* n);
 const MapInfo* hierarchy_maps(const HostHierarchy*, size_t* n);
+const uint32_t* hierarchy_cell_start(const HostHierarchy*, size_t* n);
+const Prim* hierarchy_grid_prims(const HostHierarchy*, size_t* n);
+const Node* hierarchy_large_leaves(const HostHierarchy*, size_t* n);
 
 }  // namespace pic

@@ -187,7 +187,9 @@ def test_counters_are_plausible(gu):
         assert cnt[10] <= 0.2 * V
         *_, cnt_coop = g.render(counters=True, debug_flags=4)
         assert cnt_coop[0] == V and cnt_coop[10] == V
-        assert cnt_coop[4] == cnt[4] and cnt_coop[3] == cnt[3]
+        # both routes set up the same primitives; the cull kernel finds its candidates through the uniform grid,
+        # the cooperative kernel through the box hierarchy, so the numbers of candidates tested differ
+        assert cnt_coop[4] == cnt[4] and 0 < cnt[3] < cnt_coop[3]
     finally:
         g.close()
 
