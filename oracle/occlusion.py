@@ -49,7 +49,7 @@ def occlusion_counts(scene, view_ids: Optional[Sequence[int]] = None, poses: Opt
         n_map = t1 - t0
         idx = full.index[i]
         owner = np.where(idx >= n_map, (idx - n_map) // 12, -1)
-        flagged = (full.flag[i] & 15) != 0
+        flagged = (full.flag[i] & 47) != 0
         for b in range(s.A):
             if b == a or not s.active[e, b]:
                 continue

@@ -39,6 +39,16 @@
  *                 ill-conditioned in float32 -- the per-pixel kappa output lets a comparison widen
  *                 its depth tolerance to 5e-7 * kappa, and depth gaps are judged with that width.
  *  O9 stepping    explicit-Euler kinematic bicycle update (pico_step).
+ *  O10 road users and signals (Sec. 3.2, "Rendering features for driving": pedestrians, cyclists and
+ *                 vehicles each in its own hue; traffic lights as disks visible only within a limited
+ *                 angular range).  The paper gives neither formula, so the reading is: every agent may
+ *                 carry its own class id (else the scene-wide one); a map triangle may carry a limit
+ *                 c = cos(theta_max) > 0, and is then drawn in a view only if n.d >= c, where n is its
+ *                 unit normal (V1-V0)x(V2-V0) by the order of its vertices and d the unit vector from
+ *                 its centroid to the camera centre -- otherwise it is absent from that view, for all
+ *                 pixels.  c = 0 (or no array) is the ordinary two-sided triangle.  A triangle within
+ *                 1e-5 of its limit is drawn according to the exact comparison, and every pixel it
+ *                 covers (or would cover) and could win is flagged (bit 32).
  *
  * Parity pins: tests/test_oracle_*.py (closed forms, invariants, an independent ray caster,
  * hand-counted tiny scenes, numpy's binary16 conversion).  No function here is unpinned.
@@ -73,6 +83,8 @@ typedef struct {
     double kappa;     /* O8 (v): max|V_i| |N| / D, how close the primitive's plane passes by the camera centre */
     int32_t index;    /* global primitive index (O3) */
     uint8_t cls;
+    uint8_t ghost;    /* O10: just outside its angular range -- not drawn, but its pixels are flagged */
+    uint8_t unsure;   /* O10: within 1e-5 of its angular limit, on either side */
 } prim_t;
 
 typedef struct {
@@ -129,6 +141,18 @@ static void setup_prim(prim_t* p, v3 V0, v3 V1, v3 V2, int32_t index, uint8_t cl
     }
     p->index = index;
     p->cls = cls;
+    p->ghost = 0;
+    p->unsure = 0;
+}
+
+/* O10: cosine of the angle between the triangle's normal (by vertex order) and the direction from its
+   centroid to the camera centre (the origin of camera space). */
+static double facing_cosine(v3 V0, v3 V1, v3 V2) {
+    v3 nrm = v3_cross(v3_sub(V1, V0), v3_sub(V2, V0));
+    v3 g = { (V0.x + V1.x + V2.x) / 3.0, (V0.y + V1.y + V2.y) / 3.0, (V0.z + V1.z + V2.z) / 3.0 };
+    double nn = v3_norm(nrm), gn = v3_norm(g);
+    if (nn == 0.0 || gn == 0.0) return -2.0;        /* degenerate, or the camera sits on the centroid: never in range */
+    return -v3_dot(nrm, g) / (nn * gn);
 }
 
 /* O3: the 12 triangles of agent b's box, in world coordinates. */
@@ -212,7 +236,9 @@ static int meets_frustum(v3 V0, v3 V1, v3 V2, double tx, double ty, double near,
  *   out_depth  f64     O5/O6 depth (metres along the optical axis)
  *   out_f16    u16     O7 binary16 bits of the depth
  *   out_index  i32     global index of the winning primitive, -1 for background
- *   out_flag   u8      O8 bit mask: 1 edge, 2 depth gap, 4 near/far plane, 8 horizon, 16 grazing plane (informative)
+ *   out_flag   u8      O8 bit mask: 1 edge, 2 depth gap, 4 near/far plane, 8 horizon, 16 grazing plane (informative),
+ *                      32 a triangle at the limit of its angular range (O10)
+ *   agent_classes u8 [E,A] or NULL (every agent has class agent_class); tri_vis_cos f32 [N] or NULL (O10)
  *   out_kappa  f64     conditioning of the winner's depth: max|V_i| |N| / D of its plane (0 for background);
  *                      a float32 renderer's depth may be off by about 5e-7 * kappa relative
  *   counts     i64 [n_views,4]: primitives meeting the frustum, primitives with >=1 kept
@@ -224,6 +250,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 const float* tri_xyz, const uint8_t* tri_class,
                 int agent_class, int sky_class, int ground_class,
                 const float* poses, const float* dims, const uint8_t* active, const float* rig,
+                const uint8_t* agent_classes, const float* tri_vis_cos,
                 int n_views, const int64_t* view_ids,
                 uint8_t* out_class, double* out_depth, uint16_t* out_f16, int32_t* out_index,
                 uint8_t* out_flag, double* out_kappa, int64_t* counts, int n_threads)
@@ -275,7 +302,15 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
             v3 X0 = { p[0], p[1], p[2] }, X1 = { p[3], p[4], p[5] }, X2 = { p[6], p[7], p[8] };
             v3 V0 = to_camera(&c, X0), V1 = to_camera(&c, X1), V2 = to_camera(&c, X2);
             setup_prim(&prim[np], V0, V1, V2, (int32_t)t, tri_class[t0 + t]);
-            if (prim[np].D != 0.0 && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
+            if (tri_vis_cos && tri_vis_cos[t0 + t] > 0.0f) {          /* O10: one-sided, limited angular range */
+                double lim = (double)tri_vis_cos[t0 + t], cosang = facing_cosine(V0, V1, V2);
+                if (fabs(cosang - lim) <= REL_TOL) prim[np].unsure = 1;
+                if (!(cosang >= lim)) {
+                    if (prim[np].unsure) prim[np].ghost = 1;
+                    else prim[np].D = 0.0;                             /* absent from this view */
+                }
+            }
+            if (prim[np].D != 0.0 && !prim[np].ghost && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
             ++np;
         }
         for (int b = 0; b < A; ++b) {
@@ -285,7 +320,8 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
             box_triangles(poses + 3 * ((size_t)e * A + b), dims + 3 * ((size_t)e * A + b), tri);
             for (int t = 0; t < 12; ++t) {
                 v3 V0 = to_camera(&c, tri[t][0]), V1 = to_camera(&c, tri[t][1]), V2 = to_camera(&c, tri[t][2]);
-                setup_prim(&prim[np], V0, V1, V2, (int32_t)(n_map + 12 * b + t), (uint8_t)agent_class);
+                setup_prim(&prim[np], V0, V1, V2, (int32_t)(n_map + 12 * b + t),
+                           agent_classes ? agent_classes[(size_t)e * A + b] : (uint8_t)agent_class);
                 if (prim[np].D != 0.0 && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
                 ++np;
             }
@@ -302,7 +338,7 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                 double z_win = 0.0, k_win = 0.0; int32_t i_win = -1; uint8_t c_win = 0;
                 for (int64_t j = 0; j < np; ++j) {
                     const prim_t* p = &prim[j];
-                    if (p->D == 0.0) continue;
+                    if (p->D == 0.0 || p->ghost) continue;
                     int covered = 1;
                     double S = 0.0;
                     for (int i = 0; i < 3; ++i) {
@@ -361,6 +397,9 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
                     if (inside_band && on_band && could_show &&
                         z >= near * (1.0 - REL_TOL) && z <= far * (1.0 + REL_TOL)) flag |= 1;
                     if (!covered) continue;
+                    /* (vi) O10: a triangle at the limit of its angular range that covers the pixel and could win */
+                    if (p->unsure && z >= near && z <= far && could_show) flag |= 32;
+                    if (p->ghost) continue;
                     /* (ii) a kept fragment of another class almost as near as the winner */
                     if (i_win >= 0 && z >= near && z <= far && p->cls != c_win &&
                         fabs(z - z_win) <= fmax(REL_TOL, DEPTH_KAPPA * fmax(p->kappa, k_win)) * z_win) flag |= 2;

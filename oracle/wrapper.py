@@ -31,7 +31,7 @@ def _load():
         lib = C.CDLL(_LIB)
         p = C.c_void_p
         lib.pico_render.restype = C.c_int
-        lib.pico_render.argtypes = [C.c_int] * 5 + [C.c_double] * 2 + [p] * 4 + [C.c_int] * 3 + [p] * 4 + \
+        lib.pico_render.argtypes = [C.c_int] * 5 + [C.c_double] * 2 + [p] * 4 + [C.c_int] * 3 + [p] * 6 + \
                                    [C.c_int, p] + [p] * 7 + [C.c_int]
         lib.pico_step.restype = None
         lib.pico_step.argtypes = [p, p, p, C.c_int64, C.c_double, C.c_double, C.c_double]
@@ -57,7 +57,7 @@ class OracleResult:
     depth: np.ndarray        # f64 [n,H,W]
     depth_f16: np.ndarray    # f16 [n,H,W]
     index: np.ndarray        # i32 [n,H,W]  winning primitive, -1 background
-    flag: np.ndarray         # u8  [n,H,W]  ambiguity mask bits
+    flag: np.ndarray         # u8  [n,H,W]  ambiguity mask bits (1 edge, 2 depth, 4 near/far, 8 horizon, 16 grazing, 32 angular limit)
     kappa: np.ndarray        # f64 [n,H,W]  conditioning of the winner's depth (0 for background)
     counts: np.ndarray       # i64 [n,4]    in-frustum prims, prims with a kept fragment, kept fragments, flagged px
 
@@ -80,6 +80,10 @@ def render(scene, view_ids: Optional[Sequence[int]] = None, poses: Optional[np.n
     tcl = np.ascontiguousarray(s.tri_class, dtype=np.uint8)
     emi = np.ascontiguousarray(s.env_map_id, dtype=np.int32)
     off = np.ascontiguousarray(s.map_tri_offset, dtype=np.int64)
+    acl = getattr(s, "agent_classes", None)
+    acl = None if acl is None else np.ascontiguousarray(acl, dtype=np.uint8)
+    vis = getattr(s, "tri_vis_cos", None)
+    vis = None if vis is None else np.ascontiguousarray(vis, dtype=np.float32)
     cls = np.empty((n, s.H, s.W), np.uint8)
     depth = np.empty((n, s.H, s.W), np.float64)
     f16 = np.empty((n, s.H, s.W), np.uint16)
@@ -89,7 +93,7 @@ def render(scene, view_ids: Optional[Sequence[int]] = None, poses: Optional[np.n
     counts = np.zeros((n, 4), np.int64)
     rc = lib.pico_render(s.E, s.A, s.K, s.H, s.W, float(s.near), float(s.far), _ptr(emi), _ptr(off), _ptr(tri),
                          _ptr(tcl), int(s.agent_class), int(s.sky_class), int(s.ground_class), _ptr(poses),
-                         _ptr(dims), _ptr(active), _ptr(rig), n, _ptr(view_ids), _ptr(cls), _ptr(depth),
+                         _ptr(dims), _ptr(active), _ptr(rig), _ptr(acl), _ptr(vis), n, _ptr(view_ids), _ptr(cls), _ptr(depth),
                          _ptr(f16), _ptr(index), _ptr(flag), _ptr(kappa), _ptr(counts), int(n_threads))
     if rc != 0:
         raise MemoryError("pico_render failed")

@@ -75,6 +75,9 @@ class Scene:
     ground_class: int = CLASS_GROUND
     cfg: int = -1
     meta: dict = field(default_factory=dict)
+    agent_classes: Optional[np.ndarray] = None   # u8 [E,A]: class of each agent's box (None: agent_class for all)
+    tri_vis_cos: Optional[np.ndarray] = None     # f32 [N]: cos of the largest angle off its normal from which a triangle is
+                                                 # drawn, front side only (0 or None: ordinary two-sided triangle)
 
     @property
     def n_views(self) -> int:
@@ -424,8 +427,20 @@ def make_actions(cfg: int, step: int, E: int, A: int) -> np.ndarray:
     return a
 
 
+def disk_triangles(centre, normal, radius: float, n: int = 12) -> np.ndarray:
+    """A traffic-light disk as a fan of n triangles around its centre (a regular n-gon), wound counter-clockwise
+    when seen from the side its `normal` points to; f32 [n,3,3]."""
+    c = np.asarray(centre, np.float64); nz = np.asarray(normal, np.float64); nz = nz / np.linalg.norm(nz)
+    a = np.cross(nz, [0.0, 0.0, 1.0] if abs(nz[2]) < 0.9 else [1.0, 0.0, 0.0]); a /= np.linalg.norm(a)
+    b = np.cross(nz, a)
+    ang = 2 * np.pi * np.arange(n + 1) / n
+    rim = c + radius * (np.cos(ang)[:, None] * a + np.sin(ang)[:, None] * b)
+    return np.stack([np.stack([c, rim[i], rim[i + 1]]) for i in range(n)]).astype(np.float32)
+
+
 def custom_scene(tri_xyz, tri_class, poses, dims, rig, H: int, W: int, near: float = 0.5, far: float = 100.0,
-                 active=None, env_map_id=None, map_tri_offset=None, name: str = "custom") -> Scene:
+                 active=None, env_map_id=None, map_tri_offset=None, name: str = "custom", agent_classes=None,
+                 tri_vis_cos=None) -> Scene:
     """Wrap hand-made arrays (tests) in a Scene.  poses/dims are [E,A,3]; one map unless offsets are given."""
     tri_xyz = np.asarray(tri_xyz, dtype=np.float32).reshape(-1, 3, 3)
     tri_class = np.asarray(tri_class, dtype=np.uint8).reshape(-1)
@@ -445,4 +460,6 @@ def custom_scene(tri_xyz, tri_class, poses, dims, rig, H: int, W: int, near: flo
                  env_map_id=np.asarray(env_map_id, dtype=np.int32), map_tri_offset=map_tri_offset,
                  tri_xyz=tri_xyz, tri_class=tri_class, poses=poses, dims=dims,
                  active=np.asarray(active, dtype=np.uint8), rig=rig,
-                 speed=np.zeros((E, A), dtype=np.float32))
+                 speed=np.zeros((E, A), dtype=np.float32),
+                 agent_classes=None if agent_classes is None else np.asarray(agent_classes, np.uint8).reshape(E, A),
+                 tri_vis_cos=None if tri_vis_cos is None else np.asarray(tri_vis_cos, np.float32).reshape(-1))

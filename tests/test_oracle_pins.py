@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 
 import oracle
-from scenes import make_config, make_rig, custom_scene, focal_px
+from scenes import make_config, make_rig, custom_scene, focal_px, disk_triangles
 from tests.util import single_env, compare_images
 
 HERE = os.path.dirname(os.path.abspath(__file__))
@@ -661,3 +661,87 @@ def test_occlusion_counts_closed_forms():
     assert (vis.sum(1) == (r.cls == 4).reshape(len(views), -1).sum(1)).all()
     assert (vis <= un + sv).all() and (un[vis > 0] > 0).all()
     assert ((un > 0).sum(1) >= (vis > 0).sum(1)).all() and (un > vis).any()     # heavy occlusion: somebody is partly hidden
+
+
+# ------------------------------------------------------------------------------------------------
+# road users with their own class; triangles with a limited angular range (traffic-light disks)
+# ------------------------------------------------------------------------------------------------
+def test_per_agent_classes():
+    # the 48-pixel car 12.5 m ahead, as a pedestrian (class 7); a second agent keeps class 9; the sums still hold
+    agents = np.array([ego(), ego(12.5, 0.0, 0.0), ego(14.0, 6.0, 0.0)])
+    s = custom_scene(np.zeros((0, 3, 3)), [], agents[None, :, :3], agents[None, :, 3:], make_rig((0.0,), 90.0, 90.0), 64, 64,
+                     agent_classes=[[5, 7, 9]])
+    r = oracle.render(s, [0])
+    assert (r.cls[0][32:38, 28:36] == 7).all() and (r.cls[0] == 7).sum() == 48
+    assert (r.cls[0] == 9).sum() > 0 and (r.cls[0] == 4).sum() == 0 and (r.cls[0] == 5).sum() == 0
+    vis, un, *_ = oracle.occlusion_counts(s, [0])
+    assert vis[0, 1] == 48 and vis[0, 2] == (r.cls[0] == 9).sum()
+    # seen from the third agent (view 2), the ego's own box shows the ego's class
+    assert (oracle.render(s, [2]).cls[0] == 9).sum() == 0
+
+
+def test_angular_range_of_one_sided_triangles():
+    """A wall 10 m ahead whose normal points back at the camera (-x), drawn only within 30 degrees of that normal.
+    8 x 8 image, fx = 4: camera at (0, L, 1) looking along +x.  Each of the wall's two triangles is judged from its
+    own centroid; the wall is small (1 x 1 m around the axis at camera height), so both centroids sit within
+    0.24 m of (10, 0, 1) and the angle is atan(L / 10) to within a degree and a half."""
+    lim = np.cos(np.radians(30.0))
+    # wound counter-clockwise when seen from -x (the camera's side): normal (V1-V0)x(V2-V0) = -x
+    wall = [[(10.0, -0.5, 0.5), (10.0, -0.5, 1.5), (10.0, 0.5, 1.5)], [(10.0, -0.5, 0.5), (10.0, 0.5, 1.5), (10.0, 0.5, 0.5)]]
+    n = np.cross(np.subtract(wall[0][1], wall[0][0]), np.subtract(wall[0][2], wall[0][0]))
+    assert n[0] < 0 and n[1] == 0 and n[2] == 0
+    rig = make_rig((0.0,), 90.0, 90.0, 64, 64, mount=(0.0, 0.0, 1.0))
+
+    def seen(L, yaw, vis):
+        s = single_env(wall, [5, 5], [ego(0.0, L, yaw)], rig=rig, tri_vis_cos=vis)
+        r = oracle.render(s, [0])
+        return int((r.cls[0] == 5).sum()), r
+
+    for L, want in ((0.0, True), (4.0, True), (5.0, True), (6.5, False), (10.0, False)):     # 0, 21.8, 26.6, 33.0, 45 degrees
+        yaw = np.arctan2(-L, 10.0)                                                         # keep the wall on the optical axis
+        n_on, r = seen(L, yaw, [lim, lim])
+        n_free, _ = seen(L, yaw, None)
+        assert n_free > 0 and (n_on == n_free if want else n_on == 0), (L, n_on, n_free)
+        assert (r.flag[0] & 32).sum() == 0
+    # from behind it is never drawn, whatever the angle; without a limit it is two-sided
+    s_back = single_env(wall, [5, 5], [ego(20.0, 0.0, np.pi)], rig=rig, tri_vis_cos=[lim, lim])
+    assert (oracle.render(s_back, [0]).cls[0] == 5).sum() == 0
+    s_back = single_env(wall, [5, 5], [ego(20.0, 0.0, np.pi)], rig=rig)
+    assert (oracle.render(s_back, [0]).cls[0] == 5).sum() > 0
+    # one triangle limited, the other not: only the limited one disappears at 45 degrees
+    n_half, _ = seen(10.0, np.arctan2(-10.0, 10.0), [lim, 0.0])
+    n_free, _ = seen(10.0, np.arctan2(-10.0, 10.0), None)
+    assert 0 < n_half < n_free
+    # exactly at the limit (the limit is set to the float32 of the first triangle's own cosine): decided by the exact
+    # comparison, and every pixel the triangle covers is flagged; 1e-3 away from it nothing is flagged
+    L = 5.0
+    g = np.mean(np.asarray(wall[0], np.float64), axis=0)
+    d = np.array([0.0, L, 1.0]) - g
+    c_exact = float(-d[0] / np.linalg.norm(d))
+    for delta, flagged in ((0.0, True), (3e-6, True), (-3e-6, True), (1e-3, False), (-1e-3, False)):
+        s = single_env(wall[:1], [5], [ego(0.0, L, np.arctan2(-L, 10.0))], rig=rig, tri_vis_cos=[np.float32(c_exact + delta)])
+        r = oracle.render(s, [0])
+        drawn = (r.cls[0] == 5).sum()
+        assert ((r.flag[0] & 32).sum() > 0) == flagged, (delta, drawn)
+        if not flagged:
+            assert (drawn > 0) == (delta < 0)
+
+
+def test_traffic_light_disk():
+    # a disk of radius 0.5 m, 8 m in front of the camera and facing it: a circle of radius 2 pixels (fx = 32) around
+    # the image centre; pixel centres within it: the 12 with |du|, |dv| in {0.5, 1.5} and du^2 + dv^2 < 4
+    rig = make_rig((0.0,), 90.0, 90.0, 64, 64, mount=(0.0, 0.0, 1.0))
+    tris = disk_triangles((8.0, 0.0, 1.0), (-1.0, 0.0, 0.0), 0.5, n=64)
+    lim = float(np.cos(np.radians(40.0)))
+    s = single_env(tris, [6] * len(tris), [ego()], rig=rig, tri_vis_cos=[lim] * len(tris))
+    r = oracle.render(s, [0])
+    ys, xs = np.nonzero(r.cls[0] == 6)
+    assert len(xs) == 12 and set(zip(xs.tolist(), ys.tolist())) == {(x, y) for x in range(30, 34) for y in range(30, 34)
+                                                                    if (x + 0.5 - 32) ** 2 + (y + 0.5 - 32) ** 2 < 4}
+    assert np.allclose(r.depth[0][r.cls[0] == 6], 8.0)
+    # the ego turns away until the signal's centre is 50 degrees off its normal as seen from the disk: culled
+    a = np.radians(50.0)
+    s = single_env(tris, [6] * len(tris), [ego(8.0 - 8.0 * np.cos(a), 8.0 * np.sin(a), -a)], rig=rig, tri_vis_cos=[lim] * len(tris))
+    assert (oracle.render(s, [0]).cls[0] == 6).sum() == 0
+    s = single_env(tris, [6] * len(tris), [ego(8.0 - 8.0 * np.cos(a), 8.0 * np.sin(a), -a)], rig=rig)
+    assert (oracle.render(s, [0]).cls[0] == 6).sum() > 0

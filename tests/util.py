@@ -6,7 +6,7 @@ import numpy as np
 from scenes import custom_scene, make_rig, NOMINAL_DIMS, MOUNT
 
 
-def single_env(tris, classes, agents, rig=None, H=64, W=64, near=0.5, far=100.0, active=None):
+def single_env(tris, classes, agents, rig=None, H=64, W=64, near=0.5, far=100.0, active=None, tri_vis_cos=None, agent_classes=None):
     """agents: list of (x, y, yaw, length, width, height)."""
     agents = np.asarray(agents, dtype=np.float64).reshape(-1, 6)
     poses = agents[None, :, :3]
@@ -15,7 +15,8 @@ def single_env(tris, classes, agents, rig=None, H=64, W=64, near=0.5, far=100.0,
         rig = make_rig((0.0,), 90.0, 90.0, W, H)
     tris = np.asarray(tris, dtype=np.float32).reshape(-1, 3, 3)
     return custom_scene(tris, classes, poses, dims, rig, H, W, near, far,
-                        active=None if active is None else np.asarray(active, np.uint8).reshape(1, -1))
+                        active=None if active is None else np.asarray(active, np.uint8).reshape(1, -1),
+                        tri_vis_cos=tri_vis_cos, agent_classes=agent_classes)
 
 
 def f16_ulp_distance(a: np.ndarray, b: np.ndarray) -> np.ndarray:
@@ -42,7 +43,7 @@ def compare_images(ref_cls, ref_depth, ref_flag, got_cls, got_depth32=None, got_
     bad = ref_cls != got_cls
     if got_depth32 is not None:
         bad |= np.abs(np.asarray(got_depth32, np.float64) - ref_depth) > tol * ref_depth
-    flagged = (np.asarray(ref_flag) & 15) != 0
+    flagged = (np.asarray(ref_flag) & 47) != 0
     unflagged_bad = bad & ~flagged
     stats = dict(pixels=int(n), mismatches=int(bad.sum()), flagged=int(flagged.sum()),
                  unflagged_mismatches=int(unflagged_bad.sum()))
