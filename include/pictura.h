@@ -92,6 +92,11 @@ typedef struct {
     uint8_t ground_class;          /* background below the horizon                               */
     uint8_t reserved;
     int32_t device;                /* CUDA device ordinal                                        */
+    const float* tri_vis_cos;      /* host [N] or NULL: 0 = ordinary two-sided triangle; c in (0, 1] = the triangle
+                                      is drawn in a view only from its front side (normal (V1-V0)x(V2-V0)) and only if
+                                      the direction from its centroid to the camera is within acos(c) of that normal --
+                                      the paper's traffic-light disks "visible only within a limited angular range"
+                                      (Sec. 3.2), given as triangle fans.  Such triangles are never paired into quads. */
 } pic_scene_desc;
 
 /*
@@ -133,6 +138,13 @@ pic_status pic_render_host(pic_scene* scene, const float* poses, const float* di
 pic_status pic_set_state(pic_scene* scene, const float* state, const float* dims, const uint8_t* active,
                          void* cuda_stream);
 pic_status pic_get_state(pic_scene* scene, float* state_out, void* cuda_stream);
+
+/*
+ * Class of each agent's box (Sec. 3.2: pedestrians, cyclists and vehicles each in its own hue): classes dev u8
+ * [E,A], copied into the scene on `cuda_stream`; NULL returns to desc.agent_class for every agent.  Used by all
+ * later pic_render / pic_step calls.
+ */
+pic_status pic_set_agent_classes(pic_scene* scene, const uint8_t* classes, void* cuda_stream);
 
 /*
  * One simulator step: explicit-Euler kinematic bicycle update of every active agent, everything

@@ -21,7 +21,7 @@ OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_
 FLAG_NONFINITE_POSE = 1
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
+           "pic_get_state", "pic_set_agent_classes", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
            "pic_last_error", "pic_version"]
 
 
@@ -41,7 +41,7 @@ class pic_scene_desc(C.Structure):
                 ("W", C.c_int32), ("near_z", C.c_float), ("far_z", C.c_float), ("num_maps", C.c_int32),
                 ("env_map_id", C.c_void_p), ("map_tri_offset", C.c_void_p), ("tri_xyz", C.c_void_p),
                 ("tri_class", C.c_void_p), ("agent_class", C.c_uint8), ("sky_class", C.c_uint8),
-                ("ground_class", C.c_uint8), ("reserved", C.c_uint8), ("device", C.c_int32)]
+                ("ground_class", C.c_uint8), ("reserved", C.c_uint8), ("device", C.c_int32), ("tri_vis_cos", C.c_void_p)]
 
 
 class pic_static_desc(C.Structure):
@@ -71,6 +71,7 @@ def load(path: Optional[str] = None):
     lib.pic_render_host.argtypes = [vp, vp, vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     lib.pic_set_state.argtypes = [vp, vp, vp, vp, vp]
     lib.pic_get_state.argtypes = [vp, vp, vp]
+    lib.pic_set_agent_classes.argtypes = [vp, vp, vp]
     lib.pic_step.argtypes = [vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     lib.pic_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
@@ -199,7 +200,7 @@ class Scene:
 
     def __init__(self, E: int, A: int, K: int, H: int, W: int, near: float, far: float, tri_xyz, tri_class,
                  map_tri_offset=None, env_map_id=None, agent_class: int = 4, sky_class: int = 0,
-                 ground_class: int = 1, device: int = 0):
+                 ground_class: int = 1, device: int = 0, tri_vis_cos=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the rasterizer has no CPU path")
@@ -221,6 +222,10 @@ class Scene:
         d.tri_class = tri_class.ctypes.data
         d.agent_class, d.sky_class, d.ground_class = int(agent_class), int(sky_class), int(ground_class)
         d.device = int(device)
+        vis = None if tri_vis_cos is None else np.ascontiguousarray(tri_vis_cos, dtype=np.float32).reshape(-1)
+        if vis is not None and vis.shape[0] != tri_xyz.shape[0]:
+            raise ValueError("tri_vis_cos needs one value per triangle")
+        d.tri_vis_cos = None if vis is None else vis.ctypes.data
         handle = C.c_void_p()
         _check(self._lib, self._lib.pic_scene_create(C.byref(d), C.byref(handle)))
         self._h = handle
@@ -308,6 +313,12 @@ class Scene:
         _check(self._lib, self._lib.pic_set_state(
             self._h, _dev_ptr(state, torch.float32, 4 * n), _dev_ptr(dims, torch.float32, 3 * n),
             _dev_ptr(active, torch.uint8, n) if active is not None else None, _stream_ptr(stream)))
+
+    def set_agent_classes(self, classes, stream=None):
+        """classes: CUDA u8 tensor [E,A] (class of each agent's box), or None for the scene-wide agent class."""
+        import torch
+        _check(self._lib, self._lib.pic_set_agent_classes(
+            self._h, _dev_ptr(classes, torch.uint8, self.n_agents) if classes is not None else None, _stream_ptr(stream)))
 
     def get_state(self, out=None, stream=None):
         import torch

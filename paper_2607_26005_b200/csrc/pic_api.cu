@@ -14,7 +14,7 @@ namespace pic {
 size_t max_smem_bytes();
 cudaError_t configure_kernels();
 cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses, float* state, const float* actions,
-                         const float* dims, const uint8_t* active, AgentGeom* agents_out, ViewCam* cams_out,
+                         const float* dims, const uint8_t* active, const uint8_t* agent_cls, AgentGeom* agents_out, ViewCam* cams_out,
                          float* tables, uint32_t* status, float dt, float wheelbase, float v_max, cudaStream_t stream);
 cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, int sm_count, cudaStream_t stream);
 size_t survivor_bytes_per_tile();
@@ -80,6 +80,8 @@ struct pic_scene {
     float* d_dims = nullptr;        // [E*A*3]
     uint8_t* d_active = nullptr;    // [E*A]
     bool have_active = false;
+    uint8_t* d_agent_cls = nullptr; // [E*A] class of each agent's box
+    bool have_agent_cls = false;
     uint32_t* d_status = nullptr;
     // staging for pic_render_host
     float* d_in_poses = nullptr;
@@ -115,7 +117,7 @@ struct DeviceGuard {
 
 void free_scene(pic_scene* s) {
     cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims); cudaFree(s->d_cell_start); cudaFree(s->d_grid_prims); cudaFree(s->d_large_leaves);
-    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_surv); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_status);
+    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_surv); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_agent_cls); cudaFree(s->d_status);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
     if (s->ev) {
@@ -214,7 +216,10 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     CUDA_TRY(pic::configure_kernels());
 
     char err[256] = "";
-    pic::HostHierarchy* hh = pic::build_hierarchy(d->num_maps, d->map_tri_offset, d->tri_xyz, d->tri_class, d->A, err, sizeof(err));
+    if (d->tri_vis_cos)
+        for (int64_t i = 0; i < n_tri; ++i)
+            if (!(d->tri_vis_cos[i] >= 0.f) || d->tri_vis_cos[i] > 1.f) return fail(PIC_ERR_INVALID_ARG, "tri_vis_cos[%lld] is not in [0, 1]", (long long)i);
+    pic::HostHierarchy* hh = pic::build_hierarchy(d->num_maps, d->map_tri_offset, d->tri_xyz, d->tri_class, d->tri_vis_cos, d->A, err, sizeof(err));
     if (!hh) return fail(PIC_ERR_SHAPE, "%s", err);
 
     pic_scene* s = new (std::nothrow) pic_scene();
@@ -262,6 +267,7 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_state, sizeof(float) * 4 * n_agents);
     dmalloc((void**)&s->d_dims, sizeof(float) * 3 * n_agents);
     dmalloc((void**)&s->d_active, n_agents);
+    dmalloc((void**)&s->d_agent_cls, n_agents);
     dmalloc((void**)&s->d_status, sizeof(uint32_t));
     upload(s->d_env_map, env_map, sizeof(int32_t) * d->E);
     upload(s->d_maps, maps, sizeof(pic::MapInfo) * nm);
@@ -302,7 +308,7 @@ pic_status pic_map_stats(const pic_scene_desc* d, int64_t out[8]) {
         if (d->map_tri_offset[m + 1] < d->map_tri_offset[m]) return fail(PIC_ERR_SHAPE, "map_tri_offset must be non-decreasing");
     if (d->map_tri_offset[d->num_maps] > 0 && (!d->tri_xyz || !d->tri_class)) return fail(PIC_ERR_INVALID_ARG, "triangle arrays are NULL");
     char err[256] = "";
-    pic::HostHierarchy* hh = pic::build_hierarchy(d->num_maps, d->map_tri_offset, d->tri_xyz, d->tri_class, d->A > 0 ? d->A : 0, err, sizeof(err));
+    pic::HostHierarchy* hh = pic::build_hierarchy(d->num_maps, d->map_tri_offset, d->tri_xyz, d->tri_class, d->tri_vis_cos, d->A > 0 ? d->A : 0, err, sizeof(err));
     if (!hh) return fail(PIC_ERR_SHAPE, "%s", err);
     size_t np, nl, ng, nm;
     const pic::Prim* prims = pic::hierarchy_prims(hh, &np);
@@ -385,7 +391,7 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
     DeviceGuard guard(s->device);
     if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
     const int n_agents = s->E * s->A;
-    CUDA_TRY(pic::launch_setup(P, n_agents, poses, state, actions, dims, active, s->d_agents, s->d_cams, s->d_tables,
+    CUDA_TRY(pic::launch_setup(P, n_agents, poses, state, actions, dims, active, s->have_agent_cls ? s->d_agent_cls : nullptr, s->d_agents, s->d_cams, s->d_tables,
                                s->d_status, kDt, kWheelbase, kVMax, stream));
     const long long total = (long long)s->E * s->A * s->K;
     long long count = total - s->view_first;
@@ -453,6 +459,16 @@ pic_status pic_set_state(pic_scene* s, const float* state, const float* dims, co
     CUDA_TRY(cudaMemcpyAsync(s->d_dims, dims, sizeof(float) * 3 * n, cudaMemcpyDeviceToDevice, stream));
     if (active) CUDA_TRY(cudaMemcpyAsync(s->d_active, active, n, cudaMemcpyDeviceToDevice, stream));
     else CUDA_TRY(cudaMemsetAsync(s->d_active, 1, n, stream));
+    return PIC_OK;
+}
+
+pic_status pic_set_agent_classes(pic_scene* s, const uint8_t* classes, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    s->have_agent_cls = classes != nullptr;
+    if (classes)
+        CUDA_TRY(cudaMemcpyAsync(s->d_agent_cls, classes, (size_t)s->E * s->A, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
     return PIC_OK;
 }
 

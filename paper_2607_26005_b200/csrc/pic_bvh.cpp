@@ -187,7 +187,7 @@ void build_grid(HostHierarchy& h, MapInfo& mi) {
 }  // namespace
 
 HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const float* tri_xyz,
-                               const uint8_t* tri_class, int agents_per_env, char* err, int err_len) {
+                               const uint8_t* tri_class, const float* tri_vis_cos, int agents_per_env, char* err, int err_len) {
     HostHierarchy* h = new HostHierarchy();
     h->maps.resize(num_maps);
     std::vector<Prim> local;
@@ -208,7 +208,10 @@ HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const fl
             std::memset(&p, 0, sizeof(p));
             F3 q[4];
             bool quad = false;
-            if (i + 1 < n && tri_class[t0 + i] == tri_class[t0 + i + 1]) {
+            // (a triangle with a limited angular range is judged from its own centroid: never fused)
+            const float vis = tri_vis_cos ? tri_vis_cos[t0 + i] : 0.f;
+            const bool plain = !(vis > 0.f) && !(tri_vis_cos && i + 1 < n && tri_vis_cos[t0 + i + 1] > 0.f);
+            if (plain && i + 1 < n && tri_class[t0 + i] == tri_class[t0 + i + 1]) {
                 const F3* b = reinterpret_cast<const F3*>(tri_xyz + 9 * (t0 + i + 1));
                 quad = fuse_quad(a, b, q);
             }
@@ -216,6 +219,7 @@ HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const fl
             for (int k = 0; k < 4; ++k) { p.v[3 * k] = q[k].x; p.v[3 * k + 1] = q[k].y; p.v[3 * k + 2] = q[k].z; }
             p.key_lo = ((0xFFFFFFu - (uint32_t)i) << 8) | tri_class[t0 + i];
             p.flags = quad ? 1u : 0u;
+            p.vis_cos = vis > 0.f ? vis : 0.f;
             int nv = quad ? 4 : 3;
             for (int k = 0; k < nv; ++k)
                 if (!lex_less(q[k], q[(k + 1) % nv])) p.flags |= 1u << (4 + k);

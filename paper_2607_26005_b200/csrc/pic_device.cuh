@@ -224,14 +224,36 @@ __device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const 
 }
 
 
-__device__ __forceinline__ void load_prim(const Prim* __restrict__ p, float (&v)[12], uint32_t& key_lo, uint32_t& flags) {
+__device__ __forceinline__ void load_prim(const Prim* __restrict__ p, float (&v)[12], uint32_t& key_lo, uint32_t& flags, float& vis_cos) {
     const float4* q = reinterpret_cast<const float4*>(p);
     float4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2);
     uint4 d = __ldg(reinterpret_cast<const uint4*>(q + 3));
     v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
     v[8] = c.x; v[9] = c.y; v[10] = c.z; v[11] = c.w;
-    key_lo = d.x; flags = d.y;
+    key_lo = d.x; flags = d.y; vis_cos = __uint_as_float(d.z);
 }
+__device__ __forceinline__ void load_prim(const Prim* __restrict__ p, float (&v)[12], uint32_t& key_lo, uint32_t& flags) {
+    float vis_cos;
+    load_prim(p, v, key_lo, flags, vis_cos);
+}
+
+// A triangle with vis_cos > 0 is drawn only from its front side and only if the direction from its
+// centroid to the camera (the origin of camera space) is within acos(vis_cos) of its normal P (by
+// vertex order).  Outside that range its plane normal is replaced by zero, which makes
+// prim_equations reject it as degenerate -- so every kernel that sets a primitive up drops it alike.
+__device__ __forceinline__ V3 limit_angular_range(const V3 (&V)[4], V3 P, float vis_cos) {
+    if (vis_cos > 0.f) {
+        const V3 g = {add(add(V[0].x, V[1].x), V[2].x), add(add(V[0].y, V[1].y), V[2].y), add(add(V[0].z, V[1].z), V[2].z)};   // 3 x centroid
+        const float s = -vdot(P, g);
+        const float pp = vdot(P, P), gg = vdot(g, g);
+        const bool in = s >= 0.f && mul(s, s) >= mul(mul(vis_cos, vis_cos), mul(pp, gg));
+        if (!in) P = {0.f, 0.f, 0.f};
+    }
+    return P;
+}
+
+// Class of an agent's box (AgentGeom::active = 1 | class << 8).
+__device__ __forceinline__ uint32_t agent_box_class(const AgentGeom& g) { return (g.active >> 8) & 0xffu; }
 
 // Box corner i (bit0 +x, bit1 +y, bit2 top) of agent g in camera space.
 __device__ __forceinline__ V3 box_corner(const Cam& c, const AgentGeom& g, int i) {

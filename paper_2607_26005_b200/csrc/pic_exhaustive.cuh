@@ -62,7 +62,7 @@ __device__ __forceinline__ void exhaustive_tile(ExhaustiveSmem& s, const RenderP
 #pragma unroll
                 for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
                 quad = true; flags = face_flags(corners);
-                key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+                key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | agent_box_class(g);
                 Pn = plane_normal(V, true);
             }
             PrimEq q;

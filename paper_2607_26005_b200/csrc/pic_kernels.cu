@@ -19,7 +19,7 @@ struct RigParams {
 // ------------------------------------------------------------------------------------------------
 __global__ void agent_kernel(int n, const float* __restrict__ poses, float* state, const float* __restrict__ actions,
                              const float* __restrict__ dims, const uint8_t* __restrict__ active,
-                             AgentGeom* __restrict__ out, ViewCam* __restrict__ cams, uint32_t* status,
+                             const uint8_t* __restrict__ agent_cls, uint32_t default_cls, AgentGeom* __restrict__ out, ViewCam* __restrict__ cams, uint32_t* status,
                              const __grid_constant__ RigParams R, float dt, float wheelbase, float v_max) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
@@ -59,7 +59,7 @@ __global__ void agent_kernel(int n, const float* __restrict__ poses, float* stat
     g.x = x; g.y = y;
     sincosf(th, &g.s, &g.c);
     g.hl = 0.5f * l; g.hw = 0.5f * w; g.h = h;
-    g.active = act ? 1u : 0u;
+    g.active = act ? (1u | ((agent_cls ? (uint32_t)agent_cls[i] : default_cls) << 8)) : 0u;
     out[i] = g;
     for (int k = 0; k < R.K; ++k) {
         ViewCam vc;
@@ -101,12 +101,12 @@ __global__ void __launch_bounds__(EXH_THREADS) render_brute_kernel(const __grid_
     const Prim* prims = P.prims + mi.prim_begin;
     exhaustive_tile(s, P, blockIdx.x, mi.prim_end - mi.prim_begin, mi.n_tris,
                     [prims](uint32_t i, const Cam& c, V3 (&V)[4], V3& Pn, bool& quad, uint32_t& flags, uint32_t& key_lo) {
-                        float v[12];
-                        load_prim(prims + i, v, key_lo, flags);
+                        float v[12], vis_cos;
+                        load_prim(prims + i, v, key_lo, flags, vis_cos);
                         quad = flags & 1u;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) V[j] = to_camera(c, v[3 * j], v[3 * j + 1], v[3 * j + 2]);
-                        Pn = plane_normal_world(c, v, quad);
+                        Pn = limit_angular_range(V, plane_normal_world(c, v, quad), vis_cos);
                     });
 }
 
@@ -135,7 +135,7 @@ static RigParams rig_params(const RenderParams& P) {
 
 // Per call: rig tables, then agents (+ optional bicycle step) and their cameras.
 cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses, float* state, const float* actions,
-                         const float* dims, const uint8_t* active, AgentGeom* agents_out, ViewCam* cams_out,
+                         const float* dims, const uint8_t* active, const uint8_t* agent_cls, AgentGeom* agents_out, ViewCam* cams_out,
                          float* tables, uint32_t* status, float dt, float wheelbase, float v_max, cudaStream_t stream) {
     const RigParams R = rig_params(P);
     float* ray_x = tables;
@@ -145,7 +145,7 @@ cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses
     rig_kernel<<<P.K, 256, 0, stream>>>(R, ray_x, ray_y, bg_z, bg_cls, P.overflow);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess || n_agents <= 0) return err;
-    agent_kernel<<<(n_agents + 127) / 128, 128, 0, stream>>>(n_agents, poses, state, actions, dims, active, agents_out,
+    agent_kernel<<<(n_agents + 127) / 128, 128, 0, stream>>>(n_agents, poses, state, actions, dims, active, agent_cls, P.cls_agent, agents_out,
                                                               cams_out, status, R, dt, wheelbase, v_max);
     return cudaGetLastError();
 }

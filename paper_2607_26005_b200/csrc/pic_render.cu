@@ -255,11 +255,11 @@ __device__ __forceinline__ bool fetch_candidate(const S& s, const RenderParams& 
         const uint32_t lf = s.leaf[i / LEAF_PRIMS];
         const uint32_t j = i % LEAF_PRIMS;
         if (j >= (lf & 15u)) return false;
-        float v[12];
-        load_prim(P.prims + (lf >> 4) + j, v, key_lo, flags);
+        float v[12], vis_cos;
+        load_prim(P.prims + (lf >> 4) + j, v, key_lo, flags, vis_cos);
 #pragma unroll
         for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
-        if (want_plane) Pn = plane_normal_world(c, v, flags & 1u);
+        if (want_plane) Pn = limit_angular_range(V, plane_normal_world(c, v, flags & 1u), vis_cos);
     } else {
         const uint32_t it = s.face[i - nl * LEAF_PRIMS];
         const int b = (int)(it >> 3), f = (int)(it & 7u);
@@ -267,7 +267,7 @@ __device__ __forceinline__ bool fetch_candidate(const S& s, const RenderParams& 
         const uint32_t corners = face_corners(f);
 #pragma unroll
         for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
-        key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+        key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | agent_box_class(g);
         flags = face_flags(corners);
         if (want_plane) Pn = plane_normal(V, true);
     }
@@ -1010,18 +1010,18 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
 __device__ __forceinline__ void fetch_survivor(const Cam& c, const RenderParams& P, uint32_t id, int e, uint32_t n_map_tris,
                                                V3 (&V)[4], V3& Pn, uint32_t& key_lo, uint32_t& flags) {
     if (!(id & SURV_FACE)) {
-        float v[12];
-        load_prim(P.grid_prims + id, v, key_lo, flags);
+        float v[12], vis_cos;
+        load_prim(P.grid_prims + id, v, key_lo, flags, vis_cos);
 #pragma unroll
         for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
-        Pn = plane_normal_world(c, v, flags & 1u);
+        Pn = limit_angular_range(V, plane_normal_world(c, v, flags & 1u), vis_cos);
     } else {
         const int b = (int)((id & ~SURV_FACE) >> 3), f = (int)(id & 7u);
         const AgentGeom g = P.agents[(size_t)e * P.A + b];
         const uint32_t corners = face_corners(f);
 #pragma unroll
         for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
-        key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | P.cls_agent;
+        key_lo = ((0xFFFFFFu - (n_map_tris + 12u * (uint32_t)b + 2u * (uint32_t)f)) << 8) | agent_box_class(g);
         flags = face_flags(corners);
         Pn = plane_normal(V, true);
     }

@@ -21,7 +21,7 @@
 
 namespace pic {
 cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses, float* state, const float* actions,
-                         const float* dims, const uint8_t* active, AgentGeom* agents_out, ViewCam* cams_out,
+                         const float* dims, const uint8_t* active, const uint8_t* agent_cls, AgentGeom* agents_out, ViewCam* cams_out,
                          float* tables, uint32_t* status, float dt, float wheelbase, float v_max, cudaStream_t stream);
 void set_last_error(const char* msg);
 }  // namespace pic
@@ -177,7 +177,7 @@ extern "C" pic_status pic_render_static(const pic_static_desc* d, const float* t
     }
     S.tri_xyz = tri_xyz; S.tri_class = tri_class; S.n_tris = (uint32_t)d->n_tris;
     // (the status word is sticky across calls, like a scene's: pic_static_status reads and clears it)
-    ce = pic::launch_setup(P, d->E * d->A, poses, nullptr, nullptr, dims, active, agents, cams, tables, status, 0.f, 1.f, 0.f, stream);
+    ce = pic::launch_setup(P, d->E * d->A, poses, nullptr, nullptr, dims, active, nullptr, agents, cams, tables, status, 0.f, 1.f, 0.f, stream);
     if (ce != cudaSuccess) return fail(PIC_ERR_CUDA, "set-up kernels: %s", cudaGetErrorString(ce));
     const unsigned blocks = (unsigned)(d->E * d->A * d->K * P.tiles_x * P.tiles_y);
     render_static_kernel<<<blocks, EXH_THREADS, sizeof(ExhaustiveSmem), stream>>>(S);

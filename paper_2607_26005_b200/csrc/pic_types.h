@@ -18,7 +18,8 @@ struct Prim {
     float v[12];        // 4 vertices xyz in perimeter order (triangle: the 4th repeats the 3rd)
     uint32_t key_lo;    // (0xFFFFFF - primitive index) << 8 | class : low half of the z-buffer key
     uint32_t flags;     // bit 0: quad; bits 4..7: edge i runs against its canonical direction
-    uint32_t pad[2];
+    float vis_cos;      // > 0: drawn only from its front side and within acos(vis_cos) of its normal (triangles only)
+    uint32_t pad;
 };
 static_assert(sizeof(Prim) == 64, "Prim must be 64 bytes");
 
@@ -52,7 +53,7 @@ struct AgentGeom {
     float x, y;       // box centre on the ground plane
     float c, s;       // cos, sin of the heading
     float hl, hw, h;  // half length, half width, height
-    uint32_t active;
+    uint32_t active;  // 0: inactive; else 1 | class of the agent's box << 8
 };
 
 struct CamConst {
@@ -115,7 +116,7 @@ struct RenderParams {
 // Host-side result of the hierarchy build for all maps of a scene.
 struct HostHierarchy;
 HostHierarchy* build_hierarchy(int num_maps, const int64_t* tri_offset, const float* tri_xyz,
-                               const uint8_t* tri_class, int agents_per_env, char* err, int err_len);
+                               const uint8_t* tri_class, const float* tri_vis_cos, int agents_per_env, char* err, int err_len);
 void free_hierarchy(HostHierarchy*);
 const Prim* hierarchy_prims(const HostHierarchy*, size_t* n);
 const Node* hierarchy_leaves(const HostHierarchy*, size_t* n);

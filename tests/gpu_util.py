@@ -17,10 +17,13 @@ class CudaRun:
         self.dev = torch.device("cuda", device)
         self.scene = pic.Scene(s.E, s.A, s.K, s.H, s.W, s.near, s.far, s.tri_xyz, s.tri_class,
                                map_tri_offset=s.map_tri_offset, env_map_id=s.env_map_id, agent_class=s.agent_class,
-                               sky_class=s.sky_class, ground_class=s.ground_class, device=device)
+                               sky_class=s.sky_class, ground_class=s.ground_class, device=device,
+                               tri_vis_cos=getattr(s, "tri_vis_cos", None))
         self.poses = torch.from_numpy(np.ascontiguousarray(s.poses)).to(self.dev)
         self.dims = torch.from_numpy(np.ascontiguousarray(s.dims)).to(self.dev)
         self.active = torch.from_numpy(np.ascontiguousarray(s.active)).to(self.dev)
+        if getattr(s, "agent_classes", None) is not None:
+            self.scene.set_agent_classes(torch.from_numpy(np.ascontiguousarray(s.agent_classes, dtype=np.uint8)).to(self.dev))
 
     def render(self, brute: bool = False, depth32: bool = True, poses=None, view_first: int = 0, view_count: int = 0,
                counters: bool = False, debug_flags: int = 0):
