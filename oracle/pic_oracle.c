@@ -14,7 +14,7 @@
  * frame conventions of its camera-rig table (agent frame x forward, y left, z up, yaw about z;
  * intrinsics given as a focal length in pixels, principal point at the image centre).  A rig row
  * is (mount x, y, z, yaw, pitch, fx, fy).  The paper fixes no
- * sampling, fill or depth rule; the ones used here are the steps O1..O9 below:
+ * sampling, fill or depth rule; the ones used here are the steps O1..O12 below:
  *
  *  O1 camera      q = X - P_agent; q' = q - Rz(yaw_agent) m; X_c = (r.q', d.q', f.q') with
  *                 f = (cos(pitch)cos(a), cos(pitch)sin(a), sin(pitch)), r = (sin a, -cos a, 0), d = f x r,
@@ -49,6 +49,38 @@
  *                 pixels.  c = 0 (or no array) is the ordinary two-sided triangle.  A triangle within
  *                 1e-5 of its limit is drawn according to the exact comparison, and every pixel it
  *                 covers (or would cover) and could win is flagged (bit 32).
+ *  O11 colour     (Sec. 3.2: the scene is drawn as flat-shaded primitives; agents are cuboids coloured per
+ *                 face with depth-aware brightness, each kind of road user in its own hue.)  The paper gives
+ *                 no numbers, so the reading is: a palette gives every class an 8-bit RGB triple; a map
+ *                 triangle has its class's colour; face f of an agent's box has its class's colour times
+ *                 s_f * beta(z), s = (rear 0.60, front 1.00, right 0.70, left 0.85, bottom 0.40, top 0.92),
+ *                 beta(z) = 1 - 0.5 (z - near) / (far - near) with z the fragment's depth; ground and sky
+ *                 have their classes' colours.  Without antialiasing a pixel shows the colour of its O6
+ *                 winner (or of the background), rounded to 8 bits (floor(c + 0.5)).
+ *  O12 antialiasing (Sec. 3.2: analytic-coverage antialiasing at a single sample per pixel, so that thin
+ *                 structures stay visible at low resolution.)  No formula is given; the reading is a box
+ *                 filter over the pixel's unit square, evaluated exactly:
+ *                   - the edge functions E_i = rho.N_i are linear in the pixel coordinates, so the part of
+ *                     the pixel's square inside all three edges is a convex polygon; a primitive's coverage
+ *                     alpha is that polygon's area (the square clipped by the three lines; for a single edge
+ *                     crossing the pixel this is the closed form of pico_edge_coverage);
+ *                   - it leaves a fragment at every pixel with alpha > 0 whose plane, evaluated at the pixel
+ *                     centre, has S > 0 and near <= z = D/S <= far (the centre need not be covered);
+ *                   - the pixel's fragments are sorted by z (ties to the lower index) and composited front to
+ *                     back, consecutive fragments of one surface -- map triangles of one class; the
+ *                     triangles of one box -- first being merged into one layer whose coverage A is the
+ *                     sum of theirs (at most 1) and whose colour is their coverage-weighted mean:
+ *                     C = sum_g T_g A_g C_g + T_end C_background, T_g = prod_{h<g} (1 - A_h);
+ *                   - box triangles whose outer side is turned away from the camera centre are not drawn
+ *                     (a box seen from outside looks the same without them, and they must not be merged
+ *                     with the faces in front of them).
+ *                 Pieces of one surface that tile the plane therefore add up to full coverage (no seams
+ *                 inside a mesh, none along the edge between two faces of a box), and a strip thinner than a
+ *                 pixel contributes its area.  Flags: 2 where two
+ *                 fragments of different surfaces that both show are within the O8 depth width of each
+ *                 other, 4 where a fragment that shows sits on the near or far plane, 8 on the horizon row
+ *                 of a visible background, 32 as in O10.  Edge flags (1) do not apply: the colour is
+ *                 continuous in the position of an edge.
  *
  * Parity pins: tests/test_oracle_*.py (closed forms, invariants, an independent ray caster,
  * hand-counted tiny scenes, numpy's binary16 conversion).  No function here is unpinned.
@@ -85,6 +117,7 @@ typedef struct {
     uint8_t cls;
     uint8_t ghost;    /* O10: just outside its angular range -- not drawn, but its pixels are flagged */
     uint8_t unsure;   /* O10: within 1e-5 of its angular limit, on either side */
+    uint8_t back;     /* O12: a box triangle whose outer side is turned away from the camera centre */
 } prim_t;
 
 typedef struct {
@@ -143,6 +176,7 @@ static void setup_prim(prim_t* p, v3 V0, v3 V1, v3 V2, int32_t index, uint8_t cl
     p->cls = cls;
     p->ghost = 0;
     p->unsure = 0;
+    p->back = 0;
 }
 
 /* O10: cosine of the angle between the triangle's normal (by vertex order) and the direction from its
@@ -230,6 +264,64 @@ static int meets_frustum(v3 V0, v3 V1, v3 V2, double tx, double ty, double near,
     return n > 0;
 }
 
+/* O3 + O4: every primitive of environment e as seen by camera c of ego a (the ego and inactive agents are
+   skipped), in index order; *t_vis counts those that meet the frustum (work counts only).  NULL on
+   allocation failure; the caller frees. */
+static prim_t* view_prims(const cam_t* c, int e, int a, int A, int H, int W, double near, double far,
+                          const int32_t* env_map_id, const int64_t* map_tri_offset,
+                          const float* tri_xyz, const uint8_t* tri_class, int agent_class,
+                          const float* poses, const float* dims, const uint8_t* active,
+                          const uint8_t* agent_classes, const float* tri_vis_cos,
+                          int64_t* np_out, int64_t* n_map_out, int64_t* t_vis_out)
+{
+    int m = env_map_id[e];
+    int64_t t0 = map_tri_offset[m], t1 = map_tri_offset[m + 1];
+    int64_t n_map = t1 - t0;
+    int64_t n_prim = n_map + 12 * (int64_t)A;
+    prim_t* prim = (prim_t*)malloc(sizeof(prim_t) * (size_t)(n_prim > 0 ? n_prim : 1));
+    if (!prim) return NULL;
+    int64_t np = 0, t_vis = 0;
+    double tx = (W / 2.0) / c->fx, ty = (H / 2.0) / c->fy;
+    for (int64_t t = 0; t < n_map; ++t) {
+        const float* p = tri_xyz + 9 * (size_t)(t0 + t);
+        v3 X0 = { p[0], p[1], p[2] }, X1 = { p[3], p[4], p[5] }, X2 = { p[6], p[7], p[8] };
+        v3 V0 = to_camera(c, X0), V1 = to_camera(c, X1), V2 = to_camera(c, X2);
+        setup_prim(&prim[np], V0, V1, V2, (int32_t)t, tri_class[t0 + t]);
+        if (tri_vis_cos && tri_vis_cos[t0 + t] > 0.0f) {          /* O10: one-sided, limited angular range */
+            double lim = (double)tri_vis_cos[t0 + t], cosang = facing_cosine(V0, V1, V2);
+            if (fabs(cosang - lim) <= REL_TOL) prim[np].unsure = 1;
+            if (!(cosang >= lim)) {
+                if (prim[np].unsure) prim[np].ghost = 1;
+                else prim[np].D = 0.0;                             /* absent from this view */
+            }
+        }
+        if (prim[np].D != 0.0 && !prim[np].ghost && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
+        ++np;
+    }
+    for (int b = 0; b < A; ++b) {
+        if (b == a) continue;                                   /* the ego is never drawn */
+        if (active && !active[(size_t)e * A + b]) continue;
+        v3 tri[12][3];
+        box_triangles(poses + 3 * ((size_t)e * A + b), dims + 3 * ((size_t)e * A + b), tri);
+        v3 centre = { poses[3 * ((size_t)e * A + b)], poses[3 * ((size_t)e * A + b) + 1], 0.5 * dims[3 * ((size_t)e * A + b) + 2] };
+        v3 Bc = to_camera(c, centre);
+        for (int t = 0; t < 12; ++t) {
+            v3 V0 = to_camera(c, tri[t][0]), V1 = to_camera(c, tri[t][1]), V2 = to_camera(c, tri[t][2]);
+            setup_prim(&prim[np], V0, V1, V2, (int32_t)(n_map + 12 * b + t),
+                       agent_classes ? agent_classes[(size_t)e * A + b] : (uint8_t)agent_class);
+            {   /* O12: the camera centre (the origin) and the box's centre on the same side of the triangle's plane */
+                v3 nrm = v3_cross(v3_sub(V1, V0), v3_sub(V2, V0));
+                double s_cam = -v3_dot(nrm, V0), s_box = v3_dot(nrm, v3_sub(Bc, V0));
+                prim[np].back = !(s_cam * s_box < 0.0);
+            }
+            if (prim[np].D != 0.0 && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
+            ++np;
+        }
+    }
+    *np_out = np; *n_map_out = n_map; *t_vis_out = t_vis;
+    return prim;
+}
+
 /*
  * Render the listed views.  view_ids[i] = (e*A + a)*K + k.  Outputs are [n_views, H, W]:
  *   out_class  u8      O6/O7 class
@@ -288,44 +380,11 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
         make_camera(&c, poses + 3 * ((size_t)e * A + a), cam, H, W);
 
         /* O3 + O4 set-up of every primitive of the environment */
-        int m = env_map_id[e];
-        int64_t t0 = map_tri_offset[m], t1 = map_tri_offset[m + 1];
-        int64_t n_map = t1 - t0;
-        int64_t n_prim = n_map + 12 * (int64_t)A;
-        prim_t* prim = (prim_t*)malloc(sizeof(prim_t) * (size_t)n_prim);
-        uint8_t* hit = (uint8_t*)calloc((size_t)n_prim, 1);
+        int64_t np = 0, n_map = 0, t_vis = 0;
+        prim_t* prim = view_prims(&c, e, a, A, H, W, near, far, env_map_id, map_tri_offset, tri_xyz, tri_class, agent_class,
+                                  poses, dims, active, agent_classes, tri_vis_cos, &np, &n_map, &t_vis);
+        uint8_t* hit = prim ? (uint8_t*)calloc((size_t)np + 1, 1) : NULL;
         if (!prim || !hit) { free(prim); free(hit); failed = 1; break; }
-        int64_t np = 0, t_vis = 0;
-        double tx = (W / 2.0) / c.fx, ty = (H / 2.0) / c.fy;
-        for (int64_t t = 0; t < n_map; ++t) {
-            const float* p = tri_xyz + 9 * (size_t)(t0 + t);
-            v3 X0 = { p[0], p[1], p[2] }, X1 = { p[3], p[4], p[5] }, X2 = { p[6], p[7], p[8] };
-            v3 V0 = to_camera(&c, X0), V1 = to_camera(&c, X1), V2 = to_camera(&c, X2);
-            setup_prim(&prim[np], V0, V1, V2, (int32_t)t, tri_class[t0 + t]);
-            if (tri_vis_cos && tri_vis_cos[t0 + t] > 0.0f) {          /* O10: one-sided, limited angular range */
-                double lim = (double)tri_vis_cos[t0 + t], cosang = facing_cosine(V0, V1, V2);
-                if (fabs(cosang - lim) <= REL_TOL) prim[np].unsure = 1;
-                if (!(cosang >= lim)) {
-                    if (prim[np].unsure) prim[np].ghost = 1;
-                    else prim[np].D = 0.0;                             /* absent from this view */
-                }
-            }
-            if (prim[np].D != 0.0 && !prim[np].ghost && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
-            ++np;
-        }
-        for (int b = 0; b < A; ++b) {
-            if (b == a) continue;                                   /* the ego is never drawn */
-            if (active && !active[(size_t)e * A + b]) continue;
-            v3 tri[12][3];
-            box_triangles(poses + 3 * ((size_t)e * A + b), dims + 3 * ((size_t)e * A + b), tri);
-            for (int t = 0; t < 12; ++t) {
-                v3 V0 = to_camera(&c, tri[t][0]), V1 = to_camera(&c, tri[t][1]), V2 = to_camera(&c, tri[t][2]);
-                setup_prim(&prim[np], V0, V1, V2, (int32_t)(n_map + 12 * b + t),
-                           agent_classes ? agent_classes[(size_t)e * A + b] : (uint8_t)agent_class);
-                if (prim[np].D != 0.0 && meets_frustum(V0, V1, V2, tx, ty, near, far)) ++t_vis;
-                ++np;
-            }
-        }
 
         int64_t n_frag = 0, n_flag = 0;
 #pragma omp parallel for schedule(dynamic, 1) reduction(+ : n_frag, n_flag)
@@ -427,6 +486,275 @@ int pico_render(int E, int A, int K, int H, int W, double near, double far,
         }
         free(prim);
         free(hit);
+    }
+    return failed ? -1 : 0;
+}
+
+/* O12, one edge alone (kept for the pins of the clipper below, which the renderer uses): fraction of the unit
+   square around a pixel centre on which a linear function is positive, given its
+   value e0 at the centre and its increments a, b per pixel in x and y.  With A = |a|, B = |b| the function
+   ranges over e0 +- (A + B)/2 on the square; the fraction is 1/2 + e0/max(A,B) on the middle stretch
+   |e0| <= |A - B|/2 (the boundary crosses two opposite sides) and a quadratic where it cuts off a corner. */
+double pico_edge_coverage(double e0, double a, double b) {
+    double A = fabs(a), B = fabs(b);
+    double h = 0.5 * (A + B);
+    if (e0 >= h) return (e0 > 0.0 || h > 0.0) ? 1.0 : 0.0;     /* (a constant zero function is nowhere positive) */
+    if (e0 <= -h) return 0.0;
+    double hi = fmax(A, B), lo = fmin(A, B), g = 0.5 * (hi - lo);
+    if (fabs(e0) <= g) return 0.5 + e0 / hi;
+    if (e0 < 0.0) return (e0 + h) * (e0 + h) / (2.0 * A * B);
+    return 1.0 - (h - e0) * (h - e0) / (2.0 * A * B);
+}
+
+/* O12: area of the part of the unit square around a pixel centre on which all three linear functions
+   e[i] + a[i] x + b[i] y are non-negative (Sutherland-Hodgman clipping of the square, then the shoelace formula). */
+double pico_pixel_coverage(const double e[3], const double a[3], const double b[3]) {
+    double px[16] = { -0.5, 0.5, 0.5, -0.5 }, py[16] = { -0.5, -0.5, 0.5, 0.5 };
+    int n = 4;
+    for (int i = 0; i < 3 && n > 0; ++i) {
+        double qx[16], qy[16];
+        int m = 0;
+        for (int k = 0; k < n; ++k) {
+            int k1 = (k + 1) % n;
+            double f0 = e[i] + a[i] * px[k] + b[i] * py[k], f1 = e[i] + a[i] * px[k1] + b[i] * py[k1];
+            if (f0 >= 0.0) { qx[m] = px[k]; qy[m] = py[k]; ++m; }
+            if ((f0 >= 0.0) != (f1 >= 0.0)) {
+                double t = f0 / (f0 - f1);
+                qx[m] = px[k] + t * (px[k1] - px[k]); qy[m] = py[k] + t * (py[k1] - py[k]); ++m;
+            }
+        }
+        n = m;
+        memcpy(px, qx, sizeof(double) * (size_t)n);
+        memcpy(py, qy, sizeof(double) * (size_t)n);
+    }
+    if (n < 3) return 0.0;
+    double twice = 0.0;
+    for (int k = 0; k < n; ++k) { int k1 = (k + 1) % n; twice += px[k] * py[k1] - px[k1] * py[k]; }
+    return 0.5 * fabs(twice);
+}
+
+static const double FACE_SHADE[6] = { 0.60, 1.00, 0.70, 0.85, 0.40, 0.92 };   /* rear, front, right, left, bottom, top */
+
+/* O11: colour (0..255 per channel, not yet rounded) of a fragment of primitive p at depth z. */
+static void shade(const prim_t* p, int64_t n_map, double z, double near, double far, const uint8_t* palette, double rgb[3]) {
+    double k = 1.0;
+    if (p->index >= n_map) {
+        int face = (int)((p->index - n_map) % 12) / 2;
+        k = FACE_SHADE[face] * (1.0 - 0.5 * (z - near) / (far - near));
+    }
+    for (int ch = 0; ch < 3; ++ch) rgb[ch] = k * (double)palette[3 * p->cls + ch];
+}
+
+/* O12: which fragments merge -- map triangles of one class; the triangles of one box. */
+static int64_t surface_of(const prim_t* p, int64_t n_map) {
+    return (p->index < n_map) ? (int64_t)p->cls : 256 + (p->index - n_map) / 12;
+}
+/* (ii) of O8 in colour: do two primitives show different colours -- another class, or another face of a box */
+static int64_t colour_of(const prim_t* p, int64_t n_map) {
+    return (p->index < n_map) ? (int64_t)p->cls : 256 + (p->index - n_map) / 2;
+}
+
+typedef struct { double z, alpha, kappa; int64_t j; } frag_t;
+
+static int frag_before(const frag_t* a, const frag_t* b, const prim_t* prim) {
+    return a->z < b->z || (a->z == b->z && prim[a->j].index < prim[b->j].index);
+}
+
+/*
+ * Render the listed views in colour (O11), optionally antialiased (O12).  Arguments as pico_render;
+ *   palette  u8 [256,3]  RGB of every class
+ *   aa       0: a pixel shows its O6 winner; 1: analytic coverage (O12)
+ *   out_rgb  u8  [n_views,H,W,3]   rounded colour
+ *   out_rgbf f64 [n_views,H,W,3]   the colour before rounding (0..255)
+ *   out_flag u8  [n_views,H,W]     aa 0: the O8 mask of pico_render with "another class" read as "another
+ *                                  surface or class" in (ii); aa 1: the flags listed under O12
+ * Any output pointer may be NULL.  Returns 0, or -1 on allocation failure.
+ */
+int pico_render_rgb(int E, int A, int K, int H, int W, double near, double far,
+                    const int32_t* env_map_id, const int64_t* map_tri_offset,
+                    const float* tri_xyz, const uint8_t* tri_class,
+                    int agent_class, int sky_class, int ground_class,
+                    const float* poses, const float* dims, const uint8_t* active, const float* rig,
+                    const uint8_t* agent_classes, const float* tri_vis_cos,
+                    const uint8_t* palette, int aa,
+                    int n_views, const int64_t* view_ids,
+                    uint8_t* out_rgb, double* out_rgbf, uint8_t* out_flag, int n_threads)
+{
+    (void)E;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+    int failed = 0;
+    for (int vi = 0; vi < n_views; ++vi) {
+        int64_t id = view_ids[vi];
+        int k = (int)(id % K);
+        int a = (int)((id / K) % A);
+        int e = (int)(id / ((int64_t)K * A));
+        size_t base = (size_t)vi * (size_t)H * (size_t)W;
+        const float* cam = rig + 7 * k;
+        if (active && !active[(size_t)e * A + a]) {          /* inactive ego: sky everywhere */
+            for (size_t p = 0; p < (size_t)H * W; ++p) {
+                for (int ch = 0; ch < 3; ++ch) {
+                    if (out_rgb) out_rgb[3 * (base + p) + ch] = palette[3 * sky_class + ch];
+                    if (out_rgbf) out_rgbf[3 * (base + p) + ch] = (double)palette[3 * sky_class + ch];
+                }
+                if (out_flag) out_flag[base + p] = 0;
+            }
+            continue;
+        }
+        cam_t c;
+        make_camera(&c, poses + 3 * ((size_t)e * A + a), cam, H, W);
+        int64_t np = 0, n_map = 0, t_vis = 0;
+        prim_t* prim = view_prims(&c, e, a, A, H, W, near, far, env_map_id, map_tri_offset, tri_xyz, tri_class, agent_class,
+                                  poses, dims, active, agent_classes, tri_vis_cos, &np, &n_map, &t_vis);
+        if (!prim) { failed = 1; break; }
+        int alloc_failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+        for (int v = 0; v < H; ++v) {
+            frag_t* fr = aa ? (frag_t*)malloc(sizeof(frag_t) * (size_t)(np > 0 ? np : 1)) : NULL;
+            if (aa && !fr) {
+#pragma omp atomic write
+                alloc_failed = 1;
+                continue;
+            }
+            for (int u = 0; u < W; ++u) {
+                v3 rho = { (u + 0.5 - c.cx) / c.fx, (v + 0.5 - c.cy) / c.fy, 1.0 };
+                double rho_n = v3_norm(rho);
+                double w = -rho.y * cos(c.pitch) + sin(c.pitch);
+                int bg_ground = (w < 0.0 && c.cz > 0.0);
+                int bg_class = bg_ground ? ground_class : sky_class;
+                double rgb[3] = { 0.0, 0.0, 0.0 };
+                uint8_t flag = 0;
+                if (!aa) {
+                    /* O4-O6 as in pico_render */
+                    double z_win = 0.0, k_win = 0.0; int64_t j_win = -1;
+                    for (int64_t j = 0; j < np; ++j) {
+                        const prim_t* p = &prim[j];
+                        if (p->D == 0.0 || p->ghost) continue;
+                        int covered = 1;
+                        double S = 0.0;
+                        for (int i = 0; i < 3; ++i) {
+                            double Ei = v3_dot(rho, p->N[i]);
+                            S += Ei;
+                            if (Ei > 0.0) continue;
+                            if (Ei == 0.0 && (p->N[i].x > 0.0 || (p->N[i].x == 0.0 && p->N[i].y > 0.0))) continue;
+                            covered = 0;
+                        }
+                        if (!covered || !(S > 0.0)) continue;
+                        double z = p->D / S;
+                        if (z < near || z > far) continue;
+                        if (j_win < 0 || z < z_win || (z == z_win && p->index < prim[j_win].index)) { z_win = z; j_win = j; k_win = p->kappa; }
+                    }
+                    if (j_win >= 0) shade(&prim[j_win], n_map, z_win, near, far, palette, rgb);
+                    else for (int ch = 0; ch < 3; ++ch) rgb[ch] = (double)palette[3 * bg_class + ch];
+                    /* O8 with surfaces in place of classes in (ii) */
+                    if (j_win < 0 && fabs(w) <= REL_TOL) flag |= 8;
+                    if (j_win >= 0 && k_win > GRAZING_KAPPA) flag |= 16;
+                    for (int64_t j = 0; j < np; ++j) {
+                        const prim_t* p = &prim[j];
+                        if (p->D == 0.0) continue;
+                        double S = 0.0;
+                        int inside_band = 1, on_band = 0, covered = 1;
+                        for (int i = 0; i < 3; ++i) {
+                            double Ei = v3_dot(rho, p->N[i]);
+                            S += Ei;
+                            double band = p->band[i] * rho_n;
+                            if (Ei < -band) inside_band = 0;
+                            if (fabs(Ei) <= band) on_band = 1;
+                            if (!(Ei > 0.0 || (Ei == 0.0 && (p->N[i].x > 0.0 || (p->N[i].x == 0.0 && p->N[i].y > 0.0))))) covered = 0;
+                        }
+                        if (!(S > 0.0)) continue;
+                        double z = p->D / S;
+                        int could_show = (j_win < 0) || (z <= (1.0 + REL_TOL) * z_win);
+                        if (inside_band && on_band && could_show && z >= near * (1.0 - REL_TOL) && z <= far * (1.0 + REL_TOL)) flag |= 1;
+                        if (!covered) continue;
+                        if (p->unsure && z >= near && z <= far && could_show) flag |= 32;
+                        if (p->ghost) continue;
+                        if (j_win >= 0 && z >= near && z <= far &&
+                            (p->cls != prim[j_win].cls || colour_of(p, n_map) != colour_of(&prim[j_win], n_map)) &&
+                            fabs(z - z_win) <= fmax(REL_TOL, DEPTH_KAPPA * fmax(p->kappa, k_win)) * z_win) flag |= 2;
+                        if ((fabs(z - near) <= REL_TOL * near || fabs(z - far) <= REL_TOL * far) && could_show) flag |= 4;
+                    }
+                } else {
+                    /* O12: the pixel's fragments */
+                    int64_t nf = 0;
+                    int edge_of_range = 0, unsure = 0;
+                    for (int64_t j = 0; j < np; ++j) {
+                        const prim_t* p = &prim[j];
+                        if (p->D == 0.0 || p->back) continue;
+                        double S = 0.0, Ei[3], ax[3], by[3];
+                        for (int i = 0; i < 3; ++i) {
+                            Ei[i] = v3_dot(rho, p->N[i]);
+                            ax[i] = p->N[i].x / c.fx;                /* increments of E_i per pixel in x and y */
+                            by[i] = p->N[i].y / c.fy;
+                            S += Ei[i];
+                        }
+                        if (!(S > 0.0)) continue;
+                        double alpha = pico_pixel_coverage(Ei, ax, by);
+                        if (!(alpha > 0.0)) continue;
+                        double z = p->D / S;
+                        if (alpha >= 1e-3 && (fabs(z - near) <= REL_TOL * near || fabs(z - far) <= REL_TOL * far)) edge_of_range = 1;
+                        if (z < near || z > far) continue;
+                        if (p->unsure && alpha >= 1e-3) unsure = 1;
+                        if (p->ghost) continue;
+                        fr[nf].z = z; fr[nf].alpha = alpha; fr[nf].kappa = p->kappa; fr[nf].j = j;
+                        ++nf;
+                    }
+                    for (int64_t i = 1; i < nf; ++i) {          /* insertion sort by (z, index) */
+                        frag_t x = fr[i];
+                        int64_t q = i;
+                        while (q > 0 && frag_before(&x, &fr[q - 1], prim)) { fr[q] = fr[q - 1]; --q; }
+                        fr[q] = x;
+                    }
+                    /* front to back, the fragments of one surface merged into one layer */
+                    double T = 1.0;
+                    int64_t shown_end = 0;                      /* fragments [0, shown_end) show */
+                    for (int64_t i = 0; i < nf && T > 0.0;) {
+                        int64_t surf = surface_of(&prim[fr[i].j], n_map);
+                        double Acc = 0.0, sum[3] = { 0.0, 0.0, 0.0 };
+                        int64_t q = i;
+                        while (q < nf && surface_of(&prim[fr[q].j], n_map) == surf) {
+                            double col[3];
+                            shade(&prim[fr[q].j], n_map, fr[q].z, near, far, palette, col);
+                            for (int ch = 0; ch < 3; ++ch) sum[ch] += fr[q].alpha * col[ch];
+                            Acc += fr[q].alpha;
+                            ++q;
+                        }
+                        /* the layer's colour is the coverage-weighted mean of its fragments', its coverage at most 1 */
+                        double wgt = (Acc > 1.0) ? 1.0 / Acc : 1.0;
+                        if (Acc > 1.0) Acc = 1.0;
+                        for (int ch = 0; ch < 3; ++ch) rgb[ch] += T * wgt * sum[ch];
+                        T *= 1.0 - Acc;
+                        i = q;
+                        shown_end = q;
+                    }
+                    for (int ch = 0; ch < 3; ++ch) rgb[ch] += T * (double)palette[3 * bg_class + ch];
+                    /* flags */
+                    if (T > 1e-3 && fabs(w) <= REL_TOL) flag |= 8;
+                    if (edge_of_range) flag |= 4;
+                    if (unsure) flag |= 32;
+                    for (int64_t i = 0; i + 1 < shown_end + 1 && i + 1 < nf; ++i) {
+                        /* neighbours in depth order of different surfaces, the nearer of which shows */
+                        const frag_t *x = &fr[i], *y = &fr[i + 1];
+                        if (i >= shown_end) break;
+                        if (surface_of(&prim[x->j], n_map) == surface_of(&prim[y->j], n_map)) continue;
+                        if (x->alpha < 1e-3 && y->alpha < 1e-3) continue;
+                        if (fabs(y->z - x->z) <= fmax(REL_TOL, DEPTH_KAPPA * fmax(x->kappa, y->kappa)) * x->z) flag |= 2;
+                    }
+                }
+                size_t o = base + (size_t)v * W + u;
+                for (int ch = 0; ch < 3; ++ch) {
+                    if (out_rgbf) out_rgbf[3 * o + ch] = rgb[ch];
+                    if (out_rgb) out_rgb[3 * o + ch] = (uint8_t)floor(rgb[ch] + 0.5);
+                }
+                if (out_flag) out_flag[o] = flag;
+            }
+            free(fr);
+        }
+        free(prim);
+        if (alloc_failed) { failed = 1; break; }
     }
     return failed ? -1 : 0;
 }

@@ -33,6 +33,13 @@ def _load():
         lib.pico_render.restype = C.c_int
         lib.pico_render.argtypes = [C.c_int] * 5 + [C.c_double] * 2 + [p] * 4 + [C.c_int] * 3 + [p] * 6 + \
                                    [C.c_int, p] + [p] * 7 + [C.c_int]
+        lib.pico_render_rgb.restype = C.c_int
+        lib.pico_render_rgb.argtypes = [C.c_int] * 5 + [C.c_double] * 2 + [p] * 4 + [C.c_int] * 3 + [p] * 6 + \
+                                       [p, C.c_int] + [C.c_int, p] + [p] * 3 + [C.c_int]
+        lib.pico_edge_coverage.restype = C.c_double
+        lib.pico_edge_coverage.argtypes = [C.c_double] * 3
+        lib.pico_pixel_coverage.restype = C.c_double
+        lib.pico_pixel_coverage.argtypes = [p] * 3
         lib.pico_step.restype = None
         lib.pico_step.argtypes = [p, p, p, C.c_int64, C.c_double, C.c_double, C.c_double]
         lib.pico_f64_to_f16.restype = C.c_uint16
@@ -98,6 +105,62 @@ def render(scene, view_ids: Optional[Sequence[int]] = None, poses: Optional[np.n
     if rc != 0:
         raise MemoryError("pico_render failed")
     return OracleResult(view_ids, cls, depth, f16.view(np.float16), index, flag, kappa, counts)
+
+
+@dataclass
+class OracleColour:
+    view_ids: np.ndarray     # int64 [n]
+    rgb: np.ndarray          # u8  [n,H,W,3]  rounded colour
+    rgbf: np.ndarray         # f64 [n,H,W,3]  colour before rounding, 0..255
+    flag: np.ndarray         # u8  [n,H,W]    ambiguity mask (see pico_render_rgb)
+
+
+def render_rgb(scene, palette: np.ndarray, aa: bool, view_ids: Optional[Sequence[int]] = None,
+               poses: Optional[np.ndarray] = None, n_threads: int = 0) -> OracleColour:
+    """Colour images (O11) of views of `scene`, antialiased by analytic coverage (O12) if `aa`.
+    palette: u8 [256,3], the RGB of every class."""
+    lib = _load()
+    s = scene
+    if view_ids is None:
+        view_ids = np.arange(s.E * s.A * s.K, dtype=np.int64)
+    view_ids = np.ascontiguousarray(view_ids, dtype=np.int64)
+    n = int(view_ids.shape[0])
+    poses = np.ascontiguousarray(s.poses if poses is None else poses, dtype=np.float32)
+    dims = np.ascontiguousarray(s.dims, dtype=np.float32)
+    active = np.ascontiguousarray(s.active, dtype=np.uint8)
+    rig = np.ascontiguousarray(s.rig, dtype=np.float32)
+    tri = np.ascontiguousarray(s.tri_xyz, dtype=np.float32)
+    tcl = np.ascontiguousarray(s.tri_class, dtype=np.uint8)
+    emi = np.ascontiguousarray(s.env_map_id, dtype=np.int32)
+    off = np.ascontiguousarray(s.map_tri_offset, dtype=np.int64)
+    acl = getattr(s, "agent_classes", None)
+    acl = None if acl is None else np.ascontiguousarray(acl, dtype=np.uint8)
+    vis = getattr(s, "tri_vis_cos", None)
+    vis = None if vis is None else np.ascontiguousarray(vis, dtype=np.float32)
+    pal = np.ascontiguousarray(palette, dtype=np.uint8)
+    assert pal.shape == (256, 3)
+    rgb = np.empty((n, s.H, s.W, 3), np.uint8)
+    rgbf = np.empty((n, s.H, s.W, 3), np.float64)
+    flag = np.empty((n, s.H, s.W), np.uint8)
+    rc = lib.pico_render_rgb(s.E, s.A, s.K, s.H, s.W, float(s.near), float(s.far), _ptr(emi), _ptr(off), _ptr(tri),
+                             _ptr(tcl), int(s.agent_class), int(s.sky_class), int(s.ground_class), _ptr(poses),
+                             _ptr(dims), _ptr(active), _ptr(rig), _ptr(acl), _ptr(vis), _ptr(pal), int(bool(aa)),
+                             n, _ptr(view_ids), _ptr(rgb), _ptr(rgbf), _ptr(flag), int(n_threads))
+    if rc != 0:
+        raise MemoryError("pico_render_rgb failed")
+    return OracleColour(view_ids, rgb, rgbf, flag)
+
+
+def edge_coverage(e0: float, a: float, b: float) -> float:
+    """O12: fraction of a pixel's unit square on which the linear function e0 + a x + b y is positive."""
+    return float(_load().pico_edge_coverage(float(e0), float(a), float(b)))
+
+
+def pixel_coverage(e, a, b) -> float:
+    """O12: area of the part of a pixel's unit square on which the three linear functions e[i] + a[i] x + b[i] y are >= 0."""
+    e, a, b = (np.ascontiguousarray(x, dtype=np.float64) for x in (e, a, b))
+    assert e.shape == a.shape == b.shape == (3,)
+    return float(_load().pico_pixel_coverage(_ptr(e), _ptr(a), _ptr(b)))
 
 
 def step(state: np.ndarray, actions: np.ndarray, active: Optional[np.ndarray], dt: float, wheelbase: float,

@@ -34,6 +34,29 @@ CLASS_ROAD = 2
 CLASS_MARKING = 3
 CLASS_VEHICLE = 4
 
+CLASS_SIGNAL = 6
+CLASS_CYCLIST = 7
+CLASS_PEDESTRIAN = 8
+
+
+def default_palette() -> np.ndarray:
+    """An RGB triple per class id, u8 [256,3] (input of the colour output): sky, ground, road, markings, one hue per
+    kind of road user, signals; every other class a grey that depends on its id."""
+    pal = np.zeros((256, 3), np.uint8)
+    for c in range(256):
+        pal[c] = 40 + (c * 37) % 160
+    pal[CLASS_SKY] = (135, 190, 235)
+    pal[CLASS_GROUND] = (96, 124, 84)
+    pal[CLASS_ROAD] = (72, 72, 76)
+    pal[CLASS_MARKING] = (240, 240, 230)
+    pal[CLASS_VEHICLE] = (40, 110, 220)
+    pal[5] = (150, 120, 100)
+    pal[CLASS_SIGNAL] = (230, 40, 40)
+    pal[CLASS_CYCLIST] = (240, 150, 30)
+    pal[CLASS_PEDESTRIAN] = (220, 50, 200)
+    return pal
+
+
 ROAD_WIDTH = 7.5          # two lanes
 LANE_OFFSET = 1.875       # lane centre to road centre-line
 DASH_WIDTH = 0.15
