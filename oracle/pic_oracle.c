@@ -60,12 +60,13 @@
  *  O12 antialiasing (Sec. 3.2: analytic-coverage antialiasing at a single sample per pixel, so that thin
  *                 structures stay visible at low resolution.)  No formula is given; the reading is a box
  *                 filter over the pixel's unit square, evaluated exactly:
- *                   - the edge functions E_i = rho.N_i are linear in the pixel coordinates, so the part of
- *                     the pixel's square inside all three edges is a convex polygon; a primitive's coverage
- *                     alpha is that polygon's area (the square clipped by the three lines; for a single edge
- *                     crossing the pixel this is the closed form of pico_edge_coverage);
- *                   - it leaves a fragment at every pixel with alpha > 0 whose plane, evaluated at the pixel
- *                     centre, has S > 0 and near <= z = D/S <= far (the centre need not be covered);
+ *                   - the edge functions E_i = rho.N_i and their sum S are linear in the pixel coordinates,
+ *                     so the part of the pixel's square inside all three edges and within the depth range
+ *                     (D/far <= S <= D/near) is a convex polygon; a primitive's coverage alpha is that
+ *                     polygon's area (the square clipped by the five lines; for a single line crossing the
+ *                     pixel this is the closed form of pico_edge_coverage);
+ *                   - it leaves a fragment at every pixel with alpha > 0, at the depth z of its plane at the
+ *                     pixel centre (the centre need not be covered), clamped to [near, far];
  *                   - the pixel's fragments are sorted by z (ties to the lower index) and composited front to
  *                     back, consecutive fragments of one surface -- map triangles of one class; the
  *                     triangles of one box -- first being merged into one layer whose coverage A is the
@@ -78,7 +79,7 @@
  *                 inside a mesh, none along the edge between two faces of a box), and a strip thinner than a
  *                 pixel contributes its area.  Flags: 2 where two
  *                 fragments of different surfaces that both show are within the O8 depth width of each
- *                 other, 4 where a fragment that shows sits on the near or far plane, 8 on the horizon row
+ *                 other, 8 on the horizon row
  *                 of a visible background, 32 as in O10.  Edge flags (1) do not apply: the colour is
  *                 continuous in the position of an edge.
  *
@@ -506,12 +507,12 @@ double pico_edge_coverage(double e0, double a, double b) {
     return 1.0 - (h - e0) * (h - e0) / (2.0 * A * B);
 }
 
-/* O12: area of the part of the unit square around a pixel centre on which all three linear functions
+/* O12: area of the part of the unit square around a pixel centre on which all nl (at most 8) linear functions
    e[i] + a[i] x + b[i] y are non-negative (Sutherland-Hodgman clipping of the square, then the shoelace formula). */
-double pico_pixel_coverage(const double e[3], const double a[3], const double b[3]) {
+double pico_pixel_coverage(int nl, const double* e, const double* a, const double* b) {
     double px[16] = { -0.5, 0.5, 0.5, -0.5 }, py[16] = { -0.5, -0.5, 0.5, 0.5 };
     int n = 4;
-    for (int i = 0; i < 3 && n > 0; ++i) {
+    for (int i = 0; i < nl && n > 0; ++i) {
         double qx[16], qy[16];
         int m = 0;
         for (int k = 0; k < n; ++k) {
@@ -680,23 +681,26 @@ int pico_render_rgb(int E, int A, int K, int H, int W, double near, double far,
                 } else {
                     /* O12: the pixel's fragments */
                     int64_t nf = 0;
-                    int edge_of_range = 0, unsure = 0;
+                    int unsure = 0;
                     for (int64_t j = 0; j < np; ++j) {
                         const prim_t* p = &prim[j];
                         if (p->D == 0.0 || p->back) continue;
-                        double S = 0.0, Ei[3], ax[3], by[3];
+                        double S = 0.0, Ei[5], ax[5], by[5];
+                        ax[3] = 0.0; by[3] = 0.0;
                         for (int i = 0; i < 3; ++i) {
                             Ei[i] = v3_dot(rho, p->N[i]);
                             ax[i] = p->N[i].x / c.fx;                /* increments of E_i per pixel in x and y */
                             by[i] = p->N[i].y / c.fy;
                             S += Ei[i];
+                            ax[3] += ax[i]; by[3] += by[i];
                         }
-                        if (!(S > 0.0)) continue;
-                        double alpha = pico_pixel_coverage(Ei, ax, by);
+                        Ei[3] = S - p->D / far;  /* z <= far */
+                        Ei[4] = p->D / near - S; ax[4] = -ax[3]; by[4] = -by[3];   /* z >= near */
+                        double alpha = pico_pixel_coverage(5, Ei, ax, by);
                         if (!(alpha > 0.0)) continue;
-                        double z = p->D / S;
-                        if (alpha >= 1e-3 && (fabs(z - near) <= REL_TOL * near || fabs(z - far) <= REL_TOL * far)) edge_of_range = 1;
-                        if (z < near || z > far) continue;
+                        double z = (S > 0.0) ? p->D / S : far;
+                        if (z < near) z = near;
+                        if (z > far) z = far;
                         if (p->unsure && alpha >= 1e-3) unsure = 1;
                         if (p->ghost) continue;
                         fr[nf].z = z; fr[nf].alpha = alpha; fr[nf].kappa = p->kappa; fr[nf].j = j;
@@ -733,7 +737,6 @@ int pico_render_rgb(int E, int A, int K, int H, int W, double near, double far,
                     for (int ch = 0; ch < 3; ++ch) rgb[ch] += T * (double)palette[3 * bg_class + ch];
                     /* flags */
                     if (T > 1e-3 && fabs(w) <= REL_TOL) flag |= 8;
-                    if (edge_of_range) flag |= 4;
                     if (unsure) flag |= 32;
                     for (int64_t i = 0; i + 1 < shown_end + 1 && i + 1 < nf; ++i) {
                         /* neighbours in depth order of different surfaces, the nearer of which shows */

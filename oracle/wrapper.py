@@ -39,7 +39,7 @@ def _load():
         lib.pico_edge_coverage.restype = C.c_double
         lib.pico_edge_coverage.argtypes = [C.c_double] * 3
         lib.pico_pixel_coverage.restype = C.c_double
-        lib.pico_pixel_coverage.argtypes = [p] * 3
+        lib.pico_pixel_coverage.argtypes = [C.c_int] + [p] * 3
         lib.pico_step.restype = None
         lib.pico_step.argtypes = [p, p, p, C.c_int64, C.c_double, C.c_double, C.c_double]
         lib.pico_f64_to_f16.restype = C.c_uint16
@@ -157,10 +157,10 @@ def edge_coverage(e0: float, a: float, b: float) -> float:
 
 
 def pixel_coverage(e, a, b) -> float:
-    """O12: area of the part of a pixel's unit square on which the three linear functions e[i] + a[i] x + b[i] y are >= 0."""
+    """O12: area of the part of a pixel's unit square on which the linear functions e[i] + a[i] x + b[i] y (at most 8) are >= 0."""
     e, a, b = (np.ascontiguousarray(x, dtype=np.float64) for x in (e, a, b))
-    assert e.shape == a.shape == b.shape == (3,)
-    return float(_load().pico_pixel_coverage(_ptr(e), _ptr(a), _ptr(b)))
+    assert e.ndim == 1 and e.shape == a.shape == b.shape and len(e) <= 8
+    return float(_load().pico_pixel_coverage(len(e), _ptr(e), _ptr(a), _ptr(b)))
 
 
 def step(state: np.ndarray, actions: np.ndarray, active: Optional[np.ndarray], dt: float, wheelbase: float,

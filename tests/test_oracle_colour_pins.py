@@ -292,3 +292,21 @@ def test_antialiasing_changes_only_pixels_next_to_an_edge_and_flags_are_rare():
     assert same.mean() > 0.5 and (diff[same] > 0.5).mean() < 0.02
     assert (diff[~same] > 0.5).mean() > 0.2
     assert (a.flag != 0).mean() < 5e-3 and (a.flag & 1).sum() == 0
+
+
+def test_coverage_is_cut_at_the_near_and_far_planes_inside_a_pixel():
+    # a road quad on the ground from 1 m to 50 m ahead, camera 1 m up, fy = 4: depth d shows at row 4 + 4 / d.
+    # far = 8 falls on row 4.5 and near = 1.6 on row 6.5, the middles of pixel rows 4 and 6: half of each is in range
+    quad = [[(1.0, 30.0, 0.0), (50.0, 30.0, 0.0), (50.0, -30.0, 0.0)], [(1.0, 30.0, 0.0), (50.0, -30.0, 0.0), (1.0, -30.0, 0.0)]]
+    s = single_env(quad, [2, 2], [ego()], rig=RIG8, H=8, W=8, near=1.6, far=8.0)
+    r = oracle.render_rgb(s, PAL, True)
+    road = PAL[2].astype(float)
+    for u in range(8):
+        assert np.allclose(r.rgbf[0][4, u], 0.5 * road + 0.5 * GROUND, atol=1e-6)
+        assert np.allclose(r.rgbf[0][5, u], road, atol=1e-9)
+        assert np.allclose(r.rgbf[0][6, u], 0.5 * road + 0.5 * GROUND, atol=1e-6)
+        assert np.allclose(r.rgbf[0][7, u], GROUND, atol=1e-9) and np.allclose(r.rgbf[0][3, u], SKY, atol=1e-9)
+    # whether the quad ends at the far plane or runs on beyond it makes no difference
+    cut = [[(1.0, 30.0, 0.0), (8.0, 30.0, 0.0), (8.0, -30.0, 0.0)], [(1.0, 30.0, 0.0), (8.0, -30.0, 0.0), (1.0, -30.0, 0.0)]]
+    r2 = oracle.render_rgb(single_env(cut, [2, 2], [ego()], rig=RIG8, H=8, W=8, near=1.6, far=8.0), PAL, True)
+    assert np.allclose(r.rgbf, r2.rgbf, atol=1e-6)
