@@ -67,6 +67,10 @@ typedef enum {
 #define PIC_FLAG_NONFINITE_POSE 0x1u /* a pose, size or action was NaN/Inf (or a step overflowed): that agent is treated as
                                         inactive for the call -- its images are sky, nobody sees it -- and pic_step leaves
                                         its state as it was */
+#define PIC_FLAG_COLOUR_INCOMPLETE 0x2u /* pic_render_rgb: a 64 x 64 tile saw more primitives than its list holds (254) and shows
+                                           only the background */
+#define PIC_FLAG_COLOUR_FRAGMENTS 0x4u  /* pic_render_rgb, antialiased: an 8-row strip of a tile held more than 1023 partially
+                                           covered pixel fragments in front of its opaque surfaces; the surplus was dropped */
 
 /* One pinhole camera of the rig, in the agent frame (x forward, y left, z up). */
 typedef struct {
@@ -227,6 +231,32 @@ pic_status pic_get_kernel_times(pic_scene* scene, float* ms, int32_t capacity, i
  * for checking the hierarchy's invariants (out[5] == out[6] == 0).
  */
 pic_status pic_map_stats(const pic_scene_desc* desc, int64_t out[8]);
+
+/*
+ * Colour output: the paper's image format (Sec. 3.2, "I in [0,1]^(h x w x 3)": flat-shaded primitives,
+ * cuboids coloured per face with depth-aware brightness, each kind of road user in its own hue,
+ * analytic-coverage antialiasing at one sample per pixel).  The paper gives no formulas; this library's are:
+ *   colour   pic_set_palette gives every class id an RGB triple (host u8 [256][3]; copied, the call returns
+ *            when the copy is done; until it is called class c is the grey (c, c, c)).  A map triangle has its
+ *            class's colour; face f of an agent's box has its class's colour times s_f * beta(z),
+ *            s = (rear 0.60, front 1.00, right 0.70, left 0.85, bottom 0.40, top 0.92),
+ *            beta(z) = 1 - 0.5 (z - near) / (far - near), z the fragment's depth; ground and sky have their
+ *            classes' colours.  A channel is stored as floor(c + 0.5), c in [0, 255].
+ *   antialias == 0   a pixel shows the primitive that pic_render's class image shows there.
+ *   antialias != 0   box filter over the pixel's unit square.  A primitive's coverage of a pixel is the exact
+ *            area of the square inside its edges and within [near, far] along its plane; it leaves a fragment
+ *            wherever that area is positive, at the depth of its plane at the pixel centre.  A pixel's fragments are
+ *            composited front to back; consecutive fragments of one surface -- map triangles of one class, the
+ *            faces of one box (only those turned towards the camera are drawn) -- are first merged into one
+ *            layer -- nearest first, each adds its coverage, and its colour with that weight, until the layer is
+ *            full -- so meshes show no seams and a line thinner than a pixel keeps its share.
+ *   out_rgb  dev u8 [E, A, K, H, W, 3].  Arguments, view sub-range options, PIC_OPT_OUT_RELATIVE and
+ *            PIC_OPT_TIMING as in pic_render; the other options do not apply.
+ * Limits: see PIC_FLAG_COLOUR_INCOMPLETE and PIC_FLAG_COLOUR_FRAGMENTS (reported by pic_get_status, never silently).
+ */
+pic_status pic_set_palette(pic_scene* scene, const uint8_t* rgb_host, void* cuda_stream);
+pic_status pic_render_rgb(pic_scene* scene, const float* poses, const float* dims, const uint8_t* active,
+                          const pic_camera* rig_host, int32_t antialias, uint8_t* out_rgb, void* cuda_stream);
 
 /*
  * pic_render_static -- render without a scene object and without any allocation.

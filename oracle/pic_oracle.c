@@ -69,9 +69,9 @@
  *                     pixel centre (the centre need not be covered), clamped to [near, far];
  *                   - the pixel's fragments are sorted by z (ties to the lower index) and composited front to
  *                     back, consecutive fragments of one surface -- map triangles of one class; the
- *                     triangles of one box -- first being merged into one layer whose coverage A is the
- *                     sum of theirs (at most 1) and whose colour is their coverage-weighted mean:
- *                     C = sum_g T_g A_g C_g + T_end C_background, T_g = prod_{h<g} (1 - A_h);
+ *                     triangles of one box -- first being merged into one layer: nearest first, each adds
+ *                     its coverage (and its colour with that weight) until the layer's coverage A reaches 1:
+ *                     C = sum_g T_g (sum_i a_i C_i) + T_end C_background, T_g = prod_{h<g} (1 - A_h);
  *                   - box triangles whose outer side is turned away from the camera centre are not drawn
  *                     (a box seen from outside looks the same without them, and they must not be merged
  *                     with the faces in front of them).
@@ -79,7 +79,8 @@
  *                 inside a mesh, none along the edge between two faces of a box), and a strip thinner than a
  *                 pixel contributes its area.  Flags: 2 where two
  *                 fragments of different surfaces that both show are within the O8 depth width of each
- *                 other, 8 on the horizon row
+ *                 other, or where a fragment covering less than 1e-3 of the pixel lies between two fragments of
+ *                 one surface (whether those merge hangs on it), 8 on the horizon row
  *                 of a visible background, 32 as in O10.  Edge flags (1) do not apply: the colour is
  *                 continuous in the position of an edge.
  *
@@ -720,16 +721,14 @@ int pico_render_rgb(int E, int A, int K, int H, int W, double near, double far,
                         double Acc = 0.0, sum[3] = { 0.0, 0.0, 0.0 };
                         int64_t q = i;
                         while (q < nf && surface_of(&prim[fr[q].j], n_map) == surf) {
-                            double col[3];
+                            /* nearer fragments first: each adds its coverage until the layer is full */
+                            double col[3], add = fmin(fr[q].alpha, 1.0 - Acc);
                             shade(&prim[fr[q].j], n_map, fr[q].z, near, far, palette, col);
-                            for (int ch = 0; ch < 3; ++ch) sum[ch] += fr[q].alpha * col[ch];
-                            Acc += fr[q].alpha;
+                            for (int ch = 0; ch < 3; ++ch) sum[ch] += add * col[ch];
+                            Acc += add;
                             ++q;
                         }
-                        /* the layer's colour is the coverage-weighted mean of its fragments', its coverage at most 1 */
-                        double wgt = (Acc > 1.0) ? 1.0 / Acc : 1.0;
-                        if (Acc > 1.0) Acc = 1.0;
-                        for (int ch = 0; ch < 3; ++ch) rgb[ch] += T * wgt * sum[ch];
+                        for (int ch = 0; ch < 3; ++ch) rgb[ch] += T * sum[ch];
                         T *= 1.0 - Acc;
                         i = q;
                         shown_end = q;
@@ -738,6 +737,15 @@ int pico_render_rgb(int E, int A, int K, int H, int W, double near, double far,
                     /* flags */
                     if (T > 1e-3 && fabs(w) <= REL_TOL) flag |= 8;
                     if (unsure) flag |= 32;
+                    /* a fragment of negligible coverage (below 1e-3: a renderer in float32 may not see it at all) that
+                       separates two fragments of one surface decides whether those merge: ambiguous */
+                    for (int64_t i = 0; i < nf && i <= shown_end; ++i) {
+                        if (fr[i].alpha >= 1e-3) continue;
+                        int64_t q = i + 1;
+                        while (q < nf && fr[q].alpha < 1e-3) ++q;
+                        if (i >= 1 && q < nf && surface_of(&prim[fr[i - 1].j], n_map) == surface_of(&prim[fr[q].j], n_map) &&
+                            surface_of(&prim[fr[i].j], n_map) != surface_of(&prim[fr[q].j], n_map)) flag |= 2;
+                    }
                     for (int64_t i = 0; i + 1 < shown_end + 1 && i + 1 < nf; ++i) {
                         /* neighbours in depth order of different surfaces, the nearer of which shows */
                         const frag_t *x = &fr[i], *y = &fr[i + 1];

@@ -19,9 +19,11 @@ STATUS_NAMES = {0: "PIC_OK", 1: "PIC_ERR_INVALID_ARG", 2: "PIC_ERR_SHAPE", 3: "P
                 5: "PIC_ERR_CAPACITY", 6: "PIC_ERR_NONFINITE"}
 OPT_BRUTE_FORCE, OPT_DEPTH32, OPT_COUNTERS, OPT_VIEW_FIRST, OPT_VIEW_COUNT, OPT_TIMING, OPT_DEBUG_FLAGS, OPT_OUT_RELATIVE, OPT_OCCLUSION = 1, 2, 3, 4, 5, 6, 7, 8, 9
 FLAG_NONFINITE_POSE = 1
+FLAG_COLOUR_INCOMPLETE = 2
+FLAG_COLOUR_FRAGMENTS = 4
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_set_agent_classes", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
+           "pic_get_state", "pic_set_agent_classes", "pic_set_palette", "pic_render_rgb", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
            "pic_last_error", "pic_version"]
 
 
@@ -72,6 +74,8 @@ def load(path: Optional[str] = None):
     lib.pic_set_state.argtypes = [vp, vp, vp, vp, vp]
     lib.pic_get_state.argtypes = [vp, vp, vp]
     lib.pic_set_agent_classes.argtypes = [vp, vp, vp]
+    lib.pic_set_palette.argtypes = [vp, vp, vp]
+    lib.pic_render_rgb.argtypes = [vp, vp, vp, vp, C.POINTER(pic_camera), C.c_int32, vp, vp]
     lib.pic_step.argtypes = [vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     lib.pic_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
@@ -259,6 +263,26 @@ class Scene:
             _dev_ptr(active, torch.uint8, n) if active is not None else None, _rig_array(rig),
             _dev_ptr(out_class, torch.uint8, npx), _dev_ptr(out_depth, torch.float16, npx), _stream_ptr(stream)))
         return out_class, out_depth
+
+    def set_palette(self, palette, stream=None):
+        """palette: numpy u8 [256,3], the RGB of every class id (colour output)."""
+        pal = np.ascontiguousarray(palette, dtype=np.uint8)
+        if pal.shape != (256, 3):
+            raise ValueError("palette must be u8 [256,3]")
+        _check(self._lib, self._lib.pic_set_palette(self._h, pal.ctypes.data_as(C.c_void_p), _stream_ptr(stream)))
+
+    def render_rgb(self, poses, dims, rig, active=None, out_rgb=None, antialias=False, stream=None):
+        """Colour images, u8 [E,A,K,H,W,3] (with OPT_OUT_RELATIVE: [views rendered,H,W,3], which the caller sizes);
+        antialias: analytic coverage at one sample per pixel."""
+        import torch
+        if out_rgb is None:
+            out_rgb = torch.empty(self.image_shape + (3,), dtype=torch.uint8, device=self.device)
+        n, npx = self.n_agents, self.n_agents * self.K * self.H * self.W
+        _check(self._lib, self._lib.pic_render_rgb(
+            self._h, _dev_ptr(poses, torch.float32, 3 * n), _dev_ptr(dims, torch.float32, 3 * n),
+            _dev_ptr(active, torch.uint8, n) if active is not None else None, _rig_array(rig),
+            1 if antialias else 0, _dev_ptr(out_rgb, torch.uint8), _stream_ptr(stream)))
+        return out_rgb
 
     def render_in_passes(self, poses, dims, rig, consume, max_bytes: int, active=None, stream=None) -> int:
         """Render all views in passes whose output fits `max_bytes` (class + depth bytes), into one pair of

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpictura.so")
 SOURCES = ["pic_api.cu", "pic_kernels.cu", "pic_render.cu", "pic_static.cu", "pic_probe.cu", "pic_bvh.cpp"]
-HEADERS = ["pic_types.h", "pic_device.cuh", "pic_exhaustive.cuh", os.path.join("..", "..", "include", "pictura.h")]
+HEADERS = ["pic_types.h", "pic_device.cuh", "pic_exhaustive.cuh", "pic_colour.cuh", "pic_coverage.cuh", os.path.join("..", "..", "include", "pictura.h")]
 
 
 def _stale() -> bool:

@@ -17,6 +17,7 @@ cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses
                          const float* dims, const uint8_t* active, const uint8_t* agent_cls, AgentGeom* agents_out, ViewCam* cams_out,
                          float* tables, uint32_t* status, float dt, float wheelbase, float v_max, cudaStream_t stream);
 cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, int sm_count, cudaStream_t stream);
+cudaError_t launch_colour(const RenderParams& P, long long n_views, bool antialias, cudaStream_t stream);
 size_t survivor_bytes_per_tile();
 }  // namespace pic
 
@@ -83,6 +84,7 @@ struct pic_scene {
     uint8_t* d_agent_cls = nullptr; // [E*A] class of each agent's box
     bool have_agent_cls = false;
     uint32_t* d_status = nullptr;
+    uint8_t* d_palette = nullptr;   // [256][3] RGB of every class, for the colour output
     // staging for pic_render_host
     float* d_in_poses = nullptr;
     float* d_in_dims = nullptr;
@@ -117,7 +119,7 @@ struct DeviceGuard {
 
 void free_scene(pic_scene* s) {
     cudaFree(s->d_env_map); cudaFree(s->d_env_maps); cudaFree(s->d_maps); cudaFree(s->d_groups); cudaFree(s->d_leaves); cudaFree(s->d_prims); cudaFree(s->d_cell_start); cudaFree(s->d_grid_prims); cudaFree(s->d_large_leaves);
-    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_surv); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_agent_cls); cudaFree(s->d_status);
+    cudaFree(s->d_agents); cudaFree(s->d_cams); cudaFree(s->d_overflow); cudaFree(s->d_surv); cudaFree(s->d_tables); cudaFree(s->d_state); cudaFree(s->d_dims); cudaFree(s->d_active); cudaFree(s->d_agent_cls); cudaFree(s->d_status); cudaFree(s->d_palette);
     cudaFree(s->d_in_poses); cudaFree(s->d_in_dims); cudaFree(s->d_in_active); cudaFree(s->d_out_class);
     cudaFree(s->d_out_depth);
     if (s->ev) {
@@ -128,9 +130,9 @@ void free_scene(pic_scene* s) {
 }
 
 pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth,
-                       pic::RenderParams& P) {
+                       pic::RenderParams& P, bool colour = false) {
     if (!rig) return fail(PIC_ERR_INVALID_ARG, "rig is NULL");
-    if (!out_class || !out_depth) return fail(PIC_ERR_INVALID_ARG, "output pointer is NULL");
+    if (!colour && (!out_class || !out_depth)) return fail(PIC_ERR_INVALID_ARG, "output pointer is NULL");
     if ((reinterpret_cast<uintptr_t>(out_class) & 15u) || (reinterpret_cast<uintptr_t>(out_depth) & 15u))
         return fail(PIC_ERR_INVALID_ARG, "output pointers must be 16-byte aligned");
     std::memset(&P, 0, sizeof(P));
@@ -146,6 +148,8 @@ pic_status fill_params(const pic_scene* s, const pic_camera* rig, uint8_t* out_c
     P.cams = s->d_cams;
     P.overflow = s->d_overflow;
     P.surv = s->d_surv;
+    P.palette = s->d_palette;
+    P.status = s->d_status;
     P.rig.ray_x = s->d_tables;
     P.rig.ray_y = P.rig.ray_x + (size_t)s->K * s->W;
     P.rig.bg_z = P.rig.ray_y + (size_t)s->K * s->H;
@@ -269,6 +273,7 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     dmalloc((void**)&s->d_active, n_agents);
     dmalloc((void**)&s->d_agent_cls, n_agents);
     dmalloc((void**)&s->d_status, sizeof(uint32_t));
+    dmalloc((void**)&s->d_palette, 768);
     upload(s->d_env_map, env_map, sizeof(int32_t) * d->E);
     upload(s->d_maps, maps, sizeof(pic::MapInfo) * nm);
     {
@@ -287,6 +292,11 @@ pic_status pic_scene_create(const pic_scene_desc* d, pic_scene** out) {
     upload(s->d_grid_prims, grid_prims, sizeof(pic::Prim) * ngp);
     upload(s->d_large_leaves, large_leaves, sizeof(pic::Node) * nll);
     if (ce == cudaSuccess) ce = cudaMemset(s->d_status, 0, sizeof(uint32_t));
+    if (ce == cudaSuccess) {          // until pic_set_palette: class c is the grey (c, c, c)
+        uint8_t grey[768];
+        for (int c = 0; c < 256; ++c) grey[3 * c] = grey[3 * c + 1] = grey[3 * c + 2] = (uint8_t)c;
+        ce = cudaMemcpy(s->d_palette, grey, 768, cudaMemcpyHostToDevice);
+    }
     if (ce == cudaSuccess) ce = cudaMemset(s->d_state, 0, sizeof(float) * 4 * n_agents);
     if (ce == cudaSuccess) ce = cudaMemset(s->d_dims, 0, sizeof(float) * 3 * n_agents);
     if (ce == cudaSuccess) ce = cudaMemset(s->d_active, 1, n_agents);
@@ -384,10 +394,11 @@ pic_status pic_scene_set_option(pic_scene* s, int32_t option, uint64_t value) {
 
 static pic_status render_from(pic_scene* s, const float* poses, float* state, const float* actions, const float* dims,
                               const uint8_t* active, const pic_camera* rig, uint8_t* out_class, uint16_t* out_depth,
-                              cudaStream_t stream) {
+                              cudaStream_t stream, uint8_t* out_rgb = nullptr, bool antialias = false) {
     pic::RenderParams P;
-    pic_status st = fill_params(s, rig, out_class, out_depth, P);
+    pic_status st = fill_params(s, rig, out_class, out_depth, P, out_rgb != nullptr);
     if (st != PIC_OK) return st;
+    P.out_rgb = out_rgb;
     DeviceGuard guard(s->device);
     if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
     const int n_agents = s->E * s->A;
@@ -401,14 +412,17 @@ static pic_status render_from(pic_scene* s, const float* poses, float* state, co
         // the caller's buffers start at the first rendered view: shift the bases so that the kernels'
         // absolute view indexing lands there (never dereferenced below view_first)
         const size_t off = (size_t)s->view_first * s->H * s->W;
-        P.out_class -= off; P.out_depth -= off;
+        if (P.out_class) { P.out_class -= off; P.out_depth -= off; }
         if (P.out_depth32) P.out_depth32 -= off;
+        if (P.out_rgb) P.out_rgb -= 3 * off;
     }
+    if (out_rgb) P.occlusion = nullptr;
     if (P.occlusion)    // the counts of the rendered views start at zero
         CUDA_TRY(cudaMemsetAsync(P.occlusion + (size_t)s->view_first * s->A * 2, 0, sizeof(uint32_t) * 2 * (size_t)count * s->A, stream));
     const bool timed = s->timing && s->n_timed < kMaxTimed;
     if (timed) CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed], stream));
-    CUDA_TRY(pic::launch_render(P, count, s->brute, s->sm_count, stream));
+    if (out_rgb) CUDA_TRY(pic::launch_colour(P, count, antialias, stream));
+    else CUDA_TRY(pic::launch_render(P, count, s->brute, s->sm_count, stream));
     if (timed) { CUDA_TRY(cudaEventRecord(s->ev[2 * s->n_timed + 1], stream)); ++s->n_timed; }
     return PIC_OK;
 }
@@ -418,6 +432,24 @@ pic_status pic_render(pic_scene* s, const float* poses, const float* dims, const
     if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
     if (!poses || !dims) return fail(PIC_ERR_INVALID_ARG, "poses or dims is NULL");
     return render_from(s, poses, nullptr, nullptr, dims, active, rig, out_class, out_depth, static_cast<cudaStream_t>(cuda_stream));
+}
+
+pic_status pic_set_palette(pic_scene* s, const uint8_t* rgb, void* cuda_stream) {
+    if (!s || !rgb) return fail(PIC_ERR_INVALID_ARG, "scene or palette is NULL");
+    DeviceGuard guard(s->device);
+    if (!guard.ok) return fail(PIC_ERR_CUDA, "cannot select device %d", s->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    CUDA_TRY(cudaMemcpyAsync(s->d_palette, rgb, 768, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));          // the host array may be reused by the caller
+    return PIC_OK;
+}
+
+pic_status pic_render_rgb(pic_scene* s, const float* poses, const float* dims, const uint8_t* active, const pic_camera* rig,
+                          int32_t antialias, uint8_t* out_rgb, void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!poses || !dims || !out_rgb) return fail(PIC_ERR_INVALID_ARG, "poses, dims or out_rgb is NULL");
+    return render_from(s, poses, nullptr, nullptr, dims, active, rig, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream), out_rgb,
+                       antialias != 0);
 }
 
 pic_status pic_render_host(pic_scene* s, const float* poses, const float* dims, const uint8_t* active,

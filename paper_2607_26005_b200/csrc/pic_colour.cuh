@@ -1,0 +1,417 @@
+// Colour kernel (included by pic_render.cu, inside namespace pic): the paper's output format (Sec. 3.2) --
+// 8-bit RGB images of flat-shaded primitives, box faces coloured per face with depth-aware brightness,
+// optionally antialiased by analytic coverage at one sample per pixel.
+//
+// The paper gives neither colours nor a coverage formula; the definition implemented here is:
+//   colour        a palette gives every class an RGB triple; a map primitive has its class's colour, face f of
+//                 an agent's box its class's colour times FACE_SHADE[f] * (1 - 0.5 (z - near) / (far - near));
+//   no AA         a pixel shows the nearest fragment that covers its centre (the class / depth image's winner);
+//   AA            box filter over the pixel's unit square: a primitive's coverage is the exact area of the
+//                 square inside all its edges and within the depth range of its plane; it leaves a fragment
+//                 wherever that area is positive, at its plane's depth at the pixel centre (clamped to the
+//                 range); a pixel's fragments are composited
+//                 front to back, consecutive fragments of one surface (map primitives of one class; the faces of
+//                 one box, of which only those turned towards the camera are drawn) first being merged into one
+//                 layer: nearest first, each adds its coverage, and its colour with that weight, until the layer
+//                 is full.
+//
+// Structure: the cull kernel's survivor lists (made with conservative pixel boxes when antialiasing) are set up
+// into a record pool shared by the CTA's four tiles, in rounds like render_full_kernel; 8-row strips are tasks.
+// A strip keeps, per pixel, the nearest FULLY covering fragment as a 64-bit key (unsigned max, as in the other
+// kernels, with the record's slot in the low byte) and a linked list of the partially covering fragments in
+// front of it (1/z, coverage in 14 bits, slot); the strip's warp owns both, so no atomics are needed.  The
+// resolve walks each pixel's list in depth order, merges, composites and stores 16 pixels (48 bytes) per lane.
+#pragma once
+
+constexpr int CSTRIP = 8;                       // pixel rows of a strip
+constexpr int CSTRIPS = TILE / CSTRIP;
+constexpr int CSTRIP_KEYS = TILE * CSTRIP;
+constexpr int CPOOL = 254;                      // records shared by the four tiles (a tile's survivors always fit: W_SURV < CPOOL)
+constexpr int CFRAGS = 1023;                    // partially covering fragments of a strip (10-bit links, 0 ends a list)
+constexpr uint32_t STATUS_COLOUR_INCOMPLETE = 2u;   // = PIC_FLAG_COLOUR_INCOMPLETE of the public header
+constexpr uint32_t STATUS_COLOUR_FRAGMENTS = 4u;    // = PIC_FLAG_COLOUR_FRAGMENTS
+static_assert(W_SURV <= CPOOL && CPOOL <= 256, "a tile's survivors fit the pool; a slot fits the key's low byte");
+
+__constant__ float FACE_SHADE[6] = {0.60f, 1.00f, 0.70f, 0.85f, 0.40f, 0.92f};   // rear, front, right, left, bottom, top
+
+struct __align__(16) ColourPool {
+    float4 nx[CPOOL], ny[CPOOL], nz[CPOOL];     // edge functions E_i = nx[i] rx + ny[i] ry + nz[i]
+    float4 w[CPOOL];                            // 1/z plane wx, wy, wz; key low word (index, class)
+    uint32_t box[CPOOL];                        // pixel box (6 bits per coordinate), top-left bits << 24, REC_DEAD
+    float shade[CPOOL];                         // box faces: the face's factor; map primitives: 0 (not shaded)
+    uint32_t surface[CPOOL];                    // fragments of equal surface merge: a map primitive's class, 256 + agent of a box
+};
+
+struct __align__(16) ColourSmem {
+    unsigned long long key[NW][CSTRIP_KEYS];    // warp w's strip: nearest fully covering fragment per pixel
+    unsigned long long frag[NW][CFRAGS + 1];    // its partial fragments: bits(1/z) << 32 | coverage << 18 | slot << 10 | next
+    uint16_t head[NW][CSTRIP_KEYS];             // first fragment of each pixel's list (0: none)
+    ColourPool pool;
+    float ray_x[NW][TILE], ray_y[NW][TILE];     // ray tables of tile w
+    Cam cam[NW];
+    Job job[NW];
+    int active[NW];
+    int n_surv[NW];
+    int next_task;
+};
+static_assert(sizeof(ColourSmem) <= 74 * 1024, "three CTAs per SM");
+
+struct RayView { float* ray_x; float* ray_y; };
+
+// The six lines of a record at one pixel: values at the pixel centre (edges, 1/z - 1/far, 1/near - 1/z).
+struct PixelLines { float e[CLINES]; };
+
+// Coverage (14 bits) of one pixel by a record, given its lines at the pixel centre and their half ranges hh over
+// the pixel (a line with e >= hh contains the whole pixel).
+__device__ __forceinline__ uint32_t coverage14(const PixelLines& L, const PrimEq& q, const float (&hh)[CLINES], float du, float dv, bool want) {
+    float a[CLINES], b[CLINES];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { a[i] = q.nx[i] * du; b[i] = q.ny[i] * dv; }
+    a[4] = q.wx * du; b[4] = q.wy * dv; a[5] = -a[4]; b[5] = -b[4];
+    int n_part = 0;
+    float ew = 0.f, aw = 0.f, bw = 0.f;
+#pragma unroll
+    for (int i = 0; i < CLINES; ++i)
+        if (L.e[i] < hh[i]) { ++n_part; ew = L.e[i]; aw = a[i]; bw = b[i]; }
+    float alpha = 0.f;
+    const bool general = want && n_part > 1;
+    if (want && n_part == 1) alpha = edge_coverage(ew, aw, bw);      // one line crosses the pixel, the others contain it
+    if (__any_sync(0xffffffffu, general)) {
+        if (general) alpha = pixel_coverage(L.e, a, b);
+    }
+    return (uint32_t)(alpha * 16383.f + 0.5f);
+}
+
+// A 16 x 4 pixel cell of a strip against one record; a lane handles two adjacent pixels.
+template <bool AA>
+__device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* head, unsigned long long* frag, int& n_frag,
+                                            const float* ray_x, const float* ray_y, const PrimEq& q, const float (&thr)[4],
+                                            const float (&hh)[CLINES], float du, float dv, uint32_t key_lo, uint32_t slot,
+                                            float w_near, float w_far, int xx, int yy, int lane) {
+    const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
+    const float2 rx = *reinterpret_cast<const float2*>(ray_x + x);
+    const float ry = ray_y[y];
+    const float wt = fm(q.wy, ry, q.wz);
+    const float w0 = fm(q.wx, rx.x, wt), w1 = fm(q.wx, rx.y, wt);
+    PixelLines L0, L1;
+    bool full0 = true, full1 = true, out0 = false, out1 = false;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float te = fm(q.ny[e], ry, q.nz[e]);
+        L0.e[e] = fm(q.nx[e], rx.x, te); L1.e[e] = fm(q.nx[e], rx.y, te);
+        if (!AA) { full0 = full0 && (L0.e[e] > thr[e]); full1 = full1 && (L1.e[e] > thr[e]); }
+    }
+    L0.e[4] = w0 - w_far; L0.e[5] = w_near - w0; L1.e[4] = w1 - w_far; L1.e[5] = w_near - w1;
+    if (AA) {
+#pragma unroll
+        for (int e = 0; e < CLINES; ++e) {
+            full0 = full0 && (L0.e[e] >= hh[e]); full1 = full1 && (L1.e[e] >= hh[e]);
+            out0 = out0 || (L0.e[e] <= -hh[e]); out1 = out1 || (L1.e[e] <= -hh[e]);
+        }
+    } else {
+        full0 = full0 && (w0 >= w_far) && (w0 <= w_near); full1 = full1 && (w1 >= w_far) && (w1 <= w_near);
+    }
+    unsigned long long* kp = key + key_index(x, y);
+    const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(kp);
+    // (a partially covered pixel's depth is its plane's at the pixel centre, clamped to the depth range)
+    const float c0 = AA ? fminf(fmaxf(w0, w_far), w_near) : w0, c1 = AA ? fminf(fmaxf(w1, w_far), w_near) : w1;
+    const unsigned long long k0 = make_key(__float_as_uint(c0), key_lo), k1 = make_key(__float_as_uint(c1), key_lo);
+    if (full0 && k0 > kk.x) kp[0] = k0;
+    if (full1 && k1 > kk.y) kp[1] = k1;
+    if (AA) {
+        // partially covered pixels in front of the nearest fully covering fragment seen so far
+        bool push0 = !full0 && !out0 && k0 > kk.x, push1 = !full1 && !out1 && k1 > kk.y;
+        if (__any_sync(0xffffffffu, push0 || push1)) {
+            const uint32_t a0 = coverage14(L0, q, hh, du, dv, push0), a1 = coverage14(L1, q, hh, du, dv, push1);
+            push0 = push0 && a0 != 0u; push1 = push1 && a1 != 0u;
+            const unsigned m0 = __ballot_sync(0xffffffffu, push0), m1 = __ballot_sync(0xffffffffu, push1);
+            const unsigned below = (1u << lane) - 1u;
+            const int i0 = n_frag + 1 + __popc(m0 & below), i1 = n_frag + 1 + __popc(m0) + __popc(m1 & below);
+            const int pix = y * TILE + x;
+            if (push0 && i0 <= CFRAGS) {
+                frag[i0] = ((unsigned long long)__float_as_uint(c0) << 32) | (a0 << 18) | (slot << 10) | head[pix];
+                head[pix] = (uint16_t)i0;
+            }
+            if (push1 && i1 <= CFRAGS) {
+                frag[i1] = ((unsigned long long)__float_as_uint(c1) << 32) | (a1 << 18) | (slot << 10) | head[pix + 1];
+                head[pix + 1] = (uint16_t)i1;
+            }
+            n_frag += __popc(m0) + __popc(m1);
+        }
+    }
+}
+
+// Colour of a fragment of the record in `slot` at reciprocal depth w.
+__device__ __forceinline__ void shade_fragment(const ColourPool& pool, const RenderParams& P, uint32_t slot, float w, float& r, float& g, float& b) {
+    const uint32_t cls = __float_as_uint(pool.w[slot].w) & 0xffu;
+    const float sh = pool.shade[slot];
+    float k = 1.f;
+    if (sh > 0.f) k = sh * (1.f - 0.5f * __fdividef(__fdividef(1.f, w) - P.near_z, P.far_z - P.near_z));
+    const uint8_t* pal = P.palette + 3u * cls;
+    r = k * (float)__ldg(pal); g = k * (float)__ldg(pal + 1); b = k * (float)__ldg(pal + 2);
+}
+
+// One strip of tile `jb` -> colour image: every lane resolves 16 consecutive pixels of a row, resets what it reads.
+template <bool AA>
+__device__ __forceinline__ void resolve_store_colour(unsigned long long* key, uint16_t* head, const unsigned long long* frag,
+                                                     const ColourPool& pool, const RenderParams& P, const Job& jb, bool ego_active,
+                                                     int ys, bool vec_ok, int lane) {
+    const int y = lane >> 2, xs = (lane & 3) * 16;
+    const int gy = jb.t.y0 + ys + y;
+    uint32_t bgc = P.cls_sky;
+    if (ego_active && gy < P.H) bgc = __ldg(P.rig.bg_cls + (size_t)jb.k * P.H + gy);
+    const float bgr = (float)__ldg(P.palette + 3u * bgc), bgg = (float)__ldg(P.palette + 3u * bgc + 1), bgb = (float)__ldg(P.palette + 3u * bgc + 2);
+    uint32_t ow[12];
+#pragma unroll
+    for (int i = 0; i < 12; ++i) ow[i] = 0u;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int x = xs + j;
+        unsigned long long* kp = key + key_index(x, y);
+        const unsigned long long k = *kp;
+        *kp = 0ull;
+        uint32_t hd = 0u;
+        if (AA) { hd = head[y * TILE + x]; head[y * TILE + x] = 0; }
+        float R = bgr, G = bgg, B = bgb;
+        if (hd == 0u) {
+            if (k) shade_fragment(pool, P, (uint32_t)k & 0xffu, __uint_as_float((uint32_t)(k >> 32)), R, G, B);
+        } else {
+            // front to back: the list's fragments in front of the fully covering one, then that one, then the background.
+            // Consecutive fragments of one surface form a layer: each adds its coverage until the layer is full.
+            const uint32_t w_opq = (uint32_t)(k >> 32);
+            float T = 1.f, acc = 0.f;
+            R = 0.f; G = 0.f; B = 0.f;
+            uint32_t cur = 0xffffffffu;
+            unsigned long long prev = ~0ull;
+            for (int it = 0; it < 48 && T > 0.f; ++it) {
+                // the nearest remaining fragment: the largest (1/z, entry) below the last one taken; at the end, the opaque one
+                unsigned long long best = 0ull;
+                uint32_t best_lo = 0u;
+                for (uint32_t i = hd; i;) {
+                    const unsigned long long en = frag[i];
+                    const unsigned long long cand = (en & 0xffffffff00000000ull) | i;
+                    if (cand < prev && cand > best && (uint32_t)(en >> 32) > w_opq) { best = cand; best_lo = (uint32_t)en; }
+                    i = (uint32_t)en & 1023u;
+                }
+                uint32_t slot, wb;
+                float alpha;
+                if (best) { prev = best; slot = (best_lo >> 10) & 0xffu; alpha = (float)((best_lo >> 18) & 0x3fffu) * (1.f / 16383.f); wb = (uint32_t)(best >> 32); }
+                else if (k && prev != 0ull) { prev = 0ull; slot = (uint32_t)k & 0xffu; alpha = 1.f; wb = w_opq; }
+                else break;
+                const uint32_t surf = pool.surface[slot];
+                if (surf != cur) { T *= 1.f - acc; cur = surf; acc = 0.f; }
+                const float add = fminf(alpha, 1.f - acc) * T;
+                float cr, cg, cb;
+                shade_fragment(pool, P, slot, __uint_as_float(wb), cr, cg, cb);
+                R = fm(add, cr, R); G = fm(add, cg, G); B = fm(add, cb, B);
+                acc += fminf(alpha, 1.f - acc);
+            }
+            T *= 1.f - acc;
+            R = fm(T, bgr, R); G = fm(T, bgg, G); B = fm(T, bgb, B);
+        }
+        const uint32_t r8 = (uint32_t)fminf(fmaxf(R + 0.5f, 0.f), 255.f), g8 = (uint32_t)fminf(fmaxf(G + 0.5f, 0.f), 255.f),
+                       b8 = (uint32_t)fminf(fmaxf(B + 0.5f, 0.f), 255.f);
+        ow[(3 * j) >> 2] |= r8 << (8 * ((3 * j) & 3));
+        ow[(3 * j + 1) >> 2] |= g8 << (8 * ((3 * j + 1) & 3));
+        ow[(3 * j + 2) >> 2] |= b8 << (8 * ((3 * j + 2) & 3));
+    }
+    if (ys + y >= jb.t.th || xs >= jb.t.tw) return;
+    uint8_t* dst = P.out_rgb + 3u * ((jb.view * (size_t)P.H + gy) * (size_t)P.W + jb.t.x0 + xs);
+    if (vec_ok && xs + 16 <= jb.t.tw) {
+        uint4* d4 = reinterpret_cast<uint4*>(dst);
+        d4[0] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+        d4[1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
+        d4[2] = make_uint4(ow[8], ow[9], ow[10], ow[11]);
+    } else {
+#pragma unroll
+        for (int n = 0; n < 48; ++n)
+            if (n / 3 + xs < jb.t.tw) dst[n] = (uint8_t)(ow[n >> 2] >> (8 * (n & 3)));
+    }
+}
+
+template <bool AA>
+__global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_constant__ RenderParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ColourSmem& s = *reinterpret_cast<ColourSmem*>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned id = blockIdx.x * (unsigned)NW + warp;
+    const bool valid = id < P.n_jobs;
+    const uint2* blk = P.surv + (size_t)id * SURV_STRIDE;
+    int ns = -2, n_big = 0;
+    Job job;
+    uint32_t n_map_tris = 0u;
+    if (valid) {
+        const uint4 head = __ldcg(reinterpret_cast<const uint4*>(blk));
+        job = decode_job(P, id);
+        n_map_tris = __ldg(&P.env_maps[job.e].n_tris);
+        const bool ego_active = __ldg(&P.agents[(size_t)job.e * P.A + job.a].active) != 0u;
+        RayView rv = {s.ray_x[warp], s.ray_y[warp]};
+        load_rays(rv, P, job, lane); load_rays(rv, P, job, lane + 32);
+        if (lane == 0) {
+            load_camera(s.cam[warp], P.cams[job.view], P.cam[job.k], P.W, P.H);
+            s.job[warp] = job;
+            s.active[warp] = ego_active ? 1 : 0;
+        }
+        n_big = (int)(head.x & 0xffffu);
+        ns = n_big + (int)(head.x >> 16);
+        if (head.x == SURV_OVERFLOW) {
+            // more visible primitives than the tile's list holds: the tile shows only the background, and the call says so
+            ns = 0; n_big = 0;
+            if (lane == 0) atomicOr(P.status, STATUS_COLOUR_INCOMPLETE);
+        }
+    }
+    if (lane == 0) s.n_surv[warp] = ns;
+#pragma unroll
+    for (int i = 0; i < CSTRIP_KEYS / 2 / 32; ++i)
+        reinterpret_cast<ulonglong2*>(s.key[warp])[i * 32 + lane] = make_ulonglong2(0ull, 0ull);
+#pragma unroll
+    for (int i = 0; i < CSTRIP_KEYS / 8 / 32; ++i)
+        reinterpret_cast<uint4*>(s.head[warp])[i * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    const bool vec_ok = (P.W % 16 == 0) && ((reinterpret_cast<uintptr_t>(P.out_rgb) & 15u) == 0);
+    uint32_t done = 0u;
+#pragma unroll
+    for (int j = 0; j < NW; ++j)
+        if (s.n_surv[j] < 0) done |= 1u << j;
+#pragma unroll 1
+    while (done != (1u << NW) - 1u) {
+        // this round's tiles: those not yet rendered, in order, as long as their survivors fit the pool
+        uint32_t bases = 0u, cnts = 0u, now = 0u;
+        {
+            int off = 0;
+#pragma unroll
+            for (int j = 0; j < NW; ++j) {
+                const int c = s.n_surv[j];
+                bases |= (uint32_t)off << (8 * j);
+                if (!((done >> j) & 1u) && off + c <= CPOOL) { cnts |= (uint32_t)c << (8 * j); off += c; now |= 1u << j; }
+                else cnts |= 0xffu << (8 * j);
+            }
+        }
+        // ---- set-up by the tile's warp: survivor i becomes record base + i
+        if ((now >> warp) & 1u) {
+            const int my_base = (int)((bases >> (8 * warp)) & 0xffu);
+            const Cam& c = s.cam[warp];
+            for (int i = lane; i < ns; i += 32) {
+                const uint2 svi = __ldcg(blk + 2 + (i < n_big ? i : W_SURV - 1 - (i - n_big)));
+                V3 V[4], Pn;
+                uint32_t key_lo, flags;
+                fetch_survivor(c, P, svi.x, job.e, n_map_tris, V, Pn, key_lo, flags);
+                float shade = 0.f;
+                uint32_t surface = key_lo & 0xffu;
+                bool drop = false;
+                if (svi.x & SURV_FACE) {
+                    const uint32_t b = (svi.x & ~SURV_FACE) >> 3, f = svi.x & 7u;
+                    shade = FACE_SHADE[f];
+                    surface = 256u + b;
+                    if (AA) {
+                        // faces whose outer side is turned away from the camera centre are not drawn: the camera
+                        // centre (the origin) and the box's centre lie on the same side of the face's plane
+                        const AgentGeom g = P.agents[(size_t)job.e * P.A + b];
+                        const V3 bc = rotate_to_camera(c, sub(sub(g.x, c.px), c.mwx), sub(sub(g.y, c.py), c.mwy), sub(0.5f * g.h, c.mwz));
+                        const float s_cam = -vdot(Pn, V[0]), s_box = vdot(Pn, vsub(bc, V[0]));
+                        drop = !(s_cam * s_box < 0.f);
+                    }
+                }
+                PrimEq q;
+                const int slot = my_base + i;
+                if (drop || !prim_equations(V, flags & 1u, flags, Pn, q)) { s.pool.box[slot] = REC_DEAD; continue; }
+                const uint32_t box = svi.y;
+                const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+                s.pool.nx[slot] = make_float4(q.nx[0], q.nx[1], q.nx[2], q.nx[3]);
+                s.pool.ny[slot] = make_float4(q.ny[0], q.ny[1], q.ny[2], q.ny[3]);
+                s.pool.nz[slot] = make_float4(q.nz[0], q.nz[1], q.nz[2], q.nz[3]);
+                s.pool.w[slot] = make_float4(q.wx, q.wy, q.wz, __uint_as_float(key_lo));
+                s.pool.box[slot] = bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24);
+                s.pool.shade[slot] = shade;
+                s.pool.surface[slot] = surface;
+            }
+        }
+        if (threadIdx.x == 0) s.next_task = 0;
+        __syncthreads();
+        // ---- the strips of this round's tiles are tasks that the warps draw from a counter
+        unsigned long long* key = s.key[warp];
+        uint16_t* head = s.head[warp];
+        unsigned long long* frag = s.frag[warp];
+#pragma unroll 1
+        for (;;) {
+            int task = 0;
+            if (lane == 0) task = atomicAdd(&s.next_task, 1);
+            task = __shfl_sync(0xffffffffu, task, 0);
+            if (task >= NW * CSTRIPS) break;
+            const int j = task / CSTRIPS, ys = (task % CSTRIPS) * CSTRIP;
+            const int cj = (int)((cnts >> (8 * j)) & 0xffu);
+            if (cj == 0xff) continue;
+            const Job jb = s.job[j];
+            if (ys >= jb.t.th) continue;
+            const int first = (int)((bases >> (8 * j)) & 0xffu);
+            const float* ray_x = s.ray_x[j];
+            const float* ray_y = s.ray_y[j] + ys;
+            const float du = __fdividef(1.f, s.cam[j].focx), dv = __fdividef(1.f, s.cam[j].focy);
+            int n_frag = 0;
+            for (int base = 0; base < cj; base += 32) {
+                uint32_t bw_lane = 0u;
+                bool hit = false;
+                if (base + lane < cj) {
+                    bw_lane = s.pool.box[first + base + lane];
+                    const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
+                    hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + CSTRIP;
+                }
+                for (unsigned hits = __ballot_sync(0xffffffffu, hit); hits; hits &= hits - 1) {
+                    const int src = __ffs(hits) - 1;
+                    const uint32_t bw = __shfl_sync(0xffffffffu, bw_lane, src);
+                    const int by0 = (bw >> 6) & 63, by1 = (bw >> 18) & 63, bx0 = bw & 63, bx1 = (bw >> 12) & 63;
+                    const int ly0 = max(by0, ys) - ys, ly1 = min(by1, ys + CSTRIP - 1) - ys;
+                    const uint32_t slot = (uint32_t)(first + base + src);
+                    const float4 r0 = s.pool.nx[slot], r1 = s.pool.ny[slot], r2 = s.pool.nz[slot], r3 = s.pool.w[slot];
+                    PrimEq q;
+                    q.nx[0] = r0.x; q.nx[1] = r0.y; q.nx[2] = r0.z; q.nx[3] = r0.w;
+                    q.ny[0] = r1.x; q.ny[1] = r1.y; q.ny[2] = r1.z; q.ny[3] = r1.w;
+                    q.nz[0] = r2.x; q.nz[1] = r2.y; q.nz[2] = r2.z; q.nz[3] = r2.w;
+                    q.wx = r3.x; q.wy = r3.y; q.wz = r3.z;
+                    q.tl = (bw >> 24) & 15u;
+                    const uint32_t key_lo = (__float_as_uint(r3.w) & 0xffffff00u) | slot;
+                    float thr[4], hh[CLINES];
+                    edge_thresholds(q.tl, thr);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) hh[e] = 0.5f * (fabsf(q.nx[e]) * du + fabsf(q.ny[e]) * dv);
+                    hh[4] = hh[5] = 0.5f * (fabsf(q.wx) * du + fabsf(q.wy) * dv);
+                    for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
+                        for (int xx = bx0 & ~15; xx <= bx1; xx += 16)
+                            colour_cell<AA>(key, head, frag, n_frag, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, lane);
+                }
+                __syncwarp();
+            }
+            if (AA && n_frag > CFRAGS && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);   // fragments were dropped
+            __syncwarp();
+            resolve_store_colour<AA>(key, head, frag, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
+            __syncwarp();
+        }
+        done |= now;
+        if (done != (1u << NW) - 1u) __syncthreads();        // the pool is reused by the next round
+    }
+}
+
+cudaError_t configure_colour_kernel() {
+    cudaError_t err = cudaFuncSetAttribute(colour_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ColourSmem));
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(colour_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ColourSmem));
+}
+
+// Colour images of n_views views: the cull kernel (conservative pixel boxes when antialiasing), then the colour kernel.
+cudaError_t launch_colour_kernel(const RenderParams& P0, long long n_views, bool antialias, cudaStream_t stream) {
+    RenderParams P = P0;
+    const long long jobs = n_views * P.tiles_x * P.tiles_y;
+    if (jobs > 0x7fffffffLL || (long long)P.E * P.A * P.K > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (jobs <= 0) return cudaSuccess;
+    P.n_jobs = (uint32_t)jobs;
+    P.debug_flags = 0;
+    P.counters = nullptr;
+    const unsigned grid = (unsigned)((jobs + NW - 1) / NW);
+    if (antialias) cull_kernel<NoTally, true><<<grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    else cull_kernel<NoTally, false><<<grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    if (antialias) colour_kernel<true><<<grid, NTHREADS, sizeof(ColourSmem), stream>>>(P);
+    else colour_kernel<false><<<grid, NTHREADS, sizeof(ColourSmem), stream>>>(P);
+    return cudaGetLastError();
+}

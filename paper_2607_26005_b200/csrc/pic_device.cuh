@@ -180,9 +180,9 @@ __device__ __forceinline__ unsigned long long make_key(uint32_t wbits, uint32_t 
 
 // Pixel box (inclusive, tile coordinates) of camera-space vertices, or the whole tile when a
 // vertex is too close to the camera plane to project.  Returns false if the primitive cannot
-// touch any pixel centre of the tile or lies entirely before near / beyond far.
+// touch any pixel centre of the tile (with the default margin m) or lies entirely before near / beyond far.
 // (Triangles pass their third vertex twice.)
-__device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const V3 (&V)[4], uint32_t& packed) {
+__device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const V3 (&V)[4], uint32_t& packed, const float m = 0.00390625f) {
     constexpr int n = 4;
     float zmin = V[0].z, zmax = V[0].z;
 #pragma unroll
@@ -198,8 +198,8 @@ __device__ __forceinline__ bool pixel_box(const Cam& c, const TileCtx& t, const 
             float sx = fm(c.focx, mul(V[i].x, iz), c.cx), sy = fm(c.focy, mul(V[i].y, iz), c.cy);
             sx0 = fminf(sx0, sx); sx1 = fmaxf(sx1, sx); sy0 = fminf(sy0, sy); sy1 = fmaxf(sy1, sy);
         }
-        // pixel centres u + 0.5 in [sx0, sx1], widened by 1/256 pixel against rounding
-        const float m = 0.00390625f;
+        // pixel centres u + 0.5 in [sx0, sx1], widened by m = 1/256 pixel against rounding (m = 1/2 + 1/256: every pixel
+        // whose unit square the primitive touches)
         float fx0 = ceilf(sx0 - 0.5f - m) - (float)t.x0, fx1 = floorf(sx1 - 0.5f + m) - (float)t.x0;
         float fy0 = ceilf(sy0 - 0.5f - m) - (float)t.y0, fy1 = floorf(sy1 - 0.5f + m) - (float)t.y0;
         ok = ok && (fx0 <= fx1) && (fy0 <= fy1) && (fx1 >= 0.f) && (fy1 >= 0.f) && (fx0 <= (float)(t.tw - 1)) && (fy0 <= (float)(t.th - 1));

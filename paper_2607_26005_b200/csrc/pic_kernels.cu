@@ -117,11 +117,15 @@ size_t render_smem_bytes();                       // pic_render.cu
 cudaError_t configure_render_kernel();            // pic_render.cu
 cudaError_t launch_render_kernel(const RenderParams& P, long long n_views, int sm_count, cudaStream_t stream);
 cudaError_t launch_coverage_kernel(const RenderParams& P, long long n_views, cudaStream_t stream);
+cudaError_t configure_colour_kernel();            // pic_colour.cuh (part of pic_render.cu)
+cudaError_t launch_colour_kernel(const RenderParams& P, long long n_views, bool antialias, cudaStream_t stream);
 
 size_t max_smem_bytes() { return render_smem_bytes() > sizeof(ExhaustiveSmem) ? render_smem_bytes() : sizeof(ExhaustiveSmem); }
 
 cudaError_t configure_kernels() {
     cudaError_t err = configure_render_kernel();
+    if (err != cudaSuccess) return err;
+    err = configure_colour_kernel();
     if (err != cudaSuccess) return err;
     return cudaFuncSetAttribute(render_brute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ExhaustiveSmem));
 }
@@ -148,6 +152,10 @@ cudaError_t launch_setup(const RenderParams& P, int n_agents, const float* poses
     agent_kernel<<<(n_agents + 127) / 128, 128, 0, stream>>>(n_agents, poses, state, actions, dims, active, agent_cls, P.cls_agent, agents_out,
                                                               cams_out, status, R, dt, wheelbase, v_max);
     return cudaGetLastError();
+}
+
+cudaError_t launch_colour(const RenderParams& P, long long n_views, bool antialias, cudaStream_t stream) {
+    return n_views <= 0 ? cudaSuccess : launch_colour_kernel(P, n_views, antialias, stream);
 }
 
 cudaError_t launch_render(const RenderParams& P, long long n_views, bool brute, int sm_count, cudaStream_t stream) {

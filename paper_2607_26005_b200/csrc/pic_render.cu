@@ -670,7 +670,7 @@ constexpr int W_FACE = 384;        // box-face items of a tile in the cull kerne
 // entries (id, pixel box).  Survivors whose pixel box holds more than TINY_MAX_PIXELS pixel centres
 // fill the list from the front, the others from the back; head.x = front count | back count << 16,
 // or all ones if a list overflowed.
-constexpr int SURV_STRIDE = 128;
+constexpr int SURV_STRIDE = 256;
 constexpr int W_SURV = SURV_STRIDE - 2;
 constexpr uint32_t SURV_OVERFLOW = 0xffffffffu;
 constexpr uint32_t SURV_FACE = 0x80000000u;   // survivor id: index into grid_prims, or SURV_FACE | agent << 3 | face
@@ -791,10 +791,12 @@ __device__ __forceinline__ void append_survivor(uint2* __restrict__ surv, bool k
 // candidates per lane at a time (camera space, pixel box).  The large primitives are found through
 // their leaves (a lane per leaf box against the six frustum planes), the other agents' boxes as
 // bounding spheres.  Loads that do not depend on one another are issued together.
-template <class TL>
+template <class TL, bool CONS>
 __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ surv, const RenderParams& P, const Job& job,
                                           const MapInfo& mi, int lane, TL& n) {
     const int stop = PIC_STOP(P);
+    // CONS: conservative pixel boxes -- every pixel whose unit square a primitive touches (antialiased output)
+    constexpr float BOX_MARGIN = CONS ? 0.50390625f : 0.00390625f;
     const TileCtx& t = job.t;
     const AgentGeom* env_agents = P.agents + (size_t)job.e * P.A;
     Node ln0;
@@ -952,7 +954,7 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
 #pragma unroll
                     for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[u][3 * q], v[u][3 * q + 1], v[u][3 * q + 2]);
                     ++n.tested;
-                    keep = pixel_box(c, t, V, box);
+                    keep = pixel_box(c, t, V, box, BOX_MARGIN);
                 }
                 append_survivor(surv, keep, id[u], box, n_big, n_tiny, lane);
             }
@@ -976,7 +978,7 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
 #pragma unroll
                 for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[3 * q], v[3 * q + 1], v[3 * q + 2]);
                 ++n.tested;
-                keep = pixel_box(c, t, V, box);
+                keep = pixel_box(c, t, V, box, BOX_MARGIN);
             }
         }
         append_survivor(surv, keep, id, box, n_big, n_tiny, lane);
@@ -997,7 +999,7 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
 #pragma unroll
             for (int q = 0; q < 4; ++q) V[q] = box_corner(c, g, (corners >> (4 * q)) & 7u);
             ++n.tested;
-            keep = pixel_box(c, t, V, box);
+            keep = pixel_box(c, t, V, box, BOX_MARGIN);
         }
         append_survivor(surv, keep, SURV_FACE | it, box, n_big, n_tiny, lane);
     }
@@ -1190,7 +1192,7 @@ constexpr int CULL_ROUNDS = PIC_CULL_ROUNDS;   // rounds of NW tiles per CTA of 
 #ifndef PIC_RENDER_CTAS
 #define PIC_RENDER_CTAS 5
 #endif
-template <class TL>
+template <class TL, bool CONS>
 __global__ void __launch_bounds__(NTHREADS, PIC_CULL_CTAS) cull_kernel(const __grid_constant__ RenderParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     CullSmem& s = *reinterpret_cast<CullSmem*>(smem_raw);
@@ -1209,7 +1211,7 @@ __global__ void __launch_bounds__(NTHREADS, PIC_CULL_CTAS) cull_kernel(const __g
         uint2* blk = P.surv + (size_t)id * SURV_STRIDE;
         int ns = 0;
         if (P.debug_flags & 4) ns = -1;             // test aid: every tile through cooperative_job
-        else if (ego_active && stop != 1 && !(stop >= 8 && stop <= 10)) ns = front_cull(s.lists[warp], blk + 2, P, job, mi, lane, n);
+        else if (ego_active && stop != 1 && !(stop >= 8 && stop <= 10)) ns = front_cull<TL, CONS>(s.lists[warp], blk + 2, P, job, mi, lane, n);
         // (the work counts are summed over the warp's lanes; without counters they are constants)
         const uint32_t c_grp = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.grp)), c_leaf = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.leaf)),
                        c_tested = __reduce_add_sync(0xffffffffu, (uint32_t)tally_value(n.tested));
@@ -1777,6 +1779,11 @@ __global__ void __launch_bounds__(NTHREADS) coverage_kernel(const __grid_constan
     }
 }
 
+}  // namespace pic
+#include "pic_coverage.cuh"
+namespace pic {
+#include "pic_colour.cuh"
+
 size_t survivor_bytes_per_tile() { return sizeof(uint2) * SURV_STRIDE; }
 
 cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int sm_count, cudaStream_t stream) {
@@ -1790,8 +1797,8 @@ cudaError_t launch_render_kernel(const RenderParams& P0, long long n_views, int 
                       (reinterpret_cast<uintptr_t>(P.out_depth) & 31u) == 0;   // 256-bit depth stores
     // (a) cull: survivors per tile
     const unsigned cull_grid = (unsigned)((jobs + NW * CULL_ROUNDS - 1) / (NW * CULL_ROUNDS));
-    if (P.counters) cull_kernel<Tally><<<cull_grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
-    else cull_kernel<NoTally><<<cull_grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    if (P.counters) cull_kernel<Tally, false><<<cull_grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
+    else cull_kernel<NoTally, false><<<cull_grid, NTHREADS, sizeof(CullSmem), stream>>>(P);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     // (b)-(d) set-up, raster, store

@@ -105,6 +105,9 @@ struct RenderParams {
     float* out_depth32;             // optional
     unsigned long long* counters;   // optional [16]
     uint32_t* occlusion;            // optional [E*A*K][A][2]: per view and other agent, visible pixels and pixels its box covers alone
+    uint8_t* out_rgb;               // colour output [E*A*K][H][W][3] (colour kernel only)
+    const uint8_t* palette;         // [256][3] RGB of every class (colour kernel only)
+    uint32_t* status;               // the scene's sticky status word
     uint32_t* overflow;             // [1 + tiles of all views]: count, then the tiles left to the cooperative kernel
     uint2* surv;                    // per tile: the cull kernel's survivors (head + list), read by the render kernel
     int32_t debug_flags;            // bit 0: no per-cell trivial accept/reject, bit 1: record pool / list of 2 entries, bit 2: cooperative kernel only, bit 3: pool of 40, bits 4-7: profiling stop

@@ -56,6 +56,20 @@ class CudaRun:
             out = out + (cnt.cpu().numpy(),)
         return out
 
+    def render_rgb(self, palette, antialias: bool, poses=None, view_first: int = 0, view_count: int = 0):
+        """Colour images u8 [V,H,W,3] as numpy (sentinel 7 where nothing was written), and the status flags."""
+        torch, pic, s = self.torch, self.pic, self.s
+        rgb = torch.full(self.scene.image_shape + (3,), 7, dtype=torch.uint8, device=self.dev)
+        self.scene.set_palette(palette)
+        self.scene.set_option(pic.OPT_VIEW_FIRST, view_first)
+        self.scene.set_option(pic.OPT_VIEW_COUNT, view_count)
+        p = self.poses if poses is None else torch.from_numpy(np.ascontiguousarray(poses, dtype=np.float32)).to(self.dev)
+        self.scene.render_rgb(p, self.dims, s.rig, active=self.active, out_rgb=rgb, antialias=antialias)
+        torch.cuda.synchronize()
+        self.scene.set_option(pic.OPT_VIEW_FIRST, 0)
+        self.scene.set_option(pic.OPT_VIEW_COUNT, 0)
+        return rgb.cpu().numpy().reshape(s.E * s.A * s.K, s.H, s.W, 3), self.scene.status()
+
     def close(self):
         self.scene.close()
 
