@@ -62,29 +62,99 @@ struct RayView { float* ray_x; float* ray_y; };
 struct PixelLines { float e[CLINES]; };
 
 // Coverage (14 bits) of one pixel by a record, given its lines at the pixel centre and their half ranges hh over
-// the pixel (a line with e >= hh contains the whole pixel).
-__device__ __forceinline__ uint32_t coverage14(const PixelLines& L, const PrimEq& q, const float (&hh)[CLINES], float du, float dv, bool want) {
-    float a[CLINES], b[CLINES];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { a[i] = q.nx[i] * du; b[i] = q.ny[i] * dv; }
-    a[4] = q.wx * du; b[4] = q.wy * dv; a[5] = -a[4]; b[5] = -b[4];
+// the pixel (a line with e >= hh contains the whole pixel): the closed forms for one line, or two lines that do
+// not cross inside the pixel.  Anything else (a vertex in the pixel, three lines) returns COVERAGE_PENDING: those
+// pixels are few per cell, so their areas are worked out later, a lane each (finish_coverage).
+constexpr uint32_t COVERAGE_PENDING = 0x3fffu, COVERAGE_MAX = 0x3ffeu;
+__device__ __forceinline__ uint32_t coverage14(const PixelLines& L, const PrimEq& q, const float (&hh)[CLINES], float du, float dv) {
     int n_part = 0;
-    float ew = 0.f, aw = 0.f, bw = 0.f;
+    float e1 = 0.f, a1 = 0.f, b1 = 0.f, e2 = 0.f, a2 = 0.f, b2 = 0.f;      // the last two lines that cross the pixel
 #pragma unroll
-    for (int i = 0; i < CLINES; ++i)
-        if (L.e[i] < hh[i]) { ++n_part; ew = L.e[i]; aw = a[i]; bw = b[i]; }
-    float alpha = 0.f;
-    const bool general = want && n_part > 1;
-    if (want && n_part == 1) alpha = edge_coverage(ew, aw, bw);      // one line crosses the pixel, the others contain it
-    if (__any_sync(0xffffffffu, general)) {
-        if (general) alpha = pixel_coverage(L.e, a, b);
+    for (int i = 0; i < CLINES; ++i) {
+        const float ai = (i < 4 ? q.nx[i] : i == 4 ? q.wx : -q.wx) * du, bi = (i < 4 ? q.ny[i] : i == 4 ? q.wy : -q.wy) * dv;
+        if (L.e[i] < hh[i]) { ++n_part; e2 = e1; a2 = a1; b2 = b1; e1 = L.e[i]; a1 = ai; b1 = bi; }
     }
-    return (uint32_t)(alpha * 16383.f + 0.5f);
+    float alpha = 0.f;
+    if (n_part == 1) alpha = edge_coverage(e1, a1, b1);
+    else if (n_part != 2 || !two_line_coverage(e1, a1, b1, e2, a2, b2, alpha)) return COVERAGE_PENDING;
+    return min((uint32_t)(alpha * 16383.f + 0.5f), COVERAGE_MAX);
+}
+
+// The strip's queue of pending pixels (pixel << 8 | slot; it grows down from the top of the fragment array while
+// the lists grow up from its bottom), a lane each: the record's six lines at the pixel, the exact area, the depth;
+// pixels with a positive area join their pixel's list.  The newest items -- those next to the lists' end -- go first,
+// so the entries written never reach items not yet read.
+__device__ __noinline__ void flush_pending(unsigned long long* frag, uint16_t* head, int& n_frag, int& n_pend, const ColourPool& pool,
+                                              const float* ray_x, const float* ray_y, float du, float dv, float w_near, float w_far, int lane) {
+    while (n_pend > 0) {
+        const int take = min(n_pend, 32);
+        const bool have = lane < take;
+        const uint32_t item = have ? (uint32_t)frag[CFRAGS - (n_pend - 1) + lane] : 0u;
+        __syncwarp();
+        uint32_t a14 = 0u;
+        float wc = 0.f;
+        const uint32_t pix = item >> 8, slot = item & 0xffu;
+        int n_cross = 0;
+        float area = 0.f;
+        float e[CLINES], a[CLINES], b[CLINES];
+        float w = 0.f;
+#pragma unroll
+        for (int j = 0; j < CLINES; ++j) { e[j] = 1.f; a[j] = 0.f; b[j] = 0.f; }
+        if (have) {
+            const float rx = ray_x[pix & (TILE - 1)], ry = ray_y[pix >> 6];
+            const float4 r0 = pool.nx[slot], r1 = pool.ny[slot], r2 = pool.nz[slot], r3 = pool.w[slot];
+            const float nx[4] = {r0.x, r0.y, r0.z, r0.w}, ny[4] = {r1.x, r1.y, r1.z, r1.w}, nz[4] = {r2.x, r2.y, r2.z, r2.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { e[j] = fm(nx[j], rx, fm(ny[j], ry, nz[j])); a[j] = nx[j] * du; b[j] = ny[j] * dv; }
+            w = fm(r3.x, rx, fm(r3.y, ry, r3.z));
+            e[4] = w - w_far; e[5] = w_near - w; a[4] = r3.x * du; b[4] = r3.y * dv; a[5] = -a[4]; b[5] = -b[4];
+            // the lines that cross the pixel, up to four of them, moved to the front (the others contain the pixel)
+            const float hw = 0.5f * (fabsf(a[4]) + fabsf(b[4]));
+            float e3[4] = {1.f, 1.f, 1.f, 1.f}, a3[4] = {0.f, 0.f, 0.f, 0.f}, b3[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < CLINES; ++j) {
+                const float hj = j < 4 ? 0.5f * (fabsf(a[j]) + fabsf(b[j])) : hw;
+                if (e[j] < hj) {
+                    ++n_cross;
+                    e3[3] = e3[2]; a3[3] = a3[2]; b3[3] = b3[2];
+                    e3[2] = e3[1]; a3[2] = a3[1]; b3[2] = b3[1]; e3[1] = e3[0]; a3[1] = a3[0]; b3[1] = b3[0];
+                    e3[0] = e[j]; a3[0] = a[j]; b3[0] = b[j];
+                }
+            }
+            area = pixel_coverage<4>(e3, a3, b3);
+        }
+        if (__any_sync(0xffffffffu, n_cross > 4)) {            // rare: more than four lines through one pixel
+            if (n_cross > 4) area = pixel_coverage<CLINES>(e, a, b);
+        }
+        if (have) {
+            a14 = min((uint32_t)(area * 16383.f + 0.5f), COVERAGE_MAX);
+            wc = fminf(fmaxf(w, w_far), w_near);
+        }
+        n_pend -= take;
+        // (two items of a round may belong to one pixel -- two records with a vertex there -- so the lists are
+        // extended one lane after the other)
+        const unsigned m = __ballot_sync(0xffffffffu, a14 != 0u);
+        const int idx = n_frag + 1 + __popc(m & ((1u << lane) - 1u));
+        // lanes whose pixel no other lane of the round shares link their entries at once
+        const bool alone = __popc(__match_any_sync(0xffffffffu, a14 != 0u ? pix : 0x10000u + lane)) == 1;
+        if (a14 != 0u && alone) {
+            frag[idx] = ((unsigned long long)__float_as_uint(wc) << 32) | (a14 << 18) | (slot << 10) | head[pix];
+            head[pix] = (uint16_t)idx;
+        }
+        for (unsigned rest = __ballot_sync(0xffffffffu, a14 != 0u && !alone); rest; rest &= rest - 1) {
+            if (lane == __ffs(rest) - 1) {
+                frag[idx] = ((unsigned long long)__float_as_uint(wc) << 32) | (a14 << 18) | (slot << 10) | head[pix];
+                head[pix] = (uint16_t)idx;
+            }
+            __syncwarp();
+        }
+        n_frag += __popc(m);
+    }
 }
 
 // A 16 x 4 pixel cell of a strip against one record; a lane handles two adjacent pixels.
 template <bool AA>
-__device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* head, unsigned long long* frag, int& n_frag,
+__device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* head, unsigned long long* frag, int& n_frag, int& n_pend, bool& dropped,
                                             const float* ray_x, const float* ray_y, const PrimEq& q, const float (&thr)[4],
                                             const float (&hh)[CLINES], float du, float dv, uint32_t key_lo, uint32_t slot,
                                             float w_near, float w_far, int xx, int yy, int lane) {
@@ -122,21 +192,35 @@ __device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* h
         // partially covered pixels in front of the nearest fully covering fragment seen so far
         bool push0 = !full0 && !out0 && k0 > kk.x, push1 = !full1 && !out1 && k1 > kk.y;
         if (__any_sync(0xffffffffu, push0 || push1)) {
-            const uint32_t a0 = coverage14(L0, q, hh, du, dv, push0), a1 = coverage14(L1, q, hh, du, dv, push1);
-            push0 = push0 && a0 != 0u; push1 = push1 && a1 != 0u;
+            // (one copy of the coverage code serves both pixels: the instruction cache matters more than the selects)
+            uint32_t a0 = 0u, a1 = 0u;
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                PixelLines L;
+#pragma unroll
+                for (int e = 0; e < CLINES; ++e) L.e[e] = h ? L1.e[e] : L0.e[e];
+                const uint32_t av = (h ? push1 : push0) ? coverage14(L, q, hh, du, dv) : 0u;
+                if (h) a1 = av; else a0 = av;
+            }
+            const bool pend0 = push0 && a0 == COVERAGE_PENDING, pend1 = push1 && a1 == COVERAGE_PENDING;
+            push0 = push0 && a0 != 0u && !pend0; push1 = push1 && a1 != 0u && !pend1;
             const unsigned m0 = __ballot_sync(0xffffffffu, push0), m1 = __ballot_sync(0xffffffffu, push1);
+            const unsigned q0 = __ballot_sync(0xffffffffu, pend0), q1 = __ballot_sync(0xffffffffu, pend1);
             const unsigned below = (1u << lane) - 1u;
-            const int i0 = n_frag + 1 + __popc(m0 & below), i1 = n_frag + 1 + __popc(m0) + __popc(m1 & below);
             const int pix = y * TILE + x;
-            if (push0 && i0 <= CFRAGS) {
-                frag[i0] = ((unsigned long long)__float_as_uint(c0) << 32) | (a0 << 18) | (slot << 10) | head[pix];
-                head[pix] = (uint16_t)i0;
+            // room: lists and queue share the array; what does not fit is dropped (and the call says so)
+            const bool room = n_frag + n_pend + __popc(m0) + __popc(m1) + __popc(q0) + __popc(q1) <= CFRAGS;
+            if (room) {
+                const int i0 = n_frag + 1 + __popc(m0 & below), i1 = n_frag + 1 + __popc(m0) + __popc(m1 & below);
+                if (push0) { frag[i0] = ((unsigned long long)__float_as_uint(c0) << 32) | (a0 << 18) | (slot << 10) | head[pix]; head[pix] = (uint16_t)i0; }
+                if (push1) { frag[i1] = ((unsigned long long)__float_as_uint(c1) << 32) | (a1 << 18) | (slot << 10) | head[pix + 1]; head[pix + 1] = (uint16_t)i1; }
+                n_frag += __popc(m0) + __popc(m1);
+                if (pend0) frag[CFRAGS - (n_pend + __popc(q0 & below))] = ((uint32_t)pix << 8) | slot;
+                if (pend1) frag[CFRAGS - (n_pend + __popc(q0) + __popc(q1 & below))] = ((uint32_t)(pix + 1) << 8) | slot;
+                n_pend += __popc(q0) + __popc(q1);
+            } else {
+                dropped = true;
             }
-            if (push1 && i1 <= CFRAGS) {
-                frag[i1] = ((unsigned long long)__float_as_uint(c1) << 32) | (a1 << 18) | (slot << 10) | head[pix + 1];
-                head[pix + 1] = (uint16_t)i1;
-            }
-            n_frag += __popc(m0) + __popc(m1);
         }
     }
 }
@@ -151,69 +235,97 @@ __device__ __forceinline__ void shade_fragment(const ColourPool& pool, const Ren
     r = k * (float)__ldg(pal); g = k * (float)__ldg(pal + 1); b = k * (float)__ldg(pal + 2);
 }
 
-// One strip of tile `jb` -> colour image: every lane resolves 16 consecutive pixels of a row, resets what it reads.
+// Colour of a pixel with a list of partially covering fragments: front to back, the list's fragments in front of the
+// fully covering one `k`, then that one, then the background.  Consecutive fragments of one surface form a layer:
+// each adds its coverage until the layer is full.  Returns the colour packed 8 bits per channel.
+__device__ __forceinline__ uint32_t composite_pixel(unsigned long long k, uint32_t hd, const unsigned long long* frag, const ColourPool& pool,
+                                                    const RenderParams& P, float bgr, float bgg, float bgb) {
+    const uint32_t w_opq = (uint32_t)(k >> 32);
+    float T = 1.f, acc = 0.f, R = 0.f, G = 0.f, B = 0.f;
+    uint32_t cur = 0xffffffffu;
+    unsigned long long prev = ~0ull;
+    for (int it = 0; it < 64 && T > 0.f; ++it) {
+        // the nearest remaining fragment: the largest (1/z, entry) below the last one taken; at the end, the opaque one
+        unsigned long long best = 0ull;
+        uint32_t best_lo = 0u;
+        for (uint32_t i = hd; i;) {
+            const unsigned long long en = frag[i];
+            const unsigned long long cand = (en & 0xffffffff00000000ull) | i;
+            if (cand < prev && cand > best && (uint32_t)(en >> 32) > w_opq) { best = cand; best_lo = (uint32_t)en; }
+            i = (uint32_t)en & 1023u;
+        }
+        uint32_t slot, wb;
+        float alpha;
+        if (best) { prev = best; slot = (best_lo >> 10) & 0xffu; alpha = (float)((best_lo >> 18) & 0x3fffu) * (1.f / 16383.f); wb = (uint32_t)(best >> 32); }
+        else if (k && prev != 0ull) { prev = 0ull; slot = (uint32_t)k & 0xffu; alpha = 1.f; wb = w_opq; }
+        else break;
+        const uint32_t surf = pool.surface[slot] & 0x1ffffu;
+        if (surf != cur) { T *= 1.f - acc; cur = surf; acc = 0.f; }
+        const float add = fminf(alpha, 1.f - acc) * T;
+        float cr, cg, cb;
+        shade_fragment(pool, P, slot, __uint_as_float(wb), cr, cg, cb);
+        R = fm(add, cr, R); G = fm(add, cg, G); B = fm(add, cb, B);
+        acc += fminf(alpha, 1.f - acc);
+    }
+    T *= 1.f - acc;
+    R = fm(T, bgr, R); G = fm(T, bgg, G); B = fm(T, bgb, B);
+    return (uint32_t)fminf(fmaxf(R + 0.5f, 0.f), 255.f) | ((uint32_t)fminf(fmaxf(G + 0.5f, 0.f), 255.f) << 8) |
+           ((uint32_t)fminf(fmaxf(B + 0.5f, 0.f), 255.f) << 16);
+}
+
+constexpr unsigned long long KEY_RESOLVED = 1ull << 63;     // (a key's high word is the bits of a positive float: bit 63 is free)
+
+// One strip of tile `jb` -> colour image.  First the pixels that have a list are composited, lane l taking pixels
+// l, l + 32, ... of the strip so that a row crowded with fragments (the horizon) is shared by all lanes; their colour
+// replaces the pixel's key.  Then every lane converts 16 consecutive pixels of a row, resets what it reads, and stores.
 template <bool AA>
 __device__ __forceinline__ void resolve_store_colour(unsigned long long* key, uint16_t* head, const unsigned long long* frag,
                                                      const ColourPool& pool, const RenderParams& P, const Job& jb, bool ego_active,
                                                      int ys, bool vec_ok, int lane) {
+    if (AA) {
+#pragma unroll 1
+        for (int i = 0; i < CSTRIP_KEYS / 32; ++i) {
+            const int p = i * 32 + lane, x = p & (TILE - 1), y = p >> 6;
+            const uint32_t hd = head[p];
+            if (hd) {
+                head[p] = 0;
+                const int gy = jb.t.y0 + ys + y;
+                uint32_t bgc = P.cls_sky;
+                if (ego_active && gy < P.H) bgc = __ldg(P.rig.bg_cls + (size_t)jb.k * P.H + gy);
+                unsigned long long* kp = key + key_index(x, y);
+                *kp = KEY_RESOLVED | composite_pixel(*kp, hd, frag, pool, P, (float)__ldg(P.palette + 3u * bgc), (float)__ldg(P.palette + 3u * bgc + 1),
+                                                     (float)__ldg(P.palette + 3u * bgc + 2));
+            }
+        }
+        __syncwarp();
+    }
     const int y = lane >> 2, xs = (lane & 3) * 16;
     const int gy = jb.t.y0 + ys + y;
     uint32_t bgc = P.cls_sky;
     if (ego_active && gy < P.H) bgc = __ldg(P.rig.bg_cls + (size_t)jb.k * P.H + gy);
-    const float bgr = (float)__ldg(P.palette + 3u * bgc), bgg = (float)__ldg(P.palette + 3u * bgc + 1), bgb = (float)__ldg(P.palette + 3u * bgc + 2);
+    const uint32_t bg8 = (uint32_t)__ldg(P.palette + 3u * bgc) | ((uint32_t)__ldg(P.palette + 3u * bgc + 1) << 8) | ((uint32_t)__ldg(P.palette + 3u * bgc + 2) << 16);
     uint32_t ow[12];
 #pragma unroll
     for (int i = 0; i < 12; ++i) ow[i] = 0u;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const int x = xs + j;
-        unsigned long long* kp = key + key_index(x, y);
-        const unsigned long long k = *kp;
-        *kp = 0ull;
-        uint32_t hd = 0u;
-        if (AA) { hd = head[y * TILE + x]; head[y * TILE + x] = 0; }
-        float R = bgr, G = bgg, B = bgb;
-        if (hd == 0u) {
-            if (k) shade_fragment(pool, P, (uint32_t)k & 0xffu, __uint_as_float((uint32_t)(k >> 32)), R, G, B);
-        } else {
-            // front to back: the list's fragments in front of the fully covering one, then that one, then the background.
-            // Consecutive fragments of one surface form a layer: each adds its coverage until the layer is full.
-            const uint32_t w_opq = (uint32_t)(k >> 32);
-            float T = 1.f, acc = 0.f;
-            R = 0.f; G = 0.f; B = 0.f;
-            uint32_t cur = 0xffffffffu;
-            unsigned long long prev = ~0ull;
-            for (int it = 0; it < 48 && T > 0.f; ++it) {
-                // the nearest remaining fragment: the largest (1/z, entry) below the last one taken; at the end, the opaque one
-                unsigned long long best = 0ull;
-                uint32_t best_lo = 0u;
-                for (uint32_t i = hd; i;) {
-                    const unsigned long long en = frag[i];
-                    const unsigned long long cand = (en & 0xffffffff00000000ull) | i;
-                    if (cand < prev && cand > best && (uint32_t)(en >> 32) > w_opq) { best = cand; best_lo = (uint32_t)en; }
-                    i = (uint32_t)en & 1023u;
-                }
-                uint32_t slot, wb;
-                float alpha;
-                if (best) { prev = best; slot = (best_lo >> 10) & 0xffu; alpha = (float)((best_lo >> 18) & 0x3fffu) * (1.f / 16383.f); wb = (uint32_t)(best >> 32); }
-                else if (k && prev != 0ull) { prev = 0ull; slot = (uint32_t)k & 0xffu; alpha = 1.f; wb = w_opq; }
-                else break;
-                const uint32_t surf = pool.surface[slot];
-                if (surf != cur) { T *= 1.f - acc; cur = surf; acc = 0.f; }
-                const float add = fminf(alpha, 1.f - acc) * T;
-                float cr, cg, cb;
-                shade_fragment(pool, P, slot, __uint_as_float(wb), cr, cg, cb);
-                R = fm(add, cr, R); G = fm(add, cg, G); B = fm(add, cb, B);
-                acc += fminf(alpha, 1.f - acc);
+    for (int j = 0; j < 16; j += 2) {
+        ulonglong2* kp = reinterpret_cast<ulonglong2*>(key + key_index(xs + j, y));
+        const ulonglong2 kk = *kp;
+        *kp = make_ulonglong2(0ull, 0ull);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const unsigned long long k = h ? kk.y : kk.x;
+            uint32_t c = bg8;
+            if (k & KEY_RESOLVED) c = (uint32_t)k & 0xffffffu;
+            else if (k) {
+                float R, G, B;
+                shade_fragment(pool, P, (uint32_t)k & 0xffu, __uint_as_float((uint32_t)(k >> 32)), R, G, B);
+                c = (uint32_t)fminf(R + 0.5f, 255.f) | ((uint32_t)fminf(G + 0.5f, 255.f) << 8) | ((uint32_t)fminf(B + 0.5f, 255.f) << 16);
             }
-            T *= 1.f - acc;
-            R = fm(T, bgr, R); G = fm(T, bgg, G); B = fm(T, bgb, B);
+            const int n = 3 * (j + h);           // byte offset of the pixel in the lane's 48 bytes
+            ow[n >> 2] |= c << (8 * (n & 3));
+            if ((n & 3) > 1) ow[(n >> 2) + 1] |= c >> (8 * (4 - (n & 3)));
         }
-        const uint32_t r8 = (uint32_t)fminf(fmaxf(R + 0.5f, 0.f), 255.f), g8 = (uint32_t)fminf(fmaxf(G + 0.5f, 0.f), 255.f),
-                       b8 = (uint32_t)fminf(fmaxf(B + 0.5f, 0.f), 255.f);
-        ow[(3 * j) >> 2] |= r8 << (8 * ((3 * j) & 3));
-        ow[(3 * j + 1) >> 2] |= g8 << (8 * ((3 * j + 1) & 3));
-        ow[(3 * j + 2) >> 2] |= b8 << (8 * ((3 * j + 2) & 3));
     }
     if (ys + y >= jb.t.th || xs >= jb.t.tw) return;
     uint8_t* dst = P.out_rgb + 3u * ((jb.view * (size_t)P.H + gy) * (size_t)P.W + jb.t.x0 + xs);
@@ -316,12 +428,39 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                 const int slot = my_base + i;
                 if (drop || !prim_equations(V, flags & 1u, flags, Pn, q)) { s.pool.box[slot] = REC_DEAD; continue; }
                 const uint32_t box = svi.y;
-                const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+                uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
+                uint32_t onepix = 0u;
+                if (AA) {
+                    // a primitive that lies inside one pixel and well within the depth range covers its own projected
+                    // area of that pixel and nothing else: no clipping needed (most distant primitives are of this kind)
+                    const float zlo = fminf(fminf(V[0].z, V[1].z), fminf(V[2].z, V[3].z)), zhi = fmaxf(fmaxf(V[0].z, V[1].z), fmaxf(V[2].z, V[3].z));
+                    if (zlo >= P.near_z * 1.001f && zhi <= P.far_z * 0.999f) {
+                        float sx[4], sy[4];
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            const float iz = __fdividef(1.f, V[v].z);
+                            sx[v] = fm(c.focx, V[v].x * iz, c.cx - (float)job.t.x0); sy[v] = fm(c.focy, V[v].y * iz, c.cy - (float)job.t.y0);
+                        }
+                        const float x_lo = fminf(fminf(sx[0], sx[1]), fminf(sx[2], sx[3])), x_hi = fmaxf(fmaxf(sx[0], sx[1]), fmaxf(sx[2], sx[3]));
+                        const float y_lo = fminf(fminf(sy[0], sy[1]), fminf(sy[2], sy[3])), y_hi = fmaxf(fmaxf(sy[0], sy[1]), fmaxf(sy[2], sy[3]));
+                        const float fxl = floorf(x_lo + 1e-4f), fyl = floorf(y_lo + 1e-4f);
+                        if (floorf(x_hi - 1e-4f) <= fxl && floorf(y_hi - 1e-4f) <= fyl && x_hi - x_lo < 1.f && y_hi - y_lo < 1.f) {
+                            float twice = 0.f;
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) twice += (sx[v] - x_lo) * (sy[(v + 1) & 3] - y_lo) - (sx[(v + 1) & 3] - x_lo) * (sy[v] - y_lo);
+                            const uint32_t a14 = min((uint32_t)(0.5f * fabsf(twice) * 16383.f + 0.5f), COVERAGE_MAX);
+                            if (a14 == 0u || fxl < 0.f || fyl < 0.f || fxl >= (float)job.t.tw || fyl >= (float)job.t.th) { s.pool.box[slot] = REC_DEAD; continue; }
+                            bx0 = bx1 = (uint32_t)fxl; by0 = by1 = (uint32_t)fyl;
+                            onepix = REC_TINY;
+                            surface |= a14 << 17;
+                        }
+                    }
+                }
                 s.pool.nx[slot] = make_float4(q.nx[0], q.nx[1], q.nx[2], q.nx[3]);
                 s.pool.ny[slot] = make_float4(q.ny[0], q.ny[1], q.ny[2], q.ny[3]);
                 s.pool.nz[slot] = make_float4(q.nz[0], q.nz[1], q.nz[2], q.nz[3]);
                 s.pool.w[slot] = make_float4(q.wx, q.wy, q.wz, __uint_as_float(key_lo));
-                s.pool.box[slot] = bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24);
+                s.pool.box[slot] = bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24) | onepix;
                 s.pool.shade[slot] = shade;
                 s.pool.surface[slot] = surface;
             }
@@ -347,7 +486,8 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
             const float* ray_x = s.ray_x[j];
             const float* ray_y = s.ray_y[j] + ys;
             const float du = __fdividef(1.f, s.cam[j].focx), dv = __fdividef(1.f, s.cam[j].focy);
-            int n_frag = 0;
+            int n_frag = 0, n_pend = 0;
+            bool dropped = false;
             for (int base = 0; base < cj; base += 32) {
                 uint32_t bw_lane = 0u;
                 bool hit = false;
@@ -355,6 +495,38 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     bw_lane = s.pool.box[first + base + lane];
                     const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
                     hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + CSTRIP;
+                }
+                if (AA) {
+                    // records that lie inside one pixel: their lane adds the fragment (coverage known from set-up)
+                    bool one = hit && (bw_lane & REC_TINY);
+                    hit = hit && !one;
+                    uint32_t pix = 0u, a14 = 0u, wb = 0u;
+                    const uint32_t slot = (uint32_t)(first + base + lane);
+                    if (one) {
+                        const int x = bw_lane & 63, y = ((bw_lane >> 6) & 63) - ys;
+                        pix = (uint32_t)(y * TILE + x);
+                        const float4 r3 = s.pool.w[slot];
+                        const float w = fminf(fmaxf(fm(r3.x, ray_x[x], fm(r3.y, ray_y[y], r3.z)), P.w_far), P.w_near);
+                        wb = __float_as_uint(w);
+                        a14 = s.pool.surface[slot] >> 17;
+                        one = make_key(wb, 0xffffffffu) > key[key_index(x, y)];       // in front of the nearest fully covering fragment so far
+                    }
+                    const unsigned m = __ballot_sync(0xffffffffu, one);
+                    if (m) {
+                        const bool room = n_frag + n_pend + __popc(m) <= CFRAGS;
+                        dropped = dropped || !room;
+                        const int idx = n_frag + 1 + __popc(m & ((1u << lane) - 1u));
+                        const bool alone = __popc(__match_any_sync(0xffffffffu, one ? pix : 0x10000u + lane)) == 1;
+                        if (room) {
+                            if (one && alone) { frag[idx] = ((unsigned long long)wb << 32) | (a14 << 18) | (slot << 10) | head[pix]; head[pix] = (uint16_t)idx; }
+                            for (unsigned rest = __ballot_sync(0xffffffffu, one && !alone); rest; rest &= rest - 1) {
+                                if (lane == __ffs(rest) - 1) { frag[idx] = ((unsigned long long)wb << 32) | (a14 << 18) | (slot << 10) | head[pix]; head[pix] = (uint16_t)idx; }
+                                __syncwarp();
+                            }
+                            n_frag += __popc(m);
+                        }
+                        __syncwarp();
+                    }
                 }
                 for (unsigned hits = __ballot_sync(0xffffffffu, hit); hits; hits &= hits - 1) {
                     const int src = __ffs(hits) - 1;
@@ -377,11 +549,18 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     hh[4] = hh[5] = 0.5f * (fabsf(q.wx) * du + fabsf(q.wy) * dv);
                     for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
                         for (int xx = bx0 & ~15; xx <= bx1; xx += 16)
-                            colour_cell<AA>(key, head, frag, n_frag, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, lane);
+                            colour_cell<AA>(key, head, frag, n_frag, n_pend, dropped, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, lane);
+                    // the queue is worked off when it holds a few rounds' worth (working it off frees room only for the
+                    // pixels whose area turns out to be zero, so a nearly full array is no reason to do it earlier)
+                    if (AA && n_pend >= 96) {
+                        __syncwarp();
+                        flush_pending(frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
+                    }
                 }
                 __syncwarp();
             }
-            if (AA && n_frag > CFRAGS && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);   // fragments were dropped
+            if (AA) flush_pending(frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
+            if (AA && dropped && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);
             __syncwarp();
             resolve_store_colour<AA>(key, head, frag, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
             __syncwarp();

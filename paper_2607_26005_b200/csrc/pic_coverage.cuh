@@ -17,8 +17,9 @@ __device__ __forceinline__ float edge_coverage(float e0, float a, float b) {
     return e0 < 0.f ? corner : 1.f - corner;
 }
 
-// Area of the part of the unit square around a pixel centre on which all six e[i] + a[i] x + b[i] y >= 0 (a
-// record's four edges and the two lines at which its plane reaches the far and the near depth).
+// Area of the part of the unit square around a pixel centre on which all NL lines e[i] + a[i] x + b[i] y >= 0 (of a
+// record's four edges and the two lines at which its plane reaches the far and the near depth, all six or those
+// that cross the pixel; an unused slot holds the constant 1).
 // The region is convex; its area is half the sum over its boundary lines -- the square's four sides and the
 // six lines -- of (distance of the line from the centre) x (length of the line's piece on the boundary); the
 // piece is found by cutting the line with all other constraints.  Written with t measured along (B, -A), which
@@ -28,39 +29,79 @@ __device__ __forceinline__ float edge_coverage(float e0, float a, float b) {
 // so exactly one of the two keeps the piece whatever the rounding.  (Two coinciding lines that face each
 // other bound a sliver; both keep their piece and the two contributions cancel.)
 constexpr int CLINES = 6;
-__device__ __forceinline__ float pixel_coverage(const float (&e)[CLINES], const float (&a)[CLINES], const float (&b)[CLINES]) {
-    constexpr int N = 4 + CLINES;
-    float A[N], B[N], C[N], nudge[N];
+template <int NL>
+__device__ __forceinline__ float pixel_coverage(const float (&e)[NL], const float (&a)[NL], const float (&b)[NL]) {
+    constexpr int N = 4 + NL;
+    float A[N], B[N], C[N];
     A[0] = 1.f; A[1] = -1.f; A[2] = 0.f; A[3] = 0.f;
     B[0] = 0.f; B[1] = 0.f; B[2] = 1.f; B[3] = -1.f;
 #pragma unroll
     for (int m = 0; m < 4; ++m) C[m] = 0.5f;
 #pragma unroll
-    for (int m = 0; m < CLINES; ++m) { A[4 + m] = a[m]; B[4 + m] = b[m]; C[4 + m] = e[m]; }
-#pragma unroll
-    for (int m = 0; m < N; ++m) nudge[m] = 1e-5f * (fabsf(A[m]) + fabsf(B[m]));
+    for (int m = 0; m < NL; ++m) { A[4 + m] = a[m]; B[4 + m] = b[m]; C[4 + m] = e[m]; }
     float twice = 0.f;
-#pragma unroll
+    // A loop over the boundary lines that is NOT unrolled (the code stays small enough for the instruction cache):
+    // the line in turn sits in slot 0 and the arrays are rotated by one slot per turn, so slot p holds line
+    // (j + p) mod N, which has a lower index than line j exactly when p >= N - j.
+#pragma unroll 1
     for (int j = 0; j < N; ++j) {
-        const float n2 = fm(A[j], A[j], mul(B[j], B[j]));
-        if (n2 > 0.f) {
-            const float k = -__fdividef(C[j], n2), p0x = k * A[j], p0y = k * B[j];     // the line's point nearest the centre
-            float t0 = -3e38f, t1 = 3e38f;
+        const float n2 = fm(A[0], A[0], mul(B[0], B[0]));
+        const float k = -__fdividef(C[0], n2), p0x = k * A[0], p0y = k * B[0];     // the line's point nearest the centre
+        float t0 = -3e38f, t1 = 3e38f;
 #pragma unroll
-            for (int m = 0; m < N; ++m) {
-                if (m == j) continue;
-                const float be = fm(A[m], B[j], -mul(B[m], A[j]));
-                const bool same_side = m < j && fm(A[m], A[j], mul(B[m], B[j])) > 0.f;
-                const float al = fm(A[m], p0x, fm(B[m], p0y, C[m])) + (same_side ? -nudge[m] : nudge[m]);
-                const float t = -__fdividef(al, be);
-                if (be > 0.f) t0 = fmaxf(t0, t);
-                else if (be < 0.f) t1 = fminf(t1, t);
-                else if (al < 0.f) t1 = -3e38f;                                          // parallel and outside
-            }
-            if (t1 > t0) twice = fm(C[j], t1 - t0, twice);
+        for (int p = 1; p < N; ++p) {
+            const float be = fm(A[p], B[0], -mul(B[p], A[0]));
+            const bool same_side = p >= N - j && fm(A[p], A[0], mul(B[p], B[0])) > 0.f;
+            const float nudge = 1e-5f * (fabsf(A[p]) + fabsf(B[p]));
+            const float al = fm(A[p], p0x, fm(B[p], p0y, C[p])) + (same_side ? -nudge : nudge);
+            const float t = -__fdividef(al, be);
+            // (written with selects: the lanes of a warp rarely agree on the sign of be)
+            t0 = be > 0.f ? fmaxf(t0, t) : t0;
+            t1 = be < 0.f ? fminf(t1, t) : t1;
+            t1 = (be == 0.f && al < 0.f) ? -3e38f : t1;                                  // parallel and outside
         }
+        // (a constant, n2 == 0 -- a triangle's fourth edge, an unused slot -- bounds nothing)
+        twice = (n2 > 0.f && t1 > t0) ? fm(C[0], t1 - t0, twice) : twice;
+        const float ra = A[0], rb = B[0], rc = C[0];
+#pragma unroll
+        for (int p = 0; p + 1 < N; ++p) { A[p] = A[p + 1]; B[p] = B[p + 1]; C[p] = C[p + 1]; }
+        A[N - 1] = ra; B[N - 1] = rb; C[N - 1] = rc;
     }
     return fminf(fmaxf(0.5f * twice, 0.f), 1.f);
+}
+
+// A point of the line e + a x + b y = 0 inside the pixel's square (the middle of its chord); false if it misses the square.
+__device__ __forceinline__ bool chord_point(float e, float a, float b, float& px, float& py) {
+    const float n2 = fm(a, a, mul(b, b));
+    const float k = -__fdividef(e, n2), p0x = k * a, p0y = k * b;
+    float t0 = -3e38f, t1 = 3e38f;
+    // x(t) = p0x + t b within [-1/2, 1/2], y(t) = p0y - t a within [-1/2, 1/2]
+    if (b != 0.f) { const float u = __fdividef(-0.5f - p0x, b), v = __fdividef(0.5f - p0x, b); t0 = fmaxf(t0, fminf(u, v)); t1 = fminf(t1, fmaxf(u, v)); }
+    else if (fabsf(p0x) > 0.5f) return false;
+    if (a != 0.f) { const float u = __fdividef(p0y + 0.5f, a), v = __fdividef(p0y - 0.5f, a); t0 = fmaxf(t0, fminf(u, v)); t1 = fminf(t1, fmaxf(u, v)); }
+    else if (fabsf(p0y) > 0.5f) return false;
+    const float tm = 0.5f * (t0 + t1);
+    px = fm(tm, b, p0x); py = fm(-tm, a, p0y);
+    return t1 >= t0;
+}
+
+// Area of the pixel's square inside two lines that do not cross inside it (a strip, two nested half planes, two
+// separate corners): from the two one-line coverages.  Returns false if the lines cross inside the square (or too
+// near its border to tell): then the area takes the general formula.
+__device__ __forceinline__ bool two_line_coverage(float e1, float a1, float b1, float e2, float a2, float b2, float& area) {
+    const float det = fm(a1, b2, -mul(a2, b1));
+    const float scale = (fabsf(a1) + fabsf(b1)) * (fabsf(a2) + fabsf(b2));
+    if (fabsf(det) > 1e-6f * scale) {
+        const float x = __fdividef(fm(b1, e2, -mul(b2, e1)), det), y = __fdividef(fm(a2, e1, -mul(a1, e2)), det);
+        if (fabsf(x) < 0.5001f && fabsf(y) < 0.5001f) return false;
+    }
+    float p1x, p1y, p2x, p2y;
+    if (!chord_point(e1, a1, b1, p1x, p1y) || !chord_point(e2, a2, b2, p2x, p2y)) return false;
+    const float c1 = edge_coverage(e1, a1, b1), c2 = edge_coverage(e2, a2, b2);
+    const bool in2 = fm(a2, p1x, fm(b2, p1y, e2)) >= 0.f;     // line 1's chord lies inside line 2
+    const bool in1 = fm(a1, p2x, fm(b1, p2y, e1)) >= 0.f;
+    area = (in1 && in2) ? fmaxf(c1 + c2 - 1.f, 0.f) : in1 ? c2 : in2 ? c1 : 0.f;
+    return true;
 }
 
 }  // namespace pic
