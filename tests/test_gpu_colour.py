@@ -133,3 +133,17 @@ def test_view_subrange_and_relative_output(gu):
         assert (out.cpu().numpy() == full[9:14]).all()
     finally:
         g.close()
+
+
+def test_paper_chunk_of_2048_egos_in_colour(gu):
+    # the bench's own launch: 31 map instances x 120 slots x 4 cameras at 96 x 54, antialiased; the oracle on sampled views
+    s = make_paper_workload(96, 54, egos=2048)
+    rng = np.random.default_rng(3)
+    act = np.flatnonzero(np.repeat(s.active.reshape(-1), s.K))
+    views = np.sort(rng.choice(act, size=96, replace=False))
+    st = check_colour(gu, s, views=views, modes=(True,))
+    print("paper chunk colour:", st)
+    # configs[2] at 16 environments (4 096 views of 64 x 64), plain and antialiased
+    s2 = make_config(2, E=16)
+    st2 = check_colour(gu, s2, views=np.sort(rng.choice(s2.E * s2.A * s2.K, size=64, replace=False)))
+    print("cfg2 E=16 colour:", st2)
