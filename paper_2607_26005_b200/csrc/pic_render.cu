@@ -845,7 +845,7 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
         ++n.grp;
         const float blo = gy0 + (float)row * mi.cell - margin, bhi = blo + mi.cell + 2.f * margin;
         float xlo = 3e38f, xhi = -3e38f;
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < 10; ++k) {
             const float px = f.seg[k][0], py = f.seg[k][1], dx = f.seg[k][2], dy = f.seg[k][3], idy = f.seg[k][4];
             const float ya = fminf(py, py + dy), yb = fmaxf(py, py + dy);
@@ -897,9 +897,9 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
             if (b0 + lane < P.A) ag0 = load_agent(env_agents + b0 + lane);
             if (b0 + lane + 32 < P.A) ag1 = load_agent(env_agents + b0 + lane + 32);
         }
-#pragma unroll
+#pragma unroll 1
         for (int u = 0; u < 2; ++u) {
-            const AgentGeom& g = u ? ag1 : ag0;
+            const AgentGeom g = u ? ag1 : ag0;
             const int b = b0 + lane + 32 * u;
             uint32_t faces = 0u;
             if (b < P.A && b != job.a && g.active) faces = box_faces(f, c, t, g);
@@ -945,18 +945,20 @@ __device__ __forceinline__ int front_cull(FrontLists& f, uint2* __restrict__ sur
                     load_prim(P.grid_prims + id[u], v[u], key_lo, flags);
                 }
             }
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
+#pragma unroll 1
+            for (int u = 0; u < 2; ++u) {               // (one copy of the test for both candidates: less code to fetch)
                 uint32_t box = 0;
                 bool keep = false;
-                if (have[u]) {
+                const bool hv = u ? have[1] : have[0];
+                if (hv) {
                     V3 V[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) V[q] = to_camera(c, v[u][3 * q], v[u][3 * q + 1], v[u][3 * q + 2]);
+                    for (int q = 0; q < 4; ++q)
+                        V[q] = to_camera(c, u ? v[1][3 * q] : v[0][3 * q], u ? v[1][3 * q + 1] : v[0][3 * q + 1], u ? v[1][3 * q + 2] : v[0][3 * q + 2]);
                     ++n.tested;
                     keep = pixel_box(c, t, V, box, BOX_MARGIN);
                 }
-                append_survivor(surv, keep, id[u], box, n_big, n_tiny, lane);
+                append_survivor(surv, keep, u ? id[1] : id[0], box, n_big, n_tiny, lane);
             }
         }
     }
