@@ -69,7 +69,7 @@ typedef enum {
                                         its state as it was */
 #define PIC_FLAG_COLOUR_INCOMPLETE 0x2u /* pic_render_rgb: a 64 x 64 tile saw more primitives than its list holds (254) and shows
                                            only the background */
-#define PIC_FLAG_COLOUR_FRAGMENTS 0x4u  /* pic_render_rgb, antialiased: an 8-row strip of a tile held more than 1023 partially
+#define PIC_FLAG_COLOUR_FRAGMENTS 0x4u  /* pic_render_rgb, antialiased: one row of a tile (64 pixels) held more than 1023 partially
                                            covered pixel fragments in front of its opaque surfaces; the surplus was dropped */
 
 /* One pinhole camera of the rig, in the agent frame (x forward, y left, z up). */

@@ -157,7 +157,7 @@ template <bool AA>
 __device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* head, unsigned long long* frag, int& n_frag, int& n_pend, bool& dropped,
                                             const float* ray_x, const float* ray_y, const PrimEq& q, const float (&thr)[4],
                                             const float (&hh)[CLINES], float du, float dv, uint32_t key_lo, uint32_t slot,
-                                            float w_near, float w_far, int xx, int yy, int lane) {
+                                            float w_near, float w_far, int xx, int yy, int row_lo, int row_hi, int lane) {
     const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
     const float2 rx = *reinterpret_cast<const float2*>(ray_x + x);
     const float ry = ray_y[y];
@@ -190,7 +190,8 @@ __device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* h
     if (full1 && k1 > kk.y) kp[1] = k1;
     if (AA) {
         // partially covered pixels in front of the nearest fully covering fragment seen so far
-        bool push0 = !full0 && !out0 && k0 > kk.x, push1 = !full1 && !out1 && k1 > kk.y;
+        const bool in_window = y >= row_lo && y < row_hi;      // (lists are kept for a window of the strip's rows at a time)
+        bool push0 = in_window && !full0 && !out0 && k0 > kk.x, push1 = in_window && !full1 && !out1 && k1 > kk.y;
         if (__any_sync(0xffffffffu, push0 || push1)) {
             // (one copy of the coverage code serves both pixels: the instruction cache matters more than the selects)
             uint32_t a0 = 0u, a1 = 0u;
@@ -275,16 +276,16 @@ __device__ __forceinline__ uint32_t composite_pixel(unsigned long long k, uint32
 
 constexpr unsigned long long KEY_RESOLVED = 1ull << 63;     // (a key's high word is the bits of a positive float: bit 63 is free)
 
-// One strip of tile `jb` -> colour image.  First the pixels that have a list are composited, lane l taking pixels
-// l, l + 32, ... of the strip so that a row crowded with fragments (the horizon) is shared by all lanes; their colour
-// replaces the pixel's key.  Then every lane converts 16 consecutive pixels of a row, resets what it reads, and stores.
-template <bool AA>
-__device__ __forceinline__ void resolve_store_colour(unsigned long long* key, uint16_t* head, const unsigned long long* frag,
-                                                     const ColourPool& pool, const RenderParams& P, const Job& jb, bool ego_active,
-                                                     int ys, bool vec_ok, int lane) {
-    if (AA) {
+// Rows of a strip of tile `jb` -> colours: the pixels that have a list are composited, lane l taking pixels l, l + 32, ...
+// so that a row crowded with fragments (the horizon) is shared by all lanes; their colour replaces the pixel's key
+// (composite_rows).  At the end every lane converts 16 consecutive pixels of a row, resets what it reads, and stores
+// (resolve_store_colour).
+__device__ __forceinline__ void composite_rows(unsigned long long* key, uint16_t* head, const unsigned long long* frag,
+                                               const ColourPool& pool, const RenderParams& P, const Job& jb, bool ego_active,
+                                               int ys, int row_lo, int row_hi, int lane) {
+    {
 #pragma unroll 1
-        for (int i = 0; i < CSTRIP_KEYS / 32; ++i) {
+        for (int i = row_lo * (TILE / 32); i < row_hi * (TILE / 32); ++i) {
             const int p = i * 32 + lane, x = p & (TILE - 1), y = p >> 6;
             const uint32_t hd = head[p];
             if (hd) {
@@ -299,6 +300,10 @@ __device__ __forceinline__ void resolve_store_colour(unsigned long long* key, ui
         }
         __syncwarp();
     }
+}
+
+__device__ __forceinline__ void resolve_store_colour(unsigned long long* key, const ColourPool& pool, const RenderParams& P, const Job& jb,
+                                                     bool ego_active, int ys, bool vec_ok, int lane) {
     const int y = lane >> 2, xs = (lane & 3) * 16;
     const int gy = jb.t.y0 + ys + y;
     uint32_t bgc = P.cls_sky;
@@ -486,6 +491,13 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
             const float* ray_x = s.ray_x[j];
             const float* ray_y = s.ray_y[j] + ys;
             const float du = __fdividef(1.f, s.cam[j].focx), dv = __fdividef(1.f, s.cam[j].focy);
+            // The lists of partially covering fragments are kept for a window of the strip's rows at a time: all eight,
+            // or, when the fragment array overflows (a dense soup of edges), half as many, again and again down to one
+            // row -- the window is rasterized anew, the rows before it keep their composited colours (parked in their
+            // keys, which no fragment can replace).
+            int win = CSTRIP, row_lo = 0;
+            while (row_lo < CSTRIP) {
+            const int row_hi = min(row_lo + win, CSTRIP);
             int n_frag = 0, n_pend = 0;
             bool dropped = false;
             for (int base = 0; base < cj; base += 32) {
@@ -509,7 +521,7 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                         const float w = fminf(fmaxf(fm(r3.x, ray_x[x], fm(r3.y, ray_y[y], r3.z)), P.w_far), P.w_near);
                         wb = __float_as_uint(w);
                         a14 = s.pool.surface[slot] >> 17;
-                        one = make_key(wb, 0xffffffffu) > key[key_index(x, y)];       // in front of the nearest fully covering fragment so far
+                        one = y >= row_lo && y < row_hi && make_key(wb, 0xffffffffu) > key[key_index(x, y)];   // in the window, in front of the nearest fully covering fragment so far
                     }
                     const unsigned m = __ballot_sync(0xffffffffu, one);
                     if (m) {
@@ -549,7 +561,7 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     hh[4] = hh[5] = 0.5f * (fabsf(q.wx) * du + fabsf(q.wy) * dv);
                     for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
                         for (int xx = bx0 & ~15; xx <= bx1; xx += 16)
-                            colour_cell<AA>(key, head, frag, n_frag, n_pend, dropped, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, lane);
+                            colour_cell<AA>(key, head, frag, n_frag, n_pend, dropped, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, row_lo, row_hi, lane);
                     // the queue is worked off when it holds a few rounds' worth (working it off frees room only for the
                     // pixels whose area turns out to be zero, so a nearly full array is no reason to do it earlier)
                     if (AA && n_pend >= 96) {
@@ -560,9 +572,19 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                 __syncwarp();
             }
             if (AA) flush_pending(frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
-            if (AA && dropped && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);
             __syncwarp();
-            resolve_store_colour<AA>(key, head, frag, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
+            if (AA && dropped && win > 1) {                       // too many fragments: this window again, half as many rows
+                for (int p = row_lo * TILE + lane; p < row_hi * TILE; p += 32) head[p] = 0;
+                __syncwarp();
+                win >>= 1;
+                continue;
+            }
+            if (AA && dropped && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);   // (more than 1 023 in one row of 64 pixels)
+            if (AA) composite_rows(key, head, frag, s.pool, P, jb, s.active[j] != 0, ys, row_lo, row_hi, lane);
+            row_lo = row_hi;
+            }   // (windows)
+            __syncwarp();
+            resolve_store_colour(key, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
             __syncwarp();
         }
         done |= now;

@@ -147,3 +147,27 @@ def test_paper_chunk_of_2048_egos_in_colour(gu):
     s2 = make_config(2, E=16)
     st2 = check_colour(gu, s2, views=np.sort(rng.choice(s2.E * s2.A * s2.K, size=64, replace=False)))
     print("cfg2 E=16 colour:", st2)
+
+
+def test_random_scenes_in_colour(gu):
+    # seeded random scenes (soups of triangles through the camera plane, pitched cameras, ragged sizes): plain and antialiased
+    from tests.util import random_scene
+    import oracle
+    pixels = flagged = mism = 0
+    for i, seed in enumerate([143, 209, 904, 1236] + list(range(1000, 1024))):
+        s = random_scene(seed, full_tiles=(i % 3 == 2))
+        g = gu.CudaRun(s)
+        try:
+            for aa in (False, True):
+                got, status = g.render_rgb(PAL, aa)
+                assert status == 0, f"seed {seed}: status {status}"
+                ref = oracle.render_rgb(s, PAL, aa)
+                try:
+                    st = compare_colour(ref, got, max_mismatch_frac=5e-3, max_flag_frac=0.1)
+                except AssertionError as ex:
+                    raise AssertionError(f"seed {seed}, antialias {aa}: {ex}") from ex
+                pixels += st["pixels"]; flagged += st["flagged"]; mism += st["mismatches"]
+        finally:
+            g.close()
+    print("random scenes in colour:", dict(pixels=pixels, flagged=flagged, mismatches=mism))
+    assert flagged < 0.02 * pixels
