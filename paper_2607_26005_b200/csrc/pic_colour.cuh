@@ -84,7 +84,7 @@ __device__ __forceinline__ uint32_t coverage14(const PixelLines& L, const PrimEq
 // the lists grow up from its bottom), a lane each: the record's six lines at the pixel, the exact area, the depth;
 // pixels with a positive area join their pixel's list.  The newest items -- those next to the lists' end -- go first,
 // so the entries written never reach items not yet read.
-__device__ __noinline__ void flush_pending(unsigned long long* frag, uint16_t* head, int& n_frag, int& n_pend, const ColourPool& pool,
+__device__ __noinline__ void flush_pending(const unsigned long long* key, unsigned long long* frag, uint16_t* head, int& n_frag, int& n_pend, const ColourPool& pool,
                                               const float* ray_x, const float* ray_y, float du, float dv, float w_near, float w_far, int lane) {
     while (n_pend > 0) {
         const int take = min(n_pend, 32);
@@ -129,6 +129,8 @@ __device__ __noinline__ void flush_pending(unsigned long long* frag, uint16_t* h
         if (have) {
             a14 = min((uint32_t)(area * 16383.f + 0.5f), COVERAGE_MAX);
             wc = fminf(fmaxf(w, w_far), w_near);
+            // (only fragments in front of the pixel's nearest fully covering fragment so far are kept)
+            if (!(make_key(__float_as_uint(wc), 0xffffffffu) > key[key_index((int)(pix & (TILE - 1)), (int)(pix >> 6))])) a14 = 0u;
         }
         n_pend -= take;
         // (two items of a round may belong to one pixel -- two records with a vertex there -- so the lists are
@@ -540,6 +542,37 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                         __syncwarp();
                     }
                 }
+                if (AA) {
+                    // records whose pixel box is at most 4 x 4: every pixel of the box (in this strip's window) is queued as
+                    // a (pixel, record) pair and worked off with the other pending pixels, a lane each -- far cheaper
+                    // than walking a 64-pixel cell per record for the handful of pixels a distant primitive touches
+                    const int bx0 = bw_lane & 63, bx1 = (bw_lane >> 12) & 63, by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
+                    const bool small = hit && bx1 - bx0 < 4 && by1 - by0 < 4;
+                    hit = hit && !small;
+                    const int w = bx1 - bx0 + 1, y0 = max(by0 - ys, row_lo), y1 = min(by1 - ys, row_hi - 1);
+                    const int cnt = small ? w * max(y1 - y0 + 1, 0) : 0;
+                    if (__any_sync(0xffffffffu, cnt > 0)) {
+                        int incl = cnt;
+#pragma unroll
+                        for (int d = 1; d < 32; d <<= 1) {
+                            const int up = __shfl_up_sync(0xffffffffu, incl, d);
+                            if (lane >= d) incl += up;
+                        }
+                        const int total = __shfl_sync(0xffffffffu, incl, 31);
+                        if (n_frag + n_pend + total <= CFRAGS) {
+                            const uint32_t slot = (uint32_t)(first + base + lane);
+                            for (int k = 0; k < cnt; ++k) {
+                                const uint32_t pix = (uint32_t)((y0 + k / w) * TILE + bx0 + k % w);
+                                frag[CFRAGS - (n_pend + (incl - cnt) + k)] = (pix << 8) | slot;
+                            }
+                            n_pend += total;
+                        } else {
+                            dropped = true;
+                        }
+                        __syncwarp();
+                        if (n_pend >= 96) flush_pending(key, frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
+                    }
+                }
                 for (unsigned hits = __ballot_sync(0xffffffffu, hit); hits; hits &= hits - 1) {
                     const int src = __ffs(hits) - 1;
                     const uint32_t bw = __shfl_sync(0xffffffffu, bw_lane, src);
@@ -566,12 +599,12 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     // pixels whose area turns out to be zero, so a nearly full array is no reason to do it earlier)
                     if (AA && n_pend >= 96) {
                         __syncwarp();
-                        flush_pending(frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
+                        flush_pending(key, frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
                     }
                 }
                 __syncwarp();
             }
-            if (AA) flush_pending(frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
+            if (AA) flush_pending(key, frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
             __syncwarp();
             if (AA && dropped && win > 1) {                       // too many fragments: this window again, half as many rows
                 for (int p = row_lo * TILE + lane; p < row_hi * TILE; p += 32) head[p] = 0;
