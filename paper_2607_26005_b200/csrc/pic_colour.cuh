@@ -304,7 +304,9 @@ __device__ __forceinline__ void composite_rows(unsigned long long* key, uint16_t
     }
 }
 
-__device__ __forceinline__ void resolve_store_colour(unsigned long long* key, const ColourPool& pool, const RenderParams& P, const Job& jb,
+// (the same with all 16 pixels of a lane unrolled and three 128-bit stores: faster where the kernel's code is small
+// enough anyway -- the plain instantiation)
+__device__ __forceinline__ void resolve_store_wide(unsigned long long* key, const ColourPool& pool, const RenderParams& P, const Job& jb,
                                                      bool ego_active, int ys, bool vec_ok, int lane) {
     const int y = lane >> 2, xs = (lane & 3) * 16;
     const int gy = jb.t.y0 + ys + y;
@@ -345,6 +347,53 @@ __device__ __forceinline__ void resolve_store_colour(unsigned long long* key, co
 #pragma unroll
         for (int n = 0; n < 48; ++n)
             if (n / 3 + xs < jb.t.tw) dst[n] = (uint8_t)(ow[n >> 2] >> (8 * (n & 3)));
+    }
+}
+
+__device__ __forceinline__ void resolve_store_colour(unsigned long long* key, const ColourPool& pool, const RenderParams& P, const Job& jb,
+                                                     bool ego_active, int ys, bool vec_ok, int lane) {
+    const int y = lane >> 2, xs = (lane & 3) * 16;
+    const int gy = jb.t.y0 + ys + y;
+    uint32_t bgc = P.cls_sky;
+    if (ego_active && gy < P.H) bgc = __ldg(P.rig.bg_cls + (size_t)jb.k * P.H + gy);
+    const uint32_t bg8 = (uint32_t)__ldg(P.palette + 3u * bgc) | ((uint32_t)__ldg(P.palette + 3u * bgc + 1) << 8) | ((uint32_t)__ldg(P.palette + 3u * bgc + 2) << 16);
+    const bool row_ok = ys + y < jb.t.th;
+    uint8_t* dst = P.out_rgb + 3u * ((jb.view * (size_t)P.H + gy) * (size_t)P.W + jb.t.x0 + xs);
+    // four groups of four pixels (12 bytes, three words) each; the loop is not unrolled: one copy of the shading code
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        uint32_t ow[3] = {0u, 0u, 0u};
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+            ulonglong2* kp = reinterpret_cast<ulonglong2*>(key + key_index(xs + 4 * g + 2 * h2, y));
+            const ulonglong2 kk = *kp;
+            *kp = make_ulonglong2(0ull, 0ull);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const unsigned long long k = h ? kk.y : kk.x;
+                uint32_t c = bg8;
+                if (k & KEY_RESOLVED) c = (uint32_t)k & 0xffffffu;
+                else if (k) {
+                    float R, G, B;
+                    shade_fragment(pool, P, (uint32_t)k & 0xffu, __uint_as_float((uint32_t)(k >> 32)), R, G, B);
+                    c = (uint32_t)fminf(R + 0.5f, 255.f) | ((uint32_t)fminf(G + 0.5f, 255.f) << 8) | ((uint32_t)fminf(B + 0.5f, 255.f) << 16);
+                }
+                const int n = 3 * (2 * h2 + h);      // byte offset of the pixel in the group's 12 bytes
+                ow[n >> 2] |= c << (8 * (n & 3));
+                if ((n & 3) > 1) ow[(n >> 2) + 1] |= c >> (8 * (4 - (n & 3)));
+            }
+        }
+        const int x = xs + 4 * g;
+        if (row_ok && x < jb.t.tw) {
+            if (vec_ok && x + 4 <= jb.t.tw) {
+                uint32_t* d32 = reinterpret_cast<uint32_t*>(dst + 12 * g);
+                d32[0] = ow[0]; d32[1] = ow[1]; d32[2] = ow[2];
+            } else {
+#pragma unroll
+                for (int n = 0; n < 12; ++n)
+                    if (n / 3 + x < jb.t.tw) dst[12 * g + n] = (uint8_t)(ow[n >> 2] >> (8 * (n & 3)));
+            }
+        }
     }
 }
 
@@ -617,7 +666,8 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
             row_lo = row_hi;
             }   // (windows)
             __syncwarp();
-            resolve_store_colour(key, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
+            if (AA) resolve_store_colour(key, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
+            else resolve_store_wide(key, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
             __syncwarp();
         }
         done |= now;
