@@ -94,7 +94,6 @@ __device__ __noinline__ void flush_pending(const unsigned long long* key, unsign
         uint32_t a14 = 0u;
         float wc = 0.f;
         const uint32_t pix = item >> 8, slot = item & 0xffu;
-        int n_cross = 0;
         float area = 0.f;
         float e[CLINES], a[CLINES], b[CLINES];
         float w = 0.f;
@@ -108,23 +107,7 @@ __device__ __noinline__ void flush_pending(const unsigned long long* key, unsign
             for (int j = 0; j < 4; ++j) { e[j] = fm(nx[j], rx, fm(ny[j], ry, nz[j])); a[j] = nx[j] * du; b[j] = ny[j] * dv; }
             w = fm(r3.x, rx, fm(r3.y, ry, r3.z));
             e[4] = w - w_far; e[5] = w_near - w; a[4] = r3.x * du; b[4] = r3.y * dv; a[5] = -a[4]; b[5] = -b[4];
-            // the lines that cross the pixel, up to four of them, moved to the front (the others contain the pixel)
-            const float hw = 0.5f * (fabsf(a[4]) + fabsf(b[4]));
-            float e3[4] = {1.f, 1.f, 1.f, 1.f}, a3[4] = {0.f, 0.f, 0.f, 0.f}, b3[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int j = 0; j < CLINES; ++j) {
-                const float hj = j < 4 ? 0.5f * (fabsf(a[j]) + fabsf(b[j])) : hw;
-                if (e[j] < hj) {
-                    ++n_cross;
-                    e3[3] = e3[2]; a3[3] = a3[2]; b3[3] = b3[2];
-                    e3[2] = e3[1]; a3[2] = a3[1]; b3[2] = b3[1]; e3[1] = e3[0]; a3[1] = a3[0]; b3[1] = b3[0];
-                    e3[0] = e[j]; a3[0] = a[j]; b3[0] = b[j];
-                }
-            }
-            area = pixel_coverage<4>(e3, a3, b3);
-        }
-        if (__any_sync(0xffffffffu, n_cross > 4)) {            // rare: more than four lines through one pixel
-            if (n_cross > 4) area = pixel_coverage<CLINES>(e, a, b);
+            area = pixel_coverage<CLINES>(e, a, b);
         }
         if (have) {
             a14 = min((uint32_t)(area * 16383.f + 0.5f), COVERAGE_MAX);
