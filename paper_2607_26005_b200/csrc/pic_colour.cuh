@@ -62,22 +62,21 @@ struct RayView { float* ray_x; float* ray_y; };
 struct PixelLines { float e[CLINES]; };
 
 // Coverage (14 bits) of one pixel by a record, given its lines at the pixel centre and their half ranges hh over
-// the pixel (a line with e >= hh contains the whole pixel): the closed forms for one line, or two lines that do
-// not cross inside the pixel.  Anything else (a vertex in the pixel, three lines) returns COVERAGE_PENDING: those
-// pixels are few per cell, so their areas are worked out later, a lane each (finish_coverage).
+// the pixel (a line with e >= hh contains the whole pixel): the closed form if exactly one line crosses the pixel.
+// Anything else (two or more lines: a strip, a vertex) returns COVERAGE_PENDING: those pixels are few per cell, so
+// their areas are worked out later, a lane each (flush_pending) -- which is also less code in the cell loop, and the
+// instruction cache is this kernel's bottleneck.
 constexpr uint32_t COVERAGE_PENDING = 0x3fffu, COVERAGE_MAX = 0x3ffeu;
 __device__ __forceinline__ uint32_t coverage14(const PixelLines& L, const PrimEq& q, const float (&hh)[CLINES], float du, float dv) {
     int n_part = 0;
-    float e1 = 0.f, a1 = 0.f, b1 = 0.f, e2 = 0.f, a2 = 0.f, b2 = 0.f;      // the last two lines that cross the pixel
+    float e1 = 0.f, a1 = 0.f, b1 = 0.f;      // the line that crosses the pixel
 #pragma unroll
     for (int i = 0; i < CLINES; ++i) {
         const float ai = (i < 4 ? q.nx[i] : i == 4 ? q.wx : -q.wx) * du, bi = (i < 4 ? q.ny[i] : i == 4 ? q.wy : -q.wy) * dv;
-        if (L.e[i] < hh[i]) { ++n_part; e2 = e1; a2 = a1; b2 = b1; e1 = L.e[i]; a1 = ai; b1 = bi; }
+        if (L.e[i] < hh[i]) { ++n_part; e1 = L.e[i]; a1 = ai; b1 = bi; }
     }
-    float alpha = 0.f;
-    if (n_part == 1) alpha = edge_coverage(e1, a1, b1);
-    else if (n_part != 2 || !two_line_coverage(e1, a1, b1, e2, a2, b2, alpha)) return COVERAGE_PENDING;
-    return min((uint32_t)(alpha * 16383.f + 0.5f), COVERAGE_MAX);
+    if (n_part != 1) return COVERAGE_PENDING;
+    return min((uint32_t)(edge_coverage(e1, a1, b1) * 16383.f + 0.5f), COVERAGE_MAX);
 }
 
 // The strip's queue of pending pixels (pixel << 8 | slot; it grows down from the top of the fragment array while

@@ -1,5 +1,5 @@
 // Analytic coverage of a pixel (internal; included by pic_colour.cuh): the area of the pixel's unit square on the
-// inner side of one line (closed form) or of six lines (a record's four edges and the two lines at which its
+// inner side of one line (closed form) or of several lines (a record's four edges and the two lines at which its
 // plane reaches the far and the near depth).
 #pragma once
 #include "pic_device.cuh"
@@ -68,40 +68,6 @@ __device__ __forceinline__ float pixel_coverage(const float (&e)[NL], const floa
         A[N - 1] = ra; B[N - 1] = rb; C[N - 1] = rc;
     }
     return fminf(fmaxf(0.5f * twice, 0.f), 1.f);
-}
-
-// A point of the line e + a x + b y = 0 inside the pixel's square (the middle of its chord); false if it misses the square.
-__device__ __forceinline__ bool chord_point(float e, float a, float b, float& px, float& py) {
-    const float n2 = fm(a, a, mul(b, b));
-    const float k = -__fdividef(e, n2), p0x = k * a, p0y = k * b;
-    float t0 = -3e38f, t1 = 3e38f;
-    // x(t) = p0x + t b within [-1/2, 1/2], y(t) = p0y - t a within [-1/2, 1/2]
-    if (b != 0.f) { const float u = __fdividef(-0.5f - p0x, b), v = __fdividef(0.5f - p0x, b); t0 = fmaxf(t0, fminf(u, v)); t1 = fminf(t1, fmaxf(u, v)); }
-    else if (fabsf(p0x) > 0.5f) return false;
-    if (a != 0.f) { const float u = __fdividef(p0y + 0.5f, a), v = __fdividef(p0y - 0.5f, a); t0 = fmaxf(t0, fminf(u, v)); t1 = fminf(t1, fmaxf(u, v)); }
-    else if (fabsf(p0y) > 0.5f) return false;
-    const float tm = 0.5f * (t0 + t1);
-    px = fm(tm, b, p0x); py = fm(-tm, a, p0y);
-    return t1 >= t0;
-}
-
-// Area of the pixel's square inside two lines that do not cross inside it (a strip, two nested half planes, two
-// separate corners): from the two one-line coverages.  Returns false if the lines cross inside the square (or too
-// near its border to tell): then the area takes the general formula.
-__device__ __forceinline__ bool two_line_coverage(float e1, float a1, float b1, float e2, float a2, float b2, float& area) {
-    const float det = fm(a1, b2, -mul(a2, b1));
-    const float scale = (fabsf(a1) + fabsf(b1)) * (fabsf(a2) + fabsf(b2));
-    if (fabsf(det) > 1e-6f * scale) {
-        const float x = __fdividef(fm(b1, e2, -mul(b2, e1)), det), y = __fdividef(fm(a2, e1, -mul(a1, e2)), det);
-        if (fabsf(x) < 0.5001f && fabsf(y) < 0.5001f) return false;
-    }
-    float p1x, p1y, p2x, p2y;
-    if (!chord_point(e1, a1, b1, p1x, p1y) || !chord_point(e2, a2, b2, p2x, p2y)) return false;
-    const float c1 = edge_coverage(e1, a1, b1), c2 = edge_coverage(e2, a2, b2);
-    const bool in2 = fm(a2, p1x, fm(b2, p1y, e2)) >= 0.f;     // line 1's chord lies inside line 2
-    const bool in1 = fm(a1, p2x, fm(b1, p2y, e1)) >= 0.f;
-    area = (in1 && in2) ? fmaxf(c1 + c2 - 1.f, 0.f) : in1 ? c2 : in2 ? c1 : 0.f;
-    return true;
 }
 
 }  // namespace pic
