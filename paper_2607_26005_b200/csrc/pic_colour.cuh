@@ -244,7 +244,7 @@ __device__ __forceinline__ uint32_t composite_pixel(unsigned long long k, uint32
         if (best) { prev = best; slot = (best_lo >> 10) & 0xffu; alpha = (float)((best_lo >> 18) & 0x3fffu) * (1.f / 16383.f); wb = (uint32_t)(best >> 32); }
         else if (k && prev != 0ull) { prev = 0ull; slot = (uint32_t)k & 0xffu; alpha = 1.f; wb = w_opq; }
         else break;
-        const uint32_t surf = pool.surface[slot] & 0x1ffffu;
+        const uint32_t surf = pool.surface[slot];
         if (surf != cur) { T *= 1.f - acc; cur = surf; acc = 0.f; }
         const float add = fminf(alpha, 1.f - acc) * T;
         float cr, cg, cb;
@@ -466,39 +466,12 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                 const int slot = my_base + i;
                 if (drop || !prim_equations(V, flags & 1u, flags, Pn, q)) { s.pool.box[slot] = REC_DEAD; continue; }
                 const uint32_t box = svi.y;
-                uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
-                uint32_t onepix = 0u;
-                if (AA) {
-                    // a primitive that lies inside one pixel and well within the depth range covers its own projected
-                    // area of that pixel and nothing else: no clipping needed (most distant primitives are of this kind)
-                    const float zlo = fminf(fminf(V[0].z, V[1].z), fminf(V[2].z, V[3].z)), zhi = fmaxf(fmaxf(V[0].z, V[1].z), fmaxf(V[2].z, V[3].z));
-                    if (zlo >= P.near_z * 1.001f && zhi <= P.far_z * 0.999f) {
-                        float sx[4], sy[4];
-#pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            const float iz = __fdividef(1.f, V[v].z);
-                            sx[v] = fm(c.focx, V[v].x * iz, c.cx - (float)job.t.x0); sy[v] = fm(c.focy, V[v].y * iz, c.cy - (float)job.t.y0);
-                        }
-                        const float x_lo = fminf(fminf(sx[0], sx[1]), fminf(sx[2], sx[3])), x_hi = fmaxf(fmaxf(sx[0], sx[1]), fmaxf(sx[2], sx[3]));
-                        const float y_lo = fminf(fminf(sy[0], sy[1]), fminf(sy[2], sy[3])), y_hi = fmaxf(fmaxf(sy[0], sy[1]), fmaxf(sy[2], sy[3]));
-                        const float fxl = floorf(x_lo + 1e-4f), fyl = floorf(y_lo + 1e-4f);
-                        if (floorf(x_hi - 1e-4f) <= fxl && floorf(y_hi - 1e-4f) <= fyl && x_hi - x_lo < 1.f && y_hi - y_lo < 1.f) {
-                            float twice = 0.f;
-#pragma unroll
-                            for (int v = 0; v < 4; ++v) twice += (sx[v] - x_lo) * (sy[(v + 1) & 3] - y_lo) - (sx[(v + 1) & 3] - x_lo) * (sy[v] - y_lo);
-                            const uint32_t a14 = min((uint32_t)(0.5f * fabsf(twice) * 16383.f + 0.5f), COVERAGE_MAX);
-                            if (a14 == 0u || fxl < 0.f || fyl < 0.f || fxl >= (float)job.t.tw || fyl >= (float)job.t.th) { s.pool.box[slot] = REC_DEAD; continue; }
-                            bx0 = bx1 = (uint32_t)fxl; by0 = by1 = (uint32_t)fyl;
-                            onepix = REC_TINY;
-                            surface |= a14 << 17;
-                        }
-                    }
-                }
+                const uint32_t bx0 = box & 0xff, by0 = (box >> 8) & 0xff, bx1 = (box >> 16) & 0xff, by1 = box >> 24;
                 s.pool.nx[slot] = make_float4(q.nx[0], q.nx[1], q.nx[2], q.nx[3]);
                 s.pool.ny[slot] = make_float4(q.ny[0], q.ny[1], q.ny[2], q.ny[3]);
                 s.pool.nz[slot] = make_float4(q.nz[0], q.nz[1], q.nz[2], q.nz[3]);
                 s.pool.w[slot] = make_float4(q.wx, q.wy, q.wz, __uint_as_float(key_lo));
-                s.pool.box[slot] = bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24) | onepix;
+                s.pool.box[slot] = bx0 | (by0 << 6) | (bx1 << 12) | (by1 << 18) | (q.tl << 24);
                 s.pool.shade[slot] = shade;
                 s.pool.surface[slot] = surface;
             }
@@ -540,38 +513,6 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     bw_lane = s.pool.box[first + base + lane];
                     const int by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
                     hit = !(bw_lane & REC_DEAD) && by1 >= ys && by0 < ys + CSTRIP;
-                }
-                if (AA) {
-                    // records that lie inside one pixel: their lane adds the fragment (coverage known from set-up)
-                    bool one = hit && (bw_lane & REC_TINY);
-                    hit = hit && !one;
-                    uint32_t pix = 0u, a14 = 0u, wb = 0u;
-                    const uint32_t slot = (uint32_t)(first + base + lane);
-                    if (one) {
-                        const int x = bw_lane & 63, y = ((bw_lane >> 6) & 63) - ys;
-                        pix = (uint32_t)(y * TILE + x);
-                        const float4 r3 = s.pool.w[slot];
-                        const float w = fminf(fmaxf(fm(r3.x, ray_x[x], fm(r3.y, ray_y[y], r3.z)), P.w_far), P.w_near);
-                        wb = __float_as_uint(w);
-                        a14 = s.pool.surface[slot] >> 17;
-                        one = y >= row_lo && y < row_hi && make_key(wb, 0xffffffffu) > key[key_index(x, y)];   // in the window, in front of the nearest fully covering fragment so far
-                    }
-                    const unsigned m = __ballot_sync(0xffffffffu, one);
-                    if (m) {
-                        const bool room = n_frag + n_pend + __popc(m) <= CFRAGS;
-                        dropped = dropped || !room;
-                        const int idx = n_frag + 1 + __popc(m & ((1u << lane) - 1u));
-                        const bool alone = __popc(__match_any_sync(0xffffffffu, one ? pix : 0x10000u + lane)) == 1;
-                        if (room) {
-                            if (one && alone) { frag[idx] = ((unsigned long long)wb << 32) | (a14 << 18) | (slot << 10) | head[pix]; head[pix] = (uint16_t)idx; }
-                            for (unsigned rest = __ballot_sync(0xffffffffu, one && !alone); rest; rest &= rest - 1) {
-                                if (lane == __ffs(rest) - 1) { frag[idx] = ((unsigned long long)wb << 32) | (a14 << 18) | (slot << 10) | head[pix]; head[pix] = (uint16_t)idx; }
-                                __syncwarp();
-                            }
-                            n_frag += __popc(m);
-                        }
-                        __syncwarp();
-                    }
                 }
                 if (AA) {
                     // records whose pixel box is at most 4 x 4: every pixel of the box (in this strip's window) is queued as
