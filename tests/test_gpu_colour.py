@@ -171,3 +171,14 @@ def test_random_scenes_in_colour(gu):
             g.close()
     print("random scenes in colour:", dict(pixels=pixels, flagged=flagged, mismatches=mism))
     assert flagged < 0.02 * pixels
+
+
+def test_many_tiles_per_view_in_colour(gu):
+    # configs[3] (128 x 256: 8 tiles per view, one 37 k-triangle map, far 150 m) and the paper's rig at 384 x 216 (24 tiles)
+    s = make_config(3, E=1)
+    st = check_colour(gu, s, views=[0, 101, 202])
+    print("cfg3 colour:", st)
+    s = make_paper_workload(384, 216, E=1)
+    act = np.flatnonzero(np.repeat(s.active.reshape(-1), s.K))
+    st = check_colour(gu, s, views=act[:3], modes=(True,))
+    print("paper 384x216 colour:", st)
