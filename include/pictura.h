@@ -257,6 +257,9 @@ pic_status pic_map_stats(const pic_scene_desc* desc, int64_t out[8]);
 pic_status pic_set_palette(pic_scene* scene, const uint8_t* rgb_host, void* cuda_stream);
 pic_status pic_render_rgb(pic_scene* scene, const float* poses, const float* dims, const uint8_t* active,
                           const pic_camera* rig_host, int32_t antialias, uint8_t* out_rgb, void* cuda_stream);
+/* pic_step with colour output: the bicycle update of pic_step, then pic_render_rgb from the new state. */
+pic_status pic_step_rgb(pic_scene* scene, const float* actions, const pic_camera* rig_host, int32_t antialias,
+                        uint8_t* out_rgb, void* cuda_stream);
 
 /*
  * pic_render_static -- render without a scene object and without any allocation.

@@ -23,7 +23,7 @@ FLAG_COLOUR_INCOMPLETE = 2
 FLAG_COLOUR_FRAGMENTS = 4
 
 EXPORTS = ["pic_scene_create", "pic_scene_destroy", "pic_render", "pic_render_host", "pic_set_state",
-           "pic_get_state", "pic_set_agent_classes", "pic_set_palette", "pic_render_rgb", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
+           "pic_get_state", "pic_set_agent_classes", "pic_set_palette", "pic_render_rgb", "pic_step_rgb", "pic_step", "pic_get_status", "pic_scene_set_option", "pic_get_kernel_times", "pic_map_stats", "pic_render_static", "pic_static_status", "pic_probe_fill", "pic_probe_ffma",
            "pic_last_error", "pic_version"]
 
 
@@ -76,6 +76,7 @@ def load(path: Optional[str] = None):
     lib.pic_set_agent_classes.argtypes = [vp, vp, vp]
     lib.pic_set_palette.argtypes = [vp, vp, vp]
     lib.pic_render_rgb.argtypes = [vp, vp, vp, vp, C.POINTER(pic_camera), C.c_int32, vp, vp]
+    lib.pic_step_rgb.argtypes = [vp, vp, C.POINTER(pic_camera), C.c_int32, vp, vp]
     lib.pic_step.argtypes = [vp, vp, C.POINTER(pic_camera), vp, vp, vp]
     lib.pic_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.pic_scene_set_option.argtypes = [vp, C.c_int32, C.c_uint64]
@@ -361,6 +362,16 @@ class Scene:
             self._h, _dev_ptr(actions, torch.float32, 2 * n), _rig_array(rig), _dev_ptr(out_class, torch.uint8, npx),
             _dev_ptr(out_depth, torch.float16, npx), _stream_ptr(stream)))
         return out_class, out_depth
+
+    def step_rgb(self, actions, rig, out_rgb=None, antialias=False, stream=None):
+        """One simulator step, then colour images u8 [E,A,K,H,W,3] from the new state."""
+        import torch
+        if out_rgb is None:
+            out_rgb = torch.empty(self.image_shape + (3,), dtype=torch.uint8, device=self.device)
+        _check(self._lib, self._lib.pic_step_rgb(
+            self._h, _dev_ptr(actions, torch.float32, 2 * self.n_agents), _rig_array(rig), 1 if antialias else 0,
+            _dev_ptr(out_rgb, torch.uint8), _stream_ptr(stream)))
+        return out_rgb
 
     def status(self, stream=None) -> int:
         flags = C.c_uint32(0)

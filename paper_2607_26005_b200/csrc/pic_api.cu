@@ -522,6 +522,14 @@ pic_status pic_step(pic_scene* s, const float* actions, const pic_camera* rig, u
                        static_cast<cudaStream_t>(cuda_stream));
 }
 
+pic_status pic_step_rgb(pic_scene* s, const float* actions, const pic_camera* rig, int32_t antialias, uint8_t* out_rgb,
+                        void* cuda_stream) {
+    if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
+    if (!actions || !out_rgb) return fail(PIC_ERR_INVALID_ARG, "actions or out_rgb is NULL");
+    return render_from(s, nullptr, s->d_state, actions, s->d_dims, s->d_active, rig, nullptr, nullptr,
+                       static_cast<cudaStream_t>(cuda_stream), out_rgb, antialias != 0);
+}
+
 pic_status pic_get_kernel_times(pic_scene* s, float* ms, int32_t capacity, int32_t* n) {
     if (!s) return fail(PIC_ERR_INVALID_ARG, "scene is NULL");
     if (!n || (capacity > 0 && !ms)) return fail(PIC_ERR_INVALID_ARG, "ms or n is NULL");

@@ -182,3 +182,27 @@ def test_many_tiles_per_view_in_colour(gu):
     act = np.flatnonzero(np.repeat(s.active.reshape(-1), s.K))
     st = check_colour(gu, s, views=act[:3], modes=(True,))
     print("paper 384x216 colour:", st)
+
+
+def test_step_with_colour_output(gu):
+    # pic_step_rgb = the bicycle update of pic_step, then the colour images of the new state
+    import torch
+    from scenes import make_actions
+    s = make_config(1, E=1)
+    g = gu.CudaRun(s)
+    try:
+        g.scene.set_palette(PAL)
+        state = torch.from_numpy(s.state()).to(g.dev)
+        acts = torch.from_numpy(make_actions(4, 1, s.E, s.A)).to(g.dev)
+        g.scene.set_state(state, g.dims, g.active)
+        rgb = g.scene.step_rgb(acts, s.rig, antialias=True)
+        new_state = g.scene.get_state()
+        g.scene.set_state(state, g.dims, g.active)
+        g.scene.step(acts, s.rig)
+        assert torch.equal(new_state, g.scene.get_state())                  # the same update as pic_step
+        again = g.scene.render_rgb(new_state[..., :3].contiguous(), g.dims, s.rig, active=g.active, antialias=True)
+        torch.cuda.synchronize()
+        assert torch.equal(rgb, again) and g.scene.status() == 0
+        assert not torch.equal(rgb, g.scene.render_rgb(g.poses, g.dims, s.rig, active=g.active, antialias=True))   # the agents moved
+    finally:
+        g.close()
