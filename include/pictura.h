@@ -69,8 +69,8 @@ typedef enum {
                                         its state as it was */
 #define PIC_FLAG_COLOUR_INCOMPLETE 0x2u /* pic_render_rgb: a 64 x 64 tile saw more primitives than its list holds (254) and shows
                                            only the background */
-#define PIC_FLAG_COLOUR_FRAGMENTS 0x4u  /* pic_render_rgb, antialiased: one row of a tile (64 pixels) held more than 1023 partially
-                                           covered pixel fragments in front of its opaque surfaces; the surplus was dropped */
+#define PIC_FLAG_COLOUR_FRAGMENTS 0x4u  /* pic_render_rgb, antialiased: one pixel held more than 1023 partially covering
+                                           fragments in front of its opaque surface; the surplus was dropped */
 
 /* One pinhole camera of the rig, in the agent frame (x forward, y left, z up). */
 typedef struct {

@@ -141,7 +141,7 @@ template <bool AA>
 __device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* head, unsigned long long* frag, int& n_frag, int& n_pend, bool& dropped,
                                             const float* ray_x, const float* ray_y, const PrimEq& q, const float (&thr)[4],
                                             const float (&hh)[CLINES], float du, float dv, uint32_t key_lo, uint32_t slot,
-                                            float w_near, float w_far, int xx, int yy, int row_lo, int row_hi, int lane) {
+                                            float w_near, float w_far, int xx, int yy, int row_lo, int row_hi, int col_lo, int col_hi, int lane) {
     const int x = xx + (lane & 7) * 2, y = yy + (lane >> 3);
     const float2 rx = *reinterpret_cast<const float2*>(ray_x + x);
     const float ry = ray_y[y];
@@ -174,8 +174,9 @@ __device__ __forceinline__ void colour_cell(unsigned long long* key, uint16_t* h
     if (full1 && k1 > kk.y) kp[1] = k1;
     if (AA) {
         // partially covered pixels in front of the nearest fully covering fragment seen so far
-        const bool in_window = y >= row_lo && y < row_hi;      // (lists are kept for a window of the strip's rows at a time)
-        bool push0 = in_window && !full0 && !out0 && k0 > kk.x, push1 = in_window && !full1 && !out1 && k1 > kk.y;
+        const bool in_rows = y >= row_lo && y < row_hi;        // (lists are kept for a window of the strip's pixels at a time)
+        bool push0 = in_rows && x >= col_lo && x < col_hi && !full0 && !out0 && k0 > kk.x;
+        bool push1 = in_rows && x + 1 >= col_lo && x + 1 < col_hi && !full1 && !out1 && k1 > kk.y;
         if (__any_sync(0xffffffffu, push0 || push1)) {
             // (one copy of the coverage code serves both pixels: the instruction cache matters more than the selects)
             uint32_t a0 = 0u, a1 = 0u;
@@ -500,10 +501,15 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
             // The lists of partially covering fragments are kept for a window of the strip's rows at a time: all eight,
             // or, when the fragment array overflows (a dense soup of edges), half as many, again and again down to one
             // row -- the window is rasterized anew, the rows before it keep their composited colours (parked in their
-            // keys, which no fragment can replace).
-            int win = CSTRIP, row_lo = 0;
-            while (row_lo < CSTRIP) {
-            const int row_hi = min(row_lo + win, CSTRIP);
+            // keys, which no fragment can replace).  Before the first such retry the strip is rasterized once with an
+            // empty window: that leaves every pixel's nearest fully covering fragment in its key, so the retries keep
+            // only the fragments in front of it (in a soup, few).  A single row that still overflows (many coplanar
+            // primitives cut by the near plane along it) is taken half as many columns at a time, down to one pixel.
+            int win = CSTRIP, cw = TILE, row_next = 0, col_next = 0;
+            bool prepass = false, prepass_done = false;
+            while (row_next < CSTRIP) {
+            const int row_lo = prepass ? 0 : row_next, row_hi = prepass ? 0 : min(row_next + win, CSTRIP);
+            const int col_lo = col_next, col_hi = col_next + cw;
             int n_frag = 0, n_pend = 0;
             bool dropped = false;
             for (int base = 0; base < cj; base += 32) {
@@ -521,7 +527,8 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     const int bx0 = bw_lane & 63, bx1 = (bw_lane >> 12) & 63, by0 = (bw_lane >> 6) & 63, by1 = (bw_lane >> 18) & 63;
                     const bool small = hit && bx1 - bx0 < 4 && by1 - by0 < 4;
                     hit = hit && !small;
-                    const int w = bx1 - bx0 + 1, y0 = max(by0 - ys, row_lo), y1 = min(by1 - ys, row_hi - 1);
+                    const int x0 = max(bx0, col_lo), x1 = min(bx1, col_hi - 1);
+                    const int w = max(x1 - x0 + 1, 0), y0 = max(by0 - ys, row_lo), y1 = min(by1 - ys, row_hi - 1);
                     const int cnt = small ? w * max(y1 - y0 + 1, 0) : 0;
                     if (__any_sync(0xffffffffu, cnt > 0)) {
                         int incl = cnt;
@@ -534,7 +541,7 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                         if (n_frag + n_pend + total <= CFRAGS) {
                             const uint32_t slot = (uint32_t)(first + base + lane);
                             for (int k = 0; k < cnt; ++k) {
-                                const uint32_t pix = (uint32_t)((y0 + k / w) * TILE + bx0 + k % w);
+                                const uint32_t pix = (uint32_t)((y0 + k / w) * TILE + x0 + k % w);
                                 frag[CFRAGS - (n_pend + (incl - cnt) + k)] = (pix << 8) | slot;
                             }
                             n_pend += total;
@@ -566,7 +573,7 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
                     hh[4] = hh[5] = 0.5f * (fabsf(q.wx) * du + fabsf(q.wy) * dv);
                     for (int yy = ly0 & ~3; yy <= ly1; yy += 4)
                         for (int xx = bx0 & ~15; xx <= bx1; xx += 16)
-                            colour_cell<AA>(key, head, frag, n_frag, n_pend, dropped, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, row_lo, row_hi, lane);
+                            colour_cell<AA>(key, head, frag, n_frag, n_pend, dropped, ray_x, ray_y, q, thr, hh, du, dv, key_lo, slot, P.w_near, P.w_far, xx, yy, row_lo, row_hi, col_lo, col_hi, lane);
                     // the queue is worked off when it holds a few rounds' worth (working it off frees room only for the
                     // pixels whose area turns out to be zero, so a nearly full array is no reason to do it earlier)
                     if (AA && n_pend >= 96) {
@@ -578,15 +585,20 @@ __global__ void __launch_bounds__(NTHREADS, 3) colour_kernel(const __grid_consta
             }
             if (AA) flush_pending(key, frag, head, n_frag, n_pend, s.pool, ray_x, ray_y, du, dv, P.w_near, P.w_far, lane);
             __syncwarp();
-            if (AA && dropped && win > 1) {                       // too many fragments: this window again, half as many rows
-                for (int p = row_lo * TILE + lane; p < row_hi * TILE; p += 32) head[p] = 0;
+            if (AA && prepass) { prepass = false; prepass_done = true; continue; }
+            if (AA && dropped && (!prepass_done || win > 1 || cw > 1)) {    // too many fragments: this window again
+                for (int p = row_lo * TILE + lane; p < row_hi * TILE; p += 32)
+                    if ((p & (TILE - 1)) >= col_lo) head[p] = 0;  // (the columns before the window are done: their heads are 0)
                 __syncwarp();
-                win >>= 1;
+                if (!prepass_done) prepass = true;                // ... after the keys have been completed,
+                else if (win > 1) win >>= 1;                      // ... then with half as many rows,
+                else cw >>= 1;                                    // ... then with half as many columns of the one row
                 continue;
             }
-            if (AA && dropped && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);   // (more than 1 023 in one row of 64 pixels)
+            if (AA && dropped && lane == 0) atomicOr(P.status, STATUS_COLOUR_FRAGMENTS);   // (more than 1 023 in front of the opaque surface of one pixel)
             if (AA) composite_rows(key, head, frag, s.pool, P, jb, s.active[j] != 0, ys, row_lo, row_hi, lane);
-            row_lo = row_hi;
+            col_next += cw;
+            if (col_next >= TILE) { col_next = 0; row_next = row_hi; }
             }   // (windows)
             __syncwarp();
             if (AA) resolve_store_colour(key, s.pool, P, jb, s.active[j] != 0, ys, vec_ok, lane);
