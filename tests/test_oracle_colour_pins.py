@@ -217,6 +217,12 @@ def test_layers_are_composited_front_to_back():
     # two pieces of ONE surface (same class) are complementary instead: 0.2 + 0.7 of the pixel, the rest background
     r = oracle.render_rgb(single_env(pole + back, [7, 7, 7, 7], [ego()], rig=RIG8, H=8, W=8), PAL, True)
     assert np.allclose(r.rgbf[0][2, 3], 0.9 * PAL[7] + 0.1 * SKY, atol=1e-9)
+    # a layer never holds more than the whole pixel: the pole in front of a wall of its own class that covers the pixel
+    # fully adds nothing (0.2 + 1 is capped at 1), and nothing behind the layer shows
+    full = wall(4.0, 1.0, 7.0, 0.0, 8.0)
+    hidden = wall(6.0, 0.0, 8.0, 0.0, 8.0, scale=1.5)
+    r = oracle.render_rgb(single_env(pole + full + hidden, [7, 7, 7, 7, 6, 6], [ego()], rig=RIG8, H=8, W=8), PAL, True)
+    assert np.allclose(r.rgbf[0][2, 3], PAL[7], atol=1e-9) and np.allclose(r.rgbf[0][5, 3], PAL[7], atol=1e-9)
 
 
 def test_a_mesh_has_no_seams_and_does_not_depend_on_its_triangulation():
